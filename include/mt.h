@@ -1,0 +1,131 @@
+/*
+ * mt.h - C ABI of the mixed-tenant batched inference library (one B200, sm_100a).
+ *
+ * The paper (arXiv 1901.06887) frames DNN inference as a narrow interface: a
+ * tenant uploads a model as a declarative list of standard layers (Sec. 3.1:
+ * no user code, a fixed layer catalogue), then sends requests; a DNN is a
+ * stateless deterministic function evaluated layer by layer (Sec. 1.1); a
+ * worker hosts many tenants' models at once and multiplexes incoming requests
+ * across them (Sec. 3).  This library is that worker's execution step:
+ * mt_infer evaluates ONE mixed batch of requests, each tagged with the id of
+ * its model, in a single pass over all co-resident models.
+ *
+ * Threading: all calls are serialised by one internal mutex.  A context has
+ * one workspace, so two mt_infer calls must not be in flight on different
+ * streams at the same time (order them with events, or use one stream).
+ *
+ * Every function returns an mt_status; MT_OK (0) is success.  No function
+ * throws, traps or aborts.  There is no CPU fallback: on a device that is not
+ * compute capability 10.x mt_init fails with MT_ERR_ARCH.
+ */
+#ifndef MT_H_
+#define MT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MT_OK = 0,
+    MT_ERR_INVALID_ARG = 1,   /* null pointer, negative size, bad enum value */
+    MT_ERR_BAD_MODEL_ID = 2,  /* id never issued, already released, or (async) seen in a batch */
+    MT_ERR_SHAPE = 3,         /* layer chain inconsistent, or model does not match the hosted family */
+    MT_ERR_UNSUPPORTED = 4,   /* a dimension outside what the kernels handle (see mt_register_model) */
+    MT_ERR_OOM = 5,           /* device or host allocation failed, or table full */
+    MT_ERR_CUDA = 6,          /* a CUDA runtime/driver call failed */
+    MT_ERR_ARCH = 7,          /* device is not sm_100 */
+    MT_ERR_TIMEOUT = 8,       /* (async) a bounded device-side wait gave up */
+    MT_ERR_NOT_INIT = 9
+} mt_status;
+
+typedef enum { MT_DENSE = 0, MT_CONV3X3 = 1, MT_GLOBAL_AVG_POOL = 2 } mt_layer_kind;
+
+#define MT_MAX_LAYERS 8
+
+/* One layer of a declarative model description (Sec. 3.1).
+ *   MT_DENSE            y = act(W x + b), W bf16 [out_ch][in_ch] row-major (Sec. 1.1, fully-connected layer)
+ *   MT_CONV3X3          NHWC, stride 1, zero pad 1, cross-correlation; W bf16 [out_ch][3][3][in_ch];
+ *                       tap (ky,kx) reads pixel (y+ky-1, x+kx-1)
+ *   MT_GLOBAL_AVG_POOL  mean over the h*w positions of each channel; no weights
+ * weight / bias may be host or device pointers; the library copies them during mt_register_model and
+ * keeps no reference, so the caller may free them on return.  bias == NULL means zeros. */
+typedef struct {
+    int32_t kind;          /* mt_layer_kind */
+    int32_t in_ch, out_ch; /* dense: in/out features; conv: C_in/C_out; pool: in_ch == out_ch */
+    int32_t h, w;          /* conv/pool spatial size; 0 for dense */
+    int32_t relu;          /* 1: apply max(.,0) after bias */
+    const void* weight;    /* bf16 */
+    const void* bias;      /* fp32 [out_ch] */
+} mt_layer_desc;
+
+/* Create the context on CUDA device `device`.  max_models bounds the id space (<= 8192), max_batch is
+ * a hint for the first workspace allocation (the workspace grows on demand, see mt_infer).  Calling
+ * mt_register_model before mt_init initialises device 0 with defaults (1024 models).
+ * Errors: MT_ERR_ARCH, MT_ERR_CUDA, MT_ERR_OOM, MT_ERR_INVALID_ARG (already initialised with other
+ * arguments is accepted and ignored). */
+mt_status mt_init(int32_t device, int32_t max_models, int32_t max_batch);
+
+/* Release every model, workspace and the context.  Synchronises the device. */
+mt_status mt_shutdown(void);
+
+/* "Upload your model" (Sec. 1.2 / Sec. 3): validate the layer list, copy the weights to the device in
+ * the executor's tiled layout and return a small dense id (lowest free slot first) in *model_id_out.
+ * All models hosted by one context form one family: same number and kinds of layers, same input and
+ * output element counts, same conv geometry.  Hidden dense widths may differ per model.
+ * Kernel limits (else MT_ERR_UNSUPPORTED): 1..MT_MAX_LAYERS layers; dense in_ch a multiple of 64;
+ * conv in_ch == out_ch == 64, w <= 128; a pool must follow a conv; a dense layer may not precede a conv.
+ * Synchronous: returns after the copies have completed. */
+mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32_t* model_id_out);
+
+/* predict(model, input) for a whole mixed batch (Sec. 3: a worker multiplexes requests across models).
+ *   inputs    device, bf16, [n][in_elems] row-major (NHWC per request for conv), arrival order
+ *   model_ids device, int32 [n]; request i is evaluated by model model_ids[i]
+ *   outputs   device, fp32, [n][out_elems], arrival order
+ *   stream    cudaStream_t (NULL = default stream)
+ * Only enqueues work on `stream`: bucketing (histogram, exclusive scan, stable scatter, row gather), one
+ * persistent grouped launch per layer, un-permute.  No host<->device synchronisation happens unless the
+ * workspace must grow (n larger than any earlier call, or a wider model registered since): then the
+ * call synchronises the device and reallocates first - make one call at the largest n before timing.
+ * inputs must be 16-byte aligned.  n == 0 is a no-op.
+ * A request whose id is not a live model never faults: its output row is NaN, a sticky status is set
+ * (see mt_get_async_status) and all other requests complete normally. */
+mt_status mt_infer(const void* inputs, const int32_t* model_ids, int32_t n, void* outputs, void* stream);
+
+/* Same as mt_infer with HOST buffers (pinned memory recommended): copies inputs and ids to device
+ * staging buffers on `stream`, runs the pass, copies the outputs back and synchronises `stream`. */
+mt_status mt_infer_host(const void* inputs_host, const int32_t* model_ids_host, int32_t n,
+                        void* outputs_host, void* stream);
+
+/* Mark the id dead and free its weights.  Synchronises the device first, so it cannot race an
+ * mt_infer in flight.  The id may be re-issued by a later mt_register_model. */
+mt_status mt_release(int32_t model_id);
+
+/* Synchronise `stream`, then report and clear the sticky device-side status of the calls so far:
+ * *status_out is MT_OK, MT_ERR_BAD_MODEL_ID (with the smallest offending arrival index of the first
+ * such batch in *bad_request_index_out, else -1) or MT_ERR_TIMEOUT.  Either out pointer may be NULL. */
+mt_status mt_get_async_status(void* stream, int32_t* status_out, int32_t* bad_request_index_out);
+
+const char* mt_status_string(mt_status s);
+
+/* Test hook: synchronise the device and copy the bucketing results of the last mt_infer to HOST arrays:
+ * counts [T], offsets [T+2] (offsets[T+1] == n; [offsets[T], offsets[T+1]) holds rejected ids), perm [n],
+ * inv [n], with n the batch size of that call and T = highest id ever issued + 1, returned in
+ * *n_tenants_out (call once with null arrays to size them).  Any pointer may be NULL. */
+mt_status mt_debug_last_bucketing(int32_t* counts_host, int32_t* offsets_host, int32_t* perm_host,
+                                  int32_t* inv_host, int32_t* n_tenants_out);
+
+/* Per-kernel device timing.  While enabled, every kernel launch of mt_infer is bracketed by CUDA events
+ * on the caller's stream.  mt_get_kernel_times synchronises those events, then fills up to `cap`
+ * entries: names[i] (static strings), total_ms[i], launches[i]; *n_out = number of kernels seen.
+ * Reading resets the accumulators. */
+mt_status mt_set_kernel_timing(int32_t enable);
+mt_status mt_get_kernel_times(const char** names, double* total_ms, int32_t* launches, int32_t cap,
+                              int32_t* n_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MT_H_ */

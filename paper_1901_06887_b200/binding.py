@@ -1,0 +1,165 @@
+"""Thin ctypes binding of libmt.so: the same entry points as include/mt.h, argument marshalling only.
+
+Every step of the inference path runs inside the CUDA library.  There is no fallback: if libmt.so has
+not been built (``python -m paper_1901_06887_b200.build``) importing a function from here raises.
+torch is used for device memory and streams only.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmt.so")
+
+MT_OK = 0
+STATUS_NAMES = {0: "MT_OK", 1: "MT_ERR_INVALID_ARG", 2: "MT_ERR_BAD_MODEL_ID", 3: "MT_ERR_SHAPE",
+                4: "MT_ERR_UNSUPPORTED", 5: "MT_ERR_OOM", 6: "MT_ERR_CUDA", 7: "MT_ERR_ARCH",
+                8: "MT_ERR_TIMEOUT", 9: "MT_ERR_NOT_INIT"}
+
+EXPORTS = ["mt_init", "mt_shutdown", "mt_register_model", "mt_infer", "mt_infer_host", "mt_release",
+           "mt_get_async_status", "mt_status_string", "mt_debug_last_bucketing", "mt_set_kernel_timing",
+           "mt_get_kernel_times"]
+
+
+class MtError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = int(code)
+        super().__init__("%s failed: %s (%d)" % (where, STATUS_NAMES.get(int(code), "?"), int(code)))
+
+
+class LayerDesc(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int32), ("in_ch", ctypes.c_int32), ("out_ch", ctypes.c_int32),
+                ("h", ctypes.c_int32), ("w", ctypes.c_int32), ("relu", ctypes.c_int32),
+                ("weight", ctypes.c_void_p), ("bias", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libmt.so (once).  Raises if it is missing: there is no other implementation to fall back to."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("CUDA library %s not built; run `python -m paper_1901_06887_b200.build`" % LIB_PATH)
+        l = ctypes.CDLL(LIB_PATH)
+        vp, i32 = ctypes.c_void_p, ctypes.c_int32
+        l.mt_init.argtypes = [i32, i32, i32]
+        l.mt_shutdown.argtypes = []
+        l.mt_register_model.argtypes = [ctypes.POINTER(LayerDesc), i32, ctypes.POINTER(i32)]
+        l.mt_infer.argtypes = [vp, vp, i32, vp, vp]
+        l.mt_infer_host.argtypes = [vp, vp, i32, vp, vp]
+        l.mt_release.argtypes = [i32]
+        l.mt_get_async_status.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        l.mt_status_string.argtypes = [i32]
+        l.mt_status_string.restype = ctypes.c_char_p
+        l.mt_debug_last_bucketing.argtypes = [vp] * 4 + [ctypes.POINTER(i32)]
+        l.mt_set_kernel_timing.argtypes = [i32]
+        l.mt_get_kernel_times.argtypes = [ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_double),
+                                          ctypes.POINTER(i32), i32, ctypes.POINTER(i32)]
+        for name in EXPORTS:
+            if name != "mt_status_string":
+                getattr(l, name).restype = ctypes.c_int
+        _lib = l
+    return _lib
+
+
+def _check(code: int, where: str) -> None:
+    if code != MT_OK:
+        raise MtError(code, where)
+
+
+def _ptr(x) -> Optional[int]:
+    """Address of a torch tensor (device or host), a numpy array, or None."""
+    if x is None:
+        return None
+    if isinstance(x, np.ndarray):
+        return x.ctypes.data
+    return x.data_ptr()
+
+
+def _stream_handle(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def mt_init(device: int = 0, max_models: int = 1024, max_batch: int = 0) -> None:
+    _check(lib().mt_init(device, max_models, max_batch), "mt_init")
+
+
+def mt_shutdown() -> None:
+    _check(lib().mt_shutdown(), "mt_shutdown")
+
+
+def mt_register_model(layers: Sequence) -> int:
+    """layers: objects with kind, in_ch, out_ch, h, w, relu, weight, bias (weight: uint16 numpy array of bf16
+    bit patterns or a torch bf16 tensor, host or device; bias: float32 or None).  Returns the model id."""
+    arr = (LayerDesc * len(layers))()
+    keep = []
+    for i, l in enumerate(layers):
+        w, b = l.weight, l.bias
+        if isinstance(w, np.ndarray):
+            w = np.ascontiguousarray(w, dtype=np.uint16)
+        if isinstance(b, np.ndarray):
+            b = np.ascontiguousarray(b, dtype=np.float32)
+        keep += [w, b]
+        arr[i] = LayerDesc(int(l.kind), int(l.in_ch), int(l.out_ch), int(l.h), int(l.w), int(l.relu), _ptr(w), _ptr(b))
+    mid = ctypes.c_int32(-1)
+    _check(lib().mt_register_model(arr, len(layers), ctypes.byref(mid)), "mt_register_model")
+    return int(mid.value)
+
+
+def mt_release(model_id: int) -> None:
+    _check(lib().mt_release(int(model_id)), "mt_release")
+
+
+def mt_infer(inputs, model_ids, n: int, outputs, stream=None) -> None:
+    """inputs: device bf16 [n, in_elems]; model_ids: device int32 [n]; outputs: device fp32 [n, out_elems]."""
+    _check(lib().mt_infer(_ptr(inputs), _ptr(model_ids), int(n), _ptr(outputs), _stream_handle(stream)), "mt_infer")
+
+
+def mt_infer_host(inputs, model_ids, n: int, outputs, stream=None) -> None:
+    """Same with host buffers (pinned torch tensors or numpy arrays); returns after the outputs have landed."""
+    _check(lib().mt_infer_host(_ptr(inputs), _ptr(model_ids), int(n), _ptr(outputs), _stream_handle(stream)),
+           "mt_infer_host")
+
+
+def mt_get_async_status(stream=None) -> Tuple[int, int]:
+    st, bad = ctypes.c_int32(0), ctypes.c_int32(-1)
+    _check(lib().mt_get_async_status(_stream_handle(stream), ctypes.byref(st), ctypes.byref(bad)), "mt_get_async_status")
+    return int(st.value), int(bad.value)
+
+
+def mt_status_string(code: int) -> str:
+    return lib().mt_status_string(int(code)).decode()
+
+
+def mt_debug_last_bucketing(n: int):
+    """Copies of (counts[T], offsets[T+2], perm[n], inv[n]) of the last mt_infer (batch size n) as numpy int32."""
+    T = ctypes.c_int32(0)
+    _check(lib().mt_debug_last_bucketing(None, None, None, None, ctypes.byref(T)), "mt_debug_last_bucketing")
+    arrs = [np.zeros(T.value, np.int32), np.zeros(T.value + 2, np.int32), np.zeros(n, np.int32), np.zeros(n, np.int32)]
+    _check(lib().mt_debug_last_bucketing(*[a.ctypes.data for a in arrs], None), "mt_debug_last_bucketing")
+    return tuple(arrs)
+
+
+def mt_set_kernel_timing(enable: bool) -> None:
+    _check(lib().mt_set_kernel_timing(1 if enable else 0), "mt_set_kernel_timing")
+
+
+def mt_get_kernel_times() -> List[Tuple[str, float, int]]:
+    cap = 16
+    names = (ctypes.c_char_p * cap)()
+    ms = (ctypes.c_double * cap)()
+    cnt = (ctypes.c_int32 * cap)()
+    n = ctypes.c_int32(0)
+    _check(lib().mt_get_kernel_times(names, ms, cnt, cap, ctypes.byref(n)), "mt_get_kernel_times")
+    return [(names[i].decode(), float(ms[i]), int(cnt[i])) for i in range(n.value)]

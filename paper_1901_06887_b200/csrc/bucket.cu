@@ -1,0 +1,214 @@
+// Request bucketing and its inverse: group the requests of one mixed batch by model id into
+// contiguous segments (a stable counting sort), keep the permutation back to arrival order,
+// move payload rows into bucketed order, and restore arrival order at the end.
+//
+// The paper (Sec. 3) has a worker receive requests for many tenants' models; grouping them by model is a
+// pure re-ordering, made unique by stability: inside a segment, requests keep their arrival order.
+//
+//   pass 1  bucket_block_hist   per-block histogram of ids (warp-level match + one shared atomic per group)
+//   pass 2  bucket_scan         per-tenant exclusive scan over blocks, exclusive scan over tenants
+//                               (offsets), per-layer tile prefix sums for the grouped executors
+//   pass 3  bucket_scatter      stable position of every request -> perm / inv
+//           gather_rows         X_b[j, :] = X[perm[j], :]          (128-bit copies)
+//           unpermute_rows      out[perm[j], :] = out_b[j, :]      (128-bit copies where rows allow)
+#include <limits>
+
+#include "mt_device.cuh"
+#include "mt_host.h"
+
+namespace mt {
+
+constexpr int kScanThreads = 1024;
+
+// ids outside [0, T) or of dead models go to the extra bucket T, so they sort behind every live segment.
+__device__ __forceinline__ int classify(int id, int T, const ModelDev* models) {
+    if (id < 0 || id >= T) return T;
+    return models[id].alive ? id : T;
+}
+
+__global__ void __launch_bounds__(kBucketChunk)
+bucket_block_hist(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models,
+                  int32_t* __restrict__ block_hist, int32_t* __restrict__ status) {
+    extern __shared__ int32_t s_hist[];   // T + 1
+    const int T1 = T + 1;
+    for (int t = threadIdx.x; t < T1; t += blockDim.x) s_hist[t] = 0;
+    __syncthreads();
+    const int i = blockIdx.x * kBucketChunk + threadIdx.x;
+    if (i < n) {
+        const int b = classify(ids[i], T, models);
+        if (b == T) {
+            atomicCAS(&status[ST_CODE], MT_OK, MT_ERR_BAD_MODEL_ID);
+            atomicMin(&status[ST_BAD_INDEX], i);
+        }
+        const unsigned peers = __match_any_sync(__activemask(), b);
+        if ((__ffs(peers) - 1) == (threadIdx.x & 31)) atomicAdd(&s_hist[b], __popc(peers));
+    }
+    __syncthreads();
+    for (int t = threadIdx.x; t < T1; t += blockDim.x) block_hist[(size_t)blockIdx.x * T1 + t] = s_hist[t];
+}
+
+// Exclusive scan of `n_items` ints held in global memory by one CTA of kScanThreads threads.
+// out[0..n_items] (n_items + 1 entries; the last is the total).  in and out may alias only if equal offsets
+// are not needed afterwards.  s_tmp: kScanThreads ints of shared memory.
+__device__ void cta_exclusive_scan(const int32_t* in, int32_t* out, int n_items, int32_t* s_tmp) {
+    const int tid = threadIdx.x;
+    const int per = (n_items + kScanThreads - 1) / kScanThreads;
+    const int lo = min(tid * per, n_items), hi = min(lo + per, n_items);
+    int sum = 0;
+    for (int j = lo; j < hi; ++j) sum += in[j];
+    s_tmp[tid] = sum;
+    __syncthreads();
+    // Hillis-Steele inclusive scan over the per-thread sums
+    for (int d = 1; d < kScanThreads; d <<= 1) {
+        const int v = (tid >= d) ? s_tmp[tid - d] : 0;
+        __syncthreads();
+        s_tmp[tid] += v;
+        __syncthreads();
+    }
+    int run = s_tmp[tid] - sum;
+    for (int j = lo; j < hi; ++j) {
+        const int v = in[j];
+        out[j] = run;
+        run += v;
+    }
+    if (tid == kScanThreads - 1) out[n_items] = s_tmp[tid];
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(kScanThreads)
+bucket_scan(int n_blocks, int T, const ModelDev* __restrict__ models, int n_layers, int rows_per_unit,
+            int32_t* __restrict__ block_hist, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
+            int32_t* __restrict__ tile_prefix, int32_t* __restrict__ tmp) {
+    __shared__ int32_t s_tmp[kScanThreads];
+    const int T1 = T + 1;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // (1) per bucket: counts[t] = sum over blocks; block_hist[b][t] <- exclusive prefix over blocks
+    for (int t = warp; t < T1; t += kScanThreads / 32) {
+        int carry = 0;
+        for (int b0 = 0; b0 < n_blocks; b0 += 32) {
+            const int b = b0 + lane;
+            const int v = (b < n_blocks) ? block_hist[(size_t)b * T1 + t] : 0;
+            int incl = v;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int u = __shfl_up_sync(0xffffffffu, incl, d);
+                if (lane >= d) incl += u;
+            }
+            if (b < n_blocks) block_hist[(size_t)b * T1 + t] = carry + incl - v;
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) counts[t] = carry;
+    }
+    __syncthreads();
+    // (2) offsets = exclusive scan of counts over the T + 1 buckets (offsets[T + 1] = n)
+    cta_exclusive_scan(counts, offsets, T1, s_tmp);
+    // (3) per layer: prefix sums of the work units (tiles) each tenant contributes
+    for (int l = 0; l < n_layers; ++l) {
+        for (int t = threadIdx.x; t < T; t += kScanThreads) {
+            int units = 0;
+            const int c = counts[t];
+            if (c > 0) {
+                const LayerDev& L = models[t].layer[l];
+                if (L.kind == MT_DENSE) units = ((c + BM - 1) / BM) * L.n_tiles;
+                else if (L.kind == MT_CONV3X3) units = c * rows_per_unit;   // rows_per_unit = tiles per image
+            }
+            tmp[t] = units;
+        }
+        __syncthreads();
+        cta_exclusive_scan(tmp, tile_prefix + (size_t)l * (T + 1), T, s_tmp);
+    }
+}
+
+__global__ void __launch_bounds__(kBucketChunk)
+bucket_scatter(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models,
+               const int32_t* __restrict__ block_hist, const int32_t* __restrict__ offsets,
+               int32_t* __restrict__ perm, int32_t* __restrict__ inv) {
+    extern __shared__ int32_t s_next[];   // next free position of every bucket for this block
+    const int T1 = T + 1;
+    for (int t = threadIdx.x; t < T1; t += blockDim.x)
+        s_next[t] = offsets[t] + block_hist[(size_t)blockIdx.x * T1 + t];
+    __syncthreads();
+    const int i = blockIdx.x * kBucketChunk + threadIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = (i < n) ? classify(ids[i], T, models) : -1;
+    // warps take turns in arrival order, so positions inside a bucket ascend with the arrival index
+    for (int w = 0; w < kBucketChunk / 32; ++w) {
+        if (warp == w && i < n) {
+            const unsigned peers = __match_any_sync(__activemask(), b);
+            const int rank = __popc(peers & ((1u << lane) - 1u));
+            const int pos = s_next[b] + rank;
+            __syncwarp(__activemask());
+            if (rank == 0) s_next[b] += __popc(peers);
+            perm[pos] = i;
+            inv[i] = pos;
+        }
+        __syncthreads();
+    }
+}
+
+// X_b[j, :] = X[perm[j], :]; rows of `row_vec` 16-byte vectors; dst rows `dst_ld_vec` vectors apart.
+__global__ void gather_rows(const uint4* __restrict__ src, const int32_t* __restrict__ perm, int n, int row_vec,
+                            uint4* __restrict__ dst, int dst_ld_vec) {
+    const long long total = (long long)n * row_vec;
+    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int j = (int)(idx / row_vec), v = (int)(idx % row_vec);
+        dst[(size_t)j * dst_ld_vec + v] = __ldg(&src[(size_t)perm[j] * row_vec + v]);
+    }
+}
+
+// out[perm[j], :] = out_b[j, :] for j < n_valid; rows of rejected requests (j >= n_valid) become NaN.
+template <typename V>
+__global__ void unpermute_rows(const V* __restrict__ src, const int32_t* __restrict__ perm,
+                               const int32_t* __restrict__ offsets, int T, int n, int row_vec,
+                               V* __restrict__ dst, V nan_v) {
+    const int n_valid = offsets[T];
+    const long long total = (long long)n * row_vec;
+    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int j = (int)(idx / row_vec), v = (int)(idx % row_vec);
+        dst[(size_t)perm[j] * row_vec + v] = (j < n_valid) ? src[idx] : nan_v;
+    }
+}
+
+// ------------------------------------------------------------------------------------------ launchers
+static int grid_for(long long total, int threads, int sm_count) {
+    long long blocks = (total + threads - 1) / threads;
+    const long long cap = (long long)sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (int)blocks;
+}
+
+void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
+    const int n_blocks = (a.n + kBucketChunk - 1) / kBucketChunk;
+    const size_t smem = sizeof(int32_t) * (size_t)(a.T + 1);
+    bucket_block_hist<<<n_blocks, kBucketChunk, smem, s>>>(a.ids, a.n, a.T, a.models, a.block_hist, a.status);
+    bucket_scan<<<1, kScanThreads, 0, s>>>(n_blocks, a.T, a.models, a.n_layers, a.rows_per_unit, a.block_hist,
+                                           a.counts, a.offsets, a.tile_prefix, a.tmp);
+    bucket_scatter<<<n_blocks, kBucketChunk, smem, s>>>(a.ids, a.n, a.T, a.models, a.block_hist, a.offsets, a.perm,
+                                                        a.inv);
+}
+
+void launch_gather_rows(const void* src, const int32_t* perm, int n, int row_bytes, void* dst, int dst_ld_bytes,
+                        int sm_count, cudaStream_t s) {
+    const int row_vec = row_bytes / 16;
+    gather_rows<<<grid_for((long long)n * row_vec, 256, sm_count), 256, 0, s>>>(
+        (const uint4*)src, perm, n, row_vec, (uint4*)dst, dst_ld_bytes / 16);
+}
+
+void launch_unpermute(const float* src, const int32_t* perm, const int32_t* offsets, int T, int n, int out_elems,
+                      float* dst, int sm_count, cudaStream_t s) {
+    const float qnan = std::numeric_limits<float>::quiet_NaN();
+    const bool vec_ok = (out_elems % 4 == 0) && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0);
+    if (vec_ok) {
+        const int row_vec = out_elems / 4;
+        unpermute_rows<float4><<<grid_for((long long)n * row_vec, 256, sm_count), 256, 0, s>>>(
+            (const float4*)src, perm, offsets, T, n, row_vec, (float4*)dst, make_float4(qnan, qnan, qnan, qnan));
+    } else {
+        unpermute_rows<float><<<grid_for((long long)n * out_elems, 256, sm_count), 256, 0, s>>>(
+            src, perm, offsets, T, n, out_elems, dst, qnan);
+    }
+}
+
+}  // namespace mt

@@ -1,0 +1,273 @@
+// Grouped dense-layer executor: ONE persistent launch evaluates a layer for every tenant of the batch,
+//     H_out[seg t] = act(H_in[seg t] . W_t^T + b_t)        (bf16 x bf16 -> fp32, bias + ReLU in fp32)
+// where seg t is the contiguous block of bucketed rows of tenant t.  This is the fully-connected layer of
+// the paper's primer (Sec. 1.1) applied across co-resident models (Sec. 3); since every tenant has its own
+// weights (Sec. 4: "model weights are unique"), the launch walks a device-built list of
+// (tenant, row tile, column tile) work items instead of one GEMM.
+//
+// CTA = 6 warps: warp 0 issues TMA loads (activation tile through a tensor map, weight tile as one 16 KiB
+// bulk copy of a pre-swizzled image), warp 1 issues tcgen05.mma into one of two TMEM accumulators, warps
+// 2..5 drain the other accumulator (tcgen05.ld -> bias -> ReLU -> convert -> 128-bit stores), so the
+// epilogue of tile i overlaps the main loop of tile i+1.  Rows of a tile beyond the tenant's segment are
+// computed on whatever follows in memory and never stored (rows of a GEMM are independent).
+#include "mt_device.cuh"
+#include "mt_host.h"
+
+namespace mt {
+
+constexpr int kStages = 6;
+constexpr int kStageBytes = 2 * TILE_BYTES;           // A tile + B tile
+constexpr int kGemmThreads = 192;
+constexpr int kAccCols = BN;                          // fp32 columns of one accumulator
+constexpr int kTmemCols = 2 * kAccCols;               // two accumulators (power of two >= 32)
+constexpr int kBarBytes = 256;
+constexpr int kGemmSmem = kStages * kStageBytes + kBarBytes + 1024;   // + slack for 1024-byte alignment
+
+struct TileCoord {
+    int t, m_tile, n_tile, row0, rows_valid;
+};
+
+__device__ __forceinline__ TileCoord decode_tile(int item, int T, const int32_t* __restrict__ prefix,
+                                                 const int32_t* __restrict__ offsets, const ModelDev* models,
+                                                 int layer) {
+    int lo = 0, hi = T;   // largest t with prefix[t] <= item
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (prefix[mid] <= item) lo = mid; else hi = mid;
+    }
+    TileCoord c;
+    c.t = lo;
+    const int seg0 = offsets[lo], n_t = offsets[lo + 1] - seg0;
+    const int m_tiles = (n_t + BM - 1) / BM;
+    const int local = item - prefix[lo];
+    c.n_tile = local / m_tiles;      // row tiles of one weight slab are adjacent items: the slab stays in L2
+    c.m_tile = local - c.n_tile * m_tiles;
+    c.row0 = seg0 + c.m_tile * BM;
+    c.rows_valid = min(BM, n_t - c.m_tile * BM);
+    return c;
+}
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmArgs p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+    const uint32_t bar0 = base + kStages * kStageBytes;
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
+        *abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tensormap(&tmap_a);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int total = p.tile_prefix[p.T];
+    const ModelDev* models = p.models;
+
+    if (warp == 0) {
+        if (lane == 0) {   // ------------------------------------------------ TMA producer
+            int stage = 0; uint32_t phase = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < total; item += gridDim.x) {
+                const TileCoord c = decode_tile(item, p.T, p.tile_prefix, p.offsets, models, p.layer);
+                const LayerDev& L = models[c.t].layer[p.layer];
+                const int kblocks = L.k_blocks;
+                const uint16_t* wsrc = L.w + (size_t)c.n_tile * kblocks * (BN * BK);
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
+                    const uint32_t a_dst = base + stage * kStageBytes;
+                    mbar_expect_tx(full_bar(stage), kStageBytes);
+                    tma_load_2d(a_dst, &tmap_a, kb * BK, c.row0, full_bar(stage));
+                    bulk_load(a_dst + TILE_BYTES, wsrc + (size_t)kb * (BN * BK), TILE_BYTES, full_bar(stage));
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {   // ------------------------------------------------ MMA issuer
+            constexpr uint32_t idesc = make_idesc_bf16(BM, BN);
+            int stage = 0; uint32_t phase = 0;
+            int it = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < total; item += gridDim.x, ++it) {
+                const TileCoord c = decode_tile(item, p.T, p.tile_prefix, p.offsets, models, p.layer);
+                const int kblocks = models[c.t].layer[p.layer].k_blocks;
+                const int acc = it & 1;
+                const uint32_t acc_phase = (it >> 1) & 1;
+                if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, 2)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * kAccCols;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_src = base + stage * kStageBytes;
+                    const uint64_t a_desc = make_kmajor_sw128_desc(a_src, 1024);
+                    const uint64_t b_desc = make_kmajor_sw128_desc(a_src + TILE_BYTES, 1024);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        // advancing K by 16 elements = 32 bytes inside the swizzle row: +2 in the address field
+                        umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+                    }
+                    umma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(tfull_bar(acc));
+            }
+        }
+    } else {               // ---------------------------------------------------- epilogue (warps 2..5)
+        const int q = warp & 3;                 // TMEM lane quarter this warp may read
+        const int r = q * 32 + lane;            // accumulator row of this thread
+        int it = 0;
+        for (int item = blockIdx.x; item < total; item += gridDim.x, ++it) {
+            const TileCoord c = decode_tile(item, p.T, p.tile_prefix, p.offsets, models, p.layer);
+            const LayerDev& L = models[c.t].layer[p.layer];
+            const int acc = it & 1;
+            const uint32_t acc_phase = (it >> 1) & 1;
+            if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 4)) break;
+            tc_fence_after();
+            const bool row_ok = r < c.rows_valid;
+            const size_t grow = (size_t)(c.row0 + r);
+            const int N = L.N, relu = L.relu;
+#pragma unroll 1
+            for (int ch = 0; ch < BN / 32; ++ch) {
+                uint32_t v[32];
+                __syncwarp();   // tcgen05.ld is warp-collective: reconverge after the per-row stores
+                tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccCols + ch * 32, v);
+                tmem_ld_wait();
+                const int n0 = c.n_tile * BN + ch * 32;
+                if (n0 >= N) break;
+                const float4* b4 = reinterpret_cast<const float4*>(L.bias + n0);
+                float f[32];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float4 b = __ldg(b4 + j);
+                    f[4 * j + 0] = __uint_as_float(v[4 * j + 0]) + b.x;
+                    f[4 * j + 1] = __uint_as_float(v[4 * j + 1]) + b.y;
+                    f[4 * j + 2] = __uint_as_float(v[4 * j + 2]) + b.z;
+                    f[4 * j + 3] = __uint_as_float(v[4 * j + 3]) + b.w;
+                }
+                if (relu) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) f[j] = fmaxf(f[j], 0.0f);
+                }
+                const bool full_chunk = (n0 + 32 <= N);
+                if (!row_ok) {
+                    // rows past the tenant's segment belong to someone else: never stored
+                } else if (p.out_fp32) {
+                    float* dst = reinterpret_cast<float*>(p.out) + grow * p.ld_out + n0;
+                    if (full_chunk && (p.ld_out & 3) == 0) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            reinterpret_cast<float4*>(dst)[j] = make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (n0 + j < N) dst[j] = f[j];
+                    }
+                } else {
+                    uint16_t* dst = reinterpret_cast<uint16_t*>(p.out) + grow * p.ld_out + n0;
+                    if (full_chunk && (p.ld_out & 7) == 0) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            uint4 o;
+                            o.x = pack_bf16x2(f[8 * j + 0], f[8 * j + 1]);
+                            o.y = pack_bf16x2(f[8 * j + 2], f[8 * j + 3]);
+                            o.z = pack_bf16x2(f[8 * j + 4], f[8 * j + 5]);
+                            o.w = pack_bf16x2(f[8 * j + 6], f[8 * j + 7]);
+                            reinterpret_cast<uint4*>(dst)[j] = o;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (n0 + j < N) dst[j] = static_cast<uint16_t>(pack_bf16x2(f[j], 0.0f) & 0xFFFFu);
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(tempty_bar(acc));
+        }
+    }
+
+    // ---- tear-down: every thread gets here, also after an abandoned wait
+    if (*abort_flag) {   // give copies and MMAs still in flight a bounded time to finish
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------------------------------ weight re-layout
+__global__ void pretile_dense_kernel(const uint16_t* __restrict__ w, int N, int K, uint4* __restrict__ out,
+                                     long long total_chunks) {
+    const int kblocks = K / BK;
+    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total_chunks;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const long long tile = idx >> 10;            // 1024 chunks of 16 bytes per tile
+        const int within = (int)(idx & 1023);
+        const int r = within >> 3, cpos = within & 7;
+        const int c = cpos ^ (r & 7);                // logical chunk stored at physical position cpos
+        const int nt = (int)(tile / kblocks), kb = (int)(tile % kblocks);
+        const int row = nt * BN + r;
+        uint4 val = make_uint4(0, 0, 0, 0);
+        if (row < N) val = *reinterpret_cast<const uint4*>(w + (size_t)row * K + kb * BK + c * 8);
+        out[idx] = val;
+    }
+}
+
+__global__ void pretile_conv_kernel(const uint16_t* __restrict__ w, int C_out, int C_in, uint4* __restrict__ out,
+                                    int total_chunks) {
+    // 9 tap tiles; tile `tap` holds rows o = 0..C_out-1 of 64 input channels: 64 rows x 128 bytes, swizzled
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total_chunks; idx += gridDim.x * blockDim.x) {
+        const int tap = idx / (C_out * 8);
+        const int within = idx % (C_out * 8);
+        const int r = within >> 3, cpos = within & 7;
+        const int c = cpos ^ (r & 7);
+        out[idx] = *reinterpret_cast<const uint4*>(w + ((size_t)r * 9 + tap) * C_in + c * 8);
+    }
+}
+
+void launch_pretile_dense(const uint16_t* w, int N, int K, uint16_t* out, cudaStream_t s) {
+    const long long n_tiles = (N + BN - 1) / BN;
+    const long long total = n_tiles * (K / BK) * 1024;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 4096) blocks = 4096;
+    pretile_dense_kernel<<<(int)blocks, 256, 0, s>>>(w, N, K, reinterpret_cast<uint4*>(out), total);
+}
+
+void launch_pretile_conv(const uint16_t* w, int C_out, int C_in, uint16_t* out, cudaStream_t s) {
+    const int total = 9 * C_out * 8;
+    pretile_conv_kernel<<<(total + 255) / 256, 256, 0, s>>>(w, C_out, C_in, reinterpret_cast<uint4*>(out), total);
+}
+
+cudaError_t configure_grouped_gemm() {
+    return cudaFuncSetAttribute(grouped_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
+}
+
+void launch_grouped_gemm(const CUtensorMap& tmap_a, const GemmArgs& a, int sm_count, cudaStream_t s) {
+    grouped_gemm_kernel<<<sm_count, kGemmThreads, kGemmSmem, s>>>(tmap_a, a);
+}
+
+}  // namespace mt

@@ -1,0 +1,629 @@
+// C-ABI layer: model registry, device workspace, tensor maps and the per-batch launch sequence.
+// Everything that computes runs in the CUDA kernels of the other files; this file only validates,
+// allocates, copies weights at registration and enqueues launches.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <climits>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "../../include/mt.h"
+#include "mt_device.cuh"
+#include "mt_host.h"
+
+namespace {
+
+using namespace mt;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct HostLayer {
+    int kind, in_ch, out_ch, h, w, relu;
+};
+
+struct HostModel {
+    bool alive = false;
+    std::vector<HostLayer> layers;
+    void* dev_block = nullptr;
+};
+
+enum KernelId { K_HIST = 0, K_SCAN, K_SCATTER, K_GATHER, K_GEMM, K_CONV, K_POOL, K_UNPERMUTE, K_COUNT };
+const char* const kKernelNames[K_COUNT] = {"bucket_block_hist+scan+scatter", "", "", "gather_rows",
+                                           "grouped_gemm", "grouped_conv3x3", "global_avg_pool", "unpermute_rows"};
+
+struct TimedLaunch {
+    int kernel;
+    cudaEvent_t start, stop;
+};
+
+struct Ctx {
+    bool init = false;
+    int device = 0, sm_count = 0, max_models = 0;
+    int T = 0;                           // id slots in use (highest issued id + 1)
+    std::vector<HostModel> models;
+    ModelDev* d_models = nullptr;
+    EncodeTiledFn encode = nullptr;
+
+    // the hosted family (fixed by the first registered model)
+    bool has_family = false;
+    std::vector<HostLayer> family;       // kinds and geometry; dense hidden widths are per model
+    int in_elems = 0, out_elems = 0;
+    int width[MT_MAX_LAYERS + 1] = {0};  // per layer boundary: widest input row (elements) over all models
+    int live = 0;
+
+    // workspace
+    int cap_n = 0;
+    bool ws_dirty = true;
+    int32_t *d_block_hist = nullptr, *d_counts = nullptr, *d_offsets = nullptr, *d_tile_prefix = nullptr,
+            *d_tmp = nullptr, *d_perm = nullptr, *d_inv = nullptr, *d_status = nullptr;
+    void* act[MT_MAX_LAYERS + 1] = {nullptr};
+    int act_ld[MT_MAX_LAYERS + 1] = {0};
+    CUtensorMap act_map[MT_MAX_LAYERS + 1];
+    float* d_out_b = nullptr;
+    int last_n = 0;
+
+    // staging for mt_infer_host
+    void* st_in = nullptr;
+    int32_t* st_ids = nullptr;
+    float* st_out = nullptr;
+    int st_cap = 0;
+
+    // timing
+    bool timing = false;
+    std::vector<TimedLaunch> timed;
+    std::vector<cudaEvent_t> event_pool;
+};
+
+Ctx g;
+std::mutex g_mu;
+
+#define CU_OK(call)                                                   \
+    do {                                                              \
+        cudaError_t e__ = (call);                                     \
+        if (e__ != cudaSuccess) {                                     \
+            if (getenv("MT_LOG"))                                     \
+                fprintf(stderr, "[mt] %s:%d %s -> %s\n", __FILE__, __LINE__, #call, cudaGetErrorString(e__)); \
+            return (e__ == cudaErrorMemoryAllocation) ? MT_ERR_OOM : MT_ERR_CUDA; \
+        }                                                             \
+    } while (0)
+
+int conv_rows_per_tile(int w, int h) { int r = BM / w; return r < h ? r : h; }
+
+mt_status reset_status_word() {
+    const int32_t init[ST_WORDS] = {MT_OK, INT_MAX, 0, 0};
+    CU_OK(cudaMemcpy(g.d_status, init, sizeof init, cudaMemcpyHostToDevice));
+    return MT_OK;
+}
+
+mt_status do_init(int device, int max_models, int /*max_batch*/) {
+    if (g.init) return MT_OK;
+    if (max_models <= 0 || max_models > 8192) return MT_ERR_INVALID_ARG;
+    int n_dev = 0;
+    CU_OK(cudaGetDeviceCount(&n_dev));
+    if (device < 0 || device >= n_dev) return MT_ERR_INVALID_ARG;
+    cudaDeviceProp prop;
+    CU_OK(cudaGetDeviceProperties(&prop, device));
+    if (prop.major != 10) return MT_ERR_ARCH;
+    CU_OK(cudaSetDevice(device));
+    g.device = device;
+    g.sm_count = prop.multiProcessorCount;
+    g.max_models = max_models;
+    g.models.assign(max_models, HostModel());
+    CU_OK(cudaMalloc(&g.d_models, sizeof(ModelDev) * (size_t)max_models));
+    CU_OK(cudaMemset(g.d_models, 0, sizeof(ModelDev) * (size_t)max_models));
+    CU_OK(cudaMalloc(&g.d_status, sizeof(int32_t) * ST_WORDS));
+    CU_OK(cudaMalloc(&g.d_counts, sizeof(int32_t) * (size_t)(max_models + 1)));
+    CU_OK(cudaMalloc(&g.d_offsets, sizeof(int32_t) * (size_t)(max_models + 2)));
+    CU_OK(cudaMalloc(&g.d_tmp, sizeof(int32_t) * (size_t)(max_models + 1)));
+    CU_OK(cudaMalloc(&g.d_tile_prefix, sizeof(int32_t) * (size_t)MT_MAX_LAYERS * (max_models + 1)));
+    CU_OK(cudaMemset(g.d_offsets, 0, sizeof(int32_t) * (size_t)(max_models + 2)));
+    mt_status st = reset_status_word();
+    if (st != MT_OK) return st;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    CU_OK(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) return MT_ERR_CUDA;
+    g.encode = reinterpret_cast<EncodeTiledFn>(fn);
+    CU_OK(configure_grouped_gemm());
+    CU_OK(configure_grouped_conv());
+    g.T = 0;
+    g.live = 0;
+    g.has_family = false;
+    g.cap_n = 0;
+    g.ws_dirty = true;
+    g.init = true;
+    return MT_OK;
+}
+
+void free_workspace() {
+    cudaFree(g.d_block_hist); g.d_block_hist = nullptr;
+    cudaFree(g.d_perm); g.d_perm = nullptr;
+    cudaFree(g.d_inv); g.d_inv = nullptr;
+    cudaFree(g.d_out_b); g.d_out_b = nullptr;
+    for (int b = 0; b <= MT_MAX_LAYERS; ++b) { cudaFree(g.act[b]); g.act[b] = nullptr; }
+    g.cap_n = 0;
+}
+
+mt_status encode_2d(CUtensorMap* map, void* ptr, int ld, int rows) {
+    cuuint64_t dims[2] = {(cuuint64_t)ld, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {BK, BM};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g.encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ptr, dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? MT_OK : MT_ERR_CUDA;
+}
+
+mt_status encode_nhwc(CUtensorMap* map, const void* ptr, int C, int W, int H, int n_img, int rows_per_tile) {
+    cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)n_img};
+    cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
+    cuuint32_t box[4] = {(cuuint32_t)C, (cuuint32_t)W, (cuuint32_t)rows_per_tile, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = g.encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? MT_OK : MT_ERR_CUDA;
+}
+
+// (Re)allocate everything whose size depends on the batch size or on the family's widest rows.
+mt_status ensure_workspace(int n) {
+    if (!g.ws_dirty && n <= g.cap_n) return MT_OK;
+    CU_OK(cudaDeviceSynchronize());
+    int cap = g.cap_n > n ? g.cap_n : n;
+    free_workspace();
+    const int L = (int)g.family.size();
+    const size_t n_blocks = (size_t)(cap + kBucketChunk - 1) / kBucketChunk;
+    CU_OK(cudaMalloc(&g.d_block_hist, sizeof(int32_t) * n_blocks * (size_t)(g.max_models + 1)));
+    CU_OK(cudaMalloc(&g.d_perm, sizeof(int32_t) * (size_t)cap));
+    CU_OK(cudaMalloc(&g.d_inv, sizeof(int32_t) * (size_t)cap));
+    CU_OK(cudaMalloc(&g.d_out_b, sizeof(float) * (size_t)cap * g.out_elems));
+    for (int b = 0; b < L; ++b) {
+        const HostLayer& f = g.family[b];
+        if (f.kind == MT_DENSE) {
+            g.act_ld[b] = g.width[b];
+            const size_t bytes = (size_t)cap * g.act_ld[b] * 2;
+            CU_OK(cudaMalloc(&g.act[b], bytes));
+            CU_OK(cudaMemset(g.act[b], 0, bytes));
+            mt_status st = encode_2d(&g.act_map[b], g.act[b], g.act_ld[b], cap);
+            if (st != MT_OK) return st;
+        } else {
+            g.act_ld[b] = f.in_ch * f.h * f.w;
+            if (b == 0) continue;   // the first conv layer reads the caller's buffer through perm
+            const size_t bytes = (size_t)cap * g.act_ld[b] * 2;
+            CU_OK(cudaMalloc(&g.act[b], bytes));
+            CU_OK(cudaMemset(g.act[b], 0, bytes));
+            if (f.kind == MT_CONV3X3) {
+                mt_status st = encode_nhwc(&g.act_map[b], g.act[b], f.in_ch, f.w, f.h, cap, conv_rows_per_tile(f.w, f.h));
+                if (st != MT_OK) return st;
+            }
+        }
+    }
+    g.cap_n = cap;
+    g.ws_dirty = false;
+    return MT_OK;
+}
+
+bool is_device_pointer(const void* p) {
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, p) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return attr.type == cudaMemoryTypeDevice || attr.type == cudaMemoryTypeManaged;
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+mt_status validate_layers(const mt_layer_desc* layers, int n_layers) {
+    if (!layers || n_layers < 1 || n_layers > MT_MAX_LAYERS) return n_layers > MT_MAX_LAYERS ? MT_ERR_UNSUPPORTED : MT_ERR_INVALID_ARG;
+    for (int l = 0; l < n_layers; ++l) {
+        const mt_layer_desc& d = layers[l];
+        if (d.kind < MT_DENSE || d.kind > MT_GLOBAL_AVG_POOL) return MT_ERR_INVALID_ARG;
+        if (d.in_ch <= 0 || d.out_ch <= 0) return MT_ERR_INVALID_ARG;
+        if (d.kind != MT_GLOBAL_AVG_POOL && !d.weight) return MT_ERR_INVALID_ARG;
+        if (d.kind == MT_DENSE) {
+            if (l > 0) {
+                const mt_layer_desc& p = layers[l - 1];
+                if (p.kind == MT_CONV3X3) return MT_ERR_UNSUPPORTED;   // needs a pool in between
+                if (p.out_ch != d.in_ch) return MT_ERR_SHAPE;
+            }
+            if (d.in_ch % BK != 0) return MT_ERR_UNSUPPORTED;
+        } else {
+            if (d.h <= 0 || d.w <= 0) return MT_ERR_INVALID_ARG;
+            if (l > 0) {
+                const mt_layer_desc& p = layers[l - 1];
+                if (p.kind != MT_CONV3X3) return MT_ERR_UNSUPPORTED;    // conv/pool only after a conv
+                if (p.out_ch != d.in_ch || p.h != d.h || p.w != d.w) return MT_ERR_SHAPE;
+            } else if (d.kind == MT_GLOBAL_AVG_POOL) {
+                return MT_ERR_UNSUPPORTED;
+            }
+            if (d.kind == MT_CONV3X3 && (d.in_ch != 64 || d.out_ch != 64 || d.w > BM)) return MT_ERR_UNSUPPORTED;
+            if (d.kind == MT_GLOBAL_AVG_POOL && d.in_ch != d.out_ch) return MT_ERR_SHAPE;
+        }
+    }
+    if (layers[n_layers - 1].kind != MT_DENSE) return MT_ERR_UNSUPPORTED;   // the last layer writes the fp32 output
+    return MT_OK;
+}
+
+int layer_in_elems(const HostLayer& l) { return l.kind == MT_DENSE ? l.in_ch : l.in_ch * l.h * l.w; }
+
+mt_status check_family(const std::vector<HostLayer>& m) {
+    if (!g.has_family || g.live == 0) return MT_OK;
+    if (m.size() != g.family.size()) return MT_ERR_SHAPE;
+    for (size_t l = 0; l < m.size(); ++l) {
+        const HostLayer &a = m[l], &f = g.family[l];
+        if (a.kind != f.kind) return MT_ERR_SHAPE;
+        if (a.kind != MT_DENSE && (a.in_ch != f.in_ch || a.out_ch != f.out_ch || a.h != f.h || a.w != f.w)) return MT_ERR_SHAPE;
+    }
+    if (layer_in_elems(m[0]) != g.in_elems || m.back().out_ch != g.out_elems) return MT_ERR_SHAPE;
+    return MT_OK;
+}
+
+struct Timer {
+    int kernel;
+    cudaStream_t s;
+    bool on;
+    cudaEvent_t start = nullptr, stop = nullptr;
+    Timer(int k, cudaStream_t st) : kernel(k), s(st), on(g.timing) {
+        if (!on) return;
+        auto get = [&]() {
+            cudaEvent_t e;
+            if (!g.event_pool.empty()) { e = g.event_pool.back(); g.event_pool.pop_back(); }
+            else cudaEventCreate(&e);
+            return e;
+        };
+        start = get(); stop = get();
+        cudaEventRecord(start, s);
+    }
+    ~Timer() {
+        if (!on) return;
+        cudaEventRecord(stop, s);
+        g.timed.push_back({kernel, start, stop});
+    }
+};
+
+mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outputs, cudaStream_t s) {
+    if (!g.init) return MT_ERR_NOT_INIT;
+    if (n < 0) return MT_ERR_INVALID_ARG;
+    if (n == 0) return MT_OK;
+    if (!inputs || !ids || !outputs) return MT_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(inputs) & 15) return MT_ERR_INVALID_ARG;
+    if (!g.has_family || g.live == 0) return MT_ERR_BAD_MODEL_ID;
+    CU_OK(cudaSetDevice(g.device));
+    mt_status st = ensure_workspace(n);
+    if (st != MT_OK) return st;
+    const int L = (int)g.family.size();
+    const HostLayer& f0 = g.family[0];
+    int tiles_per_image = 0, rows_per_tile = 0;
+    for (const HostLayer& f : g.family)
+        if (f.kind == MT_CONV3X3) {
+            rows_per_tile = conv_rows_per_tile(f.w, f.h);
+            tiles_per_image = (f.h + rows_per_tile - 1) / rows_per_tile;
+        }
+
+    {
+        Timer t(K_HIST, s);
+        BucketArgs a;
+        a.ids = ids; a.n = n; a.T = g.T; a.models = g.d_models; a.n_layers = L; a.rows_per_unit = tiles_per_image;
+        a.block_hist = g.d_block_hist; a.counts = g.d_counts; a.offsets = g.d_offsets; a.tile_prefix = g.d_tile_prefix;
+        a.tmp = g.d_tmp; a.perm = g.d_perm; a.inv = g.d_inv; a.status = g.d_status;
+        launch_bucketing(a, s);
+    }
+    CUtensorMap in_map;
+    if (f0.kind == MT_DENSE) {
+        Timer t(K_GATHER, s);
+        launch_gather_rows(inputs, g.d_perm, n, g.in_elems * 2, g.act[0], g.act_ld[0] * 2, g.sm_count, s);
+    } else {
+        st = encode_nhwc(&in_map, inputs, f0.in_ch, f0.w, f0.h, n, rows_per_tile);
+        if (st != MT_OK) return st;
+    }
+    for (int l = 0; l < L; ++l) {
+        const HostLayer& f = g.family[l];
+        const bool last = (l == L - 1);
+        if (f.kind == MT_DENSE) {
+            Timer t(K_GEMM, s);
+            GemmArgs a;
+            a.models = g.d_models; a.layer = l; a.T = g.T; a.offsets = g.d_offsets;
+            a.tile_prefix = g.d_tile_prefix + (size_t)l * (g.T + 1);
+            a.out = last ? (void*)g.d_out_b : g.act[l + 1];
+            a.ld_out = last ? g.out_elems : g.act_ld[l + 1];
+            a.out_fp32 = last ? 1 : 0;
+            a.status = g.d_status;
+            launch_grouped_gemm(g.act_map[l], a, g.sm_count, s);
+        } else if (f.kind == MT_CONV3X3) {
+            Timer t(K_CONV, s);
+            ConvArgs a;
+            a.models = g.d_models; a.layer = l; a.T = g.T; a.offsets = g.d_offsets;
+            a.tile_prefix = g.d_tile_prefix + (size_t)l * (g.T + 1);
+            a.perm = (l == 0) ? g.d_perm : nullptr;
+            a.out = (uint16_t*)g.act[l + 1];
+            a.H = f.h; a.W = f.w; a.rows_per_tile = rows_per_tile; a.tiles_per_image = tiles_per_image;
+            a.status = g.d_status;
+            launch_grouped_conv(l == 0 ? in_map : g.act_map[l], a, g.sm_count, s);
+        } else {
+            Timer t(K_POOL, s);
+            launch_global_avg_pool((const uint16_t*)g.act[l], n, f.h * f.w, f.in_ch, (uint16_t*)g.act[l + 1],
+                                   g.act_ld[l + 1], g.sm_count, s);
+        }
+    }
+    {
+        Timer t(K_UNPERMUTE, s);
+        launch_unpermute(g.d_out_b, g.d_perm, g.d_offsets, g.T, n, g.out_elems, (float*)outputs, g.sm_count, s);
+    }
+    g.last_n = n;
+    CU_OK(cudaGetLastError());
+    return MT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+mt_status mt_init(int32_t device, int32_t max_models, int32_t max_batch) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    return do_init(device, max_models, max_batch);
+}
+
+mt_status mt_shutdown(void) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g.init) return MT_OK;
+    cudaSetDevice(g.device);
+    cudaDeviceSynchronize();
+    for (HostModel& m : g.models)
+        if (m.dev_block) { cudaFree(m.dev_block); m.dev_block = nullptr; }
+    g.models.clear();
+    free_workspace();
+    cudaFree(g.d_models); g.d_models = nullptr;
+    cudaFree(g.d_status); g.d_status = nullptr;
+    cudaFree(g.d_counts); g.d_counts = nullptr;
+    cudaFree(g.d_offsets); g.d_offsets = nullptr;
+    cudaFree(g.d_tmp); g.d_tmp = nullptr;
+    cudaFree(g.d_tile_prefix); g.d_tile_prefix = nullptr;
+    cudaFree(g.st_in); g.st_in = nullptr;
+    cudaFree(g.st_ids); g.st_ids = nullptr;
+    cudaFree(g.st_out); g.st_out = nullptr;
+    g.st_cap = 0;
+    for (TimedLaunch& t : g.timed) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
+    g.timed.clear();
+    for (cudaEvent_t e : g.event_pool) cudaEventDestroy(e);
+    g.event_pool.clear();
+    g.timing = false;
+    g.init = false;
+    g.has_family = false;
+    g.family.clear();
+    g.live = 0;
+    g.T = 0;
+    return MT_OK;
+}
+
+mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32_t* model_id_out) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!model_id_out) return MT_ERR_INVALID_ARG;
+    mt_status st = validate_layers(layers, n_layers);
+    if (st != MT_OK) return st;
+    if (!g.init) {
+        st = do_init(0, 1024, 0);
+        if (st != MT_OK) return st;
+    }
+    CU_OK(cudaSetDevice(g.device));
+    std::vector<HostLayer> hl(n_layers);
+    for (int l = 0; l < n_layers; ++l)
+        hl[l] = {layers[l].kind, layers[l].in_ch, layers[l].out_ch, layers[l].h, layers[l].w, layers[l].relu ? 1 : 0};
+    st = check_family(hl);
+    if (st != MT_OK) return st;
+    int id = -1;
+    for (int i = 0; i < g.max_models; ++i)
+        if (!g.models[i].alive) { id = i; break; }
+    if (id < 0) return MT_ERR_OOM;
+
+    // one device block per model: [tiled weights | padded bias] per layer, 1024-byte aligned pieces
+    size_t total = 0, raw_max = 0;
+    std::vector<size_t> w_off(n_layers, 0), b_off(n_layers, 0);
+    for (int l = 0; l < n_layers; ++l) {
+        const HostLayer& h = hl[l];
+        if (h.kind == MT_GLOBAL_AVG_POOL) continue;
+        const size_t n_tiles = (h.out_ch + BN - 1) / BN;
+        size_t wbytes, raw;
+        if (h.kind == MT_DENSE) { wbytes = n_tiles * (size_t)(h.in_ch / BK) * TILE_BYTES; raw = (size_t)h.out_ch * h.in_ch * 2; }
+        else { wbytes = (size_t)9 * h.out_ch * h.in_ch * 2; raw = wbytes; }
+        w_off[l] = total; total += align_up(wbytes, 1024);
+        b_off[l] = total; total += align_up(n_tiles * BN * sizeof(float), 1024);
+        if (raw > raw_max) raw_max = raw;
+    }
+    uint8_t* block = nullptr;
+    CU_OK(cudaMalloc(&block, total));
+    cudaError_t e = cudaMemset(block, 0, total);
+    void* raw_dev = nullptr;
+    ModelDev md;
+    memset(&md, 0, sizeof md);
+    md.alive = 1;
+    md.n_layers = n_layers;
+    for (int l = 0; l < n_layers && e == cudaSuccess; ++l) {
+        const HostLayer& h = hl[l];
+        LayerDev& d = md.layer[l];
+        d.kind = h.kind; d.K = h.in_ch; d.N = h.out_ch; d.relu = h.relu;
+        d.n_tiles = (h.out_ch + BN - 1) / BN;
+        d.k_blocks = h.kind == MT_DENSE ? h.in_ch / BK : 9;
+        if (h.kind == MT_GLOBAL_AVG_POOL) continue;
+        d.w = reinterpret_cast<const uint16_t*>(block + w_off[l]);
+        d.bias = reinterpret_cast<const float*>(block + b_off[l]);
+        const size_t raw = (size_t)h.out_ch * h.in_ch * 2 * (h.kind == MT_CONV3X3 ? 9 : 1);
+        const uint16_t* src = static_cast<const uint16_t*>(layers[l].weight);
+        if (!is_device_pointer(src) || (reinterpret_cast<uintptr_t>(src) & 15)) {
+            if (!raw_dev) e = cudaMalloc(&raw_dev, raw_max);
+            if (e == cudaSuccess) e = cudaMemcpy(raw_dev, src, raw, cudaMemcpyDefault);
+            src = static_cast<const uint16_t*>(raw_dev);
+        }
+        if (e != cudaSuccess) break;
+        if (h.kind == MT_DENSE) launch_pretile_dense(src, h.out_ch, h.in_ch, (uint16_t*)(block + w_off[l]), 0);
+        else launch_pretile_conv(src, h.out_ch, h.in_ch, (uint16_t*)(block + w_off[l]), 0);
+        e = cudaGetLastError();
+        if (e == cudaSuccess && layers[l].bias)
+            e = cudaMemcpy(block + b_off[l], layers[l].bias, sizeof(float) * h.out_ch, cudaMemcpyDefault);
+        if (e == cudaSuccess) e = cudaDeviceSynchronize();   // raw_dev is reused by the next layer
+    }
+    if (e == cudaSuccess) e = cudaMemcpy(g.d_models + id, &md, sizeof md, cudaMemcpyHostToDevice);
+    if (raw_dev) cudaFree(raw_dev);
+    if (e != cudaSuccess) {
+        cudaFree(block);
+        cudaGetLastError();
+        return e == cudaErrorMemoryAllocation ? MT_ERR_OOM : MT_ERR_CUDA;
+    }
+
+    if (!g.has_family || g.live == 0) {
+        g.family = hl;
+        g.has_family = true;
+        g.in_elems = layer_in_elems(hl[0]);
+        g.out_elems = hl.back().out_ch;
+        for (int b = 0; b <= MT_MAX_LAYERS; ++b) g.width[b] = 0;
+        g.ws_dirty = true;
+    }
+    for (int l = 0; l < n_layers; ++l) {
+        const int wd = layer_in_elems(hl[l]);
+        if (wd > g.width[l]) { g.width[l] = wd; g.ws_dirty = true; }
+    }
+    HostModel& hm = g.models[id];
+    hm.alive = true;
+    hm.layers = hl;
+    hm.dev_block = block;
+    g.live += 1;
+    if (id + 1 > g.T) g.T = id + 1;
+    *model_id_out = id;
+    return MT_OK;
+}
+
+mt_status mt_release(int32_t model_id) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g.init) return MT_ERR_NOT_INIT;
+    if (model_id < 0 || model_id >= g.max_models || !g.models[model_id].alive) return MT_ERR_BAD_MODEL_ID;
+    CU_OK(cudaSetDevice(g.device));
+    CU_OK(cudaDeviceSynchronize());
+    ModelDev md;
+    memset(&md, 0, sizeof md);
+    CU_OK(cudaMemcpy(g.d_models + model_id, &md, sizeof md, cudaMemcpyHostToDevice));
+    HostModel& hm = g.models[model_id];
+    cudaFree(hm.dev_block);
+    hm.dev_block = nullptr;
+    hm.alive = false;
+    hm.layers.clear();
+    g.live -= 1;
+    return MT_OK;
+}
+
+mt_status mt_infer(const void* inputs, const int32_t* model_ids, int32_t n, void* outputs, void* stream) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    return infer_device(inputs, model_ids, n, outputs, static_cast<cudaStream_t>(stream));
+}
+
+mt_status mt_infer_host(const void* inputs_host, const int32_t* model_ids_host, int32_t n, void* outputs_host,
+                        void* stream) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g.init) return MT_ERR_NOT_INIT;
+    if (n < 0) return MT_ERR_INVALID_ARG;
+    if (n == 0) return MT_OK;
+    if (!inputs_host || !model_ids_host || !outputs_host) return MT_ERR_INVALID_ARG;
+    if (!g.has_family || g.live == 0) return MT_ERR_BAD_MODEL_ID;
+    CU_OK(cudaSetDevice(g.device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (n > g.st_cap) {
+        CU_OK(cudaDeviceSynchronize());
+        cudaFree(g.st_in); cudaFree(g.st_ids); cudaFree(g.st_out);
+        g.st_in = nullptr; g.st_ids = nullptr; g.st_out = nullptr; g.st_cap = 0;
+        CU_OK(cudaMalloc(&g.st_in, (size_t)n * g.in_elems * 2));
+        CU_OK(cudaMalloc(&g.st_ids, (size_t)n * sizeof(int32_t)));
+        CU_OK(cudaMalloc(&g.st_out, (size_t)n * g.out_elems * sizeof(float)));
+        g.st_cap = n;
+    }
+    CU_OK(cudaMemcpyAsync(g.st_in, inputs_host, (size_t)n * g.in_elems * 2, cudaMemcpyHostToDevice, s));
+    CU_OK(cudaMemcpyAsync(g.st_ids, model_ids_host, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+    mt_status st = infer_device(g.st_in, g.st_ids, n, g.st_out, s);
+    if (st != MT_OK) return st;
+    CU_OK(cudaMemcpyAsync(outputs_host, g.st_out, (size_t)n * g.out_elems * sizeof(float), cudaMemcpyDeviceToHost, s));
+    CU_OK(cudaStreamSynchronize(s));
+    return MT_OK;
+}
+
+mt_status mt_get_async_status(void* stream, int32_t* status_out, int32_t* bad_request_index_out) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g.init) return MT_ERR_NOT_INIT;
+    CU_OK(cudaSetDevice(g.device));
+    CU_OK(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    int32_t w[ST_WORDS];
+    CU_OK(cudaMemcpy(w, g.d_status, sizeof w, cudaMemcpyDeviceToHost));
+    if (status_out) *status_out = w[ST_CODE];
+    if (bad_request_index_out) *bad_request_index_out = (w[ST_BAD_INDEX] == INT_MAX) ? -1 : w[ST_BAD_INDEX];
+    if (w[ST_CODE] == MT_ERR_TIMEOUT && getenv("MT_LOG")) fprintf(stderr, "[mt] device wait gave up at site %d\n", w[ST_WHERE]);
+    return reset_status_word();
+}
+
+const char* mt_status_string(mt_status s) {
+    switch (s) {
+        case MT_OK: return "ok";
+        case MT_ERR_INVALID_ARG: return "invalid argument";
+        case MT_ERR_BAD_MODEL_ID: return "bad model id";
+        case MT_ERR_SHAPE: return "shape mismatch";
+        case MT_ERR_UNSUPPORTED: return "unsupported layer or dimension";
+        case MT_ERR_OOM: return "out of memory";
+        case MT_ERR_CUDA: return "CUDA error";
+        case MT_ERR_ARCH: return "device is not sm_100";
+        case MT_ERR_TIMEOUT: return "device-side wait timed out";
+        case MT_ERR_NOT_INIT: return "not initialised";
+    }
+    return "unknown status";
+}
+
+mt_status mt_debug_last_bucketing(int32_t* counts_host, int32_t* offsets_host, int32_t* perm_host,
+                                  int32_t* inv_host, int32_t* n_tenants_out) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g.init) return MT_ERR_NOT_INIT;
+    CU_OK(cudaSetDevice(g.device));
+    CU_OK(cudaDeviceSynchronize());
+    const size_t i4 = sizeof(int32_t);
+    if (n_tenants_out) *n_tenants_out = g.T;
+    if (counts_host && g.T) CU_OK(cudaMemcpy(counts_host, g.d_counts, i4 * g.T, cudaMemcpyDeviceToHost));
+    if (offsets_host) CU_OK(cudaMemcpy(offsets_host, g.d_offsets, i4 * (g.T + 2), cudaMemcpyDeviceToHost));
+    if (perm_host && g.last_n) CU_OK(cudaMemcpy(perm_host, g.d_perm, i4 * g.last_n, cudaMemcpyDeviceToHost));
+    if (inv_host && g.last_n) CU_OK(cudaMemcpy(inv_host, g.d_inv, i4 * g.last_n, cudaMemcpyDeviceToHost));
+    return MT_OK;
+}
+
+mt_status mt_set_kernel_timing(int32_t enable) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    g.timing = enable != 0;
+    return MT_OK;
+}
+
+mt_status mt_get_kernel_times(const char** names, double* total_ms, int32_t* launches, int32_t cap, int32_t* n_out) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!names || !total_ms || !launches || !n_out || cap < 0) return MT_ERR_INVALID_ARG;
+    double ms[K_COUNT] = {0};
+    int cnt[K_COUNT] = {0};
+    for (TimedLaunch& t : g.timed) {
+        CU_OK(cudaEventSynchronize(t.stop));
+        float f = 0.f;
+        CU_OK(cudaEventElapsedTime(&f, t.start, t.stop));
+        ms[t.kernel] += f;
+        cnt[t.kernel] += 1;
+        g.event_pool.push_back(t.start);
+        g.event_pool.push_back(t.stop);
+    }
+    g.timed.clear();
+    int k = 0;
+    for (int i = 0; i < K_COUNT && k < cap; ++i) {
+        if (cnt[i] == 0) continue;
+        names[k] = kKernelNames[i];
+        total_ms[k] = ms[i];
+        launches[k] = cnt[i];
+        ++k;
+    }
+    *n_out = k;
+    return MT_OK;
+}
+
+}  // extern "C"

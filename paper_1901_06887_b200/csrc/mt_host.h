@@ -1,0 +1,78 @@
+// Host-side declarations of the kernel launchers (one per .cu file) used by the C-ABI layer.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mt {
+
+struct ModelDev;
+
+constexpr int kBucketChunk = 256;   // requests per CTA in the bucketing passes
+
+struct BucketArgs {
+    const int32_t* ids;
+    int n;
+    int T;                    // id slots in use (highest issued id + 1)
+    const ModelDev* models;
+    int n_layers;
+    int rows_per_unit;        // conv: tiles per image
+    int32_t* block_hist;      // [ceil(n / kBucketChunk)][T + 1]
+    int32_t* counts;          // [T + 1]
+    int32_t* offsets;         // [T + 2]
+    int32_t* tile_prefix;     // [n_layers][T + 1]
+    int32_t* tmp;             // [T + 1]
+    int32_t* perm;            // [n]
+    int32_t* inv;             // [n]
+    int32_t* status;
+};
+
+void launch_bucketing(const BucketArgs& a, cudaStream_t s);
+void launch_gather_rows(const void* src, const int32_t* perm, int n, int row_bytes, void* dst, int dst_ld_bytes,
+                        int sm_count, cudaStream_t s);
+void launch_unpermute(const float* src, const int32_t* perm, const int32_t* offsets, int T, int n, int out_elems,
+                      float* dst, int sm_count, cudaStream_t s);
+
+// Re-lay a dense weight matrix W[N][K] (bf16, row-major) as ceil(N/128) x (K/64) tiles of 128 rows x 64
+// columns, each tile 16 KiB in the 128-byte-swizzled shared-memory image the tensor-core kernels consume;
+// rows >= N are zero.  Tile (nt, kb) starts at element offset (nt * (K/64) + kb) * 8192.
+void launch_pretile_dense(const uint16_t* w, int N, int K, uint16_t* out, cudaStream_t s);
+// Conv weights W[64][3][3][64] -> 9 tap tiles of 64 rows (out channel) x 64 columns (in channel), 8 KiB each.
+void launch_pretile_conv(const uint16_t* w, int C_out, int C_in, uint16_t* out, cudaStream_t s);
+
+struct GemmArgs {
+    const ModelDev* models;
+    int layer;
+    int T;
+    const int32_t* offsets;       // [T + 2]
+    const int32_t* tile_prefix;   // [T + 1] of this layer
+    void* out;                    // bf16 or fp32, rows in bucketed order
+    int ld_out;                   // elements between output rows
+    int out_fp32;
+    int32_t* status;
+};
+cudaError_t configure_grouped_gemm();
+void launch_grouped_gemm(const CUtensorMap& tmap_a, const GemmArgs& a, int sm_count, cudaStream_t s);
+
+struct ConvArgs {
+    const ModelDev* models;
+    int layer;
+    int T;
+    const int32_t* offsets;
+    const int32_t* tile_prefix;
+    const int32_t* perm;          // non-null: image index = perm[j] (first layer reads the caller's buffer)
+    uint16_t* out;                // bf16 NHWC, bucketed order
+    int H, W;
+    int rows_per_tile;            // image rows per tile: floor(128 / W)
+    int tiles_per_image;
+    int32_t* status;
+};
+cudaError_t configure_grouped_conv();
+void launch_grouped_conv(const CUtensorMap& tmap_x, const ConvArgs& a, int sm_count, cudaStream_t s);
+
+// g[j][c] = mean over the H*W positions of x[j][.][.][c]; bf16 in, fp32 sum, bf16 out (row stride ld_out).
+void launch_global_avg_pool(const uint16_t* x, int n, int HW, int C, uint16_t* out, int ld_out, int sm_count,
+                            cudaStream_t s);
+
+}  // namespace mt
