@@ -1,0 +1,171 @@
+"""Element-by-element parity of the CUDA path with the fp64 oracle on reduced workloads that still span
+several tiles and ragged tails, plus closed forms, edge cases and the properties the paper states
+(determinism, no influence between tenants).  Everything goes through the C-ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1901_06887_b200 import binding as mt, harness, synth
+from paper_1901_06887_b200.synth import CONV3X3, DENSE, GLOBAL_AVG_POOL, Layer
+
+from gpu_util import TOL, fresh, run_and_check
+
+pytestmark = pytest.mark.gpu
+
+
+def bits(a):
+    return synth.f32_to_bf16_bits(np.asarray(a, np.float32))
+
+
+def test_config1_full():
+    wl = synth.make_workload(1)
+    run_and_check(wl.models, wl.model_ids, wl.inputs)
+
+
+def test_identity_and_zero_weights_are_exact_on_the_gpu():
+    rng = np.random.default_rng(0)
+    eye = np.eye(256, dtype=np.float32)
+    ident = [Layer(DENSE, 256, 256, relu=1, weight=bits(eye), bias=None),
+             Layer(DENSE, 256, 256, relu=1, weight=bits(eye), bias=None),
+             Layer(DENSE, 256, 10, relu=0, weight=bits(eye[:10]), bias=None)]
+    b = [rng.standard_normal(256).astype(np.float32), rng.standard_normal(256).astype(np.float32),
+         rng.standard_normal(10).astype(np.float32)]
+    zero = [Layer(DENSE, 256, 256, relu=1, weight=bits(np.zeros((256, 256))), bias=b[0]),
+            Layer(DENSE, 256, 256, relu=1, weight=bits(np.zeros((256, 256))), bias=b[1]),
+            Layer(DENSE, 256, 10, relu=0, weight=bits(np.zeros((10, 256))), bias=b[2])]
+    x = bits(rng.standard_normal((300, 256)))
+    ids = (np.arange(300) % 2).astype(np.int32)
+    got, _ = run_and_check([ident, zero], ids, x)
+    xf = synth.bf16_bits_to_f32(x)
+    assert np.array_equal(got[ids == 0], np.maximum(xf[ids == 0], 0)[:, :10])   # closed form, bit for bit
+    assert np.array_equal(got[ids == 1], np.tile(b[2], (150, 1)))
+
+
+@pytest.mark.parametrize("n", [1, 2, 127, 128, 129, 385])
+def test_ragged_row_tiles_single_tenant(n):
+    rng = np.random.default_rng(n)
+    m = [Layer(DENSE, 128, 192, relu=1, weight=bits(rng.standard_normal((192, 128)) * 0.2), bias=rng.standard_normal(192).astype(np.float32)),
+         Layer(DENSE, 192, 130, relu=0, weight=bits(rng.standard_normal((130, 192)) * 0.2), bias=rng.standard_normal(130).astype(np.float32))]
+    run_and_check([m], np.zeros(n, np.int32), bits(rng.standard_normal((n, 128))))
+
+
+@pytest.mark.parametrize("K,N", [(64, 1), (64, 10), (64, 128), (128, 129), (320, 257), (1024, 96)])
+def test_one_layer_shapes(K, N):
+    rng = np.random.default_rng(K + N)
+    models = [[Layer(DENSE, K, N, relu=t % 2, weight=bits(rng.standard_normal((N, K)) / np.sqrt(K)),
+                     bias=rng.standard_normal(N).astype(np.float32))] for t in range(3)]
+    n = 300
+    ids = rng.integers(0, 3, n).astype(np.int32)
+    run_and_check(models, ids, bits(rng.standard_normal((n, K))))
+
+
+def test_config2_reduced():
+    wl = synth.make_workload(2, n=900, n_tenants=7, widths=(1024, 512, 640, 256))
+    run_and_check(wl.models, wl.model_ids, wl.inputs)
+
+
+def test_config3_reduced_heterogeneous_widths_and_empty_tenants():
+    wl = synth.make_workload(3, n=1500, n_tenants=120)
+    assert (np.bincount(wl.model_ids, minlength=120) == 0).any()        # some tenants get no request
+    run_and_check(wl.models, wl.model_ids, wl.inputs, max_models=128)
+
+
+def test_config5_reduced():
+    wl = synth.make_workload(5, n=1100, n_tenants=3, widths=(512, 2048, 512))
+    run_and_check(wl.models, wl.model_ids, wl.inputs)
+
+
+@pytest.mark.parametrize("h,w", [(8, 8), (5, 7), (56, 56), (3, 128), (17, 20)])
+def test_config4_reduced_geometries(h, w):
+    wl = synth.make_workload(4, n=7, n_tenants=3, h=h, w=w, n_conv=2)
+    run_and_check(wl.models, wl.model_ids, wl.inputs)
+
+
+def test_conv_single_tap_shift_closed_form_on_gpu():
+    # tap (ky,kx) with weight 1 on the diagonal: Y = shifted X (zero outside), exact in bf16
+    H, W = 6, 9
+    rng = np.random.default_rng(5)
+    x = rng.integers(0, 5, size=(2, H, W, 64)).astype(np.float32)
+    for ky, kx in ((0, 0), (1, 2), (2, 1), (2, 2)):
+        wgt = np.zeros((64, 3, 3, 64), np.float32)
+        wgt[np.arange(64), ky, kx, np.arange(64)] = 1.0
+        head = np.zeros((8, 64), np.float32); head[np.arange(8), np.arange(8)] = 1.0
+        m = [Layer(CONV3X3, 64, 64, h=H, w=W, relu=1, weight=bits(wgt), bias=None),
+             Layer(GLOBAL_AVG_POOL, 64, 64, h=H, w=W),
+             Layer(DENSE, 64, 8, relu=0, weight=bits(head), bias=None)]
+        got, _ = run_and_check([m], np.zeros(2, np.int32), bits(x.reshape(2, -1)))
+        shifted = np.zeros_like(x)
+        ys = slice(max(0, 1 - ky), min(H, H + 1 - ky)); xs = slice(max(0, 1 - kx), min(W, W + 1 - kx))
+        ysrc = slice(ys.start + ky - 1, ys.stop + ky - 1); xsrc = slice(xs.start + kx - 1, xs.stop + kx - 1)
+        shifted[:, ys, xs, :] = x[:, ysrc, xsrc, :]
+        want = shifted.reshape(2, H * W, 64).mean(axis=1)[:, :8]
+        assert np.allclose(got, want, rtol=4e-3, atol=0)        # only the pooled mean is rounded to bf16
+
+
+def test_batch_invariance_and_nan_isolation():
+    wl = synth.make_workload(1, n=48)
+    got, _ = run_and_check(wl.models, wl.model_ids, wl.inputs)
+    ref = oracle.forward(wl.models, wl.model_ids, wl.inputs)
+    # the same request alone, and in another mix / position
+    for i in (0, 17, 47):
+        alone = harness.run_batch(wl.model_ids[i:i + 1], wl.inputs[i:i + 1], 10)
+        assert harness.scaled_error(alone, ref[i:i + 1]).max() <= TOL
+        assert np.array_equal(alone[0], got[i])                 # same kernel path here, so also bitwise equal
+    order = np.random.default_rng(1).permutation(48)[:31]
+    mixed = harness.run_batch(wl.model_ids[order], wl.inputs[order], 10)
+    assert np.array_equal(mixed, got[order])
+    # NaN weights in another tenant must not leak
+    t0 = int(wl.model_ids[0]); other = (t0 + 1) % 4
+    mt.mt_release(other)
+    poisoned = [Layer(l.kind, l.in_ch, l.out_ch, relu=l.relu, weight=np.full_like(l.weight, 0x7FC0), bias=l.bias)
+                for l in wl.models[other]]
+    assert mt.mt_register_model(poisoned) == other
+    again = harness.run_batch(wl.model_ids, wl.inputs, 10)
+    mine = wl.model_ids != other
+    assert np.array_equal(again[mine], got[mine])
+    assert np.isnan(again[~mine]).all()
+
+
+def test_repeat_runs_are_bitwise_identical_and_host_entry_matches():
+    wl = synth.make_workload(2, n=600, n_tenants=5, widths=(256, 512, 384, 64))
+    got, _ = run_and_check(wl.models, wl.model_ids, wl.inputs)
+    for _ in range(3):
+        assert np.array_equal(harness.run_batch(wl.model_ids, wl.inputs, 64), got)
+    x = torch.from_numpy(wl.inputs.view(np.int16)).pin_memory()
+    ids = torch.from_numpy(wl.model_ids).pin_memory()
+    out = torch.empty((wl.n, 64), dtype=torch.float32).pin_memory()
+    mt.mt_infer_host(x, ids, wl.n, out)
+    assert np.array_equal(out.numpy(), got)
+    # a model re-registered after release gives the same outputs (stateless function of weights and input)
+    mt.mt_release(2)
+    assert mt.mt_register_model(wl.models[2]) == 2
+    assert np.array_equal(harness.run_batch(wl.model_ids, wl.inputs, 64), got)
+
+
+def test_growing_batches_and_wider_models_reallocate_correctly():
+    rng = np.random.default_rng(9)
+    mk = lambda h: synth.make_mlp(3, h, (128, h, 64))
+    fresh()
+    models = [mk(128)]
+    assert mt.mt_register_model(models[0]) == 0
+    for n, add in ((10, None), (300, 256), (50, None), (700, 1024)):
+        if add:
+            models.append(mk(add))
+            assert mt.mt_register_model(models[-1]) == len(models) - 1
+        ids = rng.integers(0, len(models), n).astype(np.int32)
+        x = bits(rng.standard_normal((n, 128)))
+        run_and_check(models, ids, x, register=False)
+
+
+def test_family_mismatch_is_rejected():
+    fresh()
+    assert mt.mt_register_model(synth.make_mlp(1, 0, (64, 128, 10))) == 0
+    for widths in ((128, 128, 10), (64, 128, 12), (64, 10)):
+        with pytest.raises(mt.MtError) as e:
+            mt.mt_register_model(synth.make_mlp(1, 1, widths))
+        assert e.value.code == 3
+    assert mt.mt_register_model(synth.make_mlp(1, 1, (64, 512, 10))) == 1      # hidden width may differ
+    with pytest.raises(mt.MtError) as e:
+        mt.mt_release(5)
+    assert e.value.code == 2
