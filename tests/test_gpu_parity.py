@@ -45,16 +45,16 @@ def test_identity_and_zero_weights_are_exact_on_the_gpu():
 @pytest.mark.parametrize("n", [1, 2, 127, 128, 129, 385])
 def test_ragged_row_tiles_single_tenant(n):
     rng = np.random.default_rng(n)
-    m = [Layer(DENSE, 128, 192, relu=1, weight=bits(rng.standard_normal((192, 128)) * 0.2), bias=rng.standard_normal(192).astype(np.float32)),
-         Layer(DENSE, 192, 130, relu=0, weight=bits(rng.standard_normal((130, 192)) * 0.2), bias=rng.standard_normal(130).astype(np.float32))]
+    m = synth.make_mlp(1, n, (128, 192, 130))       # He-uniform weights, as in the workloads
     run_and_check([m], np.zeros(n, np.int32), bits(rng.standard_normal((n, 128))))
 
 
 @pytest.mark.parametrize("K,N", [(64, 1), (64, 10), (64, 128), (128, 129), (320, 257), (1024, 96)])
 def test_one_layer_shapes(K, N):
     rng = np.random.default_rng(K + N)
-    models = [[Layer(DENSE, K, N, relu=t % 2, weight=bits(rng.standard_normal((N, K)) / np.sqrt(K)),
-                     bias=rng.standard_normal(N).astype(np.float32))] for t in range(3)]
+    models = [synth.make_mlp(1, 10 * K + t, (K, N)) for t in range(3)]
+    for t, m in enumerate(models):
+        m[0].relu = t % 2
     n = 300
     ids = rng.integers(0, 3, n).astype(np.int32)
     run_and_check(models, ids, bits(rng.standard_normal((n, K))))
