@@ -31,7 +31,7 @@ from paper_1901_06887_b200 import synth  # noqa: E402
 METRIC = "mixed-tenant requests/sec"
 UNIT = "requests/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-DEFAULT_STEPS = {1: 2000, 2: 400, 3: 1000, 4: 300, 5: 20}
+DEFAULT_STEPS = {1: 5000, 2: 1500, 3: 2500, 4: 1500, 5: 50}
 ORACLE_SAMPLE = {1: 64, 2: 2048, 3: 16384, 4: 24, 5: 96}      # requests of the batch the CPU baseline times
 N_INPUT_BUFFERS = 3
 
@@ -64,10 +64,10 @@ def aggregate(local_units: float, local_ms: float, world: int):
     return float(u.item()), float(t.item())
 
 
-def result_line(metric_units: float, ms_total: float, steps: int, **extra):
+def result_line(metric_units: float, ms_total: float, n_steps: int, **extra):
     """units/s over the timed region and ms per step."""
     value = metric_units / (ms_total * 1e-3) if ms_total > 0 else 0.0
-    d = {"metric": METRIC, "value": value, "unit": UNIT, "ms_per_step": ms_total / max(steps, 1),
+    d = {"metric": METRIC, "value": value, "unit": UNIT, "ms_per_step": ms_total / max(n_steps, 1),
          "higher_is_better": True}
     d.update(extra)
     return d
