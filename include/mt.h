@@ -125,6 +125,38 @@ mt_status mt_set_kernel_timing(int32_t enable);
 mt_status mt_get_kernel_times(const char** names, double* total_ms, int32_t* launches, int32_t cap,
                               int32_t* n_out);
 
+/* Bucketing without any allocation.  (The paper has no counterpart to this call; it exists for callers
+ * of this library that are not allowed to allocate device memory.)
+ *
+ * Who needs it: code that runs where cudaMalloc / cudaFree are off limits - inside another allocator's
+ * callback or a framework memory-pool hook, in a serving loop that froze its memory map after start-up, or
+ * in a process whose device memory belongs wholly to a different allocator.  mt_infer cannot serve them,
+ * because its workspace is allocated (and grown) with cudaMalloc.  This call does the same stable counting
+ * sort of a batch by model id, using a fixed scratch array that is part of the library image: each GPU that
+ * loads the library holds about 1.03 MiB for it until the process exits.  It never calls cudaMalloc,
+ * cudaFree or any allocating routine, and needs no mt_init.
+ *
+ *   model_ids   device, int32 [n]
+ *   n           0 .. MT_NOALLOC_MAX_BATCH        (larger: MT_ERR_UNSUPPORTED, nothing enqueued)
+ *   n_models    1 .. MT_NOALLOC_MAX_MODELS       (larger: MT_ERR_UNSUPPORTED, nothing enqueued)
+ *   counts_out  device, int32 [n_models]         requests per id
+ *   offsets_out device, int32 [n_models + 1]     exclusive prefix of counts; [n_models] = number of valid requests
+ *   perm_out    device, int32 [n]                arrival index at each bucketed position (arrival order kept
+ *                                                inside a segment); ids outside [0, n_models) sort behind all
+ *                                                valid segments, in arrival order
+ *   inv_out     device, int32 [n]                bucketed position of each arrival index
+ *   stream      cudaStream_t; the work is enqueued there and runs on the CURRENT device
+ *
+ * The first call on each device looks up the scratch array's device address (with that device current);
+ * make that first call before starting any stream capture.  All calls on a device share the one scratch
+ * array, which still holds the previous call's contents when the next one starts; every entry a call reads
+ * is written by that call first, so nothing needs clearing, but two calls whose kernels overlap on the GPU
+ * (different streams without ordering) race and give wrong results - serialise them. */
+#define MT_NOALLOC_MAX_BATCH 65536
+#define MT_NOALLOC_MAX_MODELS 1024
+mt_status mt_bucket_noalloc(const int32_t* model_ids, int32_t n, int32_t n_models, int32_t* counts_out,
+                            int32_t* offsets_out, int32_t* perm_out, int32_t* inv_out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

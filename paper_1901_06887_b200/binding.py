@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "MT_OK", 1: "MT_ERR_INVALID_ARG", 2: "MT_ERR_BAD_MODEL_ID", 3
 
 EXPORTS = ["mt_init", "mt_shutdown", "mt_register_model", "mt_infer", "mt_infer_host", "mt_release",
            "mt_get_async_status", "mt_status_string", "mt_debug_last_bucketing", "mt_set_kernel_timing",
-           "mt_get_kernel_times"]
+           "mt_get_kernel_times", "mt_bucket_noalloc"]
 
 
 class MtError(RuntimeError):
@@ -61,6 +61,7 @@ def lib() -> ctypes.CDLL:
         l.mt_set_kernel_timing.argtypes = [i32]
         l.mt_get_kernel_times.argtypes = [ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_double),
                                           ctypes.POINTER(i32), i32, ctypes.POINTER(i32)]
+        l.mt_bucket_noalloc.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
         for name in EXPORTS:
             if name != "mt_status_string":
                 getattr(l, name).restype = ctypes.c_int
@@ -163,3 +164,12 @@ def mt_get_kernel_times() -> List[Tuple[str, float, int]]:
     n = ctypes.c_int32(0)
     _check(lib().mt_get_kernel_times(names, ms, cnt, cap, ctypes.byref(n)), "mt_get_kernel_times")
     return [(names[i].decode(), float(ms[i]), int(cnt[i])) for i in range(n.value)]
+
+
+def mt_bucket_noalloc(model_ids, n: int, n_models: int, counts_out, offsets_out, perm_out, inv_out, stream=None) -> None:
+    """Stable bucketing of a batch by model id for callers that must not allocate device memory (allocator
+    hooks, frozen-memory serving loops): all six buffers are the caller's device tensors, the scratch is a
+    fixed array inside the library.  Limits: n <= 65536, n_models <= 1024 (else MtError MT_ERR_UNSUPPORTED).
+    Calls that overlap on the GPU share that scratch and race."""
+    _check(lib().mt_bucket_noalloc(_ptr(model_ids), int(n), int(n_models), _ptr(counts_out), _ptr(offsets_out),
+                                   _ptr(perm_out), _ptr(inv_out), _stream_handle(stream)), "mt_bucket_noalloc")
