@@ -200,6 +200,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=None)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tenants", type=int, default=None, help="reduced case: number of tenants (profiling captures)")
+    ap.add_argument("--requests", type=int, default=None, help="reduced case: requests per batch")
+    ap.add_argument("--profile", action="store_true", help="timed loop only (no e2e, CPU baseline or clock sampler)")
     args = ap.parse_args()
     if args.steps is None:
         args.steps = DEFAULT_STEPS[args.config]
@@ -222,8 +225,9 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     cfg = args.config
-    models = synth.make_models(cfg)
-    batches = [synth.make_requests(cfg, models, salt=1000 * rank + b) for b in range(N_INPUT_BUFFERS)]
+    over = {"n_tenants": args.tenants} if args.tenants else {}
+    models = synth.make_models(cfg, **over)
+    batches = [synth.make_requests(cfg, models, n=args.requests, salt=1000 * rank + b) for b in range(N_INPUT_BUFFERS)]
     wl = synth.Workload(synth.CONFIG_NAMES[cfg], cfg, models, batches[0][0], batches[0][1])
     n, out_elems = wl.n, wl.out_elems
 
@@ -253,7 +257,8 @@ def main():
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    sampler.start()
+    if not args.profile:
+        sampler.start()
     e0.record(stream)
     for i in range(args.steps):
         step(i)
@@ -266,6 +271,15 @@ def main():
     local_ms = e0.elapsed_time(e1)
     kernel_times = mt.mt_get_kernel_times()
     units, ms = aggregate(n * args.steps, local_ms, world)
+
+    if args.profile:
+        if rank == 0:
+            print(json.dumps({"profile_run": True, "ms_per_step": ms / args.steps,
+                              "kernels": {nm: t / max(c, 1) for nm, t, c in kernel_times}}), flush=True)
+        mt.mt_shutdown()
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # ---- end to end: host buffers in, host buffers out, through the public entry point
     e2e_steps = args.e2e_steps or max(3, min(args.steps, 50))
@@ -306,6 +320,7 @@ def main():
         line = result_line(units, ms, args.steps, n_gpus=world, steps=args.steps, warmup=args.warmup, scaling="weak",
                            vs_baseline=None, dtype="bf16", data="synthetic")
         line["config"] = {"workload": synth.CONFIG_NAMES[cfg], "requests_per_step_per_gpu": n, "tenants": len(models),
+                          "reduced": bool(args.tenants or args.requests),
                           "l2": "weights streamed per step exceed the 126 MB L2 only for c2/c3/c5; inputs rotate over "
                                 "%d device buffers" % N_INPUT_BUFFERS,
                           "parallelism": "replicas x%d (each GPU hosts all tenants, own batch)" % world}
