@@ -20,6 +20,8 @@ namespace mt {
 
 constexpr int kScanThreads = 1024;
 
+struct LayerTileN { int v[8]; };
+
 // ids outside [0, T) or of dead models go to the extra bucket T, so they sort behind every live segment.
 __device__ __forceinline__ int classify(int id, int T, const ModelDev* models) {
     if (id < 0 || id >= T) return T;
@@ -76,7 +78,7 @@ __device__ void cta_exclusive_scan(const int32_t* in, int32_t* out, int n_items,
 }
 
 __global__ void __launch_bounds__(kScanThreads)
-bucket_scan(int n_blocks, int T, const ModelDev* __restrict__ models, int n_layers, int rows_per_unit,
+bucket_scan(int n_blocks, int T, const ModelDev* __restrict__ models, int n_layers, int rows_per_unit, LayerTileN tn,
             int32_t* __restrict__ block_hist, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
             int32_t* __restrict__ tile_prefix, int32_t* __restrict__ tmp) {
     __shared__ int32_t s_tmp[kScanThreads];
@@ -109,7 +111,7 @@ bucket_scan(int n_blocks, int T, const ModelDev* __restrict__ models, int n_laye
             const int c = counts[t];
             if (c > 0) {
                 const LayerDev& L = models[t].layer[l];
-                if (L.kind == MT_DENSE) units = ((c + BM - 1) / BM) * L.n_tiles;
+                if (L.kind == MT_DENSE) units = ((c + BM - 1) / BM) * ((L.N + tn.v[l] - 1) / tn.v[l]);
                 else if (L.kind == MT_CONV3X3) units = c * rows_per_unit;   // rows_per_unit = tiles per image
             }
             tmp[t] = units;
@@ -184,7 +186,9 @@ void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
     const int n_blocks = (a.n + kBucketChunk - 1) / kBucketChunk;
     const size_t smem = sizeof(int32_t) * (size_t)(a.T + 1);
     bucket_block_hist<<<n_blocks, kBucketChunk, smem, s>>>(a.ids, a.n, a.T, a.models, a.block_hist, a.status);
-    bucket_scan<<<1, kScanThreads, 0, s>>>(n_blocks, a.T, a.models, a.n_layers, a.rows_per_unit, a.block_hist,
+    LayerTileN tn;
+    for (int l = 0; l < 8; ++l) tn.v[l] = a.tile_n[l] > 0 ? a.tile_n[l] : BN;
+    bucket_scan<<<1, kScanThreads, 0, s>>>(n_blocks, a.T, a.models, a.n_layers, a.rows_per_unit, tn, a.block_hist,
                                            a.counts, a.offsets, a.tile_prefix, a.tmp);
     bucket_scatter<<<n_blocks, kBucketChunk, smem, s>>>(a.ids, a.n, a.T, a.models, a.block_hist, a.offsets, a.perm,
                                                         a.inv);

@@ -15,21 +15,26 @@
 
 namespace mt {
 
-constexpr int kStages = 6;
-constexpr int kStageBytes = 2 * TILE_BYTES;           // A tile + B tile
 constexpr int kGemmThreads = 192;
-constexpr int kAccCols = BN;                          // fp32 columns of one accumulator
-constexpr int kTmemCols = 2 * kAccCols;               // two accumulators (power of two >= 32)
 constexpr int kBarBytes = 256;
-constexpr int kGemmSmem = kStages * kStageBytes + kBarBytes + 1024;   // + slack for 1024-byte alignment
+
+// TN = output columns of one work item: 128 (one weight tile per stage) or 256 (two weight tiles per stage, half
+// the activation re-reads and half the shared-memory operand traffic per flop; all of TMEM for two accumulators).
+template <int TN>
+struct GemmCfg {
+    static constexpr int kStages = (TN == 256) ? 4 : 6;
+    static constexpr int kStageBytes = TILE_BYTES + (TN / BN) * TILE_BYTES;   // A tile + TN/128 weight tiles
+    static constexpr int kAccCols = TN;                                       // fp32 columns of one accumulator
+    static constexpr int kTmemCols = 2 * TN;                                  // two accumulators: 256 or 512 columns
+    static constexpr int kSmem = kStages * kStageBytes + kBarBytes + 1024;    // + slack for 1024-byte alignment
+};
 
 struct TileCoord {
     int t, m_tile, n_tile, row0, rows_valid;
 };
 
 __device__ __forceinline__ TileCoord decode_tile(int item, int T, const int32_t* __restrict__ prefix,
-                                                 const int32_t* __restrict__ offsets, const ModelDev* models,
-                                                 int layer) {
+                                                 const int32_t* __restrict__ offsets) {
     int lo = 0, hi = T;   // largest t with prefix[t] <= item
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
@@ -47,8 +52,14 @@ __device__ __forceinline__ TileCoord decode_tile(int item, int T, const int32_t*
     return c;
 }
 
+template <int TN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmArgs p) {
+    constexpr int kStages = GemmCfg<TN>::kStages;
+    constexpr int kStageBytes = GemmCfg<TN>::kStageBytes;
+    constexpr int kAccCols = GemmCfg<TN>::kAccCols;
+    constexpr int kTmemCols = GemmCfg<TN>::kTmemCols;
+    constexpr int kWTiles = TN / BN;                  // 128-row weight tiles per stage
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -87,28 +98,32 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmArgs p
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
             for (int item = blockIdx.x; ok && item < total; item += gridDim.x) {
-                const TileCoord c = decode_tile(item, p.T, p.tile_prefix, p.offsets, models, p.layer);
+                const TileCoord c = decode_tile(item, p.T, p.tile_prefix, p.offsets);
                 const LayerDev& L = models[c.t].layer[p.layer];
                 const int kblocks = L.k_blocks;
-                const uint16_t* wsrc = L.w + (size_t)c.n_tile * kblocks * (BN * BK);
+                // weight tile (nt, kb) of 128 rows x 64 columns starts at element (nt * kblocks + kb) * 8192
+                const uint16_t* wsrc = L.w + (size_t)c.n_tile * kWTiles * kblocks * (BN * BK);
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
                     const uint32_t a_dst = base + stage * kStageBytes;
                     mbar_expect_tx(full_bar(stage), kStageBytes);
                     tma_load_2d(a_dst, &tmap_a, kb * BK, c.row0, full_bar(stage));
-                    bulk_load(a_dst + TILE_BYTES, wsrc + (size_t)kb * (BN * BK), TILE_BYTES, full_bar(stage));
+#pragma unroll
+                    for (int wt = 0; wt < kWTiles; ++wt)
+                        bulk_load(a_dst + (1 + wt) * TILE_BYTES, wsrc + ((size_t)wt * kblocks + kb) * (BN * BK),
+                                  TILE_BYTES, full_bar(stage));
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {   // ------------------------------------------------ MMA issuer
-            constexpr uint32_t idesc = make_idesc_bf16(BM, BN);
+            constexpr uint32_t idesc = make_idesc_bf16(BM, TN);
             int stage = 0; uint32_t phase = 0;
             int it = 0;
             bool ok = true;
             for (int item = blockIdx.x; ok && item < total; item += gridDim.x, ++it) {
-                const TileCoord c = decode_tile(item, p.T, p.tile_prefix, p.offsets, models, p.layer);
+                const TileCoord c = decode_tile(item, p.T, p.tile_prefix, p.offsets);
                 const int kblocks = models[c.t].layer[p.layer].k_blocks;
                 const int acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
@@ -137,7 +152,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmArgs p
         const int r = q * 32 + lane;            // accumulator row of this thread
         int it = 0;
         for (int item = blockIdx.x; item < total; item += gridDim.x, ++it) {
-            const TileCoord c = decode_tile(item, p.T, p.tile_prefix, p.offsets, models, p.layer);
+            const TileCoord c = decode_tile(item, p.T, p.tile_prefix, p.offsets);
             const LayerDev& L = models[c.t].layer[p.layer];
             const int acc = it & 1;
             const uint32_t acc_phase = (it >> 1) & 1;
@@ -147,12 +162,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmArgs p
             const size_t grow = (size_t)(c.row0 + r);
             const int N = L.N, relu = L.relu;
 #pragma unroll 1
-            for (int ch = 0; ch < BN / 32; ++ch) {
+            for (int ch = 0; ch < TN / 32; ++ch) {
                 uint32_t v[32];
                 __syncwarp();   // tcgen05.ld is warp-collective: reconverge after the per-row stores
                 tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccCols + ch * 32, v);
                 tmem_ld_wait();
-                const int n0 = c.n_tile * BN + ch * 32;
+                const int n0 = c.n_tile * TN + ch * 32;
                 if (n0 >= N) break;
                 const float4* b4 = reinterpret_cast<const float4*>(L.bias + n0);
                 float f[32];
@@ -263,11 +278,16 @@ void launch_pretile_conv(const uint16_t* w, int C_out, int C_in, uint16_t* out, 
 }
 
 cudaError_t configure_grouped_gemm() {
-    return cudaFuncSetAttribute(grouped_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
+    cudaError_t e = cudaFuncSetAttribute(grouped_gemm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         GemmCfg<128>::kSmem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(grouped_gemm_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                GemmCfg<256>::kSmem);
 }
 
-void launch_grouped_gemm(const CUtensorMap& tmap_a, const GemmArgs& a, int sm_count, cudaStream_t s) {
-    grouped_gemm_kernel<<<sm_count, kGemmThreads, kGemmSmem, s>>>(tmap_a, a);
+void launch_grouped_gemm(const CUtensorMap& tmap_a, const GemmArgs& a, int tile_n, int sm_count, cudaStream_t s) {
+    if (tile_n == 256) grouped_gemm_kernel<256><<<sm_count, kGemmThreads, GemmCfg<256>::kSmem, s>>>(tmap_a, a);
+    else grouped_gemm_kernel<128><<<sm_count, kGemmThreads, GemmCfg<128>::kSmem, s>>>(tmap_a, a);
 }
 
 }  // namespace mt

@@ -55,6 +55,7 @@ struct Ctx {
     int in_elems = 0, out_elems = 0;
     int width[MT_MAX_LAYERS + 1] = {0};  // per layer boundary: widest input row (elements) over all models
     int live = 0;
+    int tile_n[MT_MAX_LAYERS] = {0};     // per dense layer: output columns per work item (128 or 256)
 
     // workspace
     int cap_n = 0;
@@ -220,6 +221,27 @@ bool is_device_pointer(const void* p) {
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// 128-row weight tiles allocated for a layer: an even count once N >= 256, so that 256-column work items can
+// always fetch two tiles (the padding tile is zero).
+size_t padded_weight_tiles(const HostLayer& h) {
+    size_t t = (h.out_ch + BN - 1) / BN;
+    if (h.kind == MT_DENSE && h.out_ch >= 256 && (t & 1)) t += 1;
+    return t;
+}
+
+// 256-column work items for a dense layer iff every live model is at least 256 wide there.
+void recompute_tile_n() {
+    for (int l = 0; l < MT_MAX_LAYERS; ++l) g.tile_n[l] = BN;
+    if (!g.has_family) return;
+    for (size_t l = 0; l < g.family.size(); ++l) {
+        if (g.family[l].kind != MT_DENSE) continue;
+        int min_n = INT_MAX;
+        for (const HostModel& m : g.models)
+            if (m.alive && m.layers[l].out_ch < min_n) min_n = m.layers[l].out_ch;
+        g.tile_n[l] = (min_n != INT_MAX && min_n >= 256) ? 256 : BN;
+    }
+}
+
 mt_status validate_layers(const mt_layer_desc* layers, int n_layers) {
     if (!layers || n_layers < 1 || n_layers > MT_MAX_LAYERS) return n_layers > MT_MAX_LAYERS ? MT_ERR_UNSUPPORTED : MT_ERR_INVALID_ARG;
     for (int l = 0; l < n_layers; ++l) {
@@ -311,6 +333,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
         Timer t(K_HIST, s);
         BucketArgs a;
         a.ids = ids; a.n = n; a.T = g.T; a.models = g.d_models; a.n_layers = L; a.rows_per_unit = tiles_per_image;
+        for (int l = 0; l < 8; ++l) a.tile_n[l] = g.tile_n[l];
         a.block_hist = g.d_block_hist; a.counts = g.d_counts; a.offsets = g.d_offsets; a.tile_prefix = g.d_tile_prefix;
         a.tmp = g.d_tmp; a.perm = g.d_perm; a.inv = g.d_inv; a.status = g.d_status;
         launch_bucketing(a, s);
@@ -335,7 +358,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             a.ld_out = last ? g.out_elems : g.act_ld[l + 1];
             a.out_fp32 = last ? 1 : 0;
             a.status = g.d_status;
-            launch_grouped_gemm(g.act_map[l], a, g.sm_count, s);
+            launch_grouped_gemm(g.act_map[l], a, g.tile_n[l], g.sm_count, s);
         } else if (f.kind == MT_CONV3X3) {
             Timer t(K_CONV, s);
             ConvArgs a;
@@ -428,7 +451,7 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
     for (int l = 0; l < n_layers; ++l) {
         const HostLayer& h = hl[l];
         if (h.kind == MT_GLOBAL_AVG_POOL) continue;
-        const size_t n_tiles = (h.out_ch + BN - 1) / BN;
+        const size_t n_tiles = padded_weight_tiles(h);
         size_t wbytes, raw;
         if (h.kind == MT_DENSE) { wbytes = n_tiles * (size_t)(h.in_ch / BK) * TILE_BYTES; raw = (size_t)h.out_ch * h.in_ch * 2; }
         else { wbytes = (size_t)9 * h.out_ch * h.in_ch * 2; raw = wbytes; }
@@ -448,7 +471,7 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
         const HostLayer& h = hl[l];
         LayerDev& d = md.layer[l];
         d.kind = h.kind; d.K = h.in_ch; d.N = h.out_ch; d.relu = h.relu;
-        d.n_tiles = (h.out_ch + BN - 1) / BN;
+        d.n_tiles = (int)padded_weight_tiles(h);
         d.k_blocks = h.kind == MT_DENSE ? h.in_ch / BK : 9;
         if (h.kind == MT_GLOBAL_AVG_POOL) continue;
         d.w = reinterpret_cast<const uint16_t*>(block + w_off[l]);
@@ -494,6 +517,7 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
     hm.dev_block = block;
     g.live += 1;
     if (id + 1 > g.T) g.T = id + 1;
+    recompute_tile_n();
     *model_id_out = id;
     return MT_OK;
 }
@@ -513,6 +537,7 @@ mt_status mt_release(int32_t model_id) {
     hm.alive = false;
     hm.layers.clear();
     g.live -= 1;
+    recompute_tile_n();
     return MT_OK;
 }
 

@@ -18,6 +18,7 @@ struct BucketArgs {
     const ModelDev* models;
     int n_layers;
     int rows_per_unit;        // conv: tiles per image
+    int tile_n[8];            // dense: output columns per work item of each layer (128 or 256)
     int32_t* block_hist;      // [ceil(n / kBucketChunk)][T + 1]
     int32_t* counts;          // [T + 1]
     int32_t* offsets;         // [T + 2]
@@ -53,7 +54,8 @@ struct GemmArgs {
     int32_t* status;
 };
 cudaError_t configure_grouped_gemm();
-void launch_grouped_gemm(const CUtensorMap& tmap_a, const GemmArgs& a, int sm_count, cudaStream_t s);
+// tile_n: 128 or 256 output columns per work item; must match BucketArgs::tile_n of that layer.
+void launch_grouped_gemm(const CUtensorMap& tmap_a, const GemmArgs& a, int tile_n, int sm_count, cudaStream_t s);
 
 struct ConvArgs {
     const ModelDev* models;
