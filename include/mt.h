@@ -76,7 +76,7 @@ mt_status mt_shutdown(void);
  * All models hosted by one context form one family: same number and kinds of layers, same input and
  * output element counts, same conv geometry.  Hidden dense widths may differ per model.
  * Kernel limits (else MT_ERR_UNSUPPORTED): 1..MT_MAX_LAYERS layers; dense in_ch a multiple of 64;
- * conv in_ch == out_ch == 64, w <= 128; a pool must follow a conv; a dense layer may not precede a conv.
+ * conv in_ch == out_ch == 64, w <= 126; a pool must follow a conv; a dense layer may not precede a conv.
  * Synchronous: returns after the copies have completed. */
 mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32_t* model_id_out);
 

@@ -1,12 +1,29 @@
-// Grouped 3x3 convolution executor (NHWC, stride 1, zero pad 1, 64 -> 64 channels, bias + ReLU) as an
-// implicit GEMM on the tensor cores, one persistent launch per layer for all tenants of the batch:
+// Grouped 3x3 convolution executor (NHWC, stride 1, zero pad 1, 64 -> 64 channels, bias + ReLU) as an implicit
+// GEMM on the tensor cores, ONE persistent launch per layer for all tenants of the batch:
 //     Y[r, y, x, o] = act(b_t[o] + sum_{ky,kx,c} X[r, y+ky-1, x+kx-1, c] * W_t[o, ky, kx, c])
-// GEMM view per work item: M = one strip of `rows_per_tile` image rows (rows_per_tile * W <= 128 pixels),
-// N = 64 output channels, K = 9 taps x 64 input channels.  One pipeline stage = one tap: the strip shifted
-// by (ky-1, kx-1) is fetched by a 4-D TMA box whose out-of-image part is zero-filled by the hardware (that
-// IS the zero padding), and the tap's 64 x 64 weight tile arrives as an 8 KiB bulk copy of a pre-swizzled
-// image.  Images are addressed by index, so the first layer reads the caller's buffer through the bucketing
-// permutation and no image is ever moved to group requests.
+//
+// Shared-memory picture.  A strip of R output rows of one image is fetched, with its one-pixel halo, by ONE 4-D
+// TMA box of (R+2) rows x Wp pixels x 64 channels (128 bytes per pixel, 128-byte swizzle); Wp is W+2 rounded up to
+// 32, 64 or 128, and everything outside the image is zero-filled by the copy engine - that IS the zero padding.
+// The strip is addressed flat: padded pixel q = yl * Wp + x.  Output pixel q of tap (ky,kx) needs input pixel
+// q + ky*Wp + kx, so the A operand of every tap is the SAME strip started (ky*Wp + kx)*128 bytes further on: nine
+// shifted matrix descriptors instead of nine copies.  An accumulator tile is 128 consecutive padded pixels
+// (= 128/Wp image rows) x 64 output channels; pad columns (x >= W) are computed and never stored.
+//
+// Tap pairing (Wp == 64, the 56 x 56 workload).  A tcgen05.mma with M = 128 takes as long for N = 64 as for
+// N = 128, so 64 output channels alone run the tensor pipe at half rate.  With Wp = 64 a tile is exactly two image
+// rows, and the 128-pixel block that starts at an even padded row serves two tiles at once: tap row ky = 2 of the
+// tile above it and tap row ky = 0 of the tile that starts there.  Their accumulators are neighbours in TMEM
+// (a ring of eight 64-column slots), so ONE N = 128 instruction with B = [W(2,kx) ; W(0,kx)] updates both.  Six of
+// the nine taps are issued this way, across strip borders too (the last tile of a strip is completed by the first
+// block of the next strip of the same image).  The first instruction into a fresh accumulator must overwrite it,
+// which a paired instruction cannot do for one half only, so every tile starts with its (unpaired) ky = 1 taps.
+//
+// The tenant's nine 64 x 64 tap tiles (72 KiB) stay resident in shared memory while consecutive strips belong to
+// the same tenant; CTAs take contiguous ranges of strips, so they change tenant rarely.
+//
+// Roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2..9 epilogue (two warps per TMEM lane quarter, 32 output
+// channels each: tcgen05.ld -> bias (shared memory) -> ReLU -> bf16 -> 128-bit stores).
 //
 // The paper does not define convolution; it only names a catalogue of standard layers (Sec. 1.1, Sec. 3.1).
 #include "mt_device.cuh"
@@ -14,32 +31,22 @@
 
 namespace mt {
 
-constexpr int kConvStages = 6;
-constexpr int kConvN = 64;
-constexpr int kTapBytes = kConvN * BK * 2;                       // 8 KiB: 64 out channels x 64 in channels
-constexpr int kConvStageBytes = TILE_BYTES + kTapBytes;          // strip (<= 16 KiB) + tap weights
-constexpr int kConvThreads = 192;
-constexpr int kConvTmemCols = 128;                               // two 64-column accumulators
-constexpr int kConvSmem = kConvStages * kConvStageBytes + 256 + 1024;
+constexpr int kConvThreads = 320;
+constexpr int kEpiThreads = 256;
+constexpr int kCN = 64;                          // output channels
+constexpr int kTapBytes = kCN * BK * 2;          // 8 KiB: 64 out channels x 64 in channels
+constexpr int kWeightBytes = 9 * kTapBytes;      // 72 KiB, resident per tenant
+constexpr int kMaxStages = 4;
+constexpr int kSlots = 8;                        // TMEM ring: 8 accumulators of 64 columns = all 512 columns
+constexpr int kConvBarBytes = 512;
 
-struct ConvTile {
-    int t, j, y0;
+// Order of the tap tiles in the executor layout: the three ky = 1 taps, then for every kx the pair
+// W(2,kx), W(0,kx) back to back, so that one 128-row B operand covers the pair.
+__host__ __device__ constexpr int tap_slot(int ky, int kx) { return ky == 1 ? kx : (3 + 2 * kx + (ky == 0 ? 1 : 0)); }
+
+struct StripCoord {
+    int t, j, y0, strip_in_image;
 };
-
-__device__ __forceinline__ ConvTile decode_conv_tile(int item, const ConvArgs& p) {
-    int lo = 0, hi = p.T;
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (p.tile_prefix[mid] <= item) lo = mid; else hi = mid;
-    }
-    const int local = item - p.tile_prefix[lo];
-    const int img = local / p.tiles_per_image;
-    ConvTile c;
-    c.t = lo;
-    c.j = p.offsets[lo] + img;
-    c.y0 = (local - img * p.tiles_per_image) * p.rows_per_tile;
-    return c;
-}
 
 __global__ void __launch_bounds__(kConvThreads, 1)
 grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArgs p) {
@@ -47,30 +54,36 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kConvStages * kConvStageBytes);
-    const uint32_t bar0 = base + kConvStages * kConvStageBytes;
-    auto full_bar = [&](int s) { return bar0 + 8u * s; };
-    auto empty_bar = [&](int s) { return bar0 + 8u * (kConvStages + s); };
-    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kConvStages + a); };
-    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kConvStages + 2 + a); };
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kConvStages + 4);
+    const uint32_t w_smem = base;
+    const uint32_t strip0 = base + kWeightBytes;
+    const uint32_t bar0 = strip0 + p.n_stages * p.stage_bytes;
+    uint8_t* bar_ptr = smem + kWeightBytes + p.n_stages * p.stage_bytes;
+    auto sfull_bar = [&](int s) { return bar0 + 8u * s; };
+    auto sempty_bar = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kMaxStages + kSlots + a); };
+    const uint32_t wfull_bar = bar0 + 8u * (2 * kMaxStages + 2 * kSlots);
+    const uint32_t wempty_bar = wfull_bar + 8u;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * (2 * kMaxStages + 2 * kSlots + 2));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    float* s_bias = reinterpret_cast<float*>(bar_ptr + 256);          // 64 floats
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kConvStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 128); }
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(sfull_bar(s), 1); mbar_init(sempty_bar(s), 1); }
+        for (int a = 0; a < kSlots; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), kEpiThreads); }
+        mbar_init(wfull_bar, 1);
+        mbar_init(wempty_bar, 1);
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tmap_x);
     }
-    // rows of the strip buffer that no TMA box ever writes (W * rows_per_tile .. 127) must not hold NaN
-    // patterns forever: clear all stage buffers once (their accumulator rows are never stored anyway)
-    for (int i = threadIdx.x; i < kConvStages * kConvStageBytes / 16; i += blockDim.x)
-        reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+    // the last rows of every strip stage are read (for rows that are never stored) but not written by the TMA box
+    for (int i = threadIdx.x; i < (p.n_stages * p.stage_bytes) / 16; i += blockDim.x)
+        reinterpret_cast<uint4*>(smem + kWeightBytes)[i] = make_uint4(0, 0, 0, 0);
     fence_proxy_async_smem();
     if (warp == 1) {
-        tmem_alloc(smem_u32(tmem_slot), kConvTmemCols);
+        tmem_alloc(smem_u32(tmem_slot), kSlots * kCN);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -78,104 +91,187 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    // contiguous range of strips for this CTA
     const int total = p.tile_prefix[p.T];
-    const int strip_pixels = p.rows_per_tile * p.W;
-    const uint32_t strip_bytes = (uint32_t)strip_pixels * 128u;
+    const int s_begin = (int)(((long long)total * blockIdx.x) / gridDim.x);
+    const int s_end = (int)(((long long)total * (blockIdx.x + 1)) / gridDim.x);
+    const int Wp = p.Wp;
+    const int TS = p.tiles_per_strip;
+    const bool pairing = (Wp == 64);
+
+    // strip -> (tenant, image, first row); strips of one tenant are consecutive, so the tenant's range is cached
+    int cur_t = -1, cur_lo = 0, cur_hi = 0, cur_seg = 0;
+    auto locate = [&](int s) {
+        if (s < cur_lo || s >= cur_hi) {
+            int lo = 0, hi = p.T;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (p.tile_prefix[mid] <= s) lo = mid; else hi = mid;
+            }
+            cur_t = lo; cur_lo = p.tile_prefix[lo]; cur_hi = p.tile_prefix[lo + 1]; cur_seg = p.offsets[lo];
+        }
+        StripCoord c;
+        const int local = s - cur_lo;
+        const int img = local / p.strips_per_image;
+        c.t = cur_t;
+        c.j = cur_seg + img;
+        c.strip_in_image = local - img * p.strips_per_image;
+        c.y0 = c.strip_in_image * p.R;
+        return c;
+    };
 
     if (warp == 0) {
         if (lane == 0) {   // ------------------------------------------------ TMA producer
             int stage = 0; uint32_t phase = 0;
-            bool ok = true;
-            for (int item = blockIdx.x; ok && item < total; item += gridDim.x) {
-                const ConvTile c = decode_conv_tile(item, p);
-                const uint16_t* wsrc = p.models[c.t].layer[p.layer].w;
-                const int img = p.perm ? p.perm[c.j] : c.j;
-                for (int tap = 0; tap < 9; ++tap) {
-                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 11)) { ok = false; break; }
-                    const int ky = tap / 3, kx = tap - 3 * ky;
-                    const uint32_t a_dst = base + stage * kConvStageBytes;
-                    mbar_expect_tx(full_bar(stage), strip_bytes + kTapBytes);
-                    tma_load_4d(a_dst, &tmap_x, 0, kx - 1, c.y0 + ky - 1, img, full_bar(stage));
-                    bulk_load(a_dst + TILE_BYTES, wsrc + (size_t)tap * (kConvN * BK), kTapBytes, full_bar(stage));
-                    if (++stage == kConvStages) { stage = 0; phase ^= 1u; }
+            int w_loads = 0, w_tenant = -1;
+            for (int s = s_begin; s < s_end; ++s) {
+                const StripCoord c = locate(s);
+                if (c.t != w_tenant) {     // this tenant's nine tap tiles, once the MMAs on the old ones are done
+                    if (w_loads > 0 && !mbar_wait(wempty_bar, (uint32_t)((w_loads - 1) & 1), abort_flag, p.status, 21)) break;
+                    mbar_expect_tx(wfull_bar, kWeightBytes);
+                    bulk_load(w_smem, p.models[c.t].layer[p.layer].w, kWeightBytes, wfull_bar);
+                    w_tenant = c.t;
+                    ++w_loads;
                 }
+                if (!mbar_wait(sempty_bar(stage), phase ^ 1u, abort_flag, p.status, 22)) break;
+                const int img = p.perm ? p.perm[c.j] : c.j;
+                mbar_expect_tx(sfull_bar(stage), p.box_bytes);
+                tma_load_4d(strip0 + stage * p.stage_bytes, &tmap_x, 0, -1, c.y0 - 1, img, sfull_bar(stage));
+                if (++stage == p.n_stages) { stage = 0; phase ^= 1u; }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {   // ------------------------------------------------ MMA issuer
-            constexpr uint32_t idesc = make_idesc_bf16(BM, kConvN);
+            constexpr uint32_t idesc64 = make_idesc_bf16(BM, kCN);
+            constexpr uint32_t idesc128 = make_idesc_bf16(BM, 2 * kCN);
             int stage = 0; uint32_t phase = 0;
-            int it = 0;
+            int g = 0;                      // tiles started so far by this CTA; tile g lives in TMEM slot g % kSlots
+            int w_loads = 0, w_tenant = -1;
             bool ok = true;
-            for (int item = blockIdx.x; ok && item < total; item += gridDim.x, ++it) {
-                const int acc = it & 1;
-                const uint32_t acc_phase = (it >> 1) & 1;
-                if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, 12)) break;
+            // four K steps of one 128-pixel block against one (N = 64) or two stacked (N = 128) tap tiles
+            auto issue = [&](uint32_t a_addr, uint32_t b_addr, uint32_t d_tmem, uint32_t idesc, bool overwrite) {
+                const uint64_t a_desc = make_kmajor_sw128_desc(a_addr, 1024);
+                const uint64_t b_desc = make_kmajor_sw128_desc(b_addr, 1024);
+#pragma unroll
+                for (int k = 0; k < BK / UMMA_K; ++k)
+                    umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (overwrite && k == 0) ? 0u : 1u);
+            };
+            for (int s = s_begin; ok && s < s_end; ++s) {
+                const StripCoord c = locate(s);
+                if (c.t != w_tenant) {
+                    if (w_loads > 0) umma_commit(wempty_bar);      // fires when all MMAs on the old weights are done
+                    if (!mbar_wait(wfull_bar, (uint32_t)(w_loads & 1), abort_flag, p.status, 23)) break;
+                    w_tenant = c.t;
+                    ++w_loads;
+                }
+                const bool pair_top = pairing && s > s_begin && c.strip_in_image > 0;
+                const bool defer_bottom = pairing && s + 1 < s_end && c.strip_in_image + 1 < p.strips_per_image;
+                if (!mbar_wait(sfull_bar(stage), phase, abort_flag, p.status, 25)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * kConvN;
-                for (int tap = 0; tap < 9; ++tap) {
-                    if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 13)) { ok = false; break; }
+                const uint32_t strip = strip0 + stage * p.stage_bytes;
+                for (int i = 0; i < TS; ++i, ++g) {
+                    const int slot = g % kSlots;
+                    // the accumulator slot must have been drained by the epilogue of tile g - kSlots
+                    if (!mbar_wait(tempty_bar(slot), (uint32_t)(((g / kSlots) & 1) ^ 1), abort_flag, p.status, 24)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_src = base + stage * kConvStageBytes;
-                    const uint64_t a_desc = make_kmajor_sw128_desc(a_src, 1024);
-                    const uint64_t b_desc = make_kmajor_sw128_desc(a_src + TILE_BYTES, 1024);
-#pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k)
-                        umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (tap | k) != 0);
-                    umma_commit(empty_bar(stage));
-                    if (++stage == kConvStages) { stage = 0; phase ^= 1u; }
-                }
-                if (ok) umma_commit(tfull_bar(acc));
-            }
-        }
-    } else {               // ---------------------------------------------------- epilogue (warps 2..5)
-        const int q = warp & 3;
-        const int r = q * 32 + lane;            // pixel of the strip handled by this thread
-        int it = 0;
-        for (int item = blockIdx.x; item < total; item += gridDim.x, ++it) {
-            const ConvTile c = decode_conv_tile(item, p);
-            const LayerDev& L = p.models[c.t].layer[p.layer];
-            const int acc = it & 1;
-            const uint32_t acc_phase = (it >> 1) & 1;
-            if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 14)) break;
-            tc_fence_after();
-            const bool row_ok = (r < strip_pixels) && (c.y0 + r / p.W < p.H);
-            uint16_t* dst = p.out + (((size_t)c.j * p.H + c.y0) * p.W + r) * kConvN;
-            const int relu = L.relu;
-#pragma unroll 1
-            for (int ch = 0; ch < kConvN / 32; ++ch) {
-                uint32_t v[32];
-                __syncwarp();
-                tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kConvN + ch * 32, v);
-                tmem_ld_wait();
-                const float4* b4 = reinterpret_cast<const float4*>(L.bias + ch * 32);
-                float f[32];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float4 b = __ldg(b4 + j);
-                    f[4 * j + 0] = __uint_as_float(v[4 * j + 0]) + b.x;
-                    f[4 * j + 1] = __uint_as_float(v[4 * j + 1]) + b.y;
-                    f[4 * j + 2] = __uint_as_float(v[4 * j + 2]) + b.z;
-                    f[4 * j + 3] = __uint_as_float(v[4 * j + 3]) + b.w;
-                }
-                if (relu) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) f[j] = fmaxf(f[j], 0.0f);
-                }
-                if (row_ok) {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint4 o;
-                        o.x = pack_bf16x2(f[8 * j + 0], f[8 * j + 1]);
-                        o.y = pack_bf16x2(f[8 * j + 2], f[8 * j + 3]);
-                        o.z = pack_bf16x2(f[8 * j + 4], f[8 * j + 5]);
-                        o.w = pack_bf16x2(f[8 * j + 6], f[8 * j + 7]);
-                        reinterpret_cast<uint4*>(dst + ch * 32)[j] = o;
+                    const uint32_t d_this = tmem_base + slot * kCN;
+                    const uint32_t blk = strip + (uint32_t)(i * BM) * 128u;          // padded pixel i*128 of the strip
+                    if (pairing) {
+                        // ky = 1 first: these overwrite the fresh accumulator
+                        for (int kx = 0; kx < 3; ++kx)
+                            issue(blk + (uint32_t)(Wp + kx) * 128u, w_smem + tap_slot(1, kx) * kTapBytes, d_this, idesc64, kx == 0);
+                        // block at the tile's first row: ky = 0 of this tile and ky = 2 of the tile above
+                        const bool have_above = (i > 0) || pair_top;
+                        const bool adjacent = slot != 0;                              // slots g-1 and g contiguous in TMEM
+                        for (int kx = 0; kx < 3; ++kx) {
+                            const uint32_t a_addr = blk + (uint32_t)kx * 128u;
+                            if (have_above && adjacent) {
+                                issue(a_addr, w_smem + tap_slot(2, kx) * kTapBytes, d_this - kCN, idesc128, false);
+                            } else {
+                                if (have_above)
+                                    issue(a_addr, w_smem + tap_slot(2, kx) * kTapBytes, tmem_base + ((g - 1) % kSlots) * kCN, idesc64, false);
+                                issue(a_addr, w_smem + tap_slot(0, kx) * kTapBytes, d_this, idesc64, false);
+                            }
+                        }
+                        if (have_above) umma_commit(tfull_bar((g - 1) % kSlots));    // tile above is complete
+                    } else {
+                        for (int tap = 0; tap < 9; ++tap) {
+                            const int ky = tap / 3, kx = tap - 3 * ky;
+                            issue(blk + (uint32_t)(ky * Wp + kx) * 128u, w_smem + tap_slot(ky, kx) * kTapBytes, d_this, idesc64, tap == 0);
+                        }
+                        umma_commit(tfull_bar(slot));
                     }
                 }
+                if (!ok) break;
+                if (pairing && !defer_bottom) {
+                    // nobody below will finish the strip's last tile: its ky = 2 taps from the block under it
+                    const uint32_t blk = strip + (uint32_t)(TS * BM) * 128u;
+                    const int last = (g - 1) % kSlots;
+                    for (int kx = 0; kx < 3; ++kx)
+                        issue(blk + (uint32_t)kx * 128u, w_smem + tap_slot(2, kx) * kTapBytes, tmem_base + last * kCN, idesc64, false);
+                    umma_commit(tfull_bar(last));
+                }
+                umma_commit(sempty_bar(stage));     // the strip buffer is free once these MMAs have read it
+                if (++stage == p.n_stages) { stage = 0; phase ^= 1u; }
             }
-            tc_fence_before();
-            mbar_arrive(tempty_bar(acc));
+        }
+    } else {               // ---------------------------------------------------- epilogue (warps 2..9)
+        const int ew = warp - 2;
+        const int q4 = warp & 3;                    // TMEM lane quarter this warp may read
+        const int half = ew >> 2;                   // which 32 of the 64 output channels
+        const int r = q4 * 32 + lane;               // tile-local padded pixel of this thread
+        const int yl = r / Wp, x = r - yl * Wp;
+        const int rows_per_tile = BM / Wp;
+        int g = 0, b_tenant = -1, relu = 0;
+        bool ok = true;
+        for (int s = s_begin; ok && s < s_end; ++s) {
+            const StripCoord c = locate(s);
+            if (c.t != b_tenant) {                  // new tenant: its bias into shared memory, ReLU flag into a register
+                const LayerDev& L = p.models[c.t].layer[p.layer];
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");      // everyone done with the old bias
+                if (threadIdx.x - 64 < kCN) s_bias[threadIdx.x - 64] = L.bias[threadIdx.x - 64];
+                relu = L.relu;
+                b_tenant = c.t;
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+            }
+            for (int i = 0; i < TS; ++i, ++g) {
+                const int slot = g % kSlots;
+                if (!mbar_wait(tfull_bar(slot), (uint32_t)((g / kSlots) & 1), abort_flag, p.status, 26)) { ok = false; break; }
+                tc_fence_after();
+                uint32_t v[32];
+                tmem_ld32(tmem_base + (static_cast<uint32_t>(q4 * 32) << 16) + slot * kCN + half * 32, v);
+                tmem_ld_wait();
+                tc_fence_before();
+                mbar_arrive(tempty_bar(slot));      // values are in registers: the slot can be reused
+                const int y = c.y0 + i * rows_per_tile + yl;
+                if (x < p.W && y < p.H) {
+                    uint16_t* dst = p.out + (((size_t)c.j * p.H + y) * p.W + x) * kCN + half * 32;
+                    const float4* b4 = reinterpret_cast<const float4*>(s_bias + half * 32);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        float f[8];
+#pragma unroll
+                        for (int h2 = 0; h2 < 2; ++h2) {
+                            const float4 b = b4[2 * j + h2];
+                            f[4 * h2 + 0] = __uint_as_float(v[8 * j + 4 * h2 + 0]) + b.x;
+                            f[4 * h2 + 1] = __uint_as_float(v[8 * j + 4 * h2 + 1]) + b.y;
+                            f[4 * h2 + 2] = __uint_as_float(v[8 * j + 4 * h2 + 2]) + b.z;
+                            f[4 * h2 + 3] = __uint_as_float(v[8 * j + 4 * h2 + 3]) + b.w;
+                        }
+                        if (relu) {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) f[e] = fmaxf(f[e], 0.0f);
+                        }
+                        uint4 o;
+                        o.x = pack_bf16x2(f[0], f[1]);
+                        o.y = pack_bf16x2(f[2], f[3]);
+                        o.z = pack_bf16x2(f[4], f[5]);
+                        o.w = pack_bf16x2(f[6], f[7]);
+                        reinterpret_cast<uint4*>(dst)[j] = o;
+                    }
+                }
+                __syncwarp();
+            }
         }
     }
 
@@ -187,8 +283,48 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
     __syncthreads();
     if (warp == 1) {
         __syncwarp();
-        tmem_dealloc(tmem_base, kConvTmemCols);
+        tmem_dealloc(tmem_base, kSlots * kCN);
     }
+}
+
+// Strip geometry for an H x W image (W <= 126).
+bool plan_conv(int H, int W, ConvPlan* plan) {
+    if (W < 1 || H < 1 || W + 2 > 128) return false;
+    const int Wp = (W + 2 <= 32) ? 32 : (W + 2 <= 64) ? 64 : 128;
+    const int rows_per_tile = BM / Wp;
+    const int TS = 2;                                         // accumulator tiles per strip
+    const int R = TS * rows_per_tile;
+    if (R + 2 > 256) return false;
+    const int box = (R + 2) * Wp * 128;
+    const int stage = box + 1024;                             // taps shifted by up to 2 pixels read past the box
+    int stages = (227 * 1024 - kWeightBytes - kConvBarBytes - 1024) / stage;
+    if (stages < 2) return false;
+    if (stages > kMaxStages) stages = kMaxStages;
+    plan->Wp = Wp; plan->R = R; plan->tiles_per_strip = TS; plan->stage_bytes = stage; plan->n_stages = stages;
+    plan->strips_per_image = (H + R - 1) / R;
+    plan->box_bytes = box;
+    plan->smem_bytes = kWeightBytes + stages * stage + kConvBarBytes + 1024;
+    return true;
+}
+
+// Conv weights W[64][3][3][64] -> nine tap tiles of 64 rows (out channel) x 64 columns (in channel), each the
+// 8 KiB swizzled shared-memory image; tile order given by tap_slot().
+__global__ void pretile_conv_kernel(const uint16_t* __restrict__ w, int C_out, int C_in, uint4* __restrict__ out,
+                                    int total_chunks) {
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total_chunks; idx += gridDim.x * blockDim.x) {
+        const int tap = idx / (C_out * 8);                   // natural tap index ky * 3 + kx
+        const int within = idx % (C_out * 8);
+        const int r = within >> 3, cpos = within & 7;
+        const int c = cpos ^ (r & 7);
+        const int ky = tap / 3, kx = tap - 3 * ky;
+        out[tap_slot(ky, kx) * (C_out * 8) + within] =
+            *reinterpret_cast<const uint4*>(w + ((size_t)r * 9 + tap) * C_in + c * 8);
+    }
+}
+
+void launch_pretile_conv(const uint16_t* w, int C_out, int C_in, uint16_t* out, cudaStream_t s) {
+    const int total = 9 * C_out * 8;
+    pretile_conv_kernel<<<(total + 255) / 256, 256, 0, s>>>(w, C_out, C_in, reinterpret_cast<uint4*>(out), total);
 }
 
 // g[j][c] = (1 / HW) * sum_p x[j][p][c]; one CTA per image, 8 channels (16 bytes) per thread per pixel.
@@ -225,11 +361,11 @@ global_avg_pool_kernel(const uint16_t* __restrict__ x, int HW, int C, uint16_t* 
 }
 
 cudaError_t configure_grouped_conv() {
-    return cudaFuncSetAttribute(grouped_conv3x3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kConvSmem);
+    return cudaFuncSetAttribute(grouped_conv3x3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
 }
 
-void launch_grouped_conv(const CUtensorMap& tmap_x, const ConvArgs& a, int sm_count, cudaStream_t s) {
-    grouped_conv3x3_kernel<<<sm_count, kConvThreads, kConvSmem, s>>>(tmap_x, a);
+void launch_grouped_conv(const CUtensorMap& tmap_x, const ConvArgs& a, int smem_bytes, int sm_count, cudaStream_t s) {
+    grouped_conv3x3_kernel<<<sm_count, kConvThreads, smem_bytes, s>>>(tmap_x, a);
 }
 
 void launch_global_avg_pool(const uint16_t* x, int n, int HW, int C, uint16_t* out, int ld_out, int /*sm_count*/,

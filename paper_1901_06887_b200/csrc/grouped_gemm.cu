@@ -252,29 +252,12 @@ __global__ void pretile_dense_kernel(const uint16_t* __restrict__ w, int N, int 
     }
 }
 
-__global__ void pretile_conv_kernel(const uint16_t* __restrict__ w, int C_out, int C_in, uint4* __restrict__ out,
-                                    int total_chunks) {
-    // 9 tap tiles; tile `tap` holds rows o = 0..C_out-1 of 64 input channels: 64 rows x 128 bytes, swizzled
-    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total_chunks; idx += gridDim.x * blockDim.x) {
-        const int tap = idx / (C_out * 8);
-        const int within = idx % (C_out * 8);
-        const int r = within >> 3, cpos = within & 7;
-        const int c = cpos ^ (r & 7);
-        out[idx] = *reinterpret_cast<const uint4*>(w + ((size_t)r * 9 + tap) * C_in + c * 8);
-    }
-}
-
 void launch_pretile_dense(const uint16_t* w, int N, int K, uint16_t* out, cudaStream_t s) {
     const long long n_tiles = (N + BN - 1) / BN;
     const long long total = n_tiles * (K / BK) * 1024;
     long long blocks = (total + 255) / 256;
     if (blocks > 4096) blocks = 4096;
     pretile_dense_kernel<<<(int)blocks, 256, 0, s>>>(w, N, K, reinterpret_cast<uint4*>(out), total);
-}
-
-void launch_pretile_conv(const uint16_t* w, int C_out, int C_in, uint16_t* out, cudaStream_t s) {
-    const int total = 9 * C_out * 8;
-    pretile_conv_kernel<<<(total + 255) / 256, 256, 0, s>>>(w, C_out, C_in, reinterpret_cast<uint4*>(out), total);
 }
 
 cudaError_t configure_grouped_gemm() {

@@ -55,6 +55,7 @@ struct Ctx {
     int in_elems = 0, out_elems = 0;
     int width[MT_MAX_LAYERS + 1] = {0};  // per layer boundary: widest input row (elements) over all models
     int live = 0;
+    ConvPlan conv;                       // strip geometry of the conv layers (one geometry per family)
     int tile_n[MT_MAX_LAYERS] = {0};     // per dense layer: output columns per work item (128 or 256)
 
     // workspace
@@ -92,8 +93,6 @@ std::mutex g_mu;
             return (e__ == cudaErrorMemoryAllocation) ? MT_ERR_OOM : MT_ERR_CUDA; \
         }                                                             \
     } while (0)
-
-int conv_rows_per_tile(int w, int h) { int r = BM / w; return r < h ? r : h; }
 
 mt_status reset_status_word() {
     const int32_t init[ST_WORDS] = {MT_OK, INT_MAX, 0, 0};
@@ -161,10 +160,10 @@ mt_status encode_2d(CUtensorMap* map, void* ptr, int ld, int rows) {
     return r == CUDA_SUCCESS ? MT_OK : MT_ERR_CUDA;
 }
 
-mt_status encode_nhwc(CUtensorMap* map, const void* ptr, int C, int W, int H, int n_img, int rows_per_tile) {
+mt_status encode_nhwc(CUtensorMap* map, const void* ptr, int C, int W, int H, int n_img, int box_w, int box_h) {
     cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)n_img};
     cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
-    cuuint32_t box[4] = {(cuuint32_t)C, (cuuint32_t)W, (cuuint32_t)rows_per_tile, 1};
+    cuuint32_t box[4] = {(cuuint32_t)C, (cuuint32_t)box_w, (cuuint32_t)box_h, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = g.encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -200,7 +199,7 @@ mt_status ensure_workspace(int n) {
             CU_OK(cudaMalloc(&g.act[b], bytes));
             CU_OK(cudaMemset(g.act[b], 0, bytes));
             if (f.kind == MT_CONV3X3) {
-                mt_status st = encode_nhwc(&g.act_map[b], g.act[b], f.in_ch, f.w, f.h, cap, conv_rows_per_tile(f.w, f.h));
+                mt_status st = encode_nhwc(&g.act_map[b], g.act[b], f.in_ch, f.w, f.h, cap, g.conv.Wp, g.conv.R + 2);
                 if (st != MT_OK) return st;
             }
         }
@@ -265,7 +264,7 @@ mt_status validate_layers(const mt_layer_desc* layers, int n_layers) {
             } else if (d.kind == MT_GLOBAL_AVG_POOL) {
                 return MT_ERR_UNSUPPORTED;
             }
-            if (d.kind == MT_CONV3X3 && (d.in_ch != 64 || d.out_ch != 64 || d.w > BM)) return MT_ERR_UNSUPPORTED;
+            if (d.kind == MT_CONV3X3 && (d.in_ch != 64 || d.out_ch != 64 || d.w > 126)) return MT_ERR_UNSUPPORTED;
             if (d.kind == MT_GLOBAL_AVG_POOL && d.in_ch != d.out_ch) return MT_ERR_SHAPE;
         }
     }
@@ -322,12 +321,9 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
     if (st != MT_OK) return st;
     const int L = (int)g.family.size();
     const HostLayer& f0 = g.family[0];
-    int tiles_per_image = 0, rows_per_tile = 0;
+    int tiles_per_image = 0;
     for (const HostLayer& f : g.family)
-        if (f.kind == MT_CONV3X3) {
-            rows_per_tile = conv_rows_per_tile(f.w, f.h);
-            tiles_per_image = (f.h + rows_per_tile - 1) / rows_per_tile;
-        }
+        if (f.kind == MT_CONV3X3) tiles_per_image = g.conv.strips_per_image;
 
     {
         Timer t(K_HIST, s);
@@ -343,7 +339,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
         Timer t(K_GATHER, s);
         launch_gather_rows(inputs, g.d_perm, n, g.in_elems * 2, g.act[0], g.act_ld[0] * 2, g.sm_count, s);
     } else {
-        st = encode_nhwc(&in_map, inputs, f0.in_ch, f0.w, f0.h, n, rows_per_tile);
+        st = encode_nhwc(&in_map, inputs, f0.in_ch, f0.w, f0.h, n, g.conv.Wp, g.conv.R + 2);
         if (st != MT_OK) return st;
     }
     for (int l = 0; l < L; ++l) {
@@ -366,9 +362,12 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             a.tile_prefix = g.d_tile_prefix + (size_t)l * (g.T + 1);
             a.perm = (l == 0) ? g.d_perm : nullptr;
             a.out = (uint16_t*)g.act[l + 1];
-            a.H = f.h; a.W = f.w; a.rows_per_tile = rows_per_tile; a.tiles_per_image = tiles_per_image;
+            a.H = f.h; a.W = f.w;
+            a.Wp = g.conv.Wp; a.R = g.conv.R; a.tiles_per_strip = g.conv.tiles_per_strip;
+            a.stage_bytes = g.conv.stage_bytes; a.n_stages = g.conv.n_stages;
+            a.strips_per_image = g.conv.strips_per_image; a.box_bytes = g.conv.box_bytes;
             a.status = g.d_status;
-            launch_grouped_conv(l == 0 ? in_map : g.act_map[l], a, g.sm_count, s);
+            launch_grouped_conv(l == 0 ? in_map : g.act_map[l], a, g.conv.smem_bytes, g.sm_count, s);
         } else {
             Timer t(K_POOL, s);
             launch_global_avg_pool((const uint16_t*)g.act[l], n, f.h * f.w, f.in_ch, (uint16_t*)g.act[l + 1],
@@ -504,6 +503,8 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
         g.has_family = true;
         g.in_elems = layer_in_elems(hl[0]);
         g.out_elems = hl.back().out_ch;
+        for (const HostLayer& f : hl)
+            if (f.kind == MT_CONV3X3) plan_conv(f.h, f.w, &g.conv);   // cannot fail: validate_layers bounds w
         for (int b = 0; b <= MT_MAX_LAYERS; ++b) g.width[b] = 0;
         g.ws_dirty = true;
     }

@@ -39,7 +39,8 @@ void launch_unpermute(const float* src, const int32_t* perm, const int32_t* offs
 // columns, each tile 16 KiB in the 128-byte-swizzled shared-memory image the tensor-core kernels consume;
 // rows >= N are zero.  Tile (nt, kb) starts at element offset (nt * (K/64) + kb) * 8192.
 void launch_pretile_dense(const uint16_t* w, int N, int K, uint16_t* out, cudaStream_t s);
-// Conv weights W[64][3][3][64] -> 9 tap tiles of 64 rows (out channel) x 64 columns (in channel), 8 KiB each.
+// Conv weights W[64][3][3][64] -> 9 tap tiles of 64 rows (out channel) x 64 columns (in channel), 8 KiB each,
+// in the tile order the conv executor pairs them in.
 void launch_pretile_conv(const uint16_t* w, int C_out, int C_in, uint16_t* out, cudaStream_t s);
 
 struct GemmArgs {
@@ -57,21 +58,33 @@ cudaError_t configure_grouped_gemm();
 // tile_n: 128 or 256 output columns per work item; must match BucketArgs::tile_n of that layer.
 void launch_grouped_gemm(const CUtensorMap& tmap_a, const GemmArgs& a, int tile_n, int sm_count, cudaStream_t s);
 
+// Strip geometry of the conv executor (see grouped_conv.cu).
+struct ConvPlan {
+    int Wp;                // padded row length in shared memory: W + 2 rounded up to 32, 64 or 128 pixels
+    int R;                 // output rows per strip
+    int tiles_per_strip;   // 128-pixel accumulator tiles per strip
+    int stage_bytes;       // shared memory per strip stage (multiple of 1024)
+    int n_stages;
+    int strips_per_image;
+    int box_bytes;         // bytes one TMA box delivers: (R + 2) * Wp * 128
+    int smem_bytes;        // dynamic shared memory of the launch
+};
+bool plan_conv(int H, int W, ConvPlan* plan);
+
 struct ConvArgs {
     const ModelDev* models;
     int layer;
     int T;
     const int32_t* offsets;
-    const int32_t* tile_prefix;
+    const int32_t* tile_prefix;   // work units = strips
     const int32_t* perm;          // non-null: image index = perm[j] (first layer reads the caller's buffer)
     uint16_t* out;                // bf16 NHWC, bucketed order
     int H, W;
-    int rows_per_tile;            // image rows per tile: floor(128 / W)
-    int tiles_per_image;
+    int Wp, R, tiles_per_strip, stage_bytes, n_stages, strips_per_image, box_bytes;
     int32_t* status;
 };
 cudaError_t configure_grouped_conv();
-void launch_grouped_conv(const CUtensorMap& tmap_x, const ConvArgs& a, int sm_count, cudaStream_t s);
+void launch_grouped_conv(const CUtensorMap& tmap_x, const ConvArgs& a, int smem_bytes, int sm_count, cudaStream_t s);
 
 // g[j][c] = mean over the H*W positions of x[j][.][.][c]; bf16 in, fp32 sum, bf16 out (row stride ld_out).
 void launch_global_avg_pool(const uint16_t* x, int n, int HW, int C, uint16_t* out, int ld_out, int sm_count,

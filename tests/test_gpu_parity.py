@@ -76,7 +76,7 @@ def test_config5_reduced():
     run_and_check(wl.models, wl.model_ids, wl.inputs)
 
 
-@pytest.mark.parametrize("h,w", [(8, 8), (5, 7), (56, 56), (3, 128), (17, 20)])
+@pytest.mark.parametrize("h,w", [(8, 8), (5, 7), (56, 56), (3, 126), (17, 20)])
 def test_config4_reduced_geometries(h, w):
     wl = synth.make_workload(4, n=7, n_tenants=3, h=h, w=w, n_conv=2)
     run_and_check(wl.models, wl.model_ids, wl.inputs)
