@@ -121,6 +121,45 @@ bucket_scan(int n_blocks, int T, const ModelDev* __restrict__ models, int n_laye
     }
 }
 
+struct ItemPtrs { WorkItem* v[8]; };
+
+// Expand every dense layer's work list: item i of layer l -> (tenant, row tile, column tile) and everything the
+// executor needs to know about it.  Row tiles of one weight slab are adjacent items, so concurrent CTAs share it in L2.
+__global__ void build_work_items(int T, const ModelDev* __restrict__ models, int n_layers, LayerTileN tn,
+                                 const int32_t* __restrict__ offsets, const int32_t* __restrict__ tile_prefix,
+                                 ItemPtrs items) {
+    for (int l = 0; l < n_layers; ++l) {
+        WorkItem* out = items.v[l];
+        if (!out) continue;
+        const int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
+        const int total = prefix[T];
+        for (int item = blockIdx.x * blockDim.x + threadIdx.x; item < total; item += gridDim.x * blockDim.x) {
+            int lo = 0, hi = T;   // largest t with prefix[t] <= item
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (prefix[mid] <= item) lo = mid; else hi = mid;
+            }
+            const LayerDev& L = models[lo].layer[l];
+            const int seg0 = offsets[lo], n_t = offsets[lo + 1] - seg0;
+            const int m_tiles = (n_t + BM - 1) / BM;
+            const int local = item - prefix[lo];
+            const int n_tile = local / m_tiles, m_tile = local - n_tile * m_tiles;
+            WorkItem w;
+            w.row0 = seg0 + m_tile * BM;
+            w.rows_valid = min(BM, n_t - m_tile * BM);
+            w.n_tile = n_tile;
+            w.k_blocks = L.k_blocks;
+            w.w = L.w;
+            w.bias = L.bias;
+            w.N = L.N;
+            w.relu = L.relu;
+            w.t = lo;
+            w.pad = 0;
+            out[item] = w;
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kBucketChunk)
 bucket_scatter(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models,
                const int32_t* __restrict__ block_hist, const int32_t* __restrict__ offsets,
@@ -192,6 +231,10 @@ void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
                                            a.counts, a.offsets, a.tile_prefix, a.tmp);
     bucket_scatter<<<n_blocks, kBucketChunk, smem, s>>>(a.ids, a.n, a.T, a.models, a.block_hist, a.offsets, a.perm,
                                                         a.inv);
+    ItemPtrs ip;
+    bool any = false;
+    for (int l = 0; l < 8; ++l) { ip.v[l] = a.items[l]; any = any || a.items[l]; }
+    if (any) build_work_items<<<a.item_grid, 256, 0, s>>>(a.T, a.models, a.n_layers, tn, a.offsets, a.tile_prefix, ip);
 }
 
 void launch_gather_rows(const void* src, const int32_t* perm, int n, int row_bytes, void* dst, int dst_ld_bytes,

@@ -38,7 +38,8 @@ constexpr int kTapBytes = kCN * BK * 2;          // 8 KiB: 64 out channels x 64 
 constexpr int kWeightBytes = 9 * kTapBytes;      // 72 KiB, resident per tenant
 constexpr int kMaxStages = 4;
 constexpr int kSlots = 8;                        // TMEM ring: 8 accumulators of 64 columns = all 512 columns
-constexpr int kConvBarBytes = 512;
+constexpr int kConvBarBytes = 1024;
+constexpr int kRecords = 16;                     // ring of per-strip records (producer -> MMA issuer, epilogue)
 
 // Order of the tap tiles in the executor layout: the three ky = 1 taps, then for every kx the pair
 // W(2,kx), W(0,kx) back to back, so that one 128-row B operand covers the pair.
@@ -67,6 +68,11 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * (2 * kMaxStages + 2 * kSlots + 2));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     float* s_bias = reinterpret_cast<float*>(bar_ptr + 256);          // 64 floats
+    // Per-strip record written by the producer before it arms the strip's TMA load (so the mbarrier hand-over
+    // publishes it): x = flags (1 new tenant, 2 pair with the tile above, 4 the next strip finishes the last
+    // tile), y = image (bucketed index), z = first output row, w = tenant.  The issuing thread must not spend
+    // time on index arithmetic: the tensor pipe drains as soon as it stops issuing.
+    int4* s_rec = reinterpret_cast<int4*>(bar_ptr + 512);             // kRecords x 16 bytes
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -126,17 +132,24 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
             int w_loads = 0, w_tenant = -1;
             for (int s = s_begin; s < s_end; ++s) {
                 const StripCoord c = locate(s);
-                if (c.t != w_tenant) {     // this tenant's nine tap tiles, once the MMAs on the old ones are done
+                const bool new_tenant = (c.t != w_tenant);
+                if (!mbar_wait(sempty_bar(stage), phase ^ 1u, abort_flag, p.status, 22)) break;
+                const int img = p.perm ? p.perm[c.j] : c.j;
+                const bool pair_top = pairing && s > s_begin && c.strip_in_image > 0;
+                const bool defer_bottom = pairing && s + 1 < s_end && c.strip_in_image + 1 < p.strips_per_image;
+                s_rec[(s - s_begin) & (kRecords - 1)] =
+                    make_int4((new_tenant ? 1 : 0) | (pair_top ? 2 : 0) | (defer_bottom ? 4 : 0), c.j, c.y0, c.t);
+                mbar_expect_tx(sfull_bar(stage), p.box_bytes);
+                tma_load_4d(strip0 + stage * p.stage_bytes, &tmap_x, 0, -1, c.y0 - 1, img, sfull_bar(stage));
+                if (new_tenant) {
+                    // This tenant's nine tap tiles.  The issuer learns of the change from the strip's record, i.e.
+                    // after the strip has landed, and only then releases the old weights: so the strip goes first.
                     if (w_loads > 0 && !mbar_wait(wempty_bar, (uint32_t)((w_loads - 1) & 1), abort_flag, p.status, 21)) break;
                     mbar_expect_tx(wfull_bar, kWeightBytes);
                     bulk_load(w_smem, p.models[c.t].layer[p.layer].w, kWeightBytes, wfull_bar);
                     w_tenant = c.t;
                     ++w_loads;
                 }
-                if (!mbar_wait(sempty_bar(stage), phase ^ 1u, abort_flag, p.status, 22)) break;
-                const int img = p.perm ? p.perm[c.j] : c.j;
-                mbar_expect_tx(sfull_bar(stage), p.box_bytes);
-                tma_load_4d(strip0 + stage * p.stage_bytes, &tmap_x, 0, -1, c.y0 - 1, img, sfull_bar(stage));
                 if (++stage == p.n_stages) { stage = 0; phase ^= 1u; }
             }
         }
@@ -146,7 +159,7 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
             constexpr uint32_t idesc128 = make_idesc_bf16(BM, 2 * kCN);
             int stage = 0; uint32_t phase = 0;
             int g = 0;                      // tiles started so far by this CTA; tile g lives in TMEM slot g % kSlots
-            int w_loads = 0, w_tenant = -1;
+            int w_loads = 0;
             bool ok = true;
             // four K steps of one 128-pixel block against one (N = 64) or two stacked (N = 128) tap tiles
             auto issue = [&](uint32_t a_addr, uint32_t b_addr, uint32_t d_tmem, uint32_t idesc, bool overwrite) {
@@ -156,30 +169,56 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
                 for (int k = 0; k < BK / UMMA_K; ++k)
                     umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (overwrite && k == 0) ? 0u : 1u);
             };
+            // This thread is the only feeder of the tensor pipe, and its MMAs, commits and barrier polls go through one
+            // in-order queue: an instruction whose result the thread needs (a barrier poll, a shared-memory load)
+            // returns only after every MMA before it has been dispatched, and while the thread waits for it nothing
+            // new is queued - the pipe runs dry.  So (1) the strip bookkeeping (new tenant? pair with the tile above?
+            // leave the last tile to the next strip?) is kept in registers instead of being read from the producer's
+            // record, and (2) the barriers of the NEXT tile and strip are polled (non-blocking) a few MMAs into the
+            // current tile, and the answers are looked at only after the rest of the tile has been queued.
+            int t_hi = -1;                  // strips [.., t_hi) belong to the current tenant
+            int in_image = 0;               // index of the current strip inside its image
+            uint32_t strip_ready = 0, slot_ready = 0;
             for (int s = s_begin; ok && s < s_end; ++s) {
-                const StripCoord c = locate(s);
-                if (c.t != w_tenant) {
+                const bool new_tenant = (s >= t_hi);
+                if (new_tenant) {           // rare: a tenant border (or the first strip)
+                    const StripCoord c = locate(s);
+                    t_hi = cur_hi;
+                    in_image = c.strip_in_image;
+                }
+                if (!strip_ready) {
+                    if (!mbar_wait(sfull_bar(stage), phase, abort_flag, p.status, 25)) break;
+                }
+                tc_fence_after();
+                if (new_tenant) {
                     if (w_loads > 0) umma_commit(wempty_bar);      // fires when all MMAs on the old weights are done
                     if (!mbar_wait(wfull_bar, (uint32_t)(w_loads & 1), abort_flag, p.status, 23)) break;
-                    w_tenant = c.t;
                     ++w_loads;
                 }
-                const bool pair_top = pairing && s > s_begin && c.strip_in_image > 0;
-                const bool defer_bottom = pairing && s + 1 < s_end && c.strip_in_image + 1 < p.strips_per_image;
-                if (!mbar_wait(sfull_bar(stage), phase, abort_flag, p.status, 25)) break;
-                tc_fence_after();
+                const bool pair_top = pairing && s > s_begin && in_image > 0;
+                const bool defer_bottom = pairing && s + 1 < s_end && in_image + 1 < p.strips_per_image;
                 const uint32_t strip = strip0 + stage * p.stage_bytes;
+                const int next_stage = (stage + 1 == p.n_stages) ? 0 : stage + 1;
+                const uint32_t next_phase = (stage + 1 == p.n_stages) ? (phase ^ 1u) : phase;
+                strip_ready = 0;
                 for (int i = 0; i < TS; ++i, ++g) {
                     const int slot = g % kSlots;
-                    // the accumulator slot must have been drained by the epilogue of tile g - kSlots
-                    if (!mbar_wait(tempty_bar(slot), (uint32_t)(((g / kSlots) & 1) ^ 1), abort_flag, p.status, 24)) { ok = false; break; }
+                    if (!slot_ready) {   // the accumulator slot must have been drained by the epilogue of tile g - kSlots
+                        if (!mbar_wait(tempty_bar(slot), (uint32_t)(((g / kSlots) & 1) ^ 1), abort_flag, p.status, 24)) { ok = false; break; }
+                    }
                     tc_fence_after();
                     const uint32_t d_this = tmem_base + slot * kCN;
                     const uint32_t blk = strip + (uint32_t)(i * BM) * 128u;          // padded pixel i*128 of the strip
+                    const bool last_tile = (i == TS - 1);
+                    uint32_t poll_slot = 0, poll_strip = 0;
                     if (pairing) {
                         // ky = 1 first: these overwrite the fresh accumulator
-                        for (int kx = 0; kx < 3; ++kx)
-                            issue(blk + (uint32_t)(Wp + kx) * 128u, w_smem + tap_slot(1, kx) * kTapBytes, d_this, idesc64, kx == 0);
+                        issue(blk + (uint32_t)(Wp + 0) * 128u, w_smem + tap_slot(1, 0) * kTapBytes, d_this, idesc64, true);
+                        // look ahead: results are consumed after the rest of this tile has been queued
+                        poll_slot = mbar_test_wait(tempty_bar((g + 1) % kSlots), (uint32_t)((((g + 1) / kSlots) & 1) ^ 1));
+                        if (last_tile) poll_strip = mbar_test_wait(sfull_bar(next_stage), next_phase);
+                        issue(blk + (uint32_t)(Wp + 1) * 128u, w_smem + tap_slot(1, 1) * kTapBytes, d_this, idesc64, false);
+                        issue(blk + (uint32_t)(Wp + 2) * 128u, w_smem + tap_slot(1, 2) * kTapBytes, d_this, idesc64, false);
                         // block at the tile's first row: ky = 0 of this tile and ky = 2 of the tile above
                         const bool have_above = (i > 0) || pair_top;
                         const bool adjacent = slot != 0;                              // slots g-1 and g contiguous in TMEM
@@ -198,9 +237,15 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
                         for (int tap = 0; tap < 9; ++tap) {
                             const int ky = tap / 3, kx = tap - 3 * ky;
                             issue(blk + (uint32_t)(ky * Wp + kx) * 128u, w_smem + tap_slot(ky, kx) * kTapBytes, d_this, idesc64, tap == 0);
+                            if (tap == 1) {
+                                poll_slot = mbar_test_wait(tempty_bar((g + 1) % kSlots), (uint32_t)((((g + 1) / kSlots) & 1) ^ 1));
+                                if (last_tile) poll_strip = mbar_test_wait(sfull_bar(next_stage), next_phase);
+                            }
                         }
                         umma_commit(tfull_bar(slot));
                     }
+                    slot_ready = poll_slot;
+                    if (last_tile) strip_ready = (s + 1 < s_end) ? poll_strip : 0;
                 }
                 if (!ok) break;
                 if (pairing && !defer_bottom) {
@@ -211,8 +256,10 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
                         issue(blk + (uint32_t)kx * 128u, w_smem + tap_slot(2, kx) * kTapBytes, tmem_base + last * kCN, idesc64, false);
                     umma_commit(tfull_bar(last));
                 }
-                umma_commit(sempty_bar(stage));     // the strip buffer is free once these MMAs have read it
-                if (++stage == p.n_stages) { stage = 0; phase ^= 1u; }
+                // The strip buffer is released by the epilogue (see there), not by a third commit here: a commit issued
+                // while the previous one is still waiting for its MMAs stalls this thread until the queue has drained.
+                stage = next_stage; phase = next_phase;
+                if (++in_image == p.strips_per_image) in_image = 0;
             }
         }
     } else {               // ---------------------------------------------------- epilogue (warps 2..9)
@@ -222,30 +269,37 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
         const int r = q4 * 32 + lane;               // tile-local padded pixel of this thread
         const int yl = r / Wp, x = r - yl * Wp;
         const int rows_per_tile = BM / Wp;
-        int g = 0, b_tenant = -1, relu = 0;
+        int g = 0, relu = 0;
         bool ok = true;
+        int img_j = 0, y0 = 0;
         for (int s = s_begin; ok && s < s_end; ++s) {
-            const StripCoord c = locate(s);
-            if (c.t != b_tenant) {                  // new tenant: its bias into shared memory, ReLU flag into a register
-                const LayerDev& L = p.models[c.t].layer[p.layer];
-                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");      // everyone done with the old bias
-                if (threadIdx.x - 64 < kCN) s_bias[threadIdx.x - 64] = L.bias[threadIdx.x - 64];
-                relu = L.relu;
-                b_tenant = c.t;
-                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
-            }
             for (int i = 0; i < TS; ++i, ++g) {
                 const int slot = g % kSlots;
                 if (!mbar_wait(tfull_bar(slot), (uint32_t)((g / kSlots) & 1), abort_flag, p.status, 26)) { ok = false; break; }
+                // The completion of a strip's last tile is signalled after every MMA that reads the strip's buffer (by
+                // the strip's own last instruction, or by the next strip when the tile was left to it): release it.
+                if (i == TS - 1 && threadIdx.x == 64) mbar_arrive(sempty_bar((s - s_begin) % p.n_stages));
+                if (i == 0) {
+                    // the strip's record was published (with the strip's data) before any of its MMAs were issued
+                    const int4 rec = s_rec[(s - s_begin) & (kRecords - 1)];
+                    img_j = rec.y; y0 = rec.z;
+                    if (rec.x & 1) {                // new tenant: its bias into shared memory, ReLU flag into a register
+                        const LayerDev& L = p.models[rec.w].layer[p.layer];
+                        asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // everyone done with the old bias
+                        if (threadIdx.x - 64 < kCN) s_bias[threadIdx.x - 64] = L.bias[threadIdx.x - 64];
+                        relu = L.relu;
+                        asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+                    }
+                }
                 tc_fence_after();
                 uint32_t v[32];
                 tmem_ld32(tmem_base + (static_cast<uint32_t>(q4 * 32) << 16) + slot * kCN + half * 32, v);
                 tmem_ld_wait();
                 tc_fence_before();
                 mbar_arrive(tempty_bar(slot));      // values are in registers: the slot can be reused
-                const int y = c.y0 + i * rows_per_tile + yl;
+                const int y = y0 + i * rows_per_tile + yl;
                 if (x < p.W && y < p.H) {
-                    uint16_t* dst = p.out + (((size_t)c.j * p.H + y) * p.W + x) * kCN + half * 32;
+                    uint16_t* dst = p.out + (((size_t)img_j * p.H + y) * p.W + x) * kCN + half * 32;
                     const float4* b4 = reinterpret_cast<const float4*>(s_bias + half * 32);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {

@@ -29,27 +29,12 @@ struct GemmCfg {
     static constexpr int kSmem = kStages * kStageBytes + kBarBytes + 1024;    // + slack for 1024-byte alignment
 };
 
-struct TileCoord {
-    int t, m_tile, n_tile, row0, rows_valid;
-};
-
-__device__ __forceinline__ TileCoord decode_tile(int item, int T, const int32_t* __restrict__ prefix,
-                                                 const int32_t* __restrict__ offsets) {
-    int lo = 0, hi = T;   // largest t with prefix[t] <= item
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (prefix[mid] <= item) lo = mid; else hi = mid;
-    }
-    TileCoord c;
-    c.t = lo;
-    const int seg0 = offsets[lo], n_t = offsets[lo + 1] - seg0;
-    const int m_tiles = (n_t + BM - 1) / BM;
-    const int local = item - prefix[lo];
-    c.n_tile = local / m_tiles;      // row tiles of one weight slab are adjacent items: the slab stays in L2
-    c.m_tile = local - c.n_tile * m_tiles;
-    c.row0 = seg0 + c.m_tile * BM;
-    c.rows_valid = min(BM, n_t - c.m_tile * BM);
-    return c;
+// 48-byte work item as three 16-byte loads through the read-only path.
+__device__ __forceinline__ WorkItem load_item(const WorkItem* items, int idx) {
+    const int4* q = reinterpret_cast<const int4*>(items + idx);
+    union { int4 v[3]; WorkItem w; } u;
+    u.v[0] = __ldg(q); u.v[1] = __ldg(q + 1); u.v[2] = __ldg(q + 2);
+    return u.w;
 }
 
 template <int TN>
@@ -91,76 +76,92 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmArgs p
     const uint32_t tmem_base = *tmem_slot;
 
     const int total = p.tile_prefix[p.T];
-    const ModelDev* models = p.models;
 
     if (warp == 0) {
         if (lane == 0) {   // ------------------------------------------------ TMA producer
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
+            WorkItem cur = {};
+            if ((int)blockIdx.x < total) cur = load_item(p.items, blockIdx.x);
             for (int item = blockIdx.x; ok && item < total; item += gridDim.x) {
-                const TileCoord c = decode_tile(item, p.T, p.tile_prefix, p.offsets);
-                const LayerDev& L = models[c.t].layer[p.layer];
-                const int kblocks = L.k_blocks;
+                WorkItem nxt = {};
+                if (item + (int)gridDim.x < total) nxt = load_item(p.items, item + gridDim.x);   // in flight during this item
+                const int kblocks = cur.k_blocks;
                 // weight tile (nt, kb) of 128 rows x 64 columns starts at element (nt * kblocks + kb) * 8192
-                const uint16_t* wsrc = L.w + (size_t)c.n_tile * kWTiles * kblocks * (BN * BK);
+                const uint16_t* wsrc = cur.w + (size_t)cur.n_tile * kWTiles * kblocks * (BN * BK);
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
                     const uint32_t a_dst = base + stage * kStageBytes;
                     mbar_expect_tx(full_bar(stage), kStageBytes);
-                    tma_load_2d(a_dst, &tmap_a, kb * BK, c.row0, full_bar(stage));
+                    tma_load_2d(a_dst, &tmap_a, kb * BK, cur.row0, full_bar(stage));
 #pragma unroll
                     for (int wt = 0; wt < kWTiles; ++wt)
                         bulk_load(a_dst + (1 + wt) * TILE_BYTES, wsrc + ((size_t)wt * kblocks + kb) * (BN * BK),
                                   TILE_BYTES, full_bar(stage));
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
+                cur = nxt;
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {   // ------------------------------------------------ MMA issuer
+            // This thread alone feeds the tensor pipe, and it issues in order: every instruction it spends on
+            // anything else is time the pipe may run dry.  So descriptors are one 32-bit add away from a
+            // precomputed base, the next stage's barrier is polled (non-blocking) BEFORE the current stage's MMAs
+            // are issued and looked at after them, and the next item's K extent is loaded one item ahead.
             constexpr uint32_t idesc = make_idesc_bf16(BM, TN);
+            constexpr uint32_t kStageLo = kStageBytes >> 4;
+            const uint32_t a_lo0 = desc_lo(base), b_lo0 = desc_lo(base + TILE_BYTES);
             int stage = 0; uint32_t phase = 0;
             int it = 0;
             bool ok = true;
+            int kblocks = ((int)blockIdx.x < total) ? __ldg(&p.items[blockIdx.x].k_blocks) : 0;
+            uint32_t ready = 0;
             for (int item = blockIdx.x; ok && item < total; item += gridDim.x, ++it) {
-                const TileCoord c = decode_tile(item, p.T, p.tile_prefix, p.offsets);
-                const int kblocks = models[c.t].layer[p.layer].k_blocks;
+                const int next_kblocks = (item + (int)gridDim.x < total) ? __ldg(&p.items[item + gridDim.x].k_blocks) : 0;
                 const int acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
                 if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, 2)) break;
-                tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kAccCols;
                 for (int kb = 0; kb < kblocks; ++kb) {
-                    if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { ok = false; break; }
+                    if (!ready && !mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_src = base + stage * kStageBytes;
-                    const uint64_t a_desc = make_kmajor_sw128_desc(a_src, 1024);
-                    const uint64_t b_desc = make_kmajor_sw128_desc(a_src + TILE_BYTES, 1024);
-#pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        // advancing K by 16 elements = 32 bytes inside the swizzle row: +2 in the address field
-                        umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
-                    }
+                    const int next_stage = (stage + 1 == kStages) ? 0 : stage + 1;
+                    const uint32_t next_phase = (stage + 1 == kStages) ? (phase ^ 1u) : phase;
+                    const uint32_t poll = mbar_test_wait(full_bar(next_stage), next_phase);   // consumed after the MMAs
+                    const uint32_t a_lo = a_lo0 + stage * kStageLo, b_lo = b_lo0 + stage * kStageLo;
+                    // advancing K by 16 elements = 32 bytes inside the swizzle row: +2 in the address field
+                    if (kb == 0) umma_bf16_lohi<false>(d_tmem, a_lo, b_lo, idesc);
+                    else umma_bf16_lohi<true>(d_tmem, a_lo, b_lo, idesc);
+                    umma_bf16_lohi<true>(d_tmem, a_lo + 2, b_lo + 2, idesc);
+                    umma_bf16_lohi<true>(d_tmem, a_lo + 4, b_lo + 4, idesc);
+                    umma_bf16_lohi<true>(d_tmem, a_lo + 6, b_lo + 6, idesc);
                     umma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    stage = next_stage; phase = next_phase;
+                    ready = poll;
                 }
                 if (ok) umma_commit(tfull_bar(acc));
+                kblocks = next_kblocks;
             }
         }
     } else {               // ---------------------------------------------------- epilogue (warps 2..5)
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
         const int r = q * 32 + lane;            // accumulator row of this thread
         int it = 0;
+        WorkItem cur = {};
+        if ((int)blockIdx.x < total) cur = load_item(p.items, blockIdx.x);
         for (int item = blockIdx.x; item < total; item += gridDim.x, ++it) {
-            const TileCoord c = decode_tile(item, p.T, p.tile_prefix, p.offsets);
-            const LayerDev& L = models[c.t].layer[p.layer];
+            WorkItem nxt = {};
+            if (item + (int)gridDim.x < total) nxt = load_item(p.items, item + gridDim.x);
+            const WorkItem c = cur;
+            cur = nxt;
             const int acc = it & 1;
             const uint32_t acc_phase = (it >> 1) & 1;
             if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 4)) break;
             tc_fence_after();
             const bool row_ok = r < c.rows_valid;
             const size_t grow = (size_t)(c.row0 + r);
-            const int N = L.N, relu = L.relu;
+            const int N = c.N, relu = c.relu;
 #pragma unroll 1
             for (int ch = 0; ch < TN / 32; ++ch) {
                 uint32_t v[32];
@@ -169,7 +170,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmArgs p
                 tmem_ld_wait();
                 const int n0 = c.n_tile * TN + ch * 32;
                 if (n0 >= N) break;
-                const float4* b4 = reinterpret_cast<const float4*>(L.bias + n0);
+                const float4* b4 = reinterpret_cast<const float4*>(c.bias + n0);
                 float f[32];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {

@@ -67,6 +67,8 @@ struct Ctx {
     int act_ld[MT_MAX_LAYERS + 1] = {0};
     CUtensorMap act_map[MT_MAX_LAYERS + 1];
     float* d_out_b = nullptr;
+    WorkItem* d_items[MT_MAX_LAYERS] = {nullptr};   // per dense layer
+    size_t items_cap[MT_MAX_LAYERS] = {0};
     int last_n = 0;
 
     // staging for mt_infer_host
@@ -146,6 +148,7 @@ void free_workspace() {
     cudaFree(g.d_inv); g.d_inv = nullptr;
     cudaFree(g.d_out_b); g.d_out_b = nullptr;
     for (int b = 0; b <= MT_MAX_LAYERS; ++b) { cudaFree(g.act[b]); g.act[b] = nullptr; }
+    for (int l = 0; l < MT_MAX_LAYERS; ++l) { cudaFree(g.d_items[l]); g.d_items[l] = nullptr; g.items_cap[l] = 0; }
     g.cap_n = 0;
 }
 
@@ -203,6 +206,14 @@ mt_status ensure_workspace(int n) {
                 if (st != MT_OK) return st;
             }
         }
+    }
+    // work items of the dense layers: at most (row tiles + one ragged tile per tenant) x column tiles of the widest model
+    for (int l = 0; l < L; ++l) {
+        if (g.family[l].kind != MT_DENSE) continue;
+        const int out_w = (l + 1 < L) ? g.width[l + 1] : g.out_elems;
+        const size_t col_tiles = (size_t)(out_w + BN - 1) / BN;    // bound for either tile width
+        g.items_cap[l] = ((size_t)cap / BM + (size_t)g.max_models + 1) * col_tiles;
+        CU_OK(cudaMalloc(&g.d_items[l], sizeof(WorkItem) * g.items_cap[l]));
     }
     g.cap_n = cap;
     g.ws_dirty = false;
@@ -329,7 +340,8 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
         Timer t(K_HIST, s);
         BucketArgs a;
         a.ids = ids; a.n = n; a.T = g.T; a.models = g.d_models; a.n_layers = L; a.rows_per_unit = tiles_per_image;
-        for (int l = 0; l < 8; ++l) a.tile_n[l] = g.tile_n[l];
+        for (int l = 0; l < 8; ++l) { a.tile_n[l] = g.tile_n[l]; a.items[l] = (l < MT_MAX_LAYERS) ? g.d_items[l] : nullptr; }
+        a.item_grid = g.sm_count * 2;
         a.block_hist = g.d_block_hist; a.counts = g.d_counts; a.offsets = g.d_offsets; a.tile_prefix = g.d_tile_prefix;
         a.tmp = g.d_tmp; a.perm = g.d_perm; a.inv = g.d_inv; a.status = g.d_status;
         launch_bucketing(a, s);
@@ -350,6 +362,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             GemmArgs a;
             a.models = g.d_models; a.layer = l; a.T = g.T; a.offsets = g.d_offsets;
             a.tile_prefix = g.d_tile_prefix + (size_t)l * (g.T + 1);
+            a.items = g.d_items[l];
             a.out = last ? (void*)g.d_out_b : g.act[l + 1];
             a.ld_out = last ? g.out_elems : g.act_ld[l + 1];
             a.out_fp32 = last ? 1 : 0;

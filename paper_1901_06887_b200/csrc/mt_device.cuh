@@ -30,6 +30,22 @@ struct ModelDev {
     LayerDev layer[MT_MAX_LAYERS];
 };
 
+// One unit of work of the grouped dense executor: a (tenant, row tile, column tile) triple, expanded on the device
+// right after bucketing so that the executor's roles read one 48-byte record per item instead of searching the
+// per-tenant prefix sums and chasing pointers through the tenant table on their critical paths.
+struct __align__(16) WorkItem {
+    int32_t row0;        // first bucketed row of the tile
+    int32_t rows_valid;  // rows of the tile that belong to the tenant (1..128)
+    int32_t n_tile;      // column tile index (units of the launch's tile width)
+    int32_t k_blocks;    // K / 64
+    const uint16_t* w;   // tenant's weights in executor layout
+    const float* bias;   // tenant's padded bias
+    int32_t N;           // tenant's out features
+    int32_t relu;
+    int32_t t;           // tenant (model id)
+    int32_t pad;
+};
+
 // Sticky status word written by kernels: [0] status code, [1] first bad arrival index, [2] where a wait gave up.
 enum { ST_CODE = 0, ST_BAD_INDEX = 1, ST_WHERE = 2, ST_WORDS = 4 };
 
@@ -85,6 +101,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "r"(bar), "r"(parity)
         : "memory");
     return ok != 0;
+}
+
+// Non-blocking poll of a phase; the result may be consumed long after the instruction was issued, which lets a
+// single-thread MMA issuer look ahead at the barriers it will need without stalling between MMAs.
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
 }
 
 // Every wait in the executors is bounded: after kWaitLimitNs without progress the waiter raises the
@@ -206,6 +238,27 @@ __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr, u
     d |= static_cast<uint64_t>(1) << 46;                             // descriptor version for sm_100
     d |= static_cast<uint64_t>(2) << 61;                             // layout type: 128-byte swizzle
     return d;
+}
+
+// The same descriptor split in halves: the upper word is constant for a kernel, the lower word is
+// (address >> 4) | 1 << 16, so stepping through operands costs one 32-bit add in the issuing thread.
+constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t smem_addr) { return ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16); }
+
+// D[tmem] (+)= A * B with the descriptors given as (lo, hi) words.  ACC = false overwrites D.
+template <bool ACC>
+__device__ __forceinline__ void umma_bf16_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        ".reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t"
+        "}\n"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(kDescHiSw128), "r"(idesc), "n"(ACC ? 1 : 0)
+        : "memory");
 }
 
 // Instruction descriptor of tcgen05.mma kind::f16: bf16 x bf16 -> fp32, both operands K-major.

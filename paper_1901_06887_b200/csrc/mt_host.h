@@ -8,6 +8,7 @@
 namespace mt {
 
 struct ModelDev;
+struct WorkItem;
 
 constexpr int kBucketChunk = 256;   // requests per CTA in the bucketing passes
 
@@ -26,6 +27,8 @@ struct BucketArgs {
     int32_t* tmp;             // [T + 1]
     int32_t* perm;            // [n]
     int32_t* inv;             // [n]
+    int item_grid;            // CTAs of the work-item expansion kernel
+    WorkItem* items[8];       // per dense layer: expanded work items (null for other layers)
     int32_t* status;
 };
 
@@ -49,6 +52,7 @@ struct GemmArgs {
     int T;
     const int32_t* offsets;       // [T + 2]
     const int32_t* tile_prefix;   // [T + 1] of this layer
+    const WorkItem* items;        // [tile_prefix[T]] work items of this layer
     void* out;                    // bf16 or fp32, rows in bucketed order
     int ld_out;                   // elements between output rows
     int out_fp32;
