@@ -253,7 +253,7 @@ def main():
     # ---- timed region: device-resident inputs, CUDA events on the launching stream, per-kernel events inside
     sampler = ClockSampler(local_rank)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    mt.mt_set_kernel_timing(True)
+    mt.mt_set_kernel_timing(2)          # events around the grouped layer executors only (the dominant kernel)
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
@@ -267,15 +267,23 @@ def main():
     if world > 1:
         dist.barrier()
     clocks = sampler.stop()
-    mt.mt_set_kernel_timing(False)
+    mt.mt_set_kernel_timing(0)
     local_ms = e0.elapsed_time(e1)
     kernel_times = mt.mt_get_kernel_times()
+    # per-kernel breakdown of every launch of the path: a short separate pass (its events perturb small batches)
+    mt.mt_set_kernel_timing(1)
+    bd_steps = max(3, min(args.steps, 50))
+    for i in range(bd_steps):
+        step(i)
+    torch.cuda.synchronize()
+    mt.mt_set_kernel_timing(0)
+    breakdown = mt.mt_get_kernel_times()
     units, ms = aggregate(n * args.steps, local_ms, world)
 
     if args.profile:
         if rank == 0:
             print(json.dumps({"profile_run": True, "ms_per_step": ms / args.steps,
-                              "kernels": {nm: t / max(c, 1) for nm, t, c in kernel_times}}), flush=True)
+                              "kernels": {nm: t / max(c, 1) for nm, t, c in breakdown}}), flush=True)
         mt.mt_shutdown()
         if world > 1:
             dist.destroy_process_group()
@@ -307,12 +315,13 @@ def main():
 
     if rank == 0:
         peaks, peaks_kind = load_peaks()
-        per_kernel = {name: {"ms_per_step": t / args.steps, "launches_per_step": c / args.steps} for name, t, c in kernel_times}
-        launches = int(sum(c for _, _, c in kernel_times))
-        # the bucketing entry covers three kernels (histogram, scan, scatter) under one pair of events
-        launches += 2 * int(sum(c for nm, _, c in kernel_times if nm.startswith("bucket")))
+        per_kernel = {name: {"ms_per_step": t / bd_steps, "launches_per_step": c / bd_steps} for name, t, c in breakdown}
+        # launches per step: the bucketing entry covers 2 (one-CTA batch) to 5 kernels under one pair of events
+        bucket_kernels = 2 if n <= 256 else 5
+        per_step = sum(c / bd_steps for nm, _, c in breakdown if not nm.startswith("bucket")) + bucket_kernels
+        launches = int(round(per_step * args.steps))
         dom = "grouped_conv3x3" if cfg == 4 else "grouped_gemm"
-        dom_ms = per_kernel.get(dom, {"ms_per_step": 0.0})["ms_per_step"]
+        dom_ms = dict((nm, t / args.steps) for nm, t, c in kernel_times).get(dom, 0.0)
         roof = gemm_roofline(wl, dom_ms, peaks, peaks_kind, cfg)
         flops = synth.workload_flops(wl.models, wl.model_ids)
         bytes_all = synth.workload_bytes(wl.models, wl.model_ids)

@@ -117,8 +117,9 @@ const char* mt_status_string(mt_status s);
 mt_status mt_debug_last_bucketing(int32_t* counts_host, int32_t* offsets_host, int32_t* perm_host,
                                   int32_t* inv_host, int32_t* n_tenants_out);
 
-/* Per-kernel device timing.  While enabled, every kernel launch of mt_infer is bracketed by CUDA events
- * on the caller's stream.  mt_get_kernel_times synchronises those events, then fills up to `cap`
+/* Per-kernel device timing.  enable = 1: every kernel launch of mt_infer is bracketed by CUDA events on the
+ * caller's stream; enable = 2: only the grouped layer executors (dense / conv) are; 0: off.
+ * mt_get_kernel_times synchronises those events, then fills up to `cap`
  * entries: names[i] (static strings), total_ms[i], launches[i]; *n_out = number of kernels seen.
  * Reading resets the accumulators. */
 mt_status mt_set_kernel_timing(int32_t enable);

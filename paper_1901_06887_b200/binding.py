@@ -152,8 +152,9 @@ def mt_debug_last_bucketing(n: int):
     return tuple(arrs)
 
 
-def mt_set_kernel_timing(enable: bool) -> None:
-    _check(lib().mt_set_kernel_timing(1 if enable else 0), "mt_set_kernel_timing")
+def mt_set_kernel_timing(enable) -> None:
+    """0/False off, 1/True every kernel, 2 only the grouped layer executors."""
+    _check(lib().mt_set_kernel_timing(int(enable)), "mt_set_kernel_timing")
 
 
 def mt_get_kernel_times() -> List[Tuple[str, float, int]]:

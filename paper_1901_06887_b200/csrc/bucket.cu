@@ -49,75 +49,160 @@ bucket_block_hist(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
     for (int t = threadIdx.x; t < T1; t += blockDim.x) block_hist[(size_t)blockIdx.x * T1 + t] = s_hist[t];
 }
 
-// Exclusive scan of `n_items` ints held in global memory by one CTA of kScanThreads threads.
-// out[0..n_items] (n_items + 1 entries; the last is the total).  in and out may alias only if equal offsets
-// are not needed afterwards.  s_tmp: kScanThreads ints of shared memory.
-__device__ void cta_exclusive_scan(const int32_t* in, int32_t* out, int n_items, int32_t* s_tmp) {
-    const int tid = threadIdx.x;
-    const int per = (n_items + kScanThreads - 1) / kScanThreads;
-    const int lo = min(tid * per, n_items), hi = min(lo + per, n_items);
-    int sum = 0;
-    for (int j = lo; j < hi; ++j) sum += in[j];
-    s_tmp[tid] = sum;
-    __syncthreads();
-    // Hillis-Steele inclusive scan over the per-thread sums
-    for (int d = 1; d < kScanThreads; d <<= 1) {
-        const int v = (tid >= d) ? s_tmp[tid - d] : 0;
-        __syncthreads();
-        s_tmp[tid] += v;
-        __syncthreads();
+// Exclusive scan across the threads of a CTA (any multiple of 32 threads up to 1024): returns the sum of `v` over
+// all lower-numbered threads; *total = sum over the CTA.  s_warp: 33 ints of shared memory.  Two barriers.
+__device__ __forceinline__ int cta_excl_scan(int v, int32_t* s_warp, int* total) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += u;
     }
-    int run = s_tmp[tid] - sum;
-    for (int j = lo; j < hi; ++j) {
-        const int v = in[j];
-        out[j] = run;
-        run += v;
-    }
-    if (tid == kScanThreads - 1) out[n_items] = s_tmp[tid];
+    if (lane == 31) s_warp[warp] = incl;
     __syncthreads();
+    if (warp == 0) {
+        const int w = (lane < n_warps) ? s_warp[lane] : 0;
+        int wi = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int u = __shfl_up_sync(0xffffffffu, wi, d);
+            if (lane >= d) wi += u;
+        }
+        s_warp[lane] = wi - w;                 // exclusive prefix of the warp totals
+        if (lane == 31) s_warp[32] = wi;       // grand total
+    }
+    __syncthreads();
+    const int r = incl - v + s_warp[warp];
+    *total = s_warp[32];
+    __syncthreads();                           // s_warp may be reused right away
+    return r;
 }
 
+// Work units (tiles / strips) tenant t contributes to layer l, given its request count c.
+__device__ __forceinline__ int layer_units(const ModelDev* models, int t, int l, int c, int rows_per_unit, int tile_n) {
+    if (c <= 0) return 0;
+    const LayerDev& L = models[t].layer[l];
+    if (L.kind == MT_DENSE) return ((c + BM - 1) / BM) * ((L.N + tile_n - 1) / tile_n);
+    if (L.kind == MT_CONV3X3) return c * rows_per_unit;
+    return 0;
+}
+
+// Per bucket t (one warp each): counts[t] = sum over blocks, block_hist[b][t] <- exclusive prefix over blocks.
+__device__ __forceinline__ void column_scan(int t, int n_blocks, int T1, int32_t* __restrict__ block_hist,
+                                            int32_t* __restrict__ counts) {
+    const int lane = threadIdx.x & 31;
+    int carry = 0;
+    for (int b0 = 0; b0 < n_blocks; b0 += 32) {
+        const int b = b0 + lane;
+        const int v = (b < n_blocks) ? block_hist[(size_t)b * T1 + t] : 0;
+        int incl = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int u = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += u;
+        }
+        if (b < n_blocks) block_hist[(size_t)b * T1 + t] = carry + incl - v;
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) counts[t] = carry;
+}
+
+// Many tenants x many blocks: the per-tenant scans over blocks run as a grid of warps.
+__global__ void __launch_bounds__(256)
+bucket_column_scan(int n_blocks, int T, int32_t* __restrict__ block_hist, int32_t* __restrict__ counts) {
+    const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (t < T + 1) column_scan(t, n_blocks, T + 1, block_hist, counts);
+}
+
+// One CTA: (optionally the per-tenant scans over blocks,) offsets = exclusive scan of counts over the T + 1
+// buckets (offsets[T + 1] = n), and per layer the prefix sums of the work units each tenant contributes.
 __global__ void __launch_bounds__(kScanThreads)
 bucket_scan(int n_blocks, int T, const ModelDev* __restrict__ models, int n_layers, int rows_per_unit, LayerTileN tn,
-            int32_t* __restrict__ block_hist, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
-            int32_t* __restrict__ tile_prefix, int32_t* __restrict__ tmp) {
-    __shared__ int32_t s_tmp[kScanThreads];
+            int do_columns, int32_t* __restrict__ block_hist, int32_t* __restrict__ counts,
+            int32_t* __restrict__ offsets, int32_t* __restrict__ tile_prefix) {
+    __shared__ int32_t s_warp[33];
     const int T1 = T + 1;
+    if (do_columns) {
+        for (int t = threadIdx.x >> 5; t < T1; t += kScanThreads / 32) column_scan(t, n_blocks, T1, block_hist, counts);
+        __syncthreads();
+    }
+    // each thread owns `per` consecutive buckets
+    const int per = (T1 + kScanThreads - 1) / kScanThreads;
+    const int lo = min((int)threadIdx.x * per, T1), hi = min(lo + per, T1);
+    int sum = 0;
+    for (int t = lo; t < hi; ++t) sum += counts[t];
+    int total;
+    int run = cta_excl_scan(sum, s_warp, &total);
+    for (int t = lo; t < hi; ++t) { offsets[t] = run; run += counts[t]; }
+    if (threadIdx.x == 0) offsets[T1] = total;
+    for (int l = 0; l < n_layers; ++l) {
+        int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
+        const int hi_t = min(hi, T);           // the extra bucket of rejected ids contributes no work
+        int usum = 0;
+        for (int t = lo; t < hi_t; ++t) usum += layer_units(models, t, l, counts[t], rows_per_unit, tn.v[l]);
+        int urun = cta_excl_scan(usum, s_warp, &total);
+        for (int t = lo; t < hi_t; ++t) { prefix[t] = urun; urun += layer_units(models, t, l, counts[t], rows_per_unit, tn.v[l]); }
+        if (threadIdx.x == 0) prefix[T] = total;
+    }
+}
+
+// A batch that fits one CTA (n <= kBucketChunk): histogram, scans and stable scatter in ONE launch.
+__global__ void __launch_bounds__(kBucketChunk)
+bucket_small(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models, int n_layers,
+             int rows_per_unit, LayerTileN tn, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
+             int32_t* __restrict__ tile_prefix, int32_t* __restrict__ perm, int32_t* __restrict__ inv,
+             int32_t* __restrict__ status) {
+    extern __shared__ int32_t s_mem[];          // s_cnt[T + 1], s_next[T + 1]
+    __shared__ int32_t s_warp[33];
+    const int T1 = T + 1;
+    int32_t* s_cnt = s_mem;
+    int32_t* s_next = s_mem + T1;
+    for (int t = threadIdx.x; t < T1; t += blockDim.x) s_cnt[t] = 0;
+    __syncthreads();
+    const int i = threadIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // (1) per bucket: counts[t] = sum over blocks; block_hist[b][t] <- exclusive prefix over blocks
-    for (int t = warp; t < T1; t += kScanThreads / 32) {
-        int carry = 0;
-        for (int b0 = 0; b0 < n_blocks; b0 += 32) {
-            const int b = b0 + lane;
-            const int v = (b < n_blocks) ? block_hist[(size_t)b * T1 + t] : 0;
-            int incl = v;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int u = __shfl_up_sync(0xffffffffu, incl, d);
-                if (lane >= d) incl += u;
-            }
-            if (b < n_blocks) block_hist[(size_t)b * T1 + t] = carry + incl - v;
-            carry += __shfl_sync(0xffffffffu, incl, 31);
+    int b = -1;
+    if (i < n) {
+        b = classify(ids[i], T, models);
+        if (b == T) {
+            atomicCAS(&status[ST_CODE], MT_OK, MT_ERR_BAD_MODEL_ID);
+            atomicMin(&status[ST_BAD_INDEX], i);
         }
-        if (lane == 0) counts[t] = carry;
+        const unsigned peers = __match_any_sync(__activemask(), b);
+        if ((__ffs(peers) - 1) == lane) atomicAdd(&s_cnt[b], __popc(peers));
     }
     __syncthreads();
-    // (2) offsets = exclusive scan of counts over the T + 1 buckets (offsets[T + 1] = n)
-    cta_exclusive_scan(counts, offsets, T1, s_tmp);
-    // (3) per layer: prefix sums of the work units (tiles) each tenant contributes
+    const int per = (T1 + kBucketChunk - 1) / kBucketChunk;
+    const int lo = min((int)threadIdx.x * per, T1), hi = min(lo + per, T1);
+    int sum = 0;
+    for (int t = lo; t < hi; ++t) sum += s_cnt[t];
+    int total;
+    int run = cta_excl_scan(sum, s_warp, &total);
+    for (int t = lo; t < hi; ++t) { offsets[t] = run; s_next[t] = run; counts[t] = s_cnt[t]; run += s_cnt[t]; }
+    if (threadIdx.x == 0) offsets[T1] = total;
     for (int l = 0; l < n_layers; ++l) {
-        for (int t = threadIdx.x; t < T; t += kScanThreads) {
-            int units = 0;
-            const int c = counts[t];
-            if (c > 0) {
-                const LayerDev& L = models[t].layer[l];
-                if (L.kind == MT_DENSE) units = ((c + BM - 1) / BM) * ((L.N + tn.v[l] - 1) / tn.v[l]);
-                else if (L.kind == MT_CONV3X3) units = c * rows_per_unit;   // rows_per_unit = tiles per image
-            }
-            tmp[t] = units;
+        int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
+        const int hi_t = min(hi, T);
+        int usum = 0;
+        for (int t = lo; t < hi_t; ++t) usum += layer_units(models, t, l, s_cnt[t], rows_per_unit, tn.v[l]);
+        int urun = cta_excl_scan(usum, s_warp, &total);
+        for (int t = lo; t < hi_t; ++t) { prefix[t] = urun; urun += layer_units(models, t, l, s_cnt[t], rows_per_unit, tn.v[l]); }
+        if (threadIdx.x == 0) prefix[T] = total;
+    }
+    __syncthreads();
+    // warps take turns in arrival order, so positions inside a bucket ascend with the arrival index
+    for (int w = 0; w < kBucketChunk / 32; ++w) {
+        if (warp == w && i < n) {
+            const unsigned peers = __match_any_sync(__activemask(), b);
+            const int rank = __popc(peers & ((1u << lane) - 1u));
+            const int pos = s_next[b] + rank;
+            __syncwarp(__activemask());
+            if (rank == 0) s_next[b] += __popc(peers);
+            perm[pos] = i;
+            inv[i] = pos;
         }
         __syncthreads();
-        cta_exclusive_scan(tmp, tile_prefix + (size_t)l * (T + 1), T, s_tmp);
     }
 }
 
@@ -224,16 +309,26 @@ static int grid_for(long long total, int threads, int sm_count) {
 void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
     const int n_blocks = (a.n + kBucketChunk - 1) / kBucketChunk;
     const size_t smem = sizeof(int32_t) * (size_t)(a.T + 1);
-    bucket_block_hist<<<n_blocks, kBucketChunk, smem, s>>>(a.ids, a.n, a.T, a.models, a.block_hist, a.status);
     LayerTileN tn;
     for (int l = 0; l < 8; ++l) tn.v[l] = a.tile_n[l] > 0 ? a.tile_n[l] : BN;
-    bucket_scan<<<1, kScanThreads, 0, s>>>(n_blocks, a.T, a.models, a.n_layers, a.rows_per_unit, tn, a.block_hist,
-                                           a.counts, a.offsets, a.tile_prefix, a.tmp);
-    bucket_scatter<<<n_blocks, kBucketChunk, smem, s>>>(a.ids, a.n, a.T, a.models, a.block_hist, a.offsets, a.perm,
-                                                        a.inv);
     ItemPtrs ip;
     bool any = false;
     for (int l = 0; l < 8; ++l) { ip.v[l] = a.items[l]; any = any || a.items[l]; }
+    if (n_blocks == 1 && a.T + 1 <= 4096) {
+        bucket_small<<<1, kBucketChunk, 2 * smem, s>>>(a.ids, a.n, a.T, a.models, a.n_layers, a.rows_per_unit, tn, a.counts,
+                                                     a.offsets, a.tile_prefix, a.perm, a.inv, a.status);
+        if (any) build_work_items<<<a.item_grid, 256, 0, s>>>(a.T, a.models, a.n_layers, tn, a.offsets, a.tile_prefix, ip);
+        return;
+    }
+    bucket_block_hist<<<n_blocks, kBucketChunk, smem, s>>>(a.ids, a.n, a.T, a.models, a.block_hist, a.status);
+    // few buckets x few blocks: the per-tenant scans over blocks ride along in the single-CTA scan kernel
+    const int col_iters = ((a.T + 1 + 31) / 32) * ((n_blocks + 31) / 32);
+    const int fused = col_iters <= 4;
+    if (!fused) bucket_column_scan<<<(a.T + 1 + 7) / 8, 256, 0, s>>>(n_blocks, a.T, a.block_hist, a.counts);
+    bucket_scan<<<1, kScanThreads, 0, s>>>(n_blocks, a.T, a.models, a.n_layers, a.rows_per_unit, tn, fused, a.block_hist,
+                                           a.counts, a.offsets, a.tile_prefix);
+    bucket_scatter<<<n_blocks, kBucketChunk, smem, s>>>(a.ids, a.n, a.T, a.models, a.block_hist, a.offsets, a.perm,
+                                                        a.inv);
     if (any) build_work_items<<<a.item_grid, 256, 0, s>>>(a.T, a.models, a.n_layers, tn, a.offsets, a.tile_prefix, ip);
 }
 

@@ -161,13 +161,17 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
             int g = 0;                      // tiles started so far by this CTA; tile g lives in TMEM slot g % kSlots
             int w_loads = 0;
             bool ok = true;
-            // four K steps of one 128-pixel block against one (N = 64) or two stacked (N = 128) tap tiles
-            auto issue = [&](uint32_t a_addr, uint32_t b_addr, uint32_t d_tmem, uint32_t idesc, bool overwrite) {
-                const uint64_t a_desc = make_kmajor_sw128_desc(a_addr, 1024);
-                const uint64_t b_desc = make_kmajor_sw128_desc(b_addr, 1024);
-#pragma unroll
-                for (int k = 0; k < BK / UMMA_K; ++k)
-                    umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (overwrite && k == 0) ? 0u : 1u);
+            // Four K steps of one 128-pixel block against one (N = 64) or two stacked (N = 128) tap tiles.  Descriptors
+            // are handled as their low words (address >> 4 | constant): stepping costs one add.
+            const uint32_t w_lo = desc_lo(w_smem);
+            constexpr uint32_t kTapLo = kTapBytes >> 4;          // one tap tile further
+            constexpr uint32_t kPixLo = 128 >> 4;                // one pixel (128 bytes) further
+            auto issue = [&](uint32_t a_lo, uint32_t b_lo, uint32_t d_tmem, uint32_t idesc, bool overwrite) {
+                if (overwrite) umma_bf16_lohi<false>(d_tmem, a_lo, b_lo, idesc);
+                else umma_bf16_lohi<true>(d_tmem, a_lo, b_lo, idesc);
+                umma_bf16_lohi<true>(d_tmem, a_lo + 2, b_lo + 2, idesc);
+                umma_bf16_lohi<true>(d_tmem, a_lo + 4, b_lo + 4, idesc);
+                umma_bf16_lohi<true>(d_tmem, a_lo + 6, b_lo + 6, idesc);
             };
             // This thread is the only feeder of the tensor pipe, and its MMAs, commits and barrier polls go through one
             // in-order queue: an instruction whose result the thread needs (a barrier poll, a shared-memory load)
@@ -197,7 +201,7 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
                 }
                 const bool pair_top = pairing && s > s_begin && in_image > 0;
                 const bool defer_bottom = pairing && s + 1 < s_end && in_image + 1 < p.strips_per_image;
-                const uint32_t strip = strip0 + stage * p.stage_bytes;
+                const uint32_t strip_lo = desc_lo(strip0 + stage * p.stage_bytes);
                 const int next_stage = (stage + 1 == p.n_stages) ? 0 : stage + 1;
                 const uint32_t next_phase = (stage + 1 == p.n_stages) ? (phase ^ 1u) : phase;
                 strip_ready = 0;
@@ -208,35 +212,36 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
                     }
                     tc_fence_after();
                     const uint32_t d_this = tmem_base + slot * kCN;
-                    const uint32_t blk = strip + (uint32_t)(i * BM) * 128u;          // padded pixel i*128 of the strip
+                    const uint32_t blk = strip_lo + (uint32_t)(i * BM) * kPixLo;     // padded pixel i*128 of the strip
                     const bool last_tile = (i == TS - 1);
                     uint32_t poll_slot = 0, poll_strip = 0;
                     if (pairing) {
                         // ky = 1 first: these overwrite the fresh accumulator
-                        issue(blk + (uint32_t)(Wp + 0) * 128u, w_smem + tap_slot(1, 0) * kTapBytes, d_this, idesc64, true);
+                        issue(blk + (uint32_t)(Wp + 0) * kPixLo, w_lo + tap_slot(1, 0) * kTapLo, d_this, idesc64, true);
                         // look ahead: results are consumed after the rest of this tile has been queued
                         poll_slot = mbar_test_wait(tempty_bar((g + 1) % kSlots), (uint32_t)((((g + 1) / kSlots) & 1) ^ 1));
                         if (last_tile) poll_strip = mbar_test_wait(sfull_bar(next_stage), next_phase);
-                        issue(blk + (uint32_t)(Wp + 1) * 128u, w_smem + tap_slot(1, 1) * kTapBytes, d_this, idesc64, false);
-                        issue(blk + (uint32_t)(Wp + 2) * 128u, w_smem + tap_slot(1, 2) * kTapBytes, d_this, idesc64, false);
+                        issue(blk + (uint32_t)(Wp + 1) * kPixLo, w_lo + tap_slot(1, 1) * kTapLo, d_this, idesc64, false);
+                        issue(blk + (uint32_t)(Wp + 2) * kPixLo, w_lo + tap_slot(1, 2) * kTapLo, d_this, idesc64, false);
                         // block at the tile's first row: ky = 0 of this tile and ky = 2 of the tile above
                         const bool have_above = (i > 0) || pair_top;
                         const bool adjacent = slot != 0;                              // slots g-1 and g contiguous in TMEM
-                        for (int kx = 0; kx < 3; ++kx) {
-                            const uint32_t a_addr = blk + (uint32_t)kx * 128u;
-                            if (have_above && adjacent) {
-                                issue(a_addr, w_smem + tap_slot(2, kx) * kTapBytes, d_this - kCN, idesc128, false);
-                            } else {
+                        if (have_above && adjacent) {
+#pragma unroll
+                            for (int kx = 0; kx < 3; ++kx)
+                                issue(blk + kx * kPixLo, w_lo + tap_slot(2, kx) * kTapLo, d_this - kCN, idesc128, false);
+                        } else {
+                            for (int kx = 0; kx < 3; ++kx) {
                                 if (have_above)
-                                    issue(a_addr, w_smem + tap_slot(2, kx) * kTapBytes, tmem_base + ((g - 1) % kSlots) * kCN, idesc64, false);
-                                issue(a_addr, w_smem + tap_slot(0, kx) * kTapBytes, d_this, idesc64, false);
+                                    issue(blk + kx * kPixLo, w_lo + tap_slot(2, kx) * kTapLo, tmem_base + ((g - 1) % kSlots) * kCN, idesc64, false);
+                                issue(blk + kx * kPixLo, w_lo + tap_slot(0, kx) * kTapLo, d_this, idesc64, false);
                             }
                         }
                         if (have_above) umma_commit(tfull_bar((g - 1) % kSlots));    // tile above is complete
                     } else {
                         for (int tap = 0; tap < 9; ++tap) {
                             const int ky = tap / 3, kx = tap - 3 * ky;
-                            issue(blk + (uint32_t)(ky * Wp + kx) * 128u, w_smem + tap_slot(ky, kx) * kTapBytes, d_this, idesc64, tap == 0);
+                            issue(blk + (uint32_t)(ky * Wp + kx) * kPixLo, w_lo + tap_slot(ky, kx) * kTapLo, d_this, idesc64, tap == 0);
                             if (tap == 1) {
                                 poll_slot = mbar_test_wait(tempty_bar((g + 1) % kSlots), (uint32_t)((((g + 1) / kSlots) & 1) ^ 1));
                                 if (last_tile) poll_strip = mbar_test_wait(sfull_bar(next_stage), next_phase);
@@ -250,10 +255,10 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
                 if (!ok) break;
                 if (pairing && !defer_bottom) {
                     // nobody below will finish the strip's last tile: its ky = 2 taps from the block under it
-                    const uint32_t blk = strip + (uint32_t)(TS * BM) * 128u;
+                    const uint32_t blk = strip_lo + (uint32_t)(TS * BM) * kPixLo;
                     const int last = (g - 1) % kSlots;
                     for (int kx = 0; kx < 3; ++kx)
-                        issue(blk + (uint32_t)kx * 128u, w_smem + tap_slot(2, kx) * kTapBytes, tmem_base + last * kCN, idesc64, false);
+                        issue(blk + kx * kPixLo, w_lo + tap_slot(2, kx) * kTapLo, tmem_base + last * kCN, idesc64, false);
                     umma_commit(tfull_bar(last));
                 }
                 // The strip buffer is released by the epilogue (see there), not by a third commit here: a commit issued
@@ -382,7 +387,7 @@ void launch_pretile_conv(const uint16_t* w, int C_out, int C_in, uint16_t* out, 
 }
 
 // g[j][c] = (1 / HW) * sum_p x[j][p][c]; one CTA per image, 8 channels (16 bytes) per thread per pixel.
-constexpr int kPoolThreads = 256;
+constexpr int kPoolThreads = 512;
 
 __global__ void __launch_bounds__(kPoolThreads)
 global_avg_pool_kernel(const uint16_t* __restrict__ x, int HW, int C, uint16_t* __restrict__ out, int ld_out) {
@@ -393,15 +398,23 @@ global_avg_pool_kernel(const uint16_t* __restrict__ x, int HW, int C, uint16_t* 
     const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)blockIdx.x * HW * C);
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     if (g_id < groups) {
-        for (int pix = g_id; pix < HW; pix += groups) {
-            const uint4 q = __ldg(&src[(size_t)pix * vec_per_pixel + v]);
+        auto add = [&](const uint4& q) {
             const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 acc[2 * k + 0] += __uint_as_float(w[k] << 16);
                 acc[2 * k + 1] += __uint_as_float(w[k] & 0xFFFF0000u);
             }
+        };
+        int pix = g_id;
+        for (; pix + 3 * groups < HW; pix += 4 * groups) {      // four independent loads in flight per thread
+            const uint4 q0 = __ldg(&src[(size_t)pix * vec_per_pixel + v]);
+            const uint4 q1 = __ldg(&src[(size_t)(pix + groups) * vec_per_pixel + v]);
+            const uint4 q2 = __ldg(&src[(size_t)(pix + 2 * groups) * vec_per_pixel + v]);
+            const uint4 q3 = __ldg(&src[(size_t)(pix + 3 * groups) * vec_per_pixel + v]);
+            add(q0); add(q1); add(q2); add(q3);
         }
+        for (; pix < HW; pix += groups) add(__ldg(&src[(size_t)pix * vec_per_pixel + v]));
 #pragma unroll
         for (int k = 0; k < 8; ++k) s_part[g_id * C + v * 8 + k] = acc[k];
     }

@@ -78,7 +78,7 @@ struct Ctx {
     int st_cap = 0;
 
     // timing
-    bool timing = false;
+    int timing = 0;                      // 0 off, 1 every kernel, 2 only the layer executors
     std::vector<TimedLaunch> timed;
     std::vector<cudaEvent_t> event_pool;
 };
@@ -302,7 +302,8 @@ struct Timer {
     cudaStream_t s;
     bool on;
     cudaEvent_t start = nullptr, stop = nullptr;
-    Timer(int k, cudaStream_t st) : kernel(k), s(st), on(g.timing) {
+    Timer(int k, cudaStream_t st)
+        : kernel(k), s(st), on(g.timing == 1 || (g.timing == 2 && (k == K_GEMM || k == K_CONV))) {
         if (!on) return;
         auto get = [&]() {
             cudaEvent_t e;
@@ -428,7 +429,7 @@ mt_status mt_shutdown(void) {
     g.timed.clear();
     for (cudaEvent_t e : g.event_pool) cudaEventDestroy(e);
     g.event_pool.clear();
-    g.timing = false;
+    g.timing = 0;
     g.init = false;
     g.has_family = false;
     g.family.clear();
@@ -634,7 +635,7 @@ mt_status mt_debug_last_bucketing(int32_t* counts_host, int32_t* offsets_host, i
 
 mt_status mt_set_kernel_timing(int32_t enable) {
     std::lock_guard<std::mutex> lk(g_mu);
-    g.timing = enable != 0;
+    g.timing = enable < 0 ? 0 : (enable > 2 ? 1 : enable);
     return MT_OK;
 }
 
