@@ -38,7 +38,7 @@ constexpr int kTapBytes = kCN * BK * 2;          // 8 KiB: 64 out channels x 64 
 constexpr int kWeightBytes = 9 * kTapBytes;      // 72 KiB, resident per tenant
 constexpr int kMaxStages = 4;
 constexpr int kSlots = 8;                        // TMEM ring: 8 accumulators of 64 columns = all 512 columns
-constexpr int kConvBarBytes = 1024;
+constexpr int kConvBarBytes = 2048;
 constexpr int kRecords = 16;                     // ring of per-strip records (producer -> MMA issuer, epilogue)
 
 // Order of the tap tiles in the executor layout: the three ky = 1 taps, then for every kx the pair
@@ -73,6 +73,7 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
     // tile), y = image (bucketed index), z = first output row, w = tenant.  The issuing thread must not spend
     // time on index arithmetic: the tensor pipe drains as soon as it stops issuing.
     int4* s_rec = reinterpret_cast<int4*>(bar_ptr + 512);             // kRecords x 16 bytes
+    float* s_pool = reinterpret_cast<float*>(bar_ptr + 1024);         // 8 warps x 32 channel sums (fused pooling)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -277,7 +278,11 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
         int g = 0, relu = 0;
         bool ok = true;
         int img_j = 0, y0 = 0;
+        const bool pooling = (p.pool_partial != nullptr);
         for (int s = s_begin; ok && s < s_end; ++s) {
+            float psum[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) psum[e] = 0.0f;
             for (int i = 0; i < TS; ++i, ++g) {
                 const int slot = g % kSlots;
                 if (!mbar_wait(tfull_bar(slot), (uint32_t)((g / kSlots) & 1), abort_flag, p.status, 26)) { ok = false; break; }
@@ -321,15 +326,46 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
 #pragma unroll
                             for (int e = 0; e < 8; ++e) f[e] = fmaxf(f[e], 0.0f);
                         }
-                        uint4 o;
-                        o.x = pack_bf16x2(f[0], f[1]);
-                        o.y = pack_bf16x2(f[2], f[3]);
-                        o.z = pack_bf16x2(f[4], f[5]);
-                        o.w = pack_bf16x2(f[6], f[7]);
-                        reinterpret_cast<uint4*>(dst)[j] = o;
+                        if (pooling) {      // the layer feeds a global average pool: only channel sums are kept
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) psum[8 * j + e] += f[e];
+                        } else {
+                            uint4 o;
+                            o.x = pack_bf16x2(f[0], f[1]);
+                            o.y = pack_bf16x2(f[2], f[3]);
+                            o.z = pack_bf16x2(f[4], f[5]);
+                            o.w = pack_bf16x2(f[6], f[7]);
+                            reinterpret_cast<uint4*>(dst)[j] = o;
+                        }
                     }
                 }
                 __syncwarp();
+            }
+            if (pooling && ok) {
+                // Channel sums of this strip: a halving butterfly leaves lane c with the warp's total of channel c
+                // (31 shuffles), the four lane quarters are then added in a fixed order, and the strip's 64 sums are
+                // written to their own slot of pool_partial - no atomics, so the pooled value does not depend on timing.
+#pragma unroll
+                for (int step = 16; step >= 1; step >>= 1) {
+                    const bool upper = (lane & step) != 0;
+#pragma unroll
+                    for (int e = 0; e < step; ++e) {
+                        const float send = upper ? psum[e] : psum[e + step];
+                        const float recv = __shfl_xor_sync(0xffffffffu, send, step);
+                        psum[e] = (upper ? psum[e + step] : psum[e]) + recv;
+                    }
+                }
+                s_pool[ew * 32 + lane] = psum[0];
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+                const int et = threadIdx.x - 64;                    // 0..255 among the epilogue threads
+                if (et < kCN) {
+                    const int hf = et >> 5, c = et & 31;
+                    const float* q = s_pool + (hf * 4) * 32 + c;     // warps hf*4 .. hf*4+3 hold this half's quarters
+                    // quarter order by TMEM lane quarter (ew & 3 maps to q4 = (ew + 2) & 3): sum in pixel order 0,1,2,3
+                    const float t = ((q[2 * 32] + q[3 * 32]) + q[0 * 32]) + q[1 * 32];
+                    p.pool_partial[((size_t)img_j * p.strips_per_image + y0 / p.R) * kCN + et] = t;
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
             }
         }
     }
@@ -386,45 +422,20 @@ void launch_pretile_conv(const uint16_t* w, int C_out, int C_in, uint16_t* out, 
     pretile_conv_kernel<<<(total + 255) / 256, 256, 0, s>>>(w, C_out, C_in, reinterpret_cast<uint4*>(out), total);
 }
 
-// g[j][c] = (1 / HW) * sum_p x[j][p][c]; one CTA per image, 8 channels (16 bytes) per thread per pixel.
-constexpr int kPoolThreads = 512;
+// g[j][c] = (1 / HW) * sum over the image's strips of pool_partial[j][strip][c] (fixed order), rounded to bf16.
+__global__ void pool_finalize_kernel(const float* __restrict__ partial, int n, int strips, int C, float inv_hw,
+                                     uint16_t* __restrict__ out, int ld_out) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= n * C) return;
+    const int j = idx / C, c = idx - j * C;
+    float s = 0.f;
+    for (int k = 0; k < strips; ++k) s += partial[((size_t)j * strips + k) * C + c];
+    out[(size_t)j * ld_out + c] = static_cast<uint16_t>(pack_bf16x2(s * inv_hw, 0.0f) & 0xFFFFu);
+}
 
-__global__ void __launch_bounds__(kPoolThreads)
-global_avg_pool_kernel(const uint16_t* __restrict__ x, int HW, int C, uint16_t* __restrict__ out, int ld_out) {
-    extern __shared__ float s_part[];   // [groups][C]
-    const int vec_per_pixel = C / 8;
-    const int groups = kPoolThreads / vec_per_pixel;      // pixels processed per iteration
-    const int g_id = threadIdx.x / vec_per_pixel, v = threadIdx.x % vec_per_pixel;
-    const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)blockIdx.x * HW * C);
-    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    if (g_id < groups) {
-        auto add = [&](const uint4& q) {
-            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                acc[2 * k + 0] += __uint_as_float(w[k] << 16);
-                acc[2 * k + 1] += __uint_as_float(w[k] & 0xFFFF0000u);
-            }
-        };
-        int pix = g_id;
-        for (; pix + 3 * groups < HW; pix += 4 * groups) {      // four independent loads in flight per thread
-            const uint4 q0 = __ldg(&src[(size_t)pix * vec_per_pixel + v]);
-            const uint4 q1 = __ldg(&src[(size_t)(pix + groups) * vec_per_pixel + v]);
-            const uint4 q2 = __ldg(&src[(size_t)(pix + 2 * groups) * vec_per_pixel + v]);
-            const uint4 q3 = __ldg(&src[(size_t)(pix + 3 * groups) * vec_per_pixel + v]);
-            add(q0); add(q1); add(q2); add(q3);
-        }
-        for (; pix < HW; pix += groups) add(__ldg(&src[(size_t)pix * vec_per_pixel + v]));
-#pragma unroll
-        for (int k = 0; k < 8; ++k) s_part[g_id * C + v * 8 + k] = acc[k];
-    }
-    __syncthreads();
-    for (int c = threadIdx.x; c < C; c += blockDim.x) {
-        float s = 0.f;
-        for (int gi = 0; gi < groups; ++gi) s += s_part[gi * C + c];
-        const float m = s / (float)HW;
-        out[(size_t)blockIdx.x * ld_out + c] = static_cast<uint16_t>(pack_bf16x2(m, 0.0f) & 0xFFFFu);
-    }
+void launch_pool_finalize(const float* partial, int n, int strips, int C, int HW, uint16_t* out, int ld_out,
+                          cudaStream_t s) {
+    pool_finalize_kernel<<<(n * C + 255) / 256, 256, 0, s>>>(partial, n, strips, C, 1.0f / (float)HW, out, ld_out);
 }
 
 cudaError_t configure_grouped_conv() {
@@ -433,12 +444,6 @@ cudaError_t configure_grouped_conv() {
 
 void launch_grouped_conv(const CUtensorMap& tmap_x, const ConvArgs& a, int smem_bytes, int sm_count, cudaStream_t s) {
     grouped_conv3x3_kernel<<<sm_count, kConvThreads, smem_bytes, s>>>(tmap_x, a);
-}
-
-void launch_global_avg_pool(const uint16_t* x, int n, int HW, int C, uint16_t* out, int ld_out, int /*sm_count*/,
-                            cudaStream_t s) {
-    const int groups = kPoolThreads / (C / 8);
-    global_avg_pool_kernel<<<n, kPoolThreads, sizeof(float) * groups * C, s>>>(x, HW, C, out, ld_out);
 }
 
 }  // namespace mt

@@ -34,7 +34,7 @@ struct HostModel {
 
 enum KernelId { K_HIST = 0, K_SCAN, K_SCATTER, K_GATHER, K_GEMM, K_CONV, K_POOL, K_UNPERMUTE, K_COUNT };
 const char* const kKernelNames[K_COUNT] = {"bucket_block_hist+scan+scatter", "", "", "gather_rows",
-                                           "grouped_gemm", "grouped_conv3x3", "global_avg_pool", "unpermute_rows"};
+                                           "grouped_gemm", "grouped_conv3x3", "pool_finalize", "unpermute_rows"};
 
 struct TimedLaunch {
     int kernel;
@@ -67,6 +67,7 @@ struct Ctx {
     int act_ld[MT_MAX_LAYERS + 1] = {0};
     CUtensorMap act_map[MT_MAX_LAYERS + 1];
     float* d_out_b = nullptr;
+    float* d_pool_partial = nullptr;     // per-strip channel sums of a conv layer that feeds a pool
     WorkItem* d_items[MT_MAX_LAYERS] = {nullptr};   // per dense layer
     size_t items_cap[MT_MAX_LAYERS] = {0};
     int last_n = 0;
@@ -147,6 +148,7 @@ void free_workspace() {
     cudaFree(g.d_perm); g.d_perm = nullptr;
     cudaFree(g.d_inv); g.d_inv = nullptr;
     cudaFree(g.d_out_b); g.d_out_b = nullptr;
+    cudaFree(g.d_pool_partial); g.d_pool_partial = nullptr;
     for (int b = 0; b <= MT_MAX_LAYERS; ++b) { cudaFree(g.act[b]); g.act[b] = nullptr; }
     for (int l = 0; l < MT_MAX_LAYERS; ++l) { cudaFree(g.d_items[l]); g.d_items[l] = nullptr; g.items_cap[l] = 0; }
     g.cap_n = 0;
@@ -207,6 +209,9 @@ mt_status ensure_workspace(int n) {
             }
         }
     }
+    for (int l = 0; l + 1 < L; ++l)
+        if (g.family[l].kind == MT_CONV3X3 && g.family[l + 1].kind == MT_GLOBAL_AVG_POOL && !g.d_pool_partial)
+            CU_OK(cudaMalloc(&g.d_pool_partial, sizeof(float) * (size_t)cap * g.conv.strips_per_image * 64));
     // work items of the dense layers: at most (row tiles + one ragged tile per tenant) x column tiles of the widest model
     for (int l = 0; l < L; ++l) {
         if (g.family[l].kind != MT_DENSE) continue;
@@ -376,6 +381,8 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             a.tile_prefix = g.d_tile_prefix + (size_t)l * (g.T + 1);
             a.perm = (l == 0) ? g.d_perm : nullptr;
             a.out = (uint16_t*)g.act[l + 1];
+            const bool feeds_pool = (l + 1 < L) && g.family[l + 1].kind == MT_GLOBAL_AVG_POOL;
+            a.pool_partial = feeds_pool ? g.d_pool_partial : nullptr;
             a.H = f.h; a.W = f.w;
             a.Wp = g.conv.Wp; a.R = g.conv.R; a.tiles_per_strip = g.conv.tiles_per_strip;
             a.stage_bytes = g.conv.stage_bytes; a.n_stages = g.conv.n_stages;
@@ -384,8 +391,10 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             launch_grouped_conv(l == 0 ? in_map : g.act_map[l], a, g.conv.smem_bytes, g.sm_count, s);
         } else {
             Timer t(K_POOL, s);
-            launch_global_avg_pool((const uint16_t*)g.act[l], n, f.h * f.w, f.in_ch, (uint16_t*)g.act[l + 1],
-                                   g.act_ld[l + 1], g.sm_count, s);
+            // a pool always follows a conv (checked at registration), whose epilogue already reduced every strip
+            // to channel sums
+            launch_pool_finalize(g.d_pool_partial, n, g.conv.strips_per_image, f.in_ch, f.h * f.w,
+                                 (uint16_t*)g.act[l + 1], g.act_ld[l + 1], s);
         }
     }
     {

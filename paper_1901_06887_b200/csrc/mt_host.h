@@ -82,7 +82,8 @@ struct ConvArgs {
     const int32_t* offsets;
     const int32_t* tile_prefix;   // work units = strips
     const int32_t* perm;          // non-null: image index = perm[j] (first layer reads the caller's buffer)
-    uint16_t* out;                // bf16 NHWC, bucketed order
+    uint16_t* out;                // bf16 NHWC, bucketed order (unused when pool_partial is set)
+    float* pool_partial;          // non-null: the layer feeds a global average pool; [n][strips_per_image][64] sums
     int H, W;
     int Wp, R, tiles_per_strip, stage_bytes, n_stages, strips_per_image, box_bytes;
     int32_t* status;
@@ -90,8 +91,8 @@ struct ConvArgs {
 cudaError_t configure_grouped_conv();
 void launch_grouped_conv(const CUtensorMap& tmap_x, const ConvArgs& a, int smem_bytes, int sm_count, cudaStream_t s);
 
-// g[j][c] = mean over the H*W positions of x[j][.][.][c]; bf16 in, fp32 sum, bf16 out (row stride ld_out).
-void launch_global_avg_pool(const uint16_t* x, int n, int HW, int C, uint16_t* out, int ld_out, int sm_count,
-                            cudaStream_t s);
+// Second half of the fused pooling: sums the per-strip channel sums of each image and divides by H*W.
+void launch_pool_finalize(const float* partial, int n, int strips, int C, int HW, uint16_t* out, int ld_out,
+                          cudaStream_t s);
 
 }  // namespace mt

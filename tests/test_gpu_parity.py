@@ -82,6 +82,14 @@ def test_config4_reduced_geometries(h, w):
     run_and_check(wl.models, wl.model_ids, wl.inputs)
 
 
+@pytest.mark.parametrize("h,w,n,tenants", [(56, 56, 40, 5), (37, 40, 30, 4), (10, 33, 200, 3)])
+def test_conv_many_strips_per_cta(h, w, n, tenants):
+    # enough images that every CTA walks several strips: tap pairing across strip borders, the ring of TMEM
+    # accumulators wrapping around, tenant changes (weight reloads) inside a CTA's range, ragged last strips
+    wl = synth.make_workload(4, n=n, n_tenants=tenants, h=h, w=w, n_conv=3)
+    run_and_check(wl.models, wl.model_ids, wl.inputs)
+
+
 def test_conv_single_tap_shift_closed_form_on_gpu():
     # tap (ky,kx) with weight 1 on the diagonal: Y = shifted X (zero outside), exact in bf16
     H, W = 6, 9
