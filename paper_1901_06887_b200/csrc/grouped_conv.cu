@@ -155,7 +155,11 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {   // ------------------------------------------------ MMA issuer
+        {                  // ------------------------------------------------ MMA issuer
+            // The whole warp walks the loop (so that addresses and descriptors stay warp-uniform values); one elected
+            // lane issues the MMAs and commits.
+            const bool leader = elect_one();
+            const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);   // warp-uniform copy
             constexpr uint32_t idesc64 = make_idesc_bf16(BM, kCN);
             constexpr uint32_t idesc128 = make_idesc_bf16(BM, 2 * kCN);
             int stage = 0; uint32_t phase = 0;
@@ -168,6 +172,7 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
             constexpr uint32_t kTapLo = kTapBytes >> 4;          // one tap tile further
             constexpr uint32_t kPixLo = 128 >> 4;                // one pixel (128 bytes) further
             auto issue = [&](uint32_t a_lo, uint32_t b_lo, uint32_t d_tmem, uint32_t idesc, bool overwrite) {
+                if (!leader) return;
                 if (overwrite) umma_bf16_lohi<false>(d_tmem, a_lo, b_lo, idesc);
                 else umma_bf16_lohi<true>(d_tmem, a_lo, b_lo, idesc);
                 umma_bf16_lohi<true>(d_tmem, a_lo + 2, b_lo + 2, idesc);
@@ -196,7 +201,7 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
                 }
                 tc_fence_after();
                 if (new_tenant) {
-                    if (w_loads > 0) umma_commit(wempty_bar);      // fires when all MMAs on the old weights are done
+                    if (w_loads > 0 && leader) umma_commit(wempty_bar);      // fires when all MMAs on the old weights are done
                     if (!mbar_wait(wfull_bar, (uint32_t)(w_loads & 1), abort_flag, p.status, 23)) break;
                     ++w_loads;
                 }
@@ -238,7 +243,7 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
                                 issue(blk + kx * kPixLo, w_lo + tap_slot(0, kx) * kTapLo, d_this, idesc64, false);
                             }
                         }
-                        if (have_above) umma_commit(tfull_bar((g - 1) % kSlots));    // tile above is complete
+                        if (have_above && leader) umma_commit(tfull_bar((g - 1) % kSlots));    // tile above is complete
                     } else {
                         for (int tap = 0; tap < 9; ++tap) {
                             const int ky = tap / 3, kx = tap - 3 * ky;
@@ -248,7 +253,7 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
                                 if (last_tile) poll_strip = mbar_test_wait(sfull_bar(next_stage), next_phase);
                             }
                         }
-                        umma_commit(tfull_bar(slot));
+                        if (leader) umma_commit(tfull_bar(slot));
                     }
                     slot_ready = poll_slot;
                     if (last_tile) strip_ready = (s + 1 < s_end) ? poll_strip : 0;
@@ -260,7 +265,7 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
                     const int last = (g - 1) % kSlots;
                     for (int kx = 0; kx < 3; ++kx)
                         issue(blk + kx * kPixLo, w_lo + tap_slot(2, kx) * kTapLo, tmem_base + last * kCN, idesc64, false);
-                    umma_commit(tfull_bar(last));
+                    if (leader) umma_commit(tfull_bar(last));
                 }
                 // The strip buffer is released by the epilogue (see there), not by a third commit here: a commit issued
                 // while the previous one is still waiting for its MMAs stalls this thread until the queue has drained.

@@ -104,7 +104,11 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmArgs p
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {   // ------------------------------------------------ MMA issuer
+        {                  // ------------------------------------------------ MMA issuer
+            // The whole warp walks the loop, so that addresses and descriptors stay warp-uniform values; one elected
+            // lane issues the MMAs and commits.
+            const bool leader = elect_one();
+            const uint32_t tmem_base = __shfl_sync(0xffffffffu, *tmem_slot, 0);
             // This thread alone feeds the tensor pipe, and it issues in order: every instruction it spends on
             // anything else is time the pipe may run dry.  So descriptors are one 32-bit add away from a
             // precomputed base, the next stage's barrier is polled (non-blocking) BEFORE the current stage's MMAs
@@ -131,16 +135,18 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmArgs p
                     const uint32_t poll = mbar_test_wait(full_bar(next_stage), next_phase);   // consumed after the MMAs
                     const uint32_t a_lo = a_lo0 + stage * kStageLo, b_lo = b_lo0 + stage * kStageLo;
                     // advancing K by 16 elements = 32 bytes inside the swizzle row: +2 in the address field
-                    if (kb == 0) umma_bf16_lohi<false>(d_tmem, a_lo, b_lo, idesc);
-                    else umma_bf16_lohi<true>(d_tmem, a_lo, b_lo, idesc);
-                    umma_bf16_lohi<true>(d_tmem, a_lo + 2, b_lo + 2, idesc);
-                    umma_bf16_lohi<true>(d_tmem, a_lo + 4, b_lo + 4, idesc);
-                    umma_bf16_lohi<true>(d_tmem, a_lo + 6, b_lo + 6, idesc);
-                    umma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
+                    if (leader) {
+                        if (kb == 0) umma_bf16_lohi<false>(d_tmem, a_lo, b_lo, idesc);
+                        else umma_bf16_lohi<true>(d_tmem, a_lo, b_lo, idesc);
+                        umma_bf16_lohi<true>(d_tmem, a_lo + 2, b_lo + 2, idesc);
+                        umma_bf16_lohi<true>(d_tmem, a_lo + 4, b_lo + 4, idesc);
+                        umma_bf16_lohi<true>(d_tmem, a_lo + 6, b_lo + 6, idesc);
+                        umma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
+                    }
                     stage = next_stage; phase = next_phase;
                     ready = poll;
                 }
-                if (ok) umma_commit(tfull_bar(acc));
+                if (ok && leader) umma_commit(tfull_bar(acc));
                 kblocks = next_kblocks;
             }
         }
