@@ -34,6 +34,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 DEFAULT_STEPS = {1: 5000, 2: 1500, 3: 2500, 4: 1500, 5: 50}
 ORACLE_SAMPLE = {1: 64, 2: 2048, 3: 16384, 4: 24, 5: 96}      # requests of the batch the CPU baseline times
 N_INPUT_BUFFERS = 3
+# DRAM traffic of the dominant kernel from the ncu captures summarised under profiles/ (see there):
+#   config 2: measured on a reduced case, traffic / algorithmic bytes = 0.995, scaled to the full launch;
+#   config 4: measured at full size, bytes per step (four conv launches).  None = not captured.
+TRAFFIC_RATIO = {2: 0.995}
+TRAFFIC_BYTES = {4: 592.8e6}
 
 
 def load_peaks():
@@ -145,7 +150,12 @@ def gemm_roofline(wl, kernel_ms_per_launch_sum, peaks, peaks_kind, config):
         ach = flops / sec / 1e12 if sec > 0 else 0.0
         roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": ach / peaks["bf16_tflops"]}
-    roof.update(traffic=None, peak_source="of " + peaks_kind, kernel="grouped_conv3x3" if dom_kind == synth.CONV3X3 else "grouped_gemm",
+    traffic = None
+    if config in TRAFFIC_RATIO:
+        traffic = int(TRAFFIC_RATIO[config] * byts)
+    elif config in TRAFFIC_BYTES:
+        traffic = int(TRAFFIC_BYTES[config])
+    roof.update(traffic=traffic, peak_source="of " + peaks_kind, kernel="grouped_conv3x3" if dom_kind == synth.CONV3X3 else "grouped_gemm",
                 algorithmic_bytes_per_step=int(byts), flops_per_step=int(flops), kernel_ms_per_step=kernel_ms_per_launch_sum)
     return roof
 
