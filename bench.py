@@ -326,8 +326,8 @@ def main():
     if rank == 0:
         peaks, peaks_kind = load_peaks()
         per_kernel = {name: {"ms_per_step": t / bd_steps, "launches_per_step": c / bd_steps} for name, t, c in breakdown}
-        # launches per step: the bucketing entry covers 2 (one-CTA batch) to 5 kernels under one pair of events
-        bucket_kernels = 2 if n <= 256 else 5
+        # launches per step: the bucketing entry covers 1 (batch of at most 512 requests) or 5 kernels under one pair of events
+        bucket_kernels = 1 if n <= 512 else 5
         per_step = sum(c / bd_steps for nm, _, c in breakdown if not nm.startswith("bucket")) + bucket_kernels
         launches = int(round(per_step * args.steps))
         dom = "grouped_conv3x3" if cfg == 4 else "grouped_gemm"

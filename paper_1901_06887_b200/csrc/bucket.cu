@@ -147,33 +147,74 @@ bucket_scan(int n_blocks, int T, const ModelDev* __restrict__ models, int n_laye
     }
 }
 
-// A batch that fits one CTA (n <= kBucketChunk): histogram, scans and stable scatter in ONE launch.
-__global__ void __launch_bounds__(kBucketChunk)
-bucket_small(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models, int n_layers,
-             int rows_per_unit, LayerTileN tn, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
-             int32_t* __restrict__ tile_prefix, int32_t* __restrict__ perm, int32_t* __restrict__ inv,
-             int32_t* __restrict__ status) {
+struct ItemPtrs { WorkItem* v[8]; };
+
+// Work item `item` of dense layer l: (tenant, row tile, column tile) and what the executor needs to know about it.
+__device__ __forceinline__ WorkItem make_work_item(int item, int l, int T, const ModelDev* __restrict__ models,
+                                                   const int32_t* __restrict__ offsets,
+                                                   const int32_t* __restrict__ prefix) {
+    int lo = 0, hi = T;   // largest t with prefix[t] <= item
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (prefix[mid] <= item) lo = mid; else hi = mid;
+    }
+    const LayerDev& L = models[lo].layer[l];
+    const int seg0 = offsets[lo], n_t = offsets[lo + 1] - seg0;
+    const int m_tiles = (n_t + BM - 1) / BM;
+    const int local = item - prefix[lo];
+    const int n_tile = local / m_tiles, m_tile = local - n_tile * m_tiles;
+    WorkItem w;
+    w.row0 = seg0 + m_tile * BM;
+    w.rows_valid = min(BM, n_t - m_tile * BM);
+    w.n_tile = n_tile;
+    w.k_blocks = L.k_blocks;
+    w.w = L.w;
+    w.bias = L.bias;
+    w.N = L.N;
+    w.relu = L.relu;
+    w.t = lo;
+    w.pad = 0;
+    return w;
+}
+
+
+// A batch that fits one CTA (n <= kSingleCtaMax): histogram, scans, stable scatter and the work-item expansion in
+// ONE launch.  blockDim.x is 256 or 1024; the requests are taken in rounds of blockDim.x.
+constexpr int kSingleCtaMax = 4096;
+
+__global__ void __launch_bounds__(1024)
+bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models, int n_layers,
+                  int rows_per_unit, LayerTileN tn, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
+                  int32_t* __restrict__ tile_prefix, int32_t* __restrict__ perm, int32_t* __restrict__ inv,
+                  ItemPtrs items, int32_t* __restrict__ status) {
     extern __shared__ int32_t s_mem[];          // s_cnt[T + 1], s_next[T + 1]
     __shared__ int32_t s_warp[33];
     const int T1 = T + 1;
     int32_t* s_cnt = s_mem;
     int32_t* s_next = s_mem + T1;
-    for (int t = threadIdx.x; t < T1; t += blockDim.x) s_cnt[t] = 0;
-    __syncthreads();
-    const int i = threadIdx.x;
+    const int nthr = blockDim.x, n_warps = nthr >> 5;
+    const int rounds = (n + nthr - 1) / nthr;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int b = -1;
-    if (i < n) {
-        b = classify(ids[i], T, models);
-        if (b == T) {
-            atomicCAS(&status[ST_CODE], MT_OK, MT_ERR_BAD_MODEL_ID);
-            atomicMin(&status[ST_BAD_INDEX], i);
+    for (int t = threadIdx.x; t < T1; t += nthr) s_cnt[t] = 0;
+    __syncthreads();
+    int bucket[kSingleCtaMax / 256];            // this thread's requests, one per round (at most 16 rounds of 256)
+#pragma unroll
+    for (int r = 0; r < kSingleCtaMax / 256; ++r) {
+        bucket[r] = -1;
+        const int i = r * nthr + threadIdx.x;
+        if (r < rounds && i < n) {
+            const int b = classify(ids[i], T, models);
+            bucket[r] = b;
+            if (b == T) {
+                atomicCAS(&status[ST_CODE], MT_OK, MT_ERR_BAD_MODEL_ID);
+                atomicMin(&status[ST_BAD_INDEX], i);
+            }
+            const unsigned peers = __match_any_sync(__activemask(), b);
+            if ((__ffs(peers) - 1) == lane) atomicAdd(&s_cnt[b], __popc(peers));
         }
-        const unsigned peers = __match_any_sync(__activemask(), b);
-        if ((__ffs(peers) - 1) == lane) atomicAdd(&s_cnt[b], __popc(peers));
     }
     __syncthreads();
-    const int per = (T1 + kBucketChunk - 1) / kBucketChunk;
+    const int per = (T1 + nthr - 1) / nthr;
     const int lo = min((int)threadIdx.x * per, T1), hi = min(lo + per, T1);
     int sum = 0;
     for (int t = lo; t < hi; ++t) sum += s_cnt[t];
@@ -191,22 +232,36 @@ bucket_small(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __re
         if (threadIdx.x == 0) prefix[T] = total;
     }
     __syncthreads();
-    // warps take turns in arrival order, so positions inside a bucket ascend with the arrival index
-    for (int w = 0; w < kBucketChunk / 32; ++w) {
-        if (warp == w && i < n) {
-            const unsigned peers = __match_any_sync(__activemask(), b);
-            const int rank = __popc(peers & ((1u << lane) - 1u));
-            const int pos = s_next[b] + rank;
-            __syncwarp(__activemask());
-            if (rank == 0) s_next[b] += __popc(peers);
-            perm[pos] = i;
-            inv[i] = pos;
+    // rounds in order, and inside a round the warps take turns: positions inside a bucket ascend with arrival index
+#pragma unroll
+    for (int r = 0; r < kSingleCtaMax / 256; ++r) {
+        if (r >= rounds) break;
+        const int i = r * nthr + threadIdx.x;
+        const int b = bucket[r];
+        for (int w = 0; w < n_warps; ++w) {
+            if (warp == w && i < n) {
+                const unsigned peers = __match_any_sync(__activemask(), b);
+                const int rank = __popc(peers & ((1u << lane) - 1u));
+                const int pos = s_next[b] + rank;
+                __syncwarp(__activemask());
+                if (rank == 0) s_next[b] += __popc(peers);
+                perm[pos] = i;
+                inv[i] = pos;
+            }
+            __syncthreads();
         }
-        __syncthreads();
+    }
+    // work items of the dense layers (offsets and prefixes were written by this CTA: make them visible first)
+    __threadfence_block();
+    __syncthreads();
+    for (int l = 0; l < n_layers; ++l) {
+        WorkItem* out = items.v[l];
+        if (!out) continue;
+        const int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
+        const int n_items = prefix[T];
+        for (int item = threadIdx.x; item < n_items; item += nthr) out[item] = make_work_item(item, l, T, models, offsets, prefix);
     }
 }
-
-struct ItemPtrs { WorkItem* v[8]; };
 
 // Expand every dense layer's work list: item i of layer l -> (tenant, row tile, column tile) and everything the
 // executor needs to know about it.  Row tiles of one weight slab are adjacent items, so concurrent CTAs share it in L2.
@@ -219,28 +274,7 @@ __global__ void build_work_items(int T, const ModelDev* __restrict__ models, int
         const int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
         const int total = prefix[T];
         for (int item = blockIdx.x * blockDim.x + threadIdx.x; item < total; item += gridDim.x * blockDim.x) {
-            int lo = 0, hi = T;   // largest t with prefix[t] <= item
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (prefix[mid] <= item) lo = mid; else hi = mid;
-            }
-            const LayerDev& L = models[lo].layer[l];
-            const int seg0 = offsets[lo], n_t = offsets[lo + 1] - seg0;
-            const int m_tiles = (n_t + BM - 1) / BM;
-            const int local = item - prefix[lo];
-            const int n_tile = local / m_tiles, m_tile = local - n_tile * m_tiles;
-            WorkItem w;
-            w.row0 = seg0 + m_tile * BM;
-            w.rows_valid = min(BM, n_t - m_tile * BM);
-            w.n_tile = n_tile;
-            w.k_blocks = L.k_blocks;
-            w.w = L.w;
-            w.bias = L.bias;
-            w.N = L.N;
-            w.relu = L.relu;
-            w.t = lo;
-            w.pad = 0;
-            out[item] = w;
+            out[item] = make_work_item(item, l, T, models, offsets, prefix);
         }
     }
 }
@@ -314,10 +348,12 @@ void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
     ItemPtrs ip;
     bool any = false;
     for (int l = 0; l < 8; ++l) { ip.v[l] = a.items[l]; any = any || a.items[l]; }
-    if (n_blocks == 1 && a.T + 1 <= 4096) {
-        bucket_small<<<1, kBucketChunk, 2 * smem, s>>>(a.ids, a.n, a.T, a.models, a.n_layers, a.rows_per_unit, tn, a.counts,
-                                                     a.offsets, a.tile_prefix, a.perm, a.inv, a.status);
-        if (any) build_work_items<<<a.item_grid, 256, 0, s>>>(a.T, a.models, a.n_layers, tn, a.offsets, a.tile_prefix, ip);
+    // measured: one CTA wins up to a few hundred requests; beyond that its serial scatter and the item expansion
+    // by a single CTA cost more than the extra launches of the multi-CTA path
+    if (a.n <= 512 && a.T + 1 <= 4096) {
+        const int threads = (a.n <= 256) ? 256 : 1024;
+        bucket_single_cta<<<1, threads, 2 * smem, s>>>(a.ids, a.n, a.T, a.models, a.n_layers, a.rows_per_unit, tn, a.counts,
+                                                      a.offsets, a.tile_prefix, a.perm, a.inv, ip, a.status);
         return;
     }
     bucket_block_hist<<<n_blocks, kBucketChunk, smem, s>>>(a.ids, a.n, a.T, a.models, a.block_hist, a.status);
