@@ -5,11 +5,12 @@
 // weights (Sec. 4: "model weights are unique"), the launch walks a device-built list of
 // (tenant, row tile, column tile) work items instead of one GEMM.
 //
-// CTA = 6 warps: warp 0 issues TMA loads (activation tile through a tensor map, weight tile as one 16 KiB
-// bulk copy of a pre-swizzled image), warp 1 issues tcgen05.mma into one of two TMEM accumulators, warps
+// CTA = 6 warps: warp 0 issues TMA loads (activation tile through a tensor map, each 128-row weight tile as one
+// 16 KiB bulk copy of a pre-swizzled image), warp 1 issues tcgen05.mma into one of two TMEM accumulators, warps
 // 2..5 drain the other accumulator (tcgen05.ld -> bias -> ReLU -> convert -> 128-bit stores), so the
 // epilogue of tile i overlaps the main loop of tile i+1.  Rows of a tile beyond the tenant's segment are
-// computed on whatever follows in memory and never stored (rows of a GEMM are independent).
+// computed on whatever follows in memory and never stored (rows of a GEMM are independent).  The work list is
+// an array of 48-byte records expanded on the device after bucketing; CTA b takes items b, b + grid, ...
 #include "mt_device.cuh"
 #include "mt_host.h"
 

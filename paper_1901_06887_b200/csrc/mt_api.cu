@@ -32,8 +32,8 @@ struct HostModel {
     void* dev_block = nullptr;
 };
 
-enum KernelId { K_HIST = 0, K_SCAN, K_SCATTER, K_GATHER, K_GEMM, K_CONV, K_POOL, K_UNPERMUTE, K_COUNT };
-const char* const kKernelNames[K_COUNT] = {"bucket_block_hist+scan+scatter", "", "", "gather_rows",
+enum KernelId { K_BUCKET = 0, K_GATHER, K_GEMM, K_CONV, K_POOL, K_UNPERMUTE, K_COUNT };
+const char* const kKernelNames[K_COUNT] = {"bucketing (histogram, scans, scatter, work items)", "gather_rows",
                                            "grouped_gemm", "grouped_conv3x3", "pool_finalize", "unpermute_rows"};
 
 struct TimedLaunch {
@@ -62,7 +62,7 @@ struct Ctx {
     int cap_n = 0;
     bool ws_dirty = true;
     int32_t *d_block_hist = nullptr, *d_counts = nullptr, *d_offsets = nullptr, *d_tile_prefix = nullptr,
-            *d_tmp = nullptr, *d_perm = nullptr, *d_inv = nullptr, *d_status = nullptr;
+            *d_perm = nullptr, *d_inv = nullptr, *d_status = nullptr;
     void* act[MT_MAX_LAYERS + 1] = {nullptr};
     int act_ld[MT_MAX_LAYERS + 1] = {0};
     CUtensorMap act_map[MT_MAX_LAYERS + 1];
@@ -122,7 +122,6 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     CU_OK(cudaMalloc(&g.d_status, sizeof(int32_t) * ST_WORDS));
     CU_OK(cudaMalloc(&g.d_counts, sizeof(int32_t) * (size_t)(max_models + 1)));
     CU_OK(cudaMalloc(&g.d_offsets, sizeof(int32_t) * (size_t)(max_models + 2)));
-    CU_OK(cudaMalloc(&g.d_tmp, sizeof(int32_t) * (size_t)(max_models + 1)));
     CU_OK(cudaMalloc(&g.d_tile_prefix, sizeof(int32_t) * (size_t)MT_MAX_LAYERS * (max_models + 1)));
     CU_OK(cudaMemset(g.d_offsets, 0, sizeof(int32_t) * (size_t)(max_models + 2)));
     mt_status st = reset_status_word();
@@ -343,13 +342,13 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
         if (f.kind == MT_CONV3X3) tiles_per_image = g.conv.strips_per_image;
 
     {
-        Timer t(K_HIST, s);
+        Timer t(K_BUCKET, s);
         BucketArgs a;
         a.ids = ids; a.n = n; a.T = g.T; a.models = g.d_models; a.n_layers = L; a.rows_per_unit = tiles_per_image;
         for (int l = 0; l < 8; ++l) { a.tile_n[l] = g.tile_n[l]; a.items[l] = (l < MT_MAX_LAYERS) ? g.d_items[l] : nullptr; }
         a.item_grid = g.sm_count * 2;
         a.block_hist = g.d_block_hist; a.counts = g.d_counts; a.offsets = g.d_offsets; a.tile_prefix = g.d_tile_prefix;
-        a.tmp = g.d_tmp; a.perm = g.d_perm; a.inv = g.d_inv; a.status = g.d_status;
+        a.perm = g.d_perm; a.inv = g.d_inv; a.status = g.d_status;
         launch_bucketing(a, s);
     }
     CUtensorMap in_map;
@@ -366,7 +365,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
         if (f.kind == MT_DENSE) {
             Timer t(K_GEMM, s);
             GemmArgs a;
-            a.models = g.d_models; a.layer = l; a.T = g.T; a.offsets = g.d_offsets;
+            a.T = g.T;
             a.tile_prefix = g.d_tile_prefix + (size_t)l * (g.T + 1);
             a.items = g.d_items[l];
             a.out = last ? (void*)g.d_out_b : g.act[l + 1];
@@ -428,7 +427,6 @@ mt_status mt_shutdown(void) {
     cudaFree(g.d_status); g.d_status = nullptr;
     cudaFree(g.d_counts); g.d_counts = nullptr;
     cudaFree(g.d_offsets); g.d_offsets = nullptr;
-    cudaFree(g.d_tmp); g.d_tmp = nullptr;
     cudaFree(g.d_tile_prefix); g.d_tile_prefix = nullptr;
     cudaFree(g.st_in); g.st_in = nullptr;
     cudaFree(g.st_ids); g.st_ids = nullptr;

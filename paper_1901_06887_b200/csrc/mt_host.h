@@ -24,7 +24,6 @@ struct BucketArgs {
     int32_t* counts;          // [T + 1]
     int32_t* offsets;         // [T + 2]
     int32_t* tile_prefix;     // [n_layers][T + 1]
-    int32_t* tmp;             // [T + 1]
     int32_t* perm;            // [n]
     int32_t* inv;             // [n]
     int item_grid;            // CTAs of the work-item expansion kernel
@@ -47,12 +46,9 @@ void launch_pretile_dense(const uint16_t* w, int N, int K, uint16_t* out, cudaSt
 void launch_pretile_conv(const uint16_t* w, int C_out, int C_in, uint16_t* out, cudaStream_t s);
 
 struct GemmArgs {
-    const ModelDev* models;
-    int layer;
     int T;
-    const int32_t* offsets;       // [T + 2]
-    const int32_t* tile_prefix;   // [T + 1] of this layer
-    const WorkItem* items;        // [tile_prefix[T]] work items of this layer
+    const int32_t* tile_prefix;   // [T + 1] of this layer; tile_prefix[T] = number of work items
+    const WorkItem* items;        // the layer's work items
     void* out;                    // bf16 or fp32, rows in bucketed order
     int ld_out;                   // elements between output rows
     int out_fp32;
