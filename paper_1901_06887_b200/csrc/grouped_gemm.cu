@@ -40,7 +40,13 @@ __device__ __forceinline__ WorkItem load_item(const WorkItem* items, int idx) {
 
 template <int TN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmArgs p) {
+grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_a32,
+                    const GemmArgs p) {
+    // Segments of at most kSwapRows requests are computed transposed ("swap-AB"): the 128-row weight tile is the
+    // M operand and the requests are the N operand (32 or 64 columns), so only 4 or 8 KiB of activations are
+    // fetched per stage instead of a 16 KiB tile that is mostly other tenants' rows.  128-column items only.
+    constexpr bool kSwapOk = (TN == 128);
+    constexpr int kSwapRows = 64;
     constexpr int kStages = GemmCfg<TN>::kStages;
     constexpr int kStageBytes = GemmCfg<TN>::kStageBytes;
     constexpr int kAccCols = GemmCfg<TN>::kAccCols;
@@ -66,6 +72,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmArgs p
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tmap_a);
+        if (kSwapOk) prefetch_tensormap(&tmap_a32);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_slot), kTmemCols);
@@ -88,13 +95,21 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmArgs p
                 WorkItem nxt = {};
                 if (item + (int)gridDim.x < total) nxt = load_item(p.items, item + gridDim.x);   // in flight during this item
                 const int kblocks = cur.k_blocks;
+                const bool swap = kSwapOk && cur.rows_valid <= kSwapRows;
+                const int nbox = (cur.rows_valid + 31) >> 5;
                 // weight tile (nt, kb) of 128 rows x 64 columns starts at element (nt * kblocks + kb) * 8192
                 const uint16_t* wsrc = cur.w + (size_t)cur.n_tile * kWTiles * kblocks * (BN * BK);
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
                     const uint32_t a_dst = base + stage * kStageBytes;
-                    mbar_expect_tx(full_bar(stage), kStageBytes);
-                    tma_load_2d(a_dst, &tmap_a, kb * BK, cur.row0, full_bar(stage));
+                    if (swap) {          // only the 32-row boxes that hold the segment's requests
+                        mbar_expect_tx(full_bar(stage), (uint32_t)(nbox * 4096 + kWTiles * TILE_BYTES));
+                        for (int b = 0; b < nbox; ++b)
+                            tma_load_2d(a_dst + b * 4096, &tmap_a32, kb * BK, cur.row0 + b * 32, full_bar(stage));
+                    } else {
+                        mbar_expect_tx(full_bar(stage), kStageBytes);
+                        tma_load_2d(a_dst, &tmap_a, kb * BK, cur.row0, full_bar(stage));
+                    }
 #pragma unroll
                     for (int wt = 0; wt < kWTiles; ++wt)
                         bulk_load(a_dst + (1 + wt) * TILE_BYTES, wsrc + ((size_t)wt * kblocks + kb) * (BN * BK),
@@ -120,10 +135,15 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmArgs p
             int stage = 0; uint32_t phase = 0;
             int it = 0;
             bool ok = true;
-            int kblocks = ((int)blockIdx.x < total) ? __ldg(&p.items[blockIdx.x].k_blocks) : 0;
+            int4 head = ((int)blockIdx.x < total) ? __ldg(reinterpret_cast<const int4*>(p.items + blockIdx.x)) : make_int4(0, 0, 0, 0);
             uint32_t ready = 0;
             for (int item = blockIdx.x; ok && item < total; item += gridDim.x, ++it) {
-                const int next_kblocks = (item + (int)gridDim.x < total) ? __ldg(&p.items[item + gridDim.x].k_blocks) : 0;
+                const int4 next_head = (item + (int)gridDim.x < total)
+                                           ? __ldg(reinterpret_cast<const int4*>(p.items + item + gridDim.x)) : make_int4(0, 0, 0, 0);
+                const int kblocks = head.w;          // (row0, rows_valid, n_tile, k_blocks)
+                const bool swap = kSwapOk && head.y <= kSwapRows;
+                // transposed items: M = 128 weight rows, N = 32 or 64 request columns
+                const uint32_t idesc_item = swap ? make_idesc_bf16(BM, ((head.y + 31) >> 5) * 32) : idesc;
                 const int acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
                 if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, 2)) break;
@@ -134,21 +154,23 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmArgs p
                     const int next_stage = (stage + 1 == kStages) ? 0 : stage + 1;
                     const uint32_t next_phase = (stage + 1 == kStages) ? (phase ^ 1u) : phase;
                     const uint32_t poll = mbar_test_wait(full_bar(next_stage), next_phase);   // consumed after the MMAs
-                    const uint32_t a_lo = a_lo0 + stage * kStageLo, b_lo = b_lo0 + stage * kStageLo;
+                    // first operand region of the stage = activations, second = weights; swapped items swap the roles
+                    const uint32_t act_lo = a_lo0 + stage * kStageLo, w_lo = b_lo0 + stage * kStageLo;
+                    const uint32_t a_lo = swap ? w_lo : act_lo, b_lo = swap ? act_lo : w_lo;
                     // advancing K by 16 elements = 32 bytes inside the swizzle row: +2 in the address field
                     if (leader) {
-                        if (kb == 0) umma_bf16_lohi<false>(d_tmem, a_lo, b_lo, idesc);
-                        else umma_bf16_lohi<true>(d_tmem, a_lo, b_lo, idesc);
-                        umma_bf16_lohi<true>(d_tmem, a_lo + 2, b_lo + 2, idesc);
-                        umma_bf16_lohi<true>(d_tmem, a_lo + 4, b_lo + 4, idesc);
-                        umma_bf16_lohi<true>(d_tmem, a_lo + 6, b_lo + 6, idesc);
+                        if (kb == 0) umma_bf16_lohi<false>(d_tmem, a_lo, b_lo, idesc_item);
+                        else umma_bf16_lohi<true>(d_tmem, a_lo, b_lo, idesc_item);
+                        umma_bf16_lohi<true>(d_tmem, a_lo + 2, b_lo + 2, idesc_item);
+                        umma_bf16_lohi<true>(d_tmem, a_lo + 4, b_lo + 4, idesc_item);
+                        umma_bf16_lohi<true>(d_tmem, a_lo + 6, b_lo + 6, idesc_item);
                         umma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
                     }
                     stage = next_stage; phase = next_phase;
                     ready = poll;
                 }
                 if (ok && leader) umma_commit(tfull_bar(acc));
-                kblocks = next_kblocks;
+                head = next_head;
             }
         }
     } else {               // ---------------------------------------------------- epilogue (warps 2..5)
@@ -166,9 +188,41 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmArgs p
             const uint32_t acc_phase = (it >> 1) & 1;
             if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 4)) break;
             tc_fence_after();
+            const int N = c.N, relu = c.relu;
+            if (kSwapOk && c.rows_valid <= kSwapRows) {
+                // Transposed item: this thread owns output feature f, the accumulator columns are the requests.
+                // For one request the 32 lanes of a warp write 32 neighbouring features: a 64- or 128-byte run.
+                const int f = c.n_tile * TN + r;
+                const bool f_ok = f < N;
+                const float bias_f = f_ok ? __ldg(c.bias + f) : 0.0f;
+                const int nbox = (c.rows_valid + 31) >> 5;
+                for (int b = 0; b < nbox; ++b) {
+                    uint32_t v[32];
+                    __syncwarp();
+                    tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccCols + b * 32, v);
+                    tmem_ld_wait();
+                    if (f_ok) {
+                        const int n_req = min(32, c.rows_valid - b * 32);
+                        const size_t row_b = (size_t)(c.row0 + b * 32);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (j < n_req) {
+                                float val = __uint_as_float(v[j]) + bias_f;
+                                if (relu) val = fmaxf(val, 0.0f);
+                                if (p.out_fp32) reinterpret_cast<float*>(p.out)[(row_b + j) * p.ld_out + f] = val;
+                                else reinterpret_cast<uint16_t*>(p.out)[(row_b + j) * p.ld_out + f] =
+                                         static_cast<uint16_t>(pack_bf16x2(val, 0.0f) & 0xFFFFu);
+                            }
+                        }
+                    }
+                }
+                __syncwarp();
+                tc_fence_before();
+                mbar_arrive(tempty_bar(acc));
+                continue;
+            }
             const bool row_ok = r < c.rows_valid;
             const size_t grow = (size_t)(c.row0 + r);
-            const int N = c.N, relu = c.relu;
 #pragma unroll 1
             for (int ch = 0; ch < TN / 32; ++ch) {
                 uint32_t v[32];
@@ -276,9 +330,10 @@ cudaError_t configure_grouped_gemm() {
                                 GemmCfg<256>::kSmem);
 }
 
-void launch_grouped_gemm(const CUtensorMap& tmap_a, const GemmArgs& a, int tile_n, int sm_count, cudaStream_t s) {
-    if (tile_n == 256) grouped_gemm_kernel<256><<<sm_count, kGemmThreads, GemmCfg<256>::kSmem, s>>>(tmap_a, a);
-    else grouped_gemm_kernel<128><<<sm_count, kGemmThreads, GemmCfg<128>::kSmem, s>>>(tmap_a, a);
+void launch_grouped_gemm(const CUtensorMap& tmap_a, const CUtensorMap& tmap_a32, const GemmArgs& a, int tile_n,
+                         int sm_count, cudaStream_t s) {
+    if (tile_n == 256) grouped_gemm_kernel<256><<<sm_count, kGemmThreads, GemmCfg<256>::kSmem, s>>>(tmap_a, tmap_a32, a);
+    else grouped_gemm_kernel<128><<<sm_count, kGemmThreads, GemmCfg<128>::kSmem, s>>>(tmap_a, tmap_a32, a);
 }
 
 }  // namespace mt

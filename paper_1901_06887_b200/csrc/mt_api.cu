@@ -66,6 +66,7 @@ struct Ctx {
     void* act[MT_MAX_LAYERS + 1] = {nullptr};
     int act_ld[MT_MAX_LAYERS + 1] = {0};
     CUtensorMap act_map[MT_MAX_LAYERS + 1];
+    CUtensorMap act_map32[MT_MAX_LAYERS + 1];   // dense inputs again, as 32-row boxes
     float* d_out_b = nullptr;
     float* d_pool_partial = nullptr;     // per-strip channel sums of a conv layer that feeds a pool
     WorkItem* d_items[MT_MAX_LAYERS] = {nullptr};   // per dense layer
@@ -153,10 +154,10 @@ void free_workspace() {
     g.cap_n = 0;
 }
 
-mt_status encode_2d(CUtensorMap* map, void* ptr, int ld, int rows) {
+mt_status encode_2d(CUtensorMap* map, void* ptr, int ld, int rows, int box_rows = BM) {
     cuuint64_t dims[2] = {(cuuint64_t)ld, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-    cuuint32_t box[2] = {BK, BM};
+    cuuint32_t box[2] = {BK, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = g.encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ptr, dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -195,6 +196,8 @@ mt_status ensure_workspace(int n) {
             CU_OK(cudaMalloc(&g.act[b], bytes));
             CU_OK(cudaMemset(g.act[b], 0, bytes));
             mt_status st = encode_2d(&g.act_map[b], g.act[b], g.act_ld[b], cap);
+            if (st != MT_OK) return st;
+            st = encode_2d(&g.act_map32[b], g.act[b], g.act_ld[b], cap, 32);
             if (st != MT_OK) return st;
         } else {
             g.act_ld[b] = f.in_ch * f.h * f.w;
@@ -372,7 +375,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             a.ld_out = last ? g.out_elems : g.act_ld[l + 1];
             a.out_fp32 = last ? 1 : 0;
             a.status = g.d_status;
-            launch_grouped_gemm(g.act_map[l], a, g.tile_n[l], g.sm_count, s);
+            launch_grouped_gemm(g.act_map[l], g.act_map32[l], a, g.tile_n[l], g.sm_count, s);
         } else if (f.kind == MT_CONV3X3) {
             Timer t(K_CONV, s);
             ConvArgs a;

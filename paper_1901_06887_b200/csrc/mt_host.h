@@ -56,7 +56,9 @@ struct GemmArgs {
 };
 cudaError_t configure_grouped_gemm();
 // tile_n: 128 or 256 output columns per work item; must match BucketArgs::tile_n of that layer.
-void launch_grouped_gemm(const CUtensorMap& tmap_a, const GemmArgs& a, int tile_n, int sm_count, cudaStream_t s);
+// tmap_a: 128-row boxes of the layer's input; tmap_a32: 32-row boxes of the same buffer (transposed small items).
+void launch_grouped_gemm(const CUtensorMap& tmap_a, const CUtensorMap& tmap_a32, const GemmArgs& a, int tile_n,
+                         int sm_count, cudaStream_t s);
 
 // Strip geometry of the conv executor (see grouped_conv.cu).
 struct ConvPlan {
