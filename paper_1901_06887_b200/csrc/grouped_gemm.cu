@@ -44,8 +44,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                     const GemmArgs p) {
     // Segments of at most kSwapRows requests are computed transposed ("swap-AB"): the 128-row weight tile is the
     // M operand and the requests are the N operand (32 or 64 columns), so only 4 or 8 KiB of activations are
-    // fetched per stage instead of a 16 KiB tile that is mostly other tenants' rows.  128-column items only.
-    constexpr bool kSwapOk = (TN == 128);
+    // fetched per stage instead of a 16 KiB tile that is mostly other tenants' rows.  A 256-column item has two
+    // weight tiles, hence two transposed accumulators, 64 TMEM columns apart.
+    constexpr bool kSwapOk = true;
     constexpr int kSwapRows = 64;
     constexpr int kStages = GemmCfg<TN>::kStages;
     constexpr int kStageBytes = GemmCfg<TN>::kStageBytes;
@@ -156,14 +157,25 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                     const uint32_t poll = mbar_test_wait(full_bar(next_stage), next_phase);   // consumed after the MMAs
                     // first operand region of the stage = activations, second = weights; swapped items swap the roles
                     const uint32_t act_lo = a_lo0 + stage * kStageLo, w_lo = b_lo0 + stage * kStageLo;
-                    const uint32_t a_lo = swap ? w_lo : act_lo, b_lo = swap ? act_lo : w_lo;
                     // advancing K by 16 elements = 32 bytes inside the swizzle row: +2 in the address field
                     if (leader) {
-                        if (kb == 0) umma_bf16_lohi<false>(d_tmem, a_lo, b_lo, idesc_item);
-                        else umma_bf16_lohi<true>(d_tmem, a_lo, b_lo, idesc_item);
-                        umma_bf16_lohi<true>(d_tmem, a_lo + 2, b_lo + 2, idesc_item);
-                        umma_bf16_lohi<true>(d_tmem, a_lo + 4, b_lo + 4, idesc_item);
-                        umma_bf16_lohi<true>(d_tmem, a_lo + 6, b_lo + 6, idesc_item);
+                        if (swap) {
+#pragma unroll
+                            for (int wt = 0; wt < kWTiles; ++wt) {
+                                const uint32_t d = d_tmem + wt * kSwapRows, wa = w_lo + wt * (TILE_BYTES >> 4);
+                                if (kb == 0) umma_bf16_lohi<false>(d, wa, act_lo, idesc_item);
+                                else umma_bf16_lohi<true>(d, wa, act_lo, idesc_item);
+                                umma_bf16_lohi<true>(d, wa + 2, act_lo + 2, idesc_item);
+                                umma_bf16_lohi<true>(d, wa + 4, act_lo + 4, idesc_item);
+                                umma_bf16_lohi<true>(d, wa + 6, act_lo + 6, idesc_item);
+                            }
+                        } else {
+                            if (kb == 0) umma_bf16_lohi<false>(d_tmem, act_lo, w_lo, idesc_item);
+                            else umma_bf16_lohi<true>(d_tmem, act_lo, w_lo, idesc_item);
+                            umma_bf16_lohi<true>(d_tmem, act_lo + 2, w_lo + 2, idesc_item);
+                            umma_bf16_lohi<true>(d_tmem, act_lo + 4, w_lo + 4, idesc_item);
+                            umma_bf16_lohi<true>(d_tmem, act_lo + 6, w_lo + 6, idesc_item);
+                        }
                         umma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
                     }
                     stage = next_stage; phase = next_phase;
@@ -192,26 +204,29 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             if (kSwapOk && c.rows_valid <= kSwapRows) {
                 // Transposed item: this thread owns output feature f, the accumulator columns are the requests.
                 // For one request the 32 lanes of a warp write 32 neighbouring features: a 64- or 128-byte run.
-                const int f = c.n_tile * TN + r;
-                const bool f_ok = f < N;
-                const float bias_f = f_ok ? __ldg(c.bias + f) : 0.0f;
                 const int nbox = (c.rows_valid + 31) >> 5;
-                for (int b = 0; b < nbox; ++b) {
-                    uint32_t v[32];
-                    __syncwarp();
-                    tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccCols + b * 32, v);
-                    tmem_ld_wait();
-                    if (f_ok) {
-                        const int n_req = min(32, c.rows_valid - b * 32);
-                        const size_t row_b = (size_t)(c.row0 + b * 32);
+#pragma unroll 1
+                for (int wt = 0; wt < kWTiles; ++wt) {
+                    const int f = c.n_tile * TN + wt * BN + r;
+                    const bool f_ok = f < N;
+                    const float bias_f = f_ok ? __ldg(c.bias + f) : 0.0f;
+                    for (int b = 0; b < nbox; ++b) {
+                        uint32_t v[32];
+                        __syncwarp();
+                        tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccCols + wt * kSwapRows + b * 32, v);
+                        tmem_ld_wait();
+                        if (f_ok) {
+                            const int n_req = min(32, c.rows_valid - b * 32);
+                            const size_t row_b = (size_t)(c.row0 + b * 32);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (j < n_req) {
-                                float val = __uint_as_float(v[j]) + bias_f;
-                                if (relu) val = fmaxf(val, 0.0f);
-                                if (p.out_fp32) reinterpret_cast<float*>(p.out)[(row_b + j) * p.ld_out + f] = val;
-                                else reinterpret_cast<uint16_t*>(p.out)[(row_b + j) * p.ld_out + f] =
-                                         static_cast<uint16_t>(pack_bf16x2(val, 0.0f) & 0xFFFFu);
+                            for (int j = 0; j < 32; ++j) {
+                                if (j < n_req) {
+                                    float val = __uint_as_float(v[j]) + bias_f;
+                                    if (relu) val = fmaxf(val, 0.0f);
+                                    if (p.out_fp32) reinterpret_cast<float*>(p.out)[(row_b + j) * p.ld_out + f] = val;
+                                    else reinterpret_cast<uint16_t*>(p.out)[(row_b + j) * p.ld_out + f] =
+                                             static_cast<uint16_t>(pack_bf16x2(val, 0.0f) & 0xFFFFu);
+                                }
                             }
                         }
                     }
