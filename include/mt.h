@@ -117,6 +117,12 @@ const char* mt_status_string(mt_status s);
 mt_status mt_debug_last_bucketing(int32_t* counts_host, int32_t* offsets_host, int32_t* perm_host,
                                   int32_t* inv_host, int32_t* n_tenants_out);
 
+/* Test hook for the bounded device-side waits (the executors never spin forever on a barrier: after a time limit
+ * they give up, report MT_ERR_TIMEOUT and tear down normally, so a lost signal cannot hang the GPU).  Enqueues a
+ * one-thread kernel that waits, for at most limit_ms (1..1000) milliseconds, on a barrier that nothing completes.
+ * Afterwards mt_get_async_status reports MT_ERR_TIMEOUT and the context stays usable. */
+mt_status mt_debug_wait_timeout(int32_t limit_ms, void* stream);
+
 /* Per-kernel device timing.  enable = 1: every kernel launch of mt_infer is bracketed by CUDA events on the
  * caller's stream; enable = 2: only the grouped layer executors (dense / conv) are; 0: off.
  * mt_get_kernel_times synchronises those events, then fills up to `cap`

@@ -31,6 +31,8 @@ __device__ __forceinline__ int classify(int id, int T, const ModelDev* models) {
 __global__ void __launch_bounds__(kBucketChunk)
 bucket_block_hist(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models,
                   int32_t* __restrict__ block_hist, int32_t* __restrict__ status) {
+    pdl_launch_dependents();
+    pdl_wait();
     extern __shared__ int32_t s_hist[];   // T + 1
     const int T1 = T + 1;
     for (int t = threadIdx.x; t < T1; t += blockDim.x) s_hist[t] = 0;
@@ -111,6 +113,8 @@ __device__ __forceinline__ void column_scan(int t, int n_blocks, int T1, int32_t
 // Many tenants x many blocks: the per-tenant scans over blocks run as a grid of warps.
 __global__ void __launch_bounds__(256)
 bucket_column_scan(int n_blocks, int T, int32_t* __restrict__ block_hist, int32_t* __restrict__ counts) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (t < T + 1) column_scan(t, n_blocks, T + 1, block_hist, counts);
 }
@@ -121,6 +125,8 @@ __global__ void __launch_bounds__(kScanThreads)
 bucket_scan(int n_blocks, int T, const ModelDev* __restrict__ models, int n_layers, int rows_per_unit, LayerTileN tn,
             int do_columns, int32_t* __restrict__ block_hist, int32_t* __restrict__ counts,
             int32_t* __restrict__ offsets, int32_t* __restrict__ tile_prefix) {
+    pdl_launch_dependents();
+    pdl_wait();
     __shared__ int32_t s_warp[33];
     const int T1 = T + 1;
     if (do_columns) {
@@ -187,6 +193,8 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
                   int rows_per_unit, LayerTileN tn, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
                   int32_t* __restrict__ tile_prefix, int32_t* __restrict__ perm, int32_t* __restrict__ inv,
                   ItemPtrs items, int32_t* __restrict__ status) {
+    pdl_launch_dependents();
+    pdl_wait();
     extern __shared__ int32_t s_mem[];          // s_cnt[T + 1], s_next[T + 1]
     __shared__ int32_t s_warp[33];
     const int T1 = T + 1;
@@ -268,6 +276,8 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
 __global__ void build_work_items(int T, const ModelDev* __restrict__ models, int n_layers, LayerTileN tn,
                                  const int32_t* __restrict__ offsets, const int32_t* __restrict__ tile_prefix,
                                  ItemPtrs items) {
+    pdl_launch_dependents();
+    pdl_wait();
     for (int l = 0; l < n_layers; ++l) {
         WorkItem* out = items.v[l];
         if (!out) continue;
@@ -283,6 +293,8 @@ __global__ void __launch_bounds__(kBucketChunk)
 bucket_scatter(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models,
                const int32_t* __restrict__ block_hist, const int32_t* __restrict__ offsets,
                int32_t* __restrict__ perm, int32_t* __restrict__ inv) {
+    pdl_launch_dependents();
+    pdl_wait();
     extern __shared__ int32_t s_next[];   // next free position of every bucket for this block
     const int T1 = T + 1;
     for (int t = threadIdx.x; t < T1; t += blockDim.x)
@@ -309,6 +321,8 @@ bucket_scatter(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __
 // X_b[j, :] = X[perm[j], :]; rows of `row_vec` 16-byte vectors; dst rows `dst_ld_vec` vectors apart.
 __global__ void gather_rows(const uint4* __restrict__ src, const int32_t* __restrict__ perm, int n, int row_vec,
                             uint4* __restrict__ dst, int dst_ld_vec) {
+    pdl_launch_dependents();
+    pdl_wait();
     const long long total = (long long)n * row_vec;
     for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
          idx += (long long)gridDim.x * blockDim.x) {
@@ -322,6 +336,8 @@ template <typename V>
 __global__ void unpermute_rows(const V* __restrict__ src, const int32_t* __restrict__ perm,
                                const int32_t* __restrict__ offsets, int T, int n, int row_vec,
                                V* __restrict__ dst, V nan_v) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int n_valid = offsets[T];
     const long long total = (long long)n * row_vec;
     for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
@@ -329,6 +345,24 @@ __global__ void unpermute_rows(const V* __restrict__ src, const int32_t* __restr
         const int j = (int)(idx / row_vec), v = (int)(idx % row_vec);
         dst[(size_t)perm[j] * row_vec + v] = (j < n_valid) ? src[idx] : nan_v;
     }
+}
+
+// Self-test of the bounded wait every executor relies on: one thread waits on an mbarrier that nobody ever
+// completes; after limit_ns it must give up, raise the abort flag and report MT_ERR_TIMEOUT - and return.
+__global__ void wait_timeout_probe(int32_t* status, unsigned long long limit_ns, int32_t* gave_up) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        fence_mbar_init();
+        const bool done = mbar_wait(smem_u32(&bar), 0, &abort_flag, status, 99, limit_ns);
+        *gave_up = done ? 0 : 1;
+    }
+}
+
+void launch_wait_timeout_probe(int32_t* status, unsigned long long limit_ns, int32_t* gave_up, cudaStream_t s) {
+    wait_timeout_probe<<<1, 32, 0, s>>>(status, limit_ns, gave_up);
 }
 
 // ------------------------------------------------------------------------------------------ launchers
@@ -352,26 +386,26 @@ void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
     // by a single CTA cost more than the extra launches of the multi-CTA path
     if (a.n <= 512 && a.T + 1 <= 4096) {
         const int threads = (a.n <= 256) ? 256 : 1024;
-        bucket_single_cta<<<1, threads, 2 * smem, s>>>(a.ids, a.n, a.T, a.models, a.n_layers, a.rows_per_unit, tn, a.counts,
+        launch_pdl(bucket_single_cta, dim3(1), dim3(threads), 2 * smem, s, a.ids, a.n, a.T, a.models, a.n_layers, a.rows_per_unit, tn, a.counts,
                                                       a.offsets, a.tile_prefix, a.perm, a.inv, ip, a.status);
         return;
     }
-    bucket_block_hist<<<n_blocks, kBucketChunk, smem, s>>>(a.ids, a.n, a.T, a.models, a.block_hist, a.status);
+    launch_pdl(bucket_block_hist, dim3(n_blocks), dim3(kBucketChunk), smem, s, a.ids, a.n, a.T, a.models, a.block_hist, a.status);
     // few buckets x few blocks: the per-tenant scans over blocks ride along in the single-CTA scan kernel
     const int col_iters = ((a.T + 1 + 31) / 32) * ((n_blocks + 31) / 32);
     const int fused = col_iters <= 4;
-    if (!fused) bucket_column_scan<<<(a.T + 1 + 7) / 8, 256, 0, s>>>(n_blocks, a.T, a.block_hist, a.counts);
-    bucket_scan<<<1, kScanThreads, 0, s>>>(n_blocks, a.T, a.models, a.n_layers, a.rows_per_unit, tn, fused, a.block_hist,
+    if (!fused) launch_pdl(bucket_column_scan, dim3((a.T + 1 + 7) / 8), dim3(256), 0, s, n_blocks, a.T, a.block_hist, a.counts);
+    launch_pdl(bucket_scan, dim3(1), dim3(kScanThreads), 0, s, n_blocks, a.T, a.models, a.n_layers, a.rows_per_unit, tn, fused, a.block_hist,
                                            a.counts, a.offsets, a.tile_prefix);
-    bucket_scatter<<<n_blocks, kBucketChunk, smem, s>>>(a.ids, a.n, a.T, a.models, a.block_hist, a.offsets, a.perm,
+    launch_pdl(bucket_scatter, dim3(n_blocks), dim3(kBucketChunk), smem, s, a.ids, a.n, a.T, a.models, a.block_hist, a.offsets, a.perm,
                                                         a.inv);
-    if (any) build_work_items<<<a.item_grid, 256, 0, s>>>(a.T, a.models, a.n_layers, tn, a.offsets, a.tile_prefix, ip);
+    if (any) launch_pdl(build_work_items, dim3(a.item_grid), dim3(256), 0, s, a.T, a.models, a.n_layers, tn, a.offsets, a.tile_prefix, ip);
 }
 
 void launch_gather_rows(const void* src, const int32_t* perm, int n, int row_bytes, void* dst, int dst_ld_bytes,
                         int sm_count, cudaStream_t s) {
     const int row_vec = row_bytes / 16;
-    gather_rows<<<grid_for((long long)n * row_vec, 256, sm_count), 256, 0, s>>>(
+    launch_pdl(gather_rows, dim3(grid_for((long long)n * row_vec, 256, sm_count)), dim3(256), 0, s,
         (const uint4*)src, perm, n, row_vec, (uint4*)dst, dst_ld_bytes / 16);
 }
 
@@ -381,10 +415,10 @@ void launch_unpermute(const float* src, const int32_t* perm, const int32_t* offs
     const bool vec_ok = (out_elems % 4 == 0) && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0);
     if (vec_ok) {
         const int row_vec = out_elems / 4;
-        unpermute_rows<float4><<<grid_for((long long)n * row_vec, 256, sm_count), 256, 0, s>>>(
+        launch_pdl(unpermute_rows<float4>, dim3(grid_for((long long)n * row_vec, 256, sm_count)), dim3(256), 0, s,
             (const float4*)src, perm, offsets, T, n, row_vec, (float4*)dst, make_float4(qnan, qnan, qnan, qnan));
     } else {
-        unpermute_rows<float><<<grid_for((long long)n * out_elems, 256, sm_count), 256, 0, s>>>(
+        launch_pdl(unpermute_rows<float>, dim3(grid_for((long long)n * out_elems, 256, sm_count)), dim3(256), 0, s,
             src, perm, offsets, T, n, out_elems, dst, qnan);
     }
 }

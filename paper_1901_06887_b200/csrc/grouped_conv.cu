@@ -75,6 +75,7 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
     int4* s_rec = reinterpret_cast<int4*>(bar_ptr + 512);             // kRecords x 16 bytes
     float* s_pool = reinterpret_cast<float*>(bar_ptr + 1024);         // 8 warps x 32 channel sums (fused pooling)
 
+    pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(sfull_bar(s), 1); mbar_init(sempty_bar(s), 1); }
@@ -98,6 +99,7 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    pdl_wait();   // everything above overlapped the previous kernel's tail; its results are needed from here on
     // contiguous range of strips for this CTA
     const int total = p.tile_prefix[p.T];
     const int s_begin = (int)(((long long)total * blockIdx.x) / gridDim.x);
@@ -430,6 +432,8 @@ void launch_pretile_conv(const uint16_t* w, int C_out, int C_in, uint16_t* out, 
 // g[j][c] = (1 / HW) * sum over the image's strips of pool_partial[j][strip][c] (fixed order), rounded to bf16.
 __global__ void pool_finalize_kernel(const float* __restrict__ partial, int n, int strips, int C, float inv_hw,
                                      uint16_t* __restrict__ out, int ld_out) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= n * C) return;
     const int j = idx / C, c = idx - j * C;
@@ -440,7 +444,7 @@ __global__ void pool_finalize_kernel(const float* __restrict__ partial, int n, i
 
 void launch_pool_finalize(const float* partial, int n, int strips, int C, int HW, uint16_t* out, int ld_out,
                           cudaStream_t s) {
-    pool_finalize_kernel<<<(n * C + 255) / 256, 256, 0, s>>>(partial, n, strips, C, 1.0f / (float)HW, out, ld_out);
+    launch_pdl(pool_finalize_kernel, dim3((n * C + 255) / 256), dim3(256), 0, s, partial, n, strips, C, 1.0f / (float)HW, out, ld_out);
 }
 
 cudaError_t configure_grouped_conv() {
@@ -448,7 +452,7 @@ cudaError_t configure_grouped_conv() {
 }
 
 void launch_grouped_conv(const CUtensorMap& tmap_x, const ConvArgs& a, int smem_bytes, int sm_count, cudaStream_t s) {
-    grouped_conv3x3_kernel<<<sm_count, kConvThreads, smem_bytes, s>>>(tmap_x, a);
+    launch_pdl(grouped_conv3x3_kernel, dim3(sm_count), dim3(kConvThreads), (size_t)smem_bytes, s, tmap_x, a);
 }
 
 }  // namespace mt

@@ -66,6 +66,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
+    pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -84,6 +85,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    pdl_wait();   // everything above overlapped the previous kernel's tail; its results are needed from here on
     const int total = p.tile_prefix[p.T];
 
     if (warp == 0) {
@@ -347,8 +349,8 @@ cudaError_t configure_grouped_gemm() {
 
 void launch_grouped_gemm(const CUtensorMap& tmap_a, const CUtensorMap& tmap_a32, const GemmArgs& a, int tile_n,
                          int sm_count, cudaStream_t s) {
-    if (tile_n == 256) grouped_gemm_kernel<256><<<sm_count, kGemmThreads, GemmCfg<256>::kSmem, s>>>(tmap_a, tmap_a32, a);
-    else grouped_gemm_kernel<128><<<sm_count, kGemmThreads, GemmCfg<128>::kSmem, s>>>(tmap_a, tmap_a32, a);
+    if (tile_n == 256) launch_pdl(grouped_gemm_kernel<256>, dim3(sm_count), dim3(kGemmThreads), GemmCfg<256>::kSmem, s, tmap_a, tmap_a32, a);
+    else launch_pdl(grouped_gemm_kernel<128>, dim3(sm_count), dim3(kGemmThreads), GemmCfg<128>::kSmem, s, tmap_a, tmap_a32, a);
 }
 
 }  // namespace mt

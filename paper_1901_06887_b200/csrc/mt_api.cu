@@ -643,6 +643,17 @@ mt_status mt_debug_last_bucketing(int32_t* counts_host, int32_t* offsets_host, i
     return MT_OK;
 }
 
+mt_status mt_debug_wait_timeout(int32_t limit_ms, void* stream) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g.init) return MT_ERR_NOT_INIT;
+    if (limit_ms < 1 || limit_ms > 1000) return MT_ERR_INVALID_ARG;
+    CU_OK(cudaSetDevice(g.device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    launch_wait_timeout_probe(g.d_status, (unsigned long long)limit_ms * 1000000ull, g.d_status + 3, s);
+    CU_OK(cudaGetLastError());
+    return MT_OK;
+}
+
 mt_status mt_set_kernel_timing(int32_t enable) {
     std::lock_guard<std::mutex> lk(g_mu);
     g.timing = enable < 0 ? 0 : (enable > 2 ? 1 : enable);

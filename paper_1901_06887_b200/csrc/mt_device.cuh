@@ -125,7 +125,7 @@ __device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s; a whole layer takes milliseconds
 
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status, int where) {
+                                          int* status, int where, uint64_t limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     uint32_t it = 0;
@@ -133,7 +133,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((++it & 0x3FF) == 0) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            if (global_timer_ns() - t0 > limit_ns) {
                 *abort_flag = 1;
                 if (atomicCAS(&status[ST_CODE], MT_OK, MT_ERR_TIMEOUT) == MT_OK) status[ST_WHERE] = where;
                 return false;
@@ -177,6 +177,12 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
+
+// Programmatic dependent launch: every kernel of the path is launched with the stream-serialization attribute, lets
+// its successor start early (launch_dependents) and waits for its predecessor's results (wait) only after its own
+// set-up, so launch latency and prologues (barrier init, TMEM allocation) hide behind the predecessor's tail.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // One lane of a fully converged warp (the same one every time).
 __device__ __forceinline__ bool elect_one() {

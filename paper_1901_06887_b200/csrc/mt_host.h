@@ -7,6 +7,19 @@
 
 namespace mt {
 
+// Launch with programmatic stream serialization: the kernel may start while its predecessor in the stream is
+// still draining; it must call pdl_wait() before it touches anything the predecessor wrote or still reads.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 struct ModelDev;
 struct WorkItem;
 
@@ -32,6 +45,8 @@ struct BucketArgs {
 };
 
 void launch_bucketing(const BucketArgs& a, cudaStream_t s);
+// One thread waits (bounded by limit_ns) on a barrier nobody completes; *gave_up = 1 and the status word is set.
+void launch_wait_timeout_probe(int32_t* status, unsigned long long limit_ns, int32_t* gave_up, cudaStream_t s);
 void launch_gather_rows(const void* src, const int32_t* perm, int n, int row_bytes, void* dst, int dst_ld_bytes,
                         int sm_count, cudaStream_t s);
 void launch_unpermute(const float* src, const int32_t* perm, const int32_t* offsets, int T, int n, int out_elems,

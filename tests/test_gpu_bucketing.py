@@ -90,3 +90,16 @@ def test_rejected_ids_give_nan_rows_and_a_status():
     # the freed slot is re-issued, lowest first
     assert mt.mt_register_model(passthrough_models(4)[3]) == 3
     run_ids(T, [3, 3, 0])
+
+
+def test_bounded_device_wait_gives_up_and_context_survives():
+    # a wait that nothing satisfies runs into its time limit: status MT_ERR_TIMEOUT, no hang, no trap, and the
+    # next batch runs normally
+    fresh()
+    harness.register_models(passthrough_models(3))
+    run_ids(3, [0, 1, 2, 1])
+    mt.mt_debug_wait_timeout(20)
+    st, bad = mt.mt_get_async_status()
+    assert st == 8 and bad == -1                      # MT_ERR_TIMEOUT
+    assert mt.mt_get_async_status() == (0, -1)        # cleared by the read
+    run_ids(3, [2, 2, 0])
