@@ -140,16 +140,20 @@ def gemm_roofline(wl, kernel_ms_per_launch_sum, peaks, peaks_kind, config):
     counts = np.bincount(wl.model_ids, minlength=len(wl.models))
     byts = sum(b for b, k in zip(per_layer_bytes, kinds) if k == dom_kind)
     flops = sum(int(c) * sum(synth.layer_flops(l) for l in m if l.kind == dom_kind) for c, m in zip(counts, wl.models))
+    # tensor peak: the kernel is timed inside a seconds-long loop (power cap active), so the sustained cuBLAS
+    # figure is the matching denominator; the burst figure is reported beside it
+    tc_peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
     t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
-    t_tc = flops / (peaks["bf16_tflops"] * 1e12)
+    t_tc = flops / (tc_peak * 1e12)
     sec = kernel_ms_per_launch_sum * 1e-3
     if t_hbm >= t_tc:
         ach = byts / sec / 1e9 if sec > 0 else 0.0
         roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"]}
     else:
         ach = flops / sec / 1e12 if sec > 0 else 0.0
-        roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": ach / peaks["bf16_tflops"]}
+        roof = {"bound": "tensor", "achieved": ach, "peak": tc_peak, "unit": "TFLOP/s", "frac": ach / tc_peak,
+                "peak_kind": "sustained (kernel timed inside a long loop)", "burst_peak": peaks["bf16_tflops"],
+                "frac_of_burst_peak": ach / peaks["bf16_tflops"]}
     traffic = None
     if config in TRAFFIC_RATIO:
         traffic = int(TRAFFIC_RATIO[config] * byts)
@@ -335,7 +339,8 @@ def main():
         roof = gemm_roofline(wl, dom_ms, peaks, peaks_kind, cfg)
         flops = synth.workload_flops(wl.models, wl.model_ids)
         bytes_all = synth.workload_bytes(wl.models, wl.model_ids)
-        t_roof = max(flops / (peaks["bf16_tflops"] * 1e12), bytes_all / (peaks["hbm_gbs"] * 1e9))
+        t_roof = max(flops / (peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12),
+                     bytes_all / (peaks["hbm_gbs"] * 1e9))
         line = result_line(units, ms, args.steps, n_gpus=world, steps=args.steps, warmup=args.warmup, scaling="weak",
                            vs_baseline=None, dtype="bf16", data="synthetic")
         line["config"] = {"workload": synth.CONFIG_NAMES[cfg], "requests_per_step_per_gpu": n, "tenants": len(models),

@@ -20,7 +20,7 @@ namespace mt {
 
 constexpr int kScanThreads = 1024;
 
-struct LayerTileN { int v[8]; };
+struct LayerTileN { int v[8]; int m[8]; };   // per layer: columns (v) and rows (m) of one dense work item
 
 // ids outside [0, T) or of dead models go to the extra bucket T, so they sort behind every live segment.
 __device__ __forceinline__ int classify(int id, int T, const ModelDev* models) {
@@ -82,10 +82,11 @@ __device__ __forceinline__ int cta_excl_scan(int v, int32_t* s_warp, int* total)
 }
 
 // Work units (tiles / strips) tenant t contributes to layer l, given its request count c.
-__device__ __forceinline__ int layer_units(const ModelDev* models, int t, int l, int c, int rows_per_unit, int tile_n) {
+__device__ __forceinline__ int layer_units(const ModelDev* models, int t, int l, int c, int rows_per_unit, int tile_n,
+                                           int tile_m) {
     if (c <= 0) return 0;
     const LayerDev& L = models[t].layer[l];
-    if (L.kind == MT_DENSE) return ((c + BM - 1) / BM) * ((L.N + tile_n - 1) / tile_n);
+    if (L.kind == MT_DENSE) return ((c + tile_m - 1) / tile_m) * ((L.N + tile_n - 1) / tile_n);
     if (L.kind == MT_CONV3X3) return c * rows_per_unit;
     return 0;
 }
@@ -146,9 +147,9 @@ bucket_scan(int n_blocks, int T, const ModelDev* __restrict__ models, int n_laye
         int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
         const int hi_t = min(hi, T);           // the extra bucket of rejected ids contributes no work
         int usum = 0;
-        for (int t = lo; t < hi_t; ++t) usum += layer_units(models, t, l, counts[t], rows_per_unit, tn.v[l]);
+        for (int t = lo; t < hi_t; ++t) usum += layer_units(models, t, l, counts[t], rows_per_unit, tn.v[l], tn.m[l]);
         int urun = cta_excl_scan(usum, s_warp, &total);
-        for (int t = lo; t < hi_t; ++t) { prefix[t] = urun; urun += layer_units(models, t, l, counts[t], rows_per_unit, tn.v[l]); }
+        for (int t = lo; t < hi_t; ++t) { prefix[t] = urun; urun += layer_units(models, t, l, counts[t], rows_per_unit, tn.v[l], tn.m[l]); }
         if (threadIdx.x == 0) prefix[T] = total;
     }
 }
@@ -158,7 +159,7 @@ struct ItemPtrs { WorkItem* v[8]; };
 // Work item `item` of dense layer l: (tenant, row tile, column tile) and what the executor needs to know about it.
 __device__ __forceinline__ WorkItem make_work_item(int item, int l, int T, const ModelDev* __restrict__ models,
                                                    const int32_t* __restrict__ offsets,
-                                                   const int32_t* __restrict__ prefix) {
+                                                   const int32_t* __restrict__ prefix, int tile_m) {
     int lo = 0, hi = T;   // largest t with prefix[t] <= item
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
@@ -166,12 +167,12 @@ __device__ __forceinline__ WorkItem make_work_item(int item, int l, int T, const
     }
     const LayerDev& L = models[lo].layer[l];
     const int seg0 = offsets[lo], n_t = offsets[lo + 1] - seg0;
-    const int m_tiles = (n_t + BM - 1) / BM;
+    const int m_tiles = (n_t + tile_m - 1) / tile_m;
     const int local = item - prefix[lo];
     const int n_tile = local / m_tiles, m_tile = local - n_tile * m_tiles;
     WorkItem w;
-    w.row0 = seg0 + m_tile * BM;
-    w.rows_valid = min(BM, n_t - m_tile * BM);
+    w.row0 = seg0 + m_tile * tile_m;
+    w.rows_valid = min(tile_m, n_t - m_tile * tile_m);
     w.n_tile = n_tile;
     w.k_blocks = L.k_blocks;
     w.w = L.w;
@@ -234,9 +235,9 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
         int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
         const int hi_t = min(hi, T);
         int usum = 0;
-        for (int t = lo; t < hi_t; ++t) usum += layer_units(models, t, l, s_cnt[t], rows_per_unit, tn.v[l]);
+        for (int t = lo; t < hi_t; ++t) usum += layer_units(models, t, l, s_cnt[t], rows_per_unit, tn.v[l], tn.m[l]);
         int urun = cta_excl_scan(usum, s_warp, &total);
-        for (int t = lo; t < hi_t; ++t) { prefix[t] = urun; urun += layer_units(models, t, l, s_cnt[t], rows_per_unit, tn.v[l]); }
+        for (int t = lo; t < hi_t; ++t) { prefix[t] = urun; urun += layer_units(models, t, l, s_cnt[t], rows_per_unit, tn.v[l], tn.m[l]); }
         if (threadIdx.x == 0) prefix[T] = total;
     }
     __syncthreads();
@@ -267,7 +268,7 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
         if (!out) continue;
         const int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
         const int n_items = prefix[T];
-        for (int item = threadIdx.x; item < n_items; item += nthr) out[item] = make_work_item(item, l, T, models, offsets, prefix);
+        for (int item = threadIdx.x; item < n_items; item += nthr) out[item] = make_work_item(item, l, T, models, offsets, prefix, tn.m[l]);
     }
 }
 
@@ -284,7 +285,7 @@ __global__ void build_work_items(int T, const ModelDev* __restrict__ models, int
         const int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
         const int total = prefix[T];
         for (int item = blockIdx.x * blockDim.x + threadIdx.x; item < total; item += gridDim.x * blockDim.x) {
-            out[item] = make_work_item(item, l, T, models, offsets, prefix);
+            out[item] = make_work_item(item, l, T, models, offsets, prefix, tn.m[l]);
         }
     }
 }
@@ -378,7 +379,7 @@ void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
     const int n_blocks = (a.n + kBucketChunk - 1) / kBucketChunk;
     const size_t smem = sizeof(int32_t) * (size_t)(a.T + 1);
     LayerTileN tn;
-    for (int l = 0; l < 8; ++l) tn.v[l] = a.tile_n[l] > 0 ? a.tile_n[l] : BN;
+    for (int l = 0; l < 8; ++l) { tn.v[l] = a.tile_n[l] > 0 ? a.tile_n[l] : BN; tn.m[l] = a.tile_m[l] > 0 ? a.tile_m[l] : BM; }
     ItemPtrs ip;
     bool any = false;
     for (int l = 0; l < 8; ++l) { ip.v[l] = a.items[l]; any = any || a.items[l]; }

@@ -142,6 +142,28 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// Same contract as mbar_wait, but polling with the non-blocking test_wait: for barriers that are completed from
+// ANOTHER CTA of the cluster (remote arrives, multicast commits).  A thread parked in try_wait was seen to wake up
+// only at the end of its suspend interval when the completing arrival came from the peer CTA.
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                               int where, uint32_t backoff_ns = 0) {
+    if (mbar_test_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    uint32_t it = 0;
+    while (true) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if (backoff_ns) __nanosleep(backoff_ns);
+        if ((++it & 0x3FF) == 0) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                if (atomicCAS(&status[ST_CODE], MT_OK, MT_ERR_TIMEOUT) == MT_OK) status[ST_WHERE] = where;
+                return false;
+            }
+        }
+    }
+}
+
 // Wait used only during an aborted tear-down: gives in-flight copies a short, bounded time to land.
 __device__ __forceinline__ void mbar_wait_short(uint32_t bar, uint32_t parity) {
     const uint64_t t0 = global_timer_ns();

@@ -33,6 +33,7 @@ struct BucketArgs {
     int n_layers;
     int rows_per_unit;        // conv: tiles per image
     int tile_n[8];            // dense: output columns per work item of each layer (128 or 256)
+    int tile_m[8];            // dense: rows per work item of each layer (128, or 256 for the CTA-pair executor)
     int32_t* block_hist;      // [ceil(n / kBucketChunk)][T + 1]
     int32_t* counts;          // [T + 1]
     int32_t* offsets;         // [T + 2]
@@ -64,6 +65,8 @@ struct GemmArgs {
     int T;
     const int32_t* tile_prefix;   // [T + 1] of this layer; tile_prefix[T] = number of work items
     const WorkItem* items;        // the layer's work items
+    const CUtensorMap* wmaps;     // [model][MT_MAX_LAYERS] tensor maps of the tiled dense weights (CTA-pair executor)
+    int layer;
     void* out;                    // bf16 or fp32, rows in bucketed order
     int ld_out;                   // elements between output rows
     int out_fp32;
@@ -74,6 +77,10 @@ cudaError_t configure_grouped_gemm();
 // tmap_a: 128-row boxes of the layer's input; tmap_a32: 32-row boxes of the same buffer (transposed small items).
 void launch_grouped_gemm(const CUtensorMap& tmap_a, const CUtensorMap& tmap_a32, const GemmArgs& a, int tile_n,
                          int sm_count, cudaStream_t s);
+
+// CTA-pair form (grouped_gemm_pair.cu): work items of 256 rows x 256 columns (BucketArgs::tile_m = tile_n = 256).
+cudaError_t configure_grouped_gemm_pair();
+cudaError_t launch_grouped_gemm_pair(const CUtensorMap& tmap_a, const GemmArgs& a, int sm_count, cudaStream_t s);
 
 // Strip geometry of the conv executor (see grouped_conv.cu).
 struct ConvPlan {

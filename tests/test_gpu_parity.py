@@ -76,6 +76,19 @@ def test_config5_reduced():
     run_and_check(wl.models, wl.model_ids, wl.inputs)
 
 
+@pytest.mark.parametrize("n,tenants,widths", [(2500, 2, (256, 512, 256)), (3100, 3, (128, 768, 10)), (1024, 1, (64, 256, 256))])
+def test_cta_pair_executor(n, tenants, widths, monkeypatch):
+    # MT_PAIR=1, >= 1024 requests per tenant on average and layers >= 256 wide: the 256 x 256 CTA-pair executor runs
+    # those layers (ragged last row tiles, tiles whose second half is empty, bf16 and fp32 outputs); the result must
+    # also equal the one-CTA executor's bit for bit (same products, same accumulation order per output)
+    wl = synth.make_workload(5, n=n, n_tenants=tenants, widths=widths)
+    monkeypatch.setenv("MT_PAIR", "1")
+    got_pair, _ = run_and_check(wl.models, wl.model_ids, wl.inputs)
+    monkeypatch.delenv("MT_PAIR")
+    got_one, _ = run_and_check(wl.models, wl.model_ids, wl.inputs)
+    assert np.array_equal(got_pair, got_one)
+
+
 @pytest.mark.parametrize("h,w", [(8, 8), (5, 7), (56, 56), (3, 126), (17, 20)])
 def test_config4_reduced_geometries(h, w):
     wl = synth.make_workload(4, n=7, n_tenants=3, h=h, w=w, n_conv=2)
