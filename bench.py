@@ -273,11 +273,13 @@ def main():
     torch.cuda.synchronize()
     if not args.profile:
         sampler.start()
+    launches_before = mt.mt_debug_launch_count()
     e0.record(stream)
     for i in range(args.steps):
         step(i)
     e1.record(stream)
     torch.cuda.synchronize()
+    launches = mt.mt_debug_launch_count() - launches_before      # kernels the library enqueued in the timed region
     if world > 1:
         dist.barrier()
     clocks = sampler.stop()
@@ -330,13 +332,11 @@ def main():
     if rank == 0:
         peaks, peaks_kind = load_peaks()
         per_kernel = {name: {"ms_per_step": t / bd_steps, "launches_per_step": c / bd_steps} for name, t, c in breakdown}
-        # launches per step: the bucketing entry covers 1 (batch of at most 512 requests) or 5 kernels under one pair of events
-        bucket_kernels = 1 if n <= 512 else 5
-        per_step = sum(c / bd_steps for nm, _, c in breakdown if not nm.startswith("bucket")) + bucket_kernels
-        launches = int(round(per_step * args.steps))
-        dom = "grouped_conv3x3" if cfg == 4 else "grouped_gemm"
-        dom_ms = dict((nm, t / args.steps) for nm, t, c in kernel_times).get(dom, 0.0)
+        timed = dict((nm, t / args.steps) for nm, t, c in kernel_times)
+        dom = "grouped_conv3x3" if cfg == 4 else ("fused_mlp" if "fused_mlp" in timed else "grouped_gemm")
+        dom_ms = timed.get(dom, 0.0)
         roof = gemm_roofline(wl, dom_ms, peaks, peaks_kind, cfg)
+        roof["kernel"] = dom
         flops = synth.workload_flops(wl.models, wl.model_ids)
         bytes_all = synth.workload_bytes(wl.models, wl.model_ids)
         t_roof = max(flops / (peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12),
@@ -354,7 +354,7 @@ def main():
                                        "flops_per_step": int(flops), "algorithmic_bytes_per_step": int(bytes_all)}
         line["roofline"] = roof
         line["kernels"] = per_kernel
-        line["gpu_launches"] = launches
+        line["gpu_launches"] = int(launches)
         line["e2e"] = dict(result_line(e2e_units, e2e_ms, e2e_steps), steps=e2e_steps,
                            h2d_bytes_per_step=int(n * wl.in_elems * 2 + n * 4), d2h_bytes_per_step=int(n * out_elems * 4))
         for k in ("metric", "higher_is_better"):

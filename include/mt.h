@@ -86,7 +86,8 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
  *   outputs   device, fp32, [n][out_elems], arrival order
  *   stream    cudaStream_t (NULL = default stream)
  * Only enqueues work on `stream`: bucketing (histogram, exclusive scan, stable scatter, row gather), one
- * persistent grouped launch per layer, un-permute.  No host<->device synchronisation happens unless the
+ * persistent grouped launch per layer (the last one writes its rows straight back in arrival order).  A batch
+ * of at most 512 requests against dense layers at most 256 wide runs as ONE launch that does all of it.  No host<->device synchronisation happens unless the
  * workspace must grow (n larger than any earlier call, or a wider model registered since): then the
  * call synchronises the device and reallocates first - make one call at the largest n before timing.
  * inputs must be 16-byte aligned.  n == 0 is a no-op.
@@ -122,6 +123,10 @@ mt_status mt_debug_last_bucketing(int32_t* counts_host, int32_t* offsets_host, i
  * one-thread kernel that waits, for at most limit_ms (1..1000) milliseconds, on a barrier that nothing completes.
  * Afterwards mt_get_async_status reports MT_ERR_TIMEOUT and the context stays usable. */
 mt_status mt_debug_wait_timeout(int32_t limit_ms, void* stream);
+
+/* Test / bench hook: *count_out = number of kernels this library has enqueued on behalf of mt_infer and
+ * mt_infer_host since it was loaded (registration and the no-allocation call are not counted). */
+mt_status mt_debug_launch_count(int64_t* count_out);
 
 /* Per-kernel device timing.  enable = 1: every kernel launch of mt_infer is bracketed by CUDA events on the
  * caller's stream; enable = 2: only the grouped layer executors (dense / conv) are; 0: off.

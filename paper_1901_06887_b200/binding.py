@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "MT_OK", 1: "MT_ERR_INVALID_ARG", 2: "MT_ERR_BAD_MODEL_ID", 3
 
 EXPORTS = ["mt_init", "mt_shutdown", "mt_register_model", "mt_infer", "mt_infer_host", "mt_release",
            "mt_get_async_status", "mt_status_string", "mt_debug_last_bucketing", "mt_set_kernel_timing",
-           "mt_get_kernel_times", "mt_bucket_noalloc", "mt_debug_wait_timeout"]
+           "mt_get_kernel_times", "mt_bucket_noalloc", "mt_debug_wait_timeout", "mt_debug_launch_count"]
 
 
 class MtError(RuntimeError):
@@ -63,6 +63,7 @@ def lib() -> ctypes.CDLL:
                                           ctypes.POINTER(i32), i32, ctypes.POINTER(i32)]
         l.mt_bucket_noalloc.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
         l.mt_debug_wait_timeout.argtypes = [i32, vp]
+        l.mt_debug_launch_count.argtypes = [ctypes.POINTER(ctypes.c_int64)]
         for name in EXPORTS:
             if name != "mt_status_string":
                 getattr(l, name).restype = ctypes.c_int
@@ -156,6 +157,13 @@ def mt_debug_last_bucketing(n: int):
 def mt_debug_wait_timeout(limit_ms: int = 20, stream=None) -> None:
     """Enqueue the bounded-wait self-test (a wait nothing satisfies); mt_get_async_status then reports MT_ERR_TIMEOUT."""
     _check(lib().mt_debug_wait_timeout(int(limit_ms), _stream_handle(stream)), "mt_debug_wait_timeout")
+
+
+def mt_debug_launch_count() -> int:
+    """Kernels enqueued by mt_infer / mt_infer_host since the library was loaded."""
+    c = ctypes.c_int64(0)
+    _check(lib().mt_debug_launch_count(ctypes.byref(c)), "mt_debug_launch_count")
+    return int(c.value)
 
 
 def mt_set_kernel_timing(enable) -> None:

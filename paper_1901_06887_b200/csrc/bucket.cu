@@ -5,12 +5,14 @@
 // The paper (Sec. 3) has a worker receive requests for many tenants' models; grouping them by model is a
 // pure re-ordering, made unique by stability: inside a segment, requests keep their arrival order.
 //
-//   pass 1  bucket_block_hist   per-block histogram of ids (warp-level match + one shared atomic per group)
-//   pass 2  bucket_scan         per-tenant exclusive scan over blocks, exclusive scan over tenants
-//                               (offsets), per-layer tile prefix sums for the grouped executors
-//   pass 3  bucket_scatter      stable position of every request -> perm / inv
-//           gather_rows         X_b[j, :] = X[perm[j], :]          (128-bit copies)
-//           unpermute_rows      out[perm[j], :] = out_b[j, :]      (128-bit copies where rows allow)
+//   pass 1  bucket_hist_scan       per-block histogram of ids (warp-level match + one shared atomic per group); the
+//                                  CTA that finishes last scans per tenant over the blocks and over the tenants
+//                                  (offsets) and builds the per-layer unit prefix sums for the grouped executors
+//   pass 2  bucket_scatter_expand  stable position of every request -> perm / inv, payload rows moved into
+//                                  bucketed order (128-bit copies), work items of the dense layers
+//           bucket_single_cta      both passes in one CTA for batches of at most 512 requests
+//           gather_rows            X_b[j, :] = X[perm[j], :] as a pass of its own (payloads too large for pass 2)
+//           unpermute_rows         out[perm[j], :] = out_b[j, :] (executors that cannot write arrival order themselves)
 #include <limits>
 
 #include "mt_device.cuh"
@@ -18,7 +20,6 @@
 
 namespace mt {
 
-constexpr int kScanThreads = 1024;
 
 struct LayerTileN { int v[8]; int m[8]; };   // per layer: columns (v) and rows (m) of one dense work item
 
@@ -26,29 +27,6 @@ struct LayerTileN { int v[8]; int m[8]; };   // per layer: columns (v) and rows 
 __device__ __forceinline__ int classify(int id, int T, const ModelDev* models) {
     if (id < 0 || id >= T) return T;
     return models[id].alive ? id : T;
-}
-
-__global__ void __launch_bounds__(kBucketChunk)
-bucket_block_hist(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models,
-                  int32_t* __restrict__ block_hist, int32_t* __restrict__ status) {
-    pdl_launch_dependents();
-    pdl_wait();
-    extern __shared__ int32_t s_hist[];   // T + 1
-    const int T1 = T + 1;
-    for (int t = threadIdx.x; t < T1; t += blockDim.x) s_hist[t] = 0;
-    __syncthreads();
-    const int i = blockIdx.x * kBucketChunk + threadIdx.x;
-    if (i < n) {
-        const int b = classify(ids[i], T, models);
-        if (b == T) {
-            atomicCAS(&status[ST_CODE], MT_OK, MT_ERR_BAD_MODEL_ID);
-            atomicMin(&status[ST_BAD_INDEX], i);
-        }
-        const unsigned peers = __match_any_sync(__activemask(), b);
-        if ((__ffs(peers) - 1) == (threadIdx.x & 31)) atomicAdd(&s_hist[b], __popc(peers));
-    }
-    __syncthreads();
-    for (int t = threadIdx.x; t < T1; t += blockDim.x) block_hist[(size_t)blockIdx.x * T1 + t] = s_hist[t];
 }
 
 // Exclusive scan across the threads of a CTA (any multiple of 32 threads up to 1024): returns the sum of `v` over
@@ -91,51 +69,13 @@ __device__ __forceinline__ int layer_units(const ModelDev* models, int t, int l,
     return 0;
 }
 
-// Per bucket t (one warp each): counts[t] = sum over blocks, block_hist[b][t] <- exclusive prefix over blocks.
-__device__ __forceinline__ void column_scan(int t, int n_blocks, int T1, int32_t* __restrict__ block_hist,
-                                            int32_t* __restrict__ counts) {
-    const int lane = threadIdx.x & 31;
-    int carry = 0;
-    for (int b0 = 0; b0 < n_blocks; b0 += 32) {
-        const int b = b0 + lane;
-        const int v = (b < n_blocks) ? block_hist[(size_t)b * T1 + t] : 0;
-        int incl = v;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const int u = __shfl_up_sync(0xffffffffu, incl, d);
-            if (lane >= d) incl += u;
-        }
-        if (b < n_blocks) block_hist[(size_t)b * T1 + t] = carry + incl - v;
-        carry += __shfl_sync(0xffffffffu, incl, 31);
-    }
-    if (lane == 0) counts[t] = carry;
-}
-
-// Many tenants x many blocks: the per-tenant scans over blocks run as a grid of warps.
-__global__ void __launch_bounds__(256)
-bucket_column_scan(int n_blocks, int T, int32_t* __restrict__ block_hist, int32_t* __restrict__ counts) {
-    pdl_launch_dependents();
-    pdl_wait();
-    const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (t < T + 1) column_scan(t, n_blocks, T + 1, block_hist, counts);
-}
-
-// One CTA: (optionally the per-tenant scans over blocks,) offsets = exclusive scan of counts over the T + 1
-// buckets (offsets[T + 1] = n), and per layer the prefix sums of the work units each tenant contributes.
-__global__ void __launch_bounds__(kScanThreads)
-bucket_scan(int n_blocks, int T, const ModelDev* __restrict__ models, int n_layers, int rows_per_unit, LayerTileN tn,
-            int do_columns, int32_t* __restrict__ block_hist, int32_t* __restrict__ counts,
-            int32_t* __restrict__ offsets, int32_t* __restrict__ tile_prefix) {
-    pdl_launch_dependents();
-    pdl_wait();
-    __shared__ int32_t s_warp[33];
+// Offsets (exclusive scan of counts over the T + 1 buckets, offsets[T + 1] = n) and, per layer, the prefix sums of
+// the work units each tenant contributes.  Run by one CTA of any multiple of 32 threads; counts[] must be visible.
+__device__ __forceinline__ void scan_buckets(int T, const ModelDev* __restrict__ models, int n_layers, int rows_per_unit,
+                                             const LayerTileN& tn, const int32_t* counts, int32_t* __restrict__ offsets,
+                                             int32_t* __restrict__ tile_prefix, int32_t* s_warp) {
     const int T1 = T + 1;
-    if (do_columns) {
-        for (int t = threadIdx.x >> 5; t < T1; t += kScanThreads / 32) column_scan(t, n_blocks, T1, block_hist, counts);
-        __syncthreads();
-    }
-    // each thread owns `per` consecutive buckets
-    const int per = (T1 + kScanThreads - 1) / kScanThreads;
+    const int per = (T1 + (int)blockDim.x - 1) / (int)blockDim.x;     // each thread owns `per` consecutive buckets
     const int lo = min((int)threadIdx.x * per, T1), hi = min(lo + per, T1);
     int sum = 0;
     for (int t = lo; t < hi; ++t) sum += counts[t];
@@ -143,15 +83,92 @@ bucket_scan(int n_blocks, int T, const ModelDev* __restrict__ models, int n_laye
     int run = cta_excl_scan(sum, s_warp, &total);
     for (int t = lo; t < hi; ++t) { offsets[t] = run; run += counts[t]; }
     if (threadIdx.x == 0) offsets[T1] = total;
+    const int hi_t = min(hi, T);               // the extra bucket of rejected ids contributes no work
+    if (per == 1) {
+        // one bucket per thread (the usual case): the units of all layers first, so that the loads from the tenant
+        // table are in flight together instead of one round trip per layer
+        int units[MT_MAX_LAYERS];
+#pragma unroll
+        for (int l = 0; l < MT_MAX_LAYERS; ++l)
+            units[l] = (l < n_layers && lo < hi_t) ? layer_units(models, lo, l, counts[lo], rows_per_unit, tn.v[l], tn.m[l]) : 0;
+#pragma unroll
+        for (int l = 0; l < MT_MAX_LAYERS; ++l) {
+            if (l >= n_layers) break;
+            const int urun = cta_excl_scan(units[l], s_warp, &total);
+            if (lo < hi_t) tile_prefix[(size_t)l * (T + 1) + lo] = urun;
+            if (threadIdx.x == 0) tile_prefix[(size_t)l * (T + 1) + T] = total;
+        }
+        return;
+    }
     for (int l = 0; l < n_layers; ++l) {
         int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
-        const int hi_t = min(hi, T);           // the extra bucket of rejected ids contributes no work
         int usum = 0;
         for (int t = lo; t < hi_t; ++t) usum += layer_units(models, t, l, counts[t], rows_per_unit, tn.v[l], tn.m[l]);
         int urun = cta_excl_scan(usum, s_warp, &total);
         for (int t = lo; t < hi_t; ++t) { prefix[t] = urun; urun += layer_units(models, t, l, counts[t], rows_per_unit, tn.v[l], tn.m[l]); }
         if (threadIdx.x == 0) prefix[T] = total;
     }
+}
+
+// Pass 1 of a batch that needs several CTAs: per-block histogram of ids (blocks of kHistChunk requests; warp-level
+// match, one shared atomic per group of equal ids), and the CTA that finishes LAST (a ticket counter; nobody waits)
+// turns the block histograms into per-tenant exclusive prefixes over the blocks, the counts, the offsets and the
+// per-layer unit prefixes.
+__global__ void __launch_bounds__(kHistChunk)
+bucket_hist_scan(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models, int n_layers,
+                 int rows_per_unit, LayerTileN tn, int32_t* block_hist, int32_t* counts, int32_t* __restrict__ offsets,
+                 int32_t* __restrict__ tile_prefix, int32_t* ticket, int32_t* __restrict__ status) {
+    pdl_launch_dependents();
+    pdl_wait();
+    extern __shared__ int32_t s_hist[];   // T + 1
+    __shared__ int32_t s_warp[33];
+    __shared__ int s_last;
+    const int T1 = T + 1;
+    for (int t = threadIdx.x; t < T1; t += blockDim.x) s_hist[t] = 0;
+    __syncthreads();
+    const int i = blockIdx.x * kHistChunk + threadIdx.x;
+    if (i < n) {
+        const int b = classify(ids[i], T, models);
+        if (b == T) {
+            atomicCAS(&status[ST_CODE], MT_OK, MT_ERR_BAD_MODEL_ID);
+            atomicMin(&status[ST_BAD_INDEX], i);
+        }
+        const unsigned peers = __match_any_sync(__activemask(), b);
+        if ((__ffs(peers) - 1) == (threadIdx.x & 31)) atomicAdd(&s_hist[b], __popc(peers));
+    }
+    __syncthreads();
+    for (int t = threadIdx.x; t < T1; t += blockDim.x) block_hist[(size_t)blockIdx.x * T1 + t] = s_hist[t];
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int prev = atomicAdd(ticket, 1);
+        s_last = (prev == (int)gridDim.x - 1);
+        if (s_last) *ticket = 0;               // ready for the next batch
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    // per bucket (one thread each; neighbouring threads read neighbouring words): exclusive prefix over the blocks
+    const int n_blocks = gridDim.x;
+    for (int t = threadIdx.x; t < T1; t += blockDim.x) {
+        int run = 0;
+        int b = 0;
+        for (; b + 16 <= n_blocks; b += 16) {      // sixteen independent loads in flight
+            int v[16];
+#pragma unroll
+            for (int k = 0; k < 16; ++k) v[k] = __ldcg(&block_hist[(size_t)(b + k) * T1 + t]);
+#pragma unroll
+            for (int k = 0; k < 16; ++k) { block_hist[(size_t)(b + k) * T1 + t] = run; run += v[k]; }
+        }
+        for (; b < n_blocks; ++b) {
+            const int v = __ldcg(&block_hist[(size_t)b * T1 + t]);
+            block_hist[(size_t)b * T1 + t] = run;
+            run += v;
+        }
+        counts[t] = run;
+    }
+    __syncthreads();
+    scan_buckets(T, models, n_layers, rows_per_unit, tn, counts, offsets, tile_prefix, s_warp);
 }
 
 struct ItemPtrs { WorkItem* v[8]; };
@@ -272,49 +289,90 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
     }
 }
 
-// Expand every dense layer's work list: item i of layer l -> (tenant, row tile, column tile) and everything the
-// executor needs to know about it.  Row tiles of one weight slab are adjacent items, so concurrent CTAs share it in L2.
-__global__ void build_work_items(int T, const ModelDev* __restrict__ models, int n_layers, LayerTileN tn,
-                                 const int32_t* __restrict__ offsets, const int32_t* __restrict__ tile_prefix,
-                                 ItemPtrs items) {
+// Pass 2: stable position of every request (perm / inv), the move of its payload row into bucketed order
+// (X_b[pos, :] = X[i, :]: the block's source rows are contiguous, so the reads stream), and the expansion of every
+// dense layer's work list: item i of layer l -> (tenant, row tile, column tile) and everything the executor needs to
+// know about it.  Row tiles of one weight slab are adjacent items, so concurrent CTAs share the slab in L2.
+// A CTA takes kBucketChunk requests (small, so that the row move spreads over many SMs); CTAs beyond the last block
+// of requests only expand work items.
+__global__ void __launch_bounds__(kScatterThreads)
+bucket_scatter_expand(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models,
+                      const int32_t* __restrict__ block_hist, const int32_t* __restrict__ offsets,
+                      int32_t* __restrict__ perm, int32_t* __restrict__ inv, const uint4* __restrict__ rows_src,
+                      uint4* __restrict__ rows_dst, int row_vec, int dst_ld_vec, int n_layers, LayerTileN tn,
+                      const int32_t* __restrict__ tile_prefix, ItemPtrs items) {
     pdl_launch_dependents();
     pdl_wait();
+    extern __shared__ int32_t s_next[];   // T + 1: next free position of every bucket for this block; then s_pos[chunk]
+    const int T1 = T + 1;
+    int32_t* s_pos = s_next + T1;
+    const int n_blocks = (n + kBucketChunk - 1) / kBucketChunk;
+    if ((int)blockIdx.x < n_blocks) {
+        // pass 1 counted blocks of kHistChunk requests; this CTA first counts the requests of its pass-1 block that
+        // come before its own kBucketChunk
+        const int chunk0 = blockIdx.x * kBucketChunk;
+        const int hist_block = chunk0 / kHistChunk;
+        for (int t = threadIdx.x; t < T1; t += blockDim.x)
+            s_next[t] = offsets[t] + block_hist[(size_t)hist_block * T1 + t];
+        __syncthreads();
+        // (chunk0 - first id of the pass-1 block) is a multiple of kBucketChunk = 64: whole warps only
+        for (int i = hist_block * kHistChunk + threadIdx.x; i < chunk0; i += blockDim.x) {
+            const int b = classify(ids[i], T, models);
+            const unsigned peers = __match_any_sync(0xffffffffu, b);
+            if ((__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&s_next[b], __popc(peers));
+        }
+        __syncthreads();
+        const int i = chunk0 + threadIdx.x;
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        const bool mine = threadIdx.x < kBucketChunk && i < n;
+        const int b = mine ? classify(ids[i], T, models) : -1;
+        // warps take turns in arrival order, so positions inside a bucket ascend with the arrival index
+        for (int w = 0; w < kBucketChunk / 32; ++w) {
+            if (warp == w && mine) {
+                const unsigned peers = __match_any_sync(__activemask(), b);
+                const int rank = __popc(peers & ((1u << lane) - 1u));
+                const int pos = s_next[b] + rank;
+                __syncwarp(__activemask());
+                if (rank == 0) s_next[b] += __popc(peers);
+                perm[pos] = i;
+                inv[i] = pos;
+                s_pos[threadIdx.x] = pos;
+            }
+            __syncthreads();
+        }
+        if (rows_src) {
+            const int rows_here = min(kBucketChunk, n - chunk0);
+            const uint4* src = rows_src + (size_t)chunk0 * row_vec;
+            const int total = rows_here * row_vec;
+            int idx = threadIdx.x;
+            for (; idx + 3 * (int)blockDim.x < total; idx += 4 * blockDim.x) {      // four independent copies in flight
+                uint4 v[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) v[k] = __ldg(src + idx + k * blockDim.x);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int e = idx + k * blockDim.x;
+                    const int r = e / row_vec;
+                    rows_dst[(size_t)s_pos[r] * dst_ld_vec + (e - r * row_vec)] = v[k];
+                }
+            }
+            for (; idx < total; idx += blockDim.x) {
+                const int r = idx / row_vec;
+                rows_dst[(size_t)s_pos[r] * dst_ld_vec + (idx - r * row_vec)] = __ldg(src + idx);
+            }
+        }
+        __syncthreads();      // s_next is reused below
+    }
+    // work items: the layer's unit prefix sums go to shared memory first, so the search per item stays on the SM
     for (int l = 0; l < n_layers; ++l) {
         WorkItem* out = items.v[l];
         if (!out) continue;
         const int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
-        const int total = prefix[T];
-        for (int item = blockIdx.x * blockDim.x + threadIdx.x; item < total; item += gridDim.x * blockDim.x) {
-            out[item] = make_work_item(item, l, T, models, offsets, prefix, tn.m[l]);
-        }
-    }
-}
-
-__global__ void __launch_bounds__(kBucketChunk)
-bucket_scatter(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models,
-               const int32_t* __restrict__ block_hist, const int32_t* __restrict__ offsets,
-               int32_t* __restrict__ perm, int32_t* __restrict__ inv) {
-    pdl_launch_dependents();
-    pdl_wait();
-    extern __shared__ int32_t s_next[];   // next free position of every bucket for this block
-    const int T1 = T + 1;
-    for (int t = threadIdx.x; t < T1; t += blockDim.x)
-        s_next[t] = offsets[t] + block_hist[(size_t)blockIdx.x * T1 + t];
-    __syncthreads();
-    const int i = blockIdx.x * kBucketChunk + threadIdx.x;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = (i < n) ? classify(ids[i], T, models) : -1;
-    // warps take turns in arrival order, so positions inside a bucket ascend with the arrival index
-    for (int w = 0; w < kBucketChunk / 32; ++w) {
-        if (warp == w && i < n) {
-            const unsigned peers = __match_any_sync(__activemask(), b);
-            const int rank = __popc(peers & ((1u << lane) - 1u));
-            const int pos = s_next[b] + rank;
-            __syncwarp(__activemask());
-            if (rank == 0) s_next[b] += __popc(peers);
-            perm[pos] = i;
-            inv[i] = pos;
-        }
+        for (int t = threadIdx.x; t < T1; t += blockDim.x) s_next[t] = prefix[t];
+        __syncthreads();
+        const int total = s_next[T];
+        for (int item = blockIdx.x * blockDim.x + threadIdx.x; item < total; item += gridDim.x * blockDim.x)
+            out[item] = make_work_item(item, l, T, models, offsets, s_next, tn.m[l]);
         __syncthreads();
     }
 }
@@ -377,12 +435,12 @@ static int grid_for(long long total, int threads, int sm_count) {
 
 void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
     const int n_blocks = (a.n + kBucketChunk - 1) / kBucketChunk;
+    const int n_hist_blocks = (a.n + kHistChunk - 1) / kHistChunk;
     const size_t smem = sizeof(int32_t) * (size_t)(a.T + 1);
     LayerTileN tn;
     for (int l = 0; l < 8; ++l) { tn.v[l] = a.tile_n[l] > 0 ? a.tile_n[l] : BN; tn.m[l] = a.tile_m[l] > 0 ? a.tile_m[l] : BM; }
     ItemPtrs ip;
-    bool any = false;
-    for (int l = 0; l < 8; ++l) { ip.v[l] = a.items[l]; any = any || a.items[l]; }
+    for (int l = 0; l < 8; ++l) ip.v[l] = a.items[l];
     // measured: one CTA wins up to a few hundred requests; beyond that its serial scatter and the item expansion
     // by a single CTA cost more than the extra launches of the multi-CTA path
     if (a.n <= 512 && a.T + 1 <= 4096) {
@@ -391,16 +449,12 @@ void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
                                                       a.offsets, a.tile_prefix, a.perm, a.inv, ip, a.status);
         return;
     }
-    launch_pdl(bucket_block_hist, dim3(n_blocks), dim3(kBucketChunk), smem, s, a.ids, a.n, a.T, a.models, a.block_hist, a.status);
-    // few buckets x few blocks: the per-tenant scans over blocks ride along in the single-CTA scan kernel
-    const int col_iters = ((a.T + 1 + 31) / 32) * ((n_blocks + 31) / 32);
-    const int fused = col_iters <= 4;
-    if (!fused) launch_pdl(bucket_column_scan, dim3((a.T + 1 + 7) / 8), dim3(256), 0, s, n_blocks, a.T, a.block_hist, a.counts);
-    launch_pdl(bucket_scan, dim3(1), dim3(kScanThreads), 0, s, n_blocks, a.T, a.models, a.n_layers, a.rows_per_unit, tn, fused, a.block_hist,
-                                           a.counts, a.offsets, a.tile_prefix);
-    launch_pdl(bucket_scatter, dim3(n_blocks), dim3(kBucketChunk), smem, s, a.ids, a.n, a.T, a.models, a.block_hist, a.offsets, a.perm,
-                                                        a.inv);
-    if (any) launch_pdl(build_work_items, dim3(a.item_grid), dim3(256), 0, s, a.T, a.models, a.n_layers, tn, a.offsets, a.tile_prefix, ip);
+    launch_pdl(bucket_hist_scan, dim3(n_hist_blocks), dim3(kHistChunk), smem, s, a.ids, a.n, a.T, a.models, a.n_layers, a.rows_per_unit, tn,
+               a.block_hist, a.counts, a.offsets, a.tile_prefix, a.ticket, a.status);
+    const int grid2 = n_blocks > a.item_grid ? n_blocks : a.item_grid;
+    launch_pdl(bucket_scatter_expand, dim3(grid2), dim3(kScatterThreads), smem + sizeof(int32_t) * kBucketChunk, s, a.ids, a.n, a.T, a.models,
+               a.block_hist, a.offsets, a.perm, a.inv, (const uint4*)a.rows_src, (uint4*)a.rows_dst, a.row_bytes / 16,
+               a.dst_ld_bytes / 16, a.n_layers, tn, a.tile_prefix, ip);
 }
 
 void launch_gather_rows(const void* src, const int32_t* perm, int n, int row_bytes, void* dst, int dst_ld_bytes,

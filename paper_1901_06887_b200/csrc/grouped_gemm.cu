@@ -193,6 +193,16 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         int it = 0;
         WorkItem cur = {};
         if ((int)blockIdx.x < total) cur = load_item(p.items, blockIdx.x);
+        const int32_t* const perm = p.out_fp32 ? p.perm : nullptr;
+        const bool out_vec_ok = (p.ld_out & 3) == 0 && (reinterpret_cast<uintptr_t>(p.out) & 15) == 0;
+        if (perm) {
+            // requests whose id was rejected sort behind every live segment and get no work item: NaN rows
+            const int n_valid = p.offsets[p.T], n_all = p.offsets[p.T + 1];
+            for (int j = n_valid + blockIdx.x; j < n_all; j += gridDim.x) {
+                float* dst = reinterpret_cast<float*>(p.out) + (size_t)perm[j] * p.ld_out;
+                for (int e = threadIdx.x - 64; e < p.ld_out; e += 128) dst[e] = __int_as_float(0x7fc00000);
+            }
+        }
         for (int item = blockIdx.x; item < total; item += gridDim.x, ++it) {
             WorkItem nxt = {};
             if (item + (int)gridDim.x < total) nxt = load_item(p.items, item + gridDim.x);
@@ -215,20 +225,23 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                     for (int b = 0; b < nbox; ++b) {
                         uint32_t v[32];
                         __syncwarp();
+                        const int n_req = min(32, c.rows_valid - b * 32);
+                        const int row_b = c.row0 + b * 32;
+                        // output row of request j: its bucketed row, or (last layer) its arrival index - fetched by
+                        // lane j once and handed round by shuffle
+                        int my_row = row_b + lane;
+                        if (perm && lane < n_req) my_row = __ldg(perm + row_b + lane);
                         tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccCols + wt * kSwapRows + b * 32, v);
                         tmem_ld_wait();
-                        if (f_ok) {
-                            const int n_req = min(32, c.rows_valid - b * 32);
-                            const size_t row_b = (size_t)(c.row0 + b * 32);
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                if (j < n_req) {
-                                    float val = __uint_as_float(v[j]) + bias_f;
-                                    if (relu) val = fmaxf(val, 0.0f);
-                                    if (p.out_fp32) reinterpret_cast<float*>(p.out)[(row_b + j) * p.ld_out + f] = val;
-                                    else reinterpret_cast<uint16_t*>(p.out)[(row_b + j) * p.ld_out + f] =
-                                             static_cast<uint16_t>(pack_bf16x2(val, 0.0f) & 0xFFFFu);
-                                }
+                        for (int j = 0; j < 32; ++j) {
+                            const size_t orow = (size_t)__shfl_sync(0xffffffffu, my_row, j);
+                            if (f_ok && j < n_req) {
+                                float val = __uint_as_float(v[j]) + bias_f;
+                                if (relu) val = fmaxf(val, 0.0f);
+                                if (p.out_fp32) reinterpret_cast<float*>(p.out)[orow * p.ld_out + f] = val;
+                                else reinterpret_cast<uint16_t*>(p.out)[orow * p.ld_out + f] =
+                                         static_cast<uint16_t>(pack_bf16x2(val, 0.0f) & 0xFFFFu);
                             }
                         }
                     }
@@ -239,7 +252,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                 continue;
             }
             const bool row_ok = r < c.rows_valid;
-            const size_t grow = (size_t)(c.row0 + r);
+            const size_t grow = (perm && row_ok) ? (size_t)__ldg(perm + c.row0 + r) : (size_t)(c.row0 + r);
 #pragma unroll 1
             for (int ch = 0; ch < TN / 32; ++ch) {
                 uint32_t v[32];
@@ -267,7 +280,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                     // rows past the tenant's segment belong to someone else: never stored
                 } else if (p.out_fp32) {
                     float* dst = reinterpret_cast<float*>(p.out) + grow * p.ld_out + n0;
-                    if (full_chunk && (p.ld_out & 3) == 0) {
+                    if (full_chunk && out_vec_ok) {
 #pragma unroll
                         for (int j = 0; j < 8; ++j)
                             reinterpret_cast<float4*>(dst)[j] = make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);

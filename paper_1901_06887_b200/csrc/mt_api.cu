@@ -14,6 +14,10 @@
 #include "mt_device.cuh"
 #include "mt_host.h"
 
+namespace mt {
+unsigned long long g_kernel_launches = 0;
+}
+
 namespace {
 
 using namespace mt;
@@ -32,9 +36,10 @@ struct HostModel {
     void* dev_block = nullptr;
 };
 
-enum KernelId { K_BUCKET = 0, K_GATHER, K_GEMM, K_CONV, K_POOL, K_UNPERMUTE, K_COUNT };
-const char* const kKernelNames[K_COUNT] = {"bucketing (histogram, scans, scatter, work items)", "gather_rows",
-                                           "grouped_gemm", "grouped_conv3x3", "pool_finalize", "unpermute_rows"};
+enum KernelId { K_BUCKET = 0, K_GATHER, K_GEMM, K_CONV, K_POOL, K_UNPERMUTE, K_FUSED, K_COUNT };
+const char* const kKernelNames[K_COUNT] = {"bucketing (histogram, scans, scatter, row move, work items)", "gather_rows",
+                                           "grouped_gemm", "grouped_conv3x3", "pool_finalize", "unpermute_rows",
+                                           "fused_mlp"};
 
 struct TimedLaunch {
     int kernel;
@@ -63,7 +68,7 @@ struct Ctx {
     int cap_n = 0;
     bool ws_dirty = true;
     int32_t *d_block_hist = nullptr, *d_counts = nullptr, *d_offsets = nullptr, *d_tile_prefix = nullptr,
-            *d_perm = nullptr, *d_inv = nullptr, *d_status = nullptr;
+            *d_perm = nullptr, *d_inv = nullptr, *d_status = nullptr, *d_ticket = nullptr;
     void* act[MT_MAX_LAYERS + 1] = {nullptr};
     int act_ld[MT_MAX_LAYERS + 1] = {0};
     CUtensorMap act_map[MT_MAX_LAYERS + 1];
@@ -123,6 +128,8 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     CU_OK(cudaMemset(g.d_models, 0, sizeof(ModelDev) * (size_t)max_models));
     CU_OK(cudaMalloc(&g.d_wmaps, sizeof(CUtensorMap) * (size_t)max_models * MT_MAX_LAYERS));
     CU_OK(cudaMalloc(&g.d_status, sizeof(int32_t) * ST_WORDS));
+    CU_OK(cudaMalloc(&g.d_ticket, sizeof(int32_t)));
+    CU_OK(cudaMemset(g.d_ticket, 0, sizeof(int32_t)));
     CU_OK(cudaMalloc(&g.d_counts, sizeof(int32_t) * (size_t)(max_models + 1)));
     CU_OK(cudaMalloc(&g.d_offsets, sizeof(int32_t) * (size_t)(max_models + 2)));
     CU_OK(cudaMalloc(&g.d_tile_prefix, sizeof(int32_t) * (size_t)MT_MAX_LAYERS * (max_models + 1)));
@@ -137,6 +144,7 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     CU_OK(configure_grouped_gemm());
     CU_OK(configure_grouped_conv());
     CU_OK(configure_grouped_gemm_pair());
+    CU_OK(configure_fused_mlp());
     g.T = 0;
     g.live = 0;
     g.has_family = false;
@@ -199,7 +207,7 @@ mt_status ensure_workspace(int n) {
     int cap = g.cap_n > n ? g.cap_n : n;
     free_workspace();
     const int L = (int)g.family.size();
-    const size_t n_blocks = (size_t)(cap + kBucketChunk - 1) / kBucketChunk;
+    const size_t n_blocks = (size_t)(cap + kHistChunk - 1) / kHistChunk;
     CU_OK(cudaMalloc(&g.d_block_hist, sizeof(int32_t) * n_blocks * (size_t)(g.max_models + 1)));
     CU_OK(cudaMalloc(&g.d_perm, sizeof(int32_t) * (size_t)cap));
     CU_OK(cudaMalloc(&g.d_inv, sizeof(int32_t) * (size_t)cap));
@@ -326,7 +334,7 @@ struct Timer {
     bool on;
     cudaEvent_t start = nullptr, stop = nullptr;
     Timer(int k, cudaStream_t st)
-        : kernel(k), s(st), on(g.timing == 1 || (g.timing == 2 && (k == K_GEMM || k == K_CONV))) {
+        : kernel(k), s(st), on(g.timing == 1 || (g.timing == 2 && (k == K_GEMM || k == K_CONV || k == K_FUSED))) {
         if (!on) return;
         auto get = [&]() {
             cudaEvent_t e;
@@ -356,6 +364,30 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
     if (st != MT_OK) return st;
     const int L = (int)g.family.size();
     const HostLayer& f0 = g.family[0];
+    // Small batch of narrow MLPs: the whole pass in one launch (MT_FUSED=0 forces the layer-by-layer path).
+    {
+        bool all_dense = true;
+        int max_w = g.out_elems;
+        for (int l = 0; l < L; ++l) {
+            all_dense = all_dense && g.family[l].kind == MT_DENSE;
+            if (g.width[l] > max_w) max_w = g.width[l];
+        }
+        const char* fused_env = getenv("MT_FUSED");
+        if (all_dense && !(fused_env && fused_env[0] == '0') && fused_mlp_fits(n, g.T, max_w)) {
+            Timer t(K_FUSED, s);
+            FusedArgs a;
+            a.inputs = static_cast<const uint16_t*>(inputs); a.ids = ids; a.n = n; a.T = g.T; a.models = g.d_models;
+            a.n_layers = L; a.K0 = g.in_elems; a.out_elems = g.out_elems; a.out = static_cast<float*>(outputs);
+            a.counts = g.d_counts; a.offsets = g.d_offsets; a.perm = g.d_perm; a.inv = g.d_inv; a.status = g.d_status;
+            // at most one unit per request, and one per live tenant plus one per full tile
+            int grid = g.live + n / BM;
+            if (grid > n) grid = n;
+            if (grid > g.sm_count) grid = g.sm_count;
+            CU_OK(launch_fused_mlp(a, grid, s));
+            g.last_n = n;
+            return MT_OK;
+        }
+    }
     // The CTA-pair executor (256 x 256 work items, two SMs per item) fits batches whose tenants have thousands of
     // requests each; the host only knows the average, which is enough to tell that regime from the long-tail ones.
     // Under the 1 kW power cap it measured the same throughput as the one-CTA executor (at a lower clock), so it is
@@ -368,23 +400,31 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
     for (const HostLayer& f : g.family)
         if (f.kind == MT_CONV3X3) tiles_per_image = g.conv.strips_per_image;
 
+    // Dense families: the payload rows move into bucketed order inside the scatter pass when the batch is spread over
+    // enough CTAs and small enough for them; otherwise as a gather pass of its own over the whole GPU.
+    const bool rows_in_scatter = f0.kind == MT_DENSE && n > 512 && (size_t)n * g.in_elems * 2 <= ((size_t)64 << 20);
     {
         Timer t(K_BUCKET, s);
         BucketArgs a;
         a.ids = ids; a.n = n; a.T = g.T; a.models = g.d_models; a.n_layers = L; a.rows_per_unit = tiles_per_image;
+        a.ticket = g.d_ticket;
+        a.rows_src = rows_in_scatter ? inputs : nullptr; a.rows_dst = g.act[0];
+        a.row_bytes = g.in_elems * 2; a.dst_ld_bytes = g.act_ld[0] * 2;
         for (int l = 0; l < 8; ++l) {
             a.tile_n[l] = g.tile_n[l]; a.tile_m[l] = pair_mode[l] ? 2 * BM : BM;
             a.items[l] = (l < MT_MAX_LAYERS) ? g.d_items[l] : nullptr;
         }
-        a.item_grid = g.sm_count * 2;
+        a.item_grid = g.sm_count;
         a.block_hist = g.d_block_hist; a.counts = g.d_counts; a.offsets = g.d_offsets; a.tile_prefix = g.d_tile_prefix;
         a.perm = g.d_perm; a.inv = g.d_inv; a.status = g.d_status;
         launch_bucketing(a, s);
     }
     CUtensorMap in_map;
     if (f0.kind == MT_DENSE) {
-        Timer t(K_GATHER, s);
-        launch_gather_rows(inputs, g.d_perm, n, g.in_elems * 2, g.act[0], g.act_ld[0] * 2, g.sm_count, s);
+        if (!rows_in_scatter) {
+            Timer t(K_GATHER, s);
+            launch_gather_rows(inputs, g.d_perm, n, g.in_elems * 2, g.act[0], g.act_ld[0] * 2, g.sm_count, s);
+        }
     } else {
         st = encode_nhwc(&in_map, inputs, f0.in_ch, f0.w, f0.h, n, g.conv.Wp, g.conv.R + 2);
         if (st != MT_OK) return st;
@@ -399,9 +439,13 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             a.tile_prefix = g.d_tile_prefix + (size_t)l * (g.T + 1);
             a.items = g.d_items[l];
             a.wmaps = g.d_wmaps; a.layer = l;
-            a.out = last ? (void*)g.d_out_b : g.act[l + 1];
+            // the last layer of the one-CTA executor writes straight into the caller's buffer in arrival order
+            const bool direct = last && !pair_mode[l];
+            a.out = last ? (direct ? outputs : (void*)g.d_out_b) : g.act[l + 1];
             a.ld_out = last ? g.out_elems : g.act_ld[l + 1];
             a.out_fp32 = last ? 1 : 0;
+            a.perm = direct ? g.d_perm : nullptr;
+            a.offsets = g.d_offsets;
             a.status = g.d_status;
             if (pair_mode[l]) CU_OK(launch_grouped_gemm_pair(g.act_map[l], a, g.sm_count, s));
             else launch_grouped_gemm(g.act_map[l], g.act_map32[l], a, g.tile_n[l], g.sm_count, s);
@@ -428,7 +472,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
                                  (uint16_t*)g.act[l + 1], g.act_ld[l + 1], s);
         }
     }
-    {
+    if (pair_mode[L - 1]) {
         Timer t(K_UNPERMUTE, s);
         launch_unpermute(g.d_out_b, g.d_perm, g.d_offsets, g.T, n, g.out_elems, (float*)outputs, g.sm_count, s);
     }
@@ -458,6 +502,7 @@ mt_status mt_shutdown(void) {
     cudaFree(g.d_models); g.d_models = nullptr;
     cudaFree(g.d_wmaps); g.d_wmaps = nullptr;
     cudaFree(g.d_status); g.d_status = nullptr;
+    cudaFree(g.d_ticket); g.d_ticket = nullptr;
     cudaFree(g.d_counts); g.d_counts = nullptr;
     cudaFree(g.d_offsets); g.d_offsets = nullptr;
     cudaFree(g.d_tile_prefix); g.d_tile_prefix = nullptr;
@@ -690,6 +735,13 @@ mt_status mt_debug_wait_timeout(int32_t limit_ms, void* stream) {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     launch_wait_timeout_probe(g.d_status, (unsigned long long)limit_ms * 1000000ull, g.d_status + 3, s);
     CU_OK(cudaGetLastError());
+    return MT_OK;
+}
+
+mt_status mt_debug_launch_count(int64_t* count_out) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!count_out) return MT_ERR_INVALID_ARG;
+    *count_out = (int64_t)mt::g_kernel_launches;
     return MT_OK;
 }
 

@@ -9,6 +9,7 @@ namespace mt {
 
 // Launch with programmatic stream serialization: the kernel may start while its predecessor in the stream is
 // still draining; it must call pdl_wait() before it touches anything the predecessor wrote or still reads.
+extern unsigned long long g_kernel_launches;   // kernels enqueued through launch_pdl since the library was loaded
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
     cudaLaunchConfig_t cfg = {};
@@ -17,13 +18,16 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
+    ++g_kernel_launches;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 struct ModelDev;
 struct WorkItem;
 
-constexpr int kBucketChunk = 256;   // requests per CTA in the bucketing passes
+constexpr int kBucketChunk = 64;    // requests per CTA in the scatter pass (kHistChunk is a multiple of it)
+constexpr int kScatterThreads = 256;
+constexpr int kHistChunk = 1024;    // requests per CTA (and per row of block_hist) in the histogram pass
 
 struct BucketArgs {
     const int32_t* ids;
@@ -34,13 +38,18 @@ struct BucketArgs {
     int rows_per_unit;        // conv: tiles per image
     int tile_n[8];            // dense: output columns per work item of each layer (128 or 256)
     int tile_m[8];            // dense: rows per work item of each layer (128, or 256 for the CTA-pair executor)
-    int32_t* block_hist;      // [ceil(n / kBucketChunk)][T + 1]
+    int32_t* block_hist;      // [ceil(n / kHistChunk)][T + 1]
     int32_t* counts;          // [T + 1]
     int32_t* offsets;         // [T + 2]
     int32_t* tile_prefix;     // [n_layers][T + 1]
     int32_t* perm;            // [n]
     int32_t* inv;             // [n]
-    int item_grid;            // CTAs of the work-item expansion kernel
+    int32_t* ticket;          // one zero-initialised word: arrival counter of pass 1 (left at zero by every call)
+    const void* rows_src;     // non-null: payload rows [n][row_bytes] in arrival order, moved by pass 2 ...
+    void* rows_dst;           // ... to bucketed order, rows dst_ld_bytes apart (both multiples of 16 bytes)
+    int row_bytes;
+    int dst_ld_bytes;
+    int item_grid;            // least number of CTAs of pass 2 (the work-item expansion wants the whole GPU)
     WorkItem* items[8];       // per dense layer: expanded work items (null for other layers)
     int32_t* status;
 };
@@ -70,6 +79,11 @@ struct GemmArgs {
     void* out;                    // bf16 or fp32, rows in bucketed order
     int ld_out;                   // elements between output rows
     int out_fp32;
+    // Last layer only (out_fp32): non-null perm sends bucketed row j straight to row perm[j] of `out` (the caller's
+    // buffer, arrival order), and the rows of rejected requests, bucketed rows [offsets[T], offsets[T + 1]), are
+    // filled with NaN by the same launch - no separate un-permute pass.
+    const int32_t* perm;
+    const int32_t* offsets;       // [T + 2]
     int32_t* status;
 };
 cudaError_t configure_grouped_gemm();
@@ -77,6 +91,29 @@ cudaError_t configure_grouped_gemm();
 // tmap_a: 128-row boxes of the layer's input; tmap_a32: 32-row boxes of the same buffer (transposed small items).
 void launch_grouped_gemm(const CUtensorMap& tmap_a, const CUtensorMap& tmap_a32, const GemmArgs& a, int tile_n,
                          int sm_count, cudaStream_t s);
+
+// Whole-pass executor for small batches of narrow MLPs (fused_mlp.cu): bucketing, all dense layers and the return to
+// arrival order in one launch.
+struct FusedArgs {
+    const uint16_t* inputs;   // bf16 [n][K0], arrival order
+    const int32_t* ids;       // [n]
+    int n;
+    int T;
+    const ModelDev* models;
+    int n_layers;
+    int K0;                   // input features (multiple of 64, at most 256)
+    int out_elems;            // output features (at most 256)
+    float* out;               // fp32 [n][out_elems], arrival order (the caller's buffer)
+    int32_t* counts;          // [T + 1]   bucketing results, written by CTA 0
+    int32_t* offsets;         // [T + 2]
+    int32_t* perm;            // [n]
+    int32_t* inv;             // [n]
+    int32_t* status;
+};
+// n <= 512, every layer at most max_width <= 256 wide, and the per-chunk histograms fit the operand buffer
+bool fused_mlp_fits(int n, int T, int max_width);
+cudaError_t configure_fused_mlp();
+cudaError_t launch_fused_mlp(const FusedArgs& a, int grid, cudaStream_t s);
 
 // CTA-pair form (grouped_gemm_pair.cu): work items of 256 rows x 256 columns (BucketArgs::tile_m = tile_n = 256).
 cudaError_t configure_grouped_gemm_pair();

@@ -17,3 +17,12 @@ def oracle_mod():
     import oracle
     oracle.build()
     return oracle
+
+
+@pytest.fixture(params=["fused", "layered"])
+def small_batch_path(request, monkeypatch):
+    """Batches of at most 512 requests against narrow dense models run as one fused launch; MT_FUSED=0 sends the
+    same batch down the layer-by-layer path.  Tests that take this fixture run once on each."""
+    if request.param == "layered":
+        monkeypatch.setenv("MT_FUSED", "0")
+    return request.param

@@ -37,7 +37,7 @@ def run_ids(T, ids, registered=None):
 
 
 @pytest.mark.parametrize("T", [1, 4, 37, 1000])
-def test_bucketing_distributions(T):
+def test_bucketing_distributions(T, small_batch_path):
     fresh(max(64, T))
     harness.register_models(passthrough_models(T))
     rng = np.random.default_rng(T)
@@ -70,7 +70,7 @@ def test_empty_batch_is_a_noop():
     assert float(out.abs().sum()) == 0.0
 
 
-def test_rejected_ids_give_nan_rows_and_a_status():
+def test_rejected_ids_give_nan_rows_and_a_status(small_batch_path):
     T = 5
     fresh()
     harness.register_models(passthrough_models(T))

@@ -1,0 +1,97 @@
+"""The one-launch path for small batches of narrow MLPs (bucketing, all layers and the return to arrival order in a
+single kernel) and the last layer's direct write to arrival order on the layer-by-layer path: parity with the fp64
+oracle element by element, bit-exact bucketing, rejected ids, launch counts.  Everything goes through the C-ABI."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_1901_06887_b200 import binding as mt, harness, synth
+
+from gpu_util import TOL, fresh, run_and_check
+
+pytestmark = pytest.mark.gpu
+
+
+def bits(a):
+    return synth.f32_to_bf16_bits(np.asarray(a, np.float32))
+
+
+def launches_of(fn):
+    before = mt.mt_debug_launch_count()
+    r = fn()
+    return r, mt.mt_debug_launch_count() - before
+
+
+def test_config1_is_one_launch_and_layered_path_agrees(monkeypatch):
+    wl = synth.make_workload(1)
+    (got, _), k = launches_of(lambda: run_and_check(wl.models, wl.model_ids, wl.inputs))
+    assert k == 1
+    monkeypatch.setenv("MT_FUSED", "0")
+    layered, k = launches_of(lambda: harness.run_batch(wl.model_ids, wl.inputs, 10))
+    assert k == 5                                     # bucketing, gather, three layers (the last one un-permutes)
+    ref = oracle.forward(wl.models, wl.model_ids, wl.inputs)
+    assert harness.scaled_error(layered, ref).max() <= TOL
+    assert np.abs(layered - got).max() <= 1e-4        # same products; only the accumulation grouping may differ
+
+
+@pytest.mark.parametrize("n,T,hidden,out", [(1, 1, (64,), 1), (512, 1, (256, 256), 256), (512, 200, (128, 192), 200),
+                                            (300, 37, (256, 64, 256), 10), (129, 2, (192,), 72), (33, 1000, (64,), 8)])
+def test_fused_shapes_many_tenants_and_ragged_units(n, T, hidden, out):
+    # several 128-row units per tenant, tenants without requests, hidden widths that differ per tenant, outputs that
+    # are not a multiple of 8 or 32 wide, more tenants than requests
+    rng = np.random.default_rng(n + T)
+    widths_of = lambda t: (128,) + tuple(int(rng.choice([64, 128, 192, 256])) if h != 64 else 64 for h in hidden) + (out,)
+    models = [synth.make_mlp(7, 1000 * T + t, widths_of(t)) for t in range(T)]
+    ids = rng.integers(0, T, n).astype(np.int32)
+    if T > 2:
+        ids[ids == 1] = 0                             # tenant 1 gets no request
+    (_, err), k = launches_of(lambda: run_and_check(models, ids, bits(rng.standard_normal((n, 128))), max_models=max(64, T)))
+    assert k == 1
+
+
+def test_fused_rejected_ids_and_unaligned_output():
+    import torch
+    T = 6
+    rng = np.random.default_rng(3)
+    models = [synth.make_mlp(7, t, (64, 128, 12)) for t in range(T)]
+    fresh()
+    harness.register_models(models)
+    mt.mt_release(2)
+    ids = rng.integers(-1, T + 1, 200).astype(np.int32)            # -1, T and the released id 2 are rejected
+    x = bits(rng.standard_normal((200, 64)))
+    good = (ids >= 0) & (ids < T) & (ids != 2)
+    # an output buffer that is only 4-byte aligned: the vector stores must not be used
+    buf = torch.full((200 * 12 + 1,), float("nan"), dtype=torch.float32, device="cuda")
+    out = buf[1:].view(200, 12)
+    mt.mt_infer(harness.bf16_bits_to_device(x), torch.from_numpy(ids).cuda(), 200, out)
+    st, bad = mt.mt_get_async_status()
+    assert st == 2 and bad == int(np.flatnonzero(~good)[0])
+    got = out.cpu().numpy()
+    assert np.isnan(got[~good]).all()
+    ref = oracle.forward(models, ids[good], x[good])
+    assert harness.scaled_error(got[good], ref).max() <= TOL
+    counts, offsets, perm, inv = mt.mt_debug_last_bucketing(200)
+    live_ids = np.where(good, ids, T)
+    oc, oo, op, oi = oracle.bucket(live_ids, T + 1)                # rejected requests form a last bucket, arrival order kept
+    assert np.array_equal(counts, oc[:T]) and np.array_equal(offsets, oo)
+    assert np.array_equal(perm, op) and np.array_equal(inv, oi)
+
+
+@pytest.mark.parametrize("n", [513, 2000])
+def test_layered_last_layer_writes_arrival_order_with_rejected_ids(n):
+    # above the fused path's batch limit: the last grouped launch writes through perm and fills the rejected rows
+    T = 9
+    rng = np.random.default_rng(n)
+    models = [synth.make_mlp(7, t, (128, 320, 40)) for t in range(T)]
+    fresh()
+    harness.register_models(models)
+    ids = rng.integers(0, T + 2, n).astype(np.int32)
+    x = bits(rng.standard_normal((n, 128)))
+    good = ids < T
+    (got), k = launches_of(lambda: harness.run_batch(ids, x, 40))
+    assert k == 2 + 2                                 # two bucketing passes (rows move in the second), two layers; no un-permute pass
+    st, bad = mt.mt_get_async_status()
+    assert st == 2 and bad == int(np.flatnonzero(~good)[0])
+    assert np.isnan(got[~good]).all() and np.isfinite(got[good]).all()
+    ref = oracle.forward(models, ids[good], x[good])
+    assert harness.scaled_error(got[good], ref).max() <= TOL

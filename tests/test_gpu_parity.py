@@ -18,12 +18,12 @@ def bits(a):
     return synth.f32_to_bf16_bits(np.asarray(a, np.float32))
 
 
-def test_config1_full():
+def test_config1_full(small_batch_path):
     wl = synth.make_workload(1)
     run_and_check(wl.models, wl.model_ids, wl.inputs)
 
 
-def test_identity_and_zero_weights_are_exact_on_the_gpu():
+def test_identity_and_zero_weights_are_exact_on_the_gpu(small_batch_path):
     rng = np.random.default_rng(0)
     eye = np.eye(256, dtype=np.float32)
     ident = [Layer(DENSE, 256, 256, relu=1, weight=bits(eye), bias=None),
@@ -43,14 +43,14 @@ def test_identity_and_zero_weights_are_exact_on_the_gpu():
 
 
 @pytest.mark.parametrize("n", [1, 2, 127, 128, 129, 385])
-def test_ragged_row_tiles_single_tenant(n):
+def test_ragged_row_tiles_single_tenant(n, small_batch_path):
     rng = np.random.default_rng(n)
     m = synth.make_mlp(1, n, (128, 192, 130))       # He-uniform weights, as in the workloads
     run_and_check([m], np.zeros(n, np.int32), bits(rng.standard_normal((n, 128))))
 
 
 @pytest.mark.parametrize("K,N", [(64, 1), (64, 10), (64, 128), (128, 129), (320, 257), (1024, 96)])
-def test_one_layer_shapes(K, N):
+def test_one_layer_shapes(K, N, small_batch_path):
     rng = np.random.default_rng(K + N)
     models = [synth.make_mlp(1, 10 * K + t, (K, N)) for t in range(3)]
     for t, m in enumerate(models):
@@ -124,7 +124,7 @@ def test_conv_single_tap_shift_closed_form_on_gpu():
         assert np.allclose(got, want, rtol=4e-3, atol=0)        # only the pooled mean is rounded to bf16
 
 
-def test_batch_invariance_and_nan_isolation():
+def test_batch_invariance_and_nan_isolation(small_batch_path):
     wl = synth.make_workload(1, n=48)
     got, _ = run_and_check(wl.models, wl.model_ids, wl.inputs)
     ref = oracle.forward(wl.models, wl.model_ids, wl.inputs)
@@ -164,7 +164,7 @@ def test_repeat_runs_are_bitwise_identical_and_host_entry_matches():
     assert np.array_equal(harness.run_batch(wl.model_ids, wl.inputs, 64), got)
 
 
-def test_growing_batches_and_wider_models_reallocate_correctly():
+def test_growing_batches_and_wider_models_reallocate_correctly(small_batch_path):
     rng = np.random.default_rng(9)
     mk = lambda h: synth.make_mlp(3, h, (128, h, 64))
     fresh()
