@@ -44,6 +44,7 @@ const char* const kKernelNames[K_COUNT] = {"bucketing (histogram, scans, scatter
 struct TimedLaunch {
     int kernel;
     cudaEvent_t start, stop;
+    int count;                           // launches between the two events
 };
 
 struct Ctx {
@@ -328,29 +329,58 @@ mt_status check_family(const std::vector<HostLayer>& m) {
     return MT_OK;
 }
 
+cudaEvent_t pooled_event() {
+    cudaEvent_t e;
+    if (!g.event_pool.empty()) { e = g.event_pool.back(); g.event_pool.pop_back(); }
+    else cudaEventCreate(&e);
+    return e;
+}
+
+// Timing mode 1: one pair of events around every launch.  Mode 2: only the layer executors are timed, and
+// consecutive launches of the same executor share ONE pair of events (start before the first, stop after the last):
+// an event between two launches would serialise them and undo the programmatic dependent launch that lets the next
+// layer's prologue run under the previous layer's tail, i.e. it would time something the untimed path never does.
 struct Timer {
+    static int open_kernel;              // mode 2: executor whose group of launches is open (-1 none)
+    static cudaEvent_t open_start;
+    static int open_count;
     int kernel;
     cudaStream_t s;
-    bool on;
-    cudaEvent_t start = nullptr, stop = nullptr;
-    Timer(int k, cudaStream_t st)
-        : kernel(k), s(st), on(g.timing == 1 || (g.timing == 2 && (k == K_GEMM || k == K_CONV || k == K_FUSED))) {
-        if (!on) return;
-        auto get = [&]() {
-            cudaEvent_t e;
-            if (!g.event_pool.empty()) { e = g.event_pool.back(); g.event_pool.pop_back(); }
-            else cudaEventCreate(&e);
-            return e;
-        };
-        start = get(); stop = get();
-        cudaEventRecord(start, s);
+    bool each;
+    cudaEvent_t start = nullptr;
+    static void close_group(cudaStream_t st) {
+        if (open_kernel < 0) return;
+        cudaEvent_t stop = pooled_event();
+        cudaEventRecord(stop, st);
+        g.timed.push_back({open_kernel, open_start, stop, open_count});
+        open_kernel = -1;
+    }
+    Timer(int k, cudaStream_t st) : kernel(k), s(st), each(g.timing == 1) {
+        if (each) {
+            start = pooled_event();
+            cudaEventRecord(start, s);
+        } else if (g.timing == 2) {
+            const bool executor = (k == K_GEMM || k == K_CONV || k == K_FUSED);
+            if (open_kernel >= 0 && open_kernel != k) close_group(s);
+            if (executor && open_kernel < 0) {
+                open_start = pooled_event();
+                cudaEventRecord(open_start, s);
+                open_kernel = k;
+                open_count = 0;
+            }
+            if (executor) ++open_count;
+        }
     }
     ~Timer() {
-        if (!on) return;
+        if (!each) return;
+        cudaEvent_t stop = pooled_event();
         cudaEventRecord(stop, s);
-        g.timed.push_back({kernel, start, stop});
+        g.timed.push_back({kernel, start, stop, 1});
     }
 };
+int Timer::open_kernel = -1;
+cudaEvent_t Timer::open_start = nullptr;
+int Timer::open_count = 0;
 
 mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outputs, cudaStream_t s) {
     if (!g.init) return MT_ERR_NOT_INIT;
@@ -384,6 +414,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             if (grid > n) grid = n;
             if (grid > g.sm_count) grid = g.sm_count;
             CU_OK(launch_fused_mlp(a, grid, s));
+            Timer::close_group(s);
             g.last_n = n;
             return MT_OK;
         }
@@ -476,6 +507,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
         Timer t(K_UNPERMUTE, s);
         launch_unpermute(g.d_out_b, g.d_perm, g.d_offsets, g.T, n, g.out_elems, (float*)outputs, g.sm_count, s);
     }
+    Timer::close_group(s);
     g.last_n = n;
     CU_OK(cudaGetLastError());
     return MT_OK;
@@ -761,7 +793,7 @@ mt_status mt_get_kernel_times(const char** names, double* total_ms, int32_t* lau
         float f = 0.f;
         CU_OK(cudaEventElapsedTime(&f, t.start, t.stop));
         ms[t.kernel] += f;
-        cnt[t.kernel] += 1;
+        cnt[t.kernel] += t.count;
         g.event_pool.push_back(t.start);
         g.event_pool.push_back(t.stop);
     }
