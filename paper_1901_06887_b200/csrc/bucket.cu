@@ -65,7 +65,7 @@ __device__ __forceinline__ int layer_units(const ModelDev* models, int t, int l,
     if (c <= 0) return 0;
     const LayerDev& L = models[t].layer[l];
     if (L.kind == MT_DENSE) return ((c + tile_m - 1) / tile_m) * ((L.N + tile_n - 1) / tile_n);
-    if (L.kind == MT_CONV3X3) return c * rows_per_unit;
+    if (L.kind == MT_CONV3X3) return ((c + tile_m - 1) / tile_m) * rows_per_unit;   // tile_m = images per unit
     return 0;
 }
 

@@ -1,0 +1,475 @@
+// Grouped 3x3 convolution executor, CTA-pair form (images whose padded row length is 64 pixels, i.e. the 56 x 56
+// workload): the same implicit GEMM, strip geometry and tap pairing as grouped_conv.cu,
+//     Y[r, y, x, o] = act(b_t[o] + sum_{ky,kx,c} X[r, y+ky-1, x+kx-1, c] * W_t[o, ky, kx, c]),
+// but two CTAs of a cluster (two SMs) work in lockstep on the same strip of TWO images of one tenant, and ONE
+// thread of the leader CTA issues tcgen05.mma.cta_group::2 (M = 256: 128 pixels of each image) for both.
+//
+// Why: with 64 output channels an instruction is short, and the one-CTA executor is bound by what its single
+// issuing thread can feed (measured: the thread spends about 1850 cycles per 128-pixel tile, of which the tensor
+// pipe is busy about 1150).  A pair instruction costs the issuing thread the same and keeps two tensor pipes busy,
+// so the issue cost per tile halves.  Each CTA holds only its share of the B operand: for the N = 64 instructions
+// its 32 output channels of the tap, for the paired N = 128 instructions one of the two stacked tap tiles (rank 0:
+// W(2,kx), rank 1: W(0,kx)); 60 KiB per CTA instead of 72.
+//
+// Synchronisation inside the pair (every wait bounded, as everywhere):
+//   sfull[s]   in the leader: announces the bytes of BOTH CTAs' strip loads; both loads report there;
+//   sempty[s]  in each CTA: its own epilogue releases its own strip buffer;
+//   tfull[a]   in both CTAs, signalled together by a multicast commit: each CTA drains its own 128 accumulator rows;
+//   tempty[a]  in the leader: 16 arrivals (one per epilogue warp, 8 local and 8 remote);
+//   wfull      in each CTA for its own weight image; the peer then arrives on wpeer in the leader;
+//   wempty     in both CTAs, multicast commit once every MMA on the old weights is done.
+// The two CTAs meet at a cluster barrier before they exit.  A tenant with an odd number of images leaves the peer
+// of its last pair a copy of the leader's image, computed and not stored.
+//
+// The paper does not define convolution; it only names a catalogue of standard layers (Sec. 1.1, Sec. 3.1).
+#include "mt_device.cuh"
+#include "mt_host.h"
+
+namespace mt {
+
+constexpr int kCpThreads = 320;
+constexpr int kCpEpiThreads = 256;
+constexpr int kCpN = 64;                                  // output channels
+constexpr int kCpHalfTap = 32 * BK * 2;                   // 4 KiB: 32 output channels x 64 input channels
+constexpr int kCpFullTap = 64 * BK * 2;                   // 8 KiB
+constexpr int kOffMid = 0;                                // ky = 1 taps, this CTA's 32 output channels, kx = 0..2
+constexpr int kOffPair = 3 * kCpHalfTap;                  // stacked pairs: rank 0 holds W(2,kx), rank 1 W(0,kx)
+constexpr int kOffBot = kOffPair + 3 * kCpFullTap;        // ky = 2 taps alone, this CTA's 32 output channels
+constexpr int kOffTop = kOffBot + 3 * kCpHalfTap;         // ky = 0 taps alone
+static_assert(kOffTop + 3 * kCpHalfTap == kConvPairWeightBytes, "weight image layout");
+constexpr int kCpMaxStages = 4;
+constexpr int kCpSlots = 8;                               // TMEM ring: 8 accumulators of 64 columns
+constexpr int kCpBarBytes = 2048;
+constexpr int kCpRecords = 16;
+constexpr int kCpOutStageBytes = 8 * 2048;                // per epilogue warp: 32 pixels x 64 bytes
+
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                                 uint32_t leader_bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(leader_bar)
+        : "memory");
+}
+
+struct PairStrip {
+    int t, j, y0, strip_in_image, dummy;
+};
+
+__global__ void __launch_bounds__(kCpThreads, 1)
+grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_y,
+                            const ConvArgs p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+    const uint32_t w_smem = base;
+    const uint32_t strip0 = base + kConvPairWeightBytes;
+    // output staging: one 2 KiB region per epilogue warp (32 pixels x 32 channels), the source of its TMA stores
+    const uint32_t out_stage0 = strip0 + p.n_stages * p.stage_bytes;
+    uint8_t* out_stage_ptr = smem + kConvPairWeightBytes + p.n_stages * p.stage_bytes;
+    const uint32_t bar0 = out_stage0 + kCpOutStageBytes;
+    uint8_t* bar_ptr = out_stage_ptr + kCpOutStageBytes;
+    auto sfull_bar = [&](int s) { return bar0 + 8u * s; };
+    auto sempty_bar = [&](int s) { return bar0 + 8u * (kCpMaxStages + s); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kCpMaxStages + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kCpMaxStages + kCpSlots + a); };
+    const uint32_t wfull_bar = bar0 + 8u * (2 * kCpMaxStages + 2 * kCpSlots);
+    const uint32_t wempty_bar = wfull_bar + 8u;
+    const uint32_t wpeer_bar = wfull_bar + 16u;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * (2 * kCpMaxStages + 2 * kCpSlots + 3));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    float* s_bias = reinterpret_cast<float*>(bar_ptr + 256);          // 64 floats
+    // Per-strip record, producer -> epilogue of the same CTA: x = flags (1 new tenant, 8 copy of the leader's image:
+    // do not store, 4 the strip's last tile is finished by the next strip), y = image (bucketed index), z = first output row, w = tenant.
+    int4* s_rec = reinterpret_cast<int4*>(bar_ptr + 512);             // kCpRecords x 16 bytes
+    float* s_pool = reinterpret_cast<float*>(bar_ptr + 1024);         // 8 warps x 32 channel sums (fused pooling)
+
+    pdl_launch_dependents();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();          // 0 = leader (issues the MMAs), 1 = peer
+    const bool is_leader = (rank == 0);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kCpMaxStages; ++s) { mbar_init(sfull_bar(s), 1); mbar_init(sempty_bar(s), 1); }
+        for (int a = 0; a < kCpSlots; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 2 * (kCpEpiThreads / 32)); }
+        mbar_init(wfull_bar, 1);
+        mbar_init(wempty_bar, 1);
+        mbar_init(wpeer_bar, 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tensormap(&tmap_x);
+        prefetch_tensormap(&tmap_y);
+    }
+    // the last rows of every strip stage are read (for rows that are never stored) but not written by the TMA box
+    for (int i = threadIdx.x; i < (p.n_stages * p.stage_bytes) / 16; i += blockDim.x)
+        reinterpret_cast<uint4*>(smem + kConvPairWeightBytes)[i] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async_smem();
+    if (warp == 1) {                                  // the same warp of both CTAs
+        tmem_alloc_pair(smem_u32(tmem_slot), kCpSlots * kCpN);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                               // both CTAs' barriers exist before anyone signals across
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    pdl_wait();   // everything above overlapped the previous kernel's tail; its results are needed from here on
+    // contiguous range of pair-strips for this cluster: unit = (tenant, pair of images, strip of 2 tiles)
+    const int total = p.tile_prefix[p.T];
+    const int n_pairs = gridDim.x >> 1, pair_id = blockIdx.x >> 1;
+    const int s_begin = (int)(((long long)total * pair_id) / n_pairs);
+    const int s_end = (int)(((long long)total * (pair_id + 1)) / n_pairs);
+    constexpr int Wp = 64;
+    const int TS = p.tiles_per_strip;
+
+    // pair-strip -> (tenant, this CTA's image, first row); units of one tenant are consecutive: its range is cached
+    int cur_t = -1, cur_lo = 0, cur_hi = 0, cur_seg = 0, cur_n = 0;
+    auto locate = [&](int s) {
+        if (s < cur_lo || s >= cur_hi) {
+            int lo = 0, hi = p.T;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (p.tile_prefix[mid] <= s) lo = mid; else hi = mid;
+            }
+            cur_t = lo; cur_lo = p.tile_prefix[lo]; cur_hi = p.tile_prefix[lo + 1];
+            cur_seg = p.offsets[lo]; cur_n = p.offsets[lo + 1] - cur_seg;
+        }
+        PairStrip c;
+        const int local = s - cur_lo;
+        const int pr = local / p.strips_per_image;
+        const int mine = 2 * pr + (int)rank;
+        c.t = cur_t;
+        c.dummy = mine >= cur_n;
+        c.j = cur_seg + (c.dummy ? 2 * pr : mine);
+        c.strip_in_image = local - pr * p.strips_per_image;
+        c.y0 = c.strip_in_image * p.R;
+        return c;
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {   // ------------------------------------------------ TMA producer (both CTAs)
+            int stage = 0; uint32_t phase = 0;
+            int w_loads = 0, w_tenant = -1;
+            const uint32_t wpeer_leader = map_to_cta(wpeer_bar, 0);
+            for (int s = s_begin; s < s_end; ++s) {
+                const PairStrip c = locate(s);
+                const bool new_tenant = (c.t != w_tenant);
+                if (!mbar_wait(sempty_bar(stage), phase ^ 1u, abort_flag, p.status, 52)) break;
+                const int img = p.perm ? p.perm[c.j] : c.j;
+                const bool defer_bottom = s + 1 < s_end && c.strip_in_image + 1 < p.strips_per_image;
+                s_rec[(s - s_begin) & (kCpRecords - 1)] =
+                    make_int4((new_tenant ? 1 : 0) | (defer_bottom ? 4 : 0) | (c.dummy ? 8 : 0), c.j, c.y0, c.t);
+                if (is_leader) mbar_expect_tx(sfull_bar(stage), 2u * (uint32_t)p.box_bytes);   // both CTAs' bytes
+                tma_load_4d_pair(strip0 + stage * p.stage_bytes, &tmap_x, 0, -1, c.y0 - 1, img, map_to_cta(sfull_bar(stage), 0));
+                if (new_tenant) {
+                    // The issuer releases the old weights when it reaches this strip, i.e. after the strip has
+                    // landed in both CTAs: so the strip goes first.
+                    if (w_loads > 0 && !mbar_wait_spin(wempty_bar, (uint32_t)((w_loads - 1) & 1), abort_flag, p.status, 51, 64)) break;
+                    mbar_expect_tx(wfull_bar, kConvPairWeightBytes);
+                    bulk_load(w_smem, p.models[c.t].layer[p.layer].w + kConvPairImageOffset + (size_t)rank * (kConvPairWeightBytes / 2),
+                              kConvPairWeightBytes, wfull_bar);
+                    if (!is_leader) {      // tell the leader's issuer once this CTA's share has landed
+                        if (!mbar_wait(wfull_bar, (uint32_t)(w_loads & 1), abort_flag, p.status, 53)) break;
+                        mbar_arrive_remote(wpeer_leader);
+                    }
+                    w_tenant = c.t;
+                    ++w_loads;
+                }
+                if (++stage == p.n_stages) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        if (is_leader) {   // ------------------------------------------------ MMA issuer (leader CTA)
+            // The whole warp walks the loop (addresses and descriptors stay warp-uniform); one elected lane issues.
+            const bool leader = elect_one();
+            const uint32_t tb = __shfl_sync(0xffffffffu, *tmem_slot, 0);
+            constexpr uint32_t idesc64 = make_idesc_bf16(2 * BM, kCpN);
+            constexpr uint32_t idesc128 = make_idesc_bf16(2 * BM, 2 * kCpN);
+            int stage = 0; uint32_t phase = 0;
+            int g = 0;                      // tiles started so far by this pair; tile g lives in TMEM slot g % kCpSlots
+            int w_loads = 0;
+            bool ok = true;
+            const uint32_t w_lo = desc_lo(w_smem);
+            constexpr uint32_t kHalfLo = kCpHalfTap >> 4, kFullLo = kCpFullTap >> 4;
+            constexpr uint32_t kMidLo = kOffMid >> 4, kPairLo = kOffPair >> 4, kBotLo = kOffBot >> 4, kTopLo = kOffTop >> 4;
+            constexpr uint32_t kPixLo = 128 >> 4;                // one pixel (128 bytes) further
+            // four K steps of one 128-pixel block (of each CTA) against one tap operand
+            auto issue = [&](uint32_t a_lo, uint32_t b_lo, uint32_t d_tmem, uint32_t idesc, bool overwrite) {
+                if (!leader) return;
+                if (overwrite) umma_pair_lohi<false>(d_tmem, a_lo, b_lo, idesc);
+                else umma_pair_lohi<true>(d_tmem, a_lo, b_lo, idesc);
+                umma_pair_lohi<true>(d_tmem, a_lo + 2, b_lo + 2, idesc);
+                umma_pair_lohi<true>(d_tmem, a_lo + 4, b_lo + 4, idesc);
+                umma_pair_lohi<true>(d_tmem, a_lo + 6, b_lo + 6, idesc);
+            };
+            int t_hi = -1;                  // units [.., t_hi) belong to the current tenant
+            int in_image = 0;               // index of the current strip inside its image
+            uint32_t strip_ready = 0, slot_ready = 0;
+            for (int s = s_begin; ok && s < s_end; ++s) {
+                const bool new_tenant = (s >= t_hi);
+                if (new_tenant) {           // rare: a tenant border (or the first unit)
+                    const PairStrip c = locate(s);
+                    t_hi = cur_hi;
+                    in_image = c.strip_in_image;
+                }
+                if (!strip_ready) {
+                    if (!mbar_wait_spin(sfull_bar(stage), phase, abort_flag, p.status, 55)) break;
+                }
+                tc_fence_after();
+                if (new_tenant) {
+                    if (w_loads > 0 && leader) umma_commit_pair(wempty_bar);     // fires when all MMAs on the old weights are done
+                    if (!mbar_wait(wfull_bar, (uint32_t)(w_loads & 1), abort_flag, p.status, 56)) break;
+                    if (!mbar_wait_spin(wpeer_bar, (uint32_t)(w_loads & 1), abort_flag, p.status, 57)) break;
+                    ++w_loads;
+                }
+                const bool pair_top = s > s_begin && in_image > 0;
+                const bool defer_bottom = s + 1 < s_end && in_image + 1 < p.strips_per_image;
+                const uint32_t strip_lo = desc_lo(strip0 + stage * p.stage_bytes);
+                const int next_stage = (stage + 1 == p.n_stages) ? 0 : stage + 1;
+                const uint32_t next_phase = (stage + 1 == p.n_stages) ? (phase ^ 1u) : phase;
+                strip_ready = 0;
+                for (int i = 0; i < TS; ++i, ++g) {
+                    const int slot = g % kCpSlots;
+                    if (!slot_ready) {   // the slot must have been drained by both CTAs' epilogues of tile g - kCpSlots
+                        if (!mbar_wait_spin(tempty_bar(slot), (uint32_t)(((g / kCpSlots) & 1) ^ 1), abort_flag, p.status, 54)) { ok = false; break; }
+                    }
+                    tc_fence_after();
+                    const uint32_t d_this = tb + slot * kCpN;
+                    const uint32_t blk = strip_lo + (uint32_t)(i * BM) * kPixLo;     // padded pixel i*128 of the strip
+                    const bool last_tile = (i == TS - 1);
+                    // ky = 1 first: these overwrite the fresh accumulator
+                    issue(blk + (uint32_t)(Wp + 0) * kPixLo, w_lo + kMidLo + 0 * kHalfLo, d_this, idesc64, true);
+                    // look ahead: the answers are consumed after the rest of this tile has been queued
+                    const uint32_t poll_slot = mbar_test_wait(tempty_bar((g + 1) % kCpSlots), (uint32_t)((((g + 1) / kCpSlots) & 1) ^ 1));
+                    uint32_t poll_strip = 0;
+                    if (last_tile) poll_strip = mbar_test_wait(sfull_bar(next_stage), next_phase);
+                    issue(blk + (uint32_t)(Wp + 1) * kPixLo, w_lo + kMidLo + 1 * kHalfLo, d_this, idesc64, false);
+                    issue(blk + (uint32_t)(Wp + 2) * kPixLo, w_lo + kMidLo + 2 * kHalfLo, d_this, idesc64, false);
+                    // block at the tile's first row: ky = 0 of this tile and ky = 2 of the tile above
+                    const bool have_above = (i > 0) || pair_top;
+                    const bool adjacent = slot != 0;                              // slots g-1 and g contiguous in TMEM
+                    if (have_above && adjacent) {
+#pragma unroll
+                        for (int kx = 0; kx < 3; ++kx)
+                            issue(blk + kx * kPixLo, w_lo + kPairLo + kx * kFullLo, d_this - kCpN, idesc128, false);
+                    } else {
+                        for (int kx = 0; kx < 3; ++kx) {
+                            if (have_above)
+                                issue(blk + kx * kPixLo, w_lo + kBotLo + kx * kHalfLo, tb + ((g - 1) % kCpSlots) * kCpN, idesc64, false);
+                            issue(blk + kx * kPixLo, w_lo + kTopLo + kx * kHalfLo, d_this, idesc64, false);
+                        }
+                    }
+                    if (have_above && leader) umma_commit_pair(tfull_bar((g - 1) % kCpSlots));    // tile above is complete
+                    slot_ready = poll_slot;
+                    if (last_tile) strip_ready = (s + 1 < s_end) ? poll_strip : 0;
+                }
+                if (!ok) break;
+                if (!defer_bottom) {
+                    // nobody below will finish the strip's last tile: its ky = 2 taps from the block under it
+                    const uint32_t blk = strip_lo + (uint32_t)(TS * BM) * kPixLo;
+                    const int last = (g - 1) % kCpSlots;
+                    for (int kx = 0; kx < 3; ++kx)
+                        issue(blk + kx * kPixLo, w_lo + kBotLo + kx * kHalfLo, tb + last * kCpN, idesc64, false);
+                    if (leader) umma_commit_pair(tfull_bar(last));
+                }
+                stage = next_stage; phase = next_phase;
+                if (++in_image == p.strips_per_image) in_image = 0;
+            }
+        }
+    } else {               // ---------------------------------------------------- epilogue (warps 2..9, both CTAs)
+        const int ew = warp - 2;
+        const int q4 = warp & 3;                    // TMEM lane quarter this warp may read
+        const int half = ew >> 2;                   // which 32 of the 64 output channels
+        const int r = q4 * 32 + lane;               // tile-local padded pixel of this thread
+        const int yl = r / Wp, x = r - yl * Wp;
+        constexpr int rows_per_tile = BM / Wp;
+        int g = 0, relu = 0;
+        bool ok = true;
+        int img_j = 0, y0 = 0, store = 1, release_at = 0;
+        const bool pooling = (p.pool_partial != nullptr);
+        const uint32_t tempty_leader0 = map_to_cta(tempty_bar(0), 0);   // the leader's tempty barriers, 8 bytes apart
+        for (int s = s_begin; ok && s < s_end; ++s) {
+            float psum[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) psum[e] = 0.0f;
+            for (int i = 0; i < TS; ++i, ++g) {
+                const int slot = g % kCpSlots;
+                // tfull is completed by the leader's multicast commit: one lane per warp polls and tells the others
+                int got = 1;
+                if (lane == 0) got = mbar_wait_spin(tfull_bar(slot), (uint32_t)((g / kCpSlots) & 1), abort_flag, p.status, 58, 32) ? 1 : 0;
+                got = __shfl_sync(0xffffffffu, got, 0);
+                if (!got) { ok = false; break; }
+                if (i == 0) {
+                    // the strip's record was published (with the strip's data) before any of its MMAs were issued
+                    const int4 rec = s_rec[(s - s_begin) & (kCpRecords - 1)];
+                    img_j = rec.y; y0 = rec.z; store = (rec.x & 8) ? 0 : 1;
+                    // Which completion tells that no MMA will read the strip's buffer again: the strip's last tile
+                    // when the strip finishes it itself; when its ky = 2 taps are left to the next strip (which reads
+                    // its own buffer for them), already the tile before - that commit follows the last tile's other taps.
+                    release_at = ((rec.x & 4) && TS >= 2) ? TS - 2 : TS - 1;
+                    if (rec.x & 1) {                // new tenant: its bias into shared memory, ReLU flag into a register
+                        const LayerDev& L = p.models[rec.w].layer[p.layer];
+                        asm volatile("bar.sync 1, %0;" ::"n"(kCpEpiThreads) : "memory");   // everyone done with the old bias
+                        if (threadIdx.x - 64 < kCpN) s_bias[threadIdx.x - 64] = L.bias[threadIdx.x - 64];
+                        relu = L.relu;
+                        asm volatile("bar.sync 1, %0;" ::"n"(kCpEpiThreads) : "memory");
+                    }
+                }
+                if (i == release_at && threadIdx.x == 64) mbar_arrive(sempty_bar((s - s_begin) % p.n_stages));
+                tc_fence_after();
+                uint32_t v[32];
+                tmem_ld32(tmem_base + (static_cast<uint32_t>(q4 * 32) << 16) + slot * kCpN + half * 32, v);
+                tmem_ld_wait();
+                tc_fence_before();
+                // values are in registers: the slot can be reused once the eight epilogue warps of both CTAs have said
+                // so (one arrival per warp: an arrival that crosses to the other CTA is expensive)
+                __syncwarp();
+                if (lane == 0) {
+                    if (is_leader) mbar_arrive(tempty_bar(slot));
+                    else mbar_arrive_remote_relaxed(tempty_leader0 + 8u * slot);
+                }
+                const int y = y0 + i * rows_per_tile + yl;
+                // bias + ReLU in fp32 on this thread's pixel, 32 channels
+                float f[32];
+                {
+                    const float4* b4 = reinterpret_cast<const float4*>(s_bias + half * 32);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float4 b = b4[j];
+                        f[4 * j + 0] = __uint_as_float(v[4 * j + 0]) + b.x;
+                        f[4 * j + 1] = __uint_as_float(v[4 * j + 1]) + b.y;
+                        f[4 * j + 2] = __uint_as_float(v[4 * j + 2]) + b.z;
+                        f[4 * j + 3] = __uint_as_float(v[4 * j + 3]) + b.w;
+                    }
+                    if (relu) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) f[e] = fmaxf(f[e], 0.0f);
+                    }
+                }
+                if (pooling) {      // the layer feeds a global average pool: only channel sums are kept
+                    if (store && x < p.W && y < p.H) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) psum[e] += f[e];
+                    }
+                } else {
+                    // The warp's 32 pixels x 32 channels go to its staging region (64 bytes per pixel, 16-byte chunk c
+                    // of pixel q at chunk c ^ ((q >> 1) & 3): the 64-byte swizzle of the store's tensor map) and leave
+                    // as ONE tensor store, which also drops the pad columns and the rows past the image.  A row of
+                    // per-thread 64-byte global stores would cost the load/store unit 32 separate lines per instruction.
+                    if (lane == 0) bulk_wait_group_read0();      // the previous tile's store has read the region
+                    __syncwarp();
+                    uint8_t* mine = out_stage_ptr + ew * 2048 + lane * 64;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        uint4 o;
+                        o.x = pack_bf16x2(f[8 * j + 0], f[8 * j + 1]);
+                        o.y = pack_bf16x2(f[8 * j + 2], f[8 * j + 3]);
+                        o.z = pack_bf16x2(f[8 * j + 4], f[8 * j + 5]);
+                        o.w = pack_bf16x2(f[8 * j + 6], f[8 * j + 7]);
+                        *reinterpret_cast<uint4*>(mine + ((j ^ ((lane >> 1) & 3)) << 4)) = o;
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    const int yw = y0 + i * rows_per_tile + (q4 >> 1);       // the warp's image row (warp-uniform)
+                    if (lane == 0 && store && yw < p.H && (q4 & 1) * 32 < p.W) {
+                        tma_store_4d(&tmap_y, half * 32, (q4 & 1) * 32, yw, img_j, out_stage0 + ew * 2048);
+                        bulk_commit_group();
+                    }
+                }
+                __syncwarp();
+            }
+            if (pooling && ok) {
+                // Channel sums of this strip: a halving butterfly leaves lane c with the warp's total of channel c
+                // (31 shuffles), the four lane quarters are then added in a fixed order, and the strip's 64 sums are
+                // written to their own slot of pool_partial - no atomics, so the pooled value does not depend on timing.
+#pragma unroll
+                for (int step = 16; step >= 1; step >>= 1) {
+                    const bool upper = (lane & step) != 0;
+#pragma unroll
+                    for (int e = 0; e < step; ++e) {
+                        const float send = upper ? psum[e] : psum[e + step];
+                        const float recv = __shfl_xor_sync(0xffffffffu, send, step);
+                        psum[e] = (upper ? psum[e + step] : psum[e]) + recv;
+                    }
+                }
+                s_pool[ew * 32 + lane] = psum[0];
+                asm volatile("bar.sync 1, %0;" ::"n"(kCpEpiThreads) : "memory");
+                const int et = threadIdx.x - 64;                    // 0..255 among the epilogue threads
+                if (et < kCpN && store) {
+                    const int hf = et >> 5, c = et & 31;
+                    const float* q = s_pool + (hf * 4) * 32 + c;     // warps hf*4 .. hf*4+3 hold this half's quarters
+                    // quarter order by TMEM lane quarter (ew & 3 maps to q4 = (ew + 2) & 3): sum in pixel order 0,1,2,3
+                    const float t = ((q[2 * 32] + q[3 * 32]) + q[0 * 32]) + q[1 * 32];
+                    p.pool_partial[((size_t)img_j * p.strips_per_image + y0 / p.R) * kCpN + et] = t;
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(kCpEpiThreads) : "memory");
+            }
+        }
+    }
+
+    // ---- tear-down: every thread of both CTAs gets here, also after an abandoned wait
+    bulk_wait_group_read0();     // tensor stores still reading the staging regions
+    if (*abort_flag) {
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 2000000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();     // nobody signals a CTA that has left, and both are done with the pair's TMEM
+    if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc_pair(tmem_base, kCpSlots * kCpN);
+    }
+}
+
+// Conv weights W[64][3][3][64] -> the two CTAs' weight images of the pair executor (60 KiB each, rank 0 first),
+// every tile in the 128-byte-swizzled shared-memory layout: three ky = 1 taps with the CTA's 32 output channels,
+// three full 64-channel tiles (rank 0: W(2,kx), rank 1: W(0,kx)), three ky = 2 and three ky = 0 taps with the CTA's
+// 32 output channels.
+__global__ void pretile_conv_pair_kernel(const uint16_t* __restrict__ w, uint4* __restrict__ out) {
+    constexpr int kChunksPerRank = kConvPairWeightBytes / 16;
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < 2 * kChunksPerRank; idx += gridDim.x * blockDim.x) {
+        const int rank = idx / kChunksPerRank;
+        const int off = (idx - rank * kChunksPerRank) * 16;      // byte offset inside the rank's image
+        int ky, kx, row0, local;
+        if (off < kOffPair) { ky = 1; kx = off / kCpHalfTap; local = off - kx * kCpHalfTap; row0 = 32 * rank; }
+        else if (off < kOffBot) { const int o = off - kOffPair; ky = rank == 0 ? 2 : 0; kx = o / kCpFullTap; local = o - kx * kCpFullTap; row0 = 0; }
+        else if (off < kOffTop) { const int o = off - kOffBot; ky = 2; kx = o / kCpHalfTap; local = o - kx * kCpHalfTap; row0 = 32 * rank; }
+        else { const int o = off - kOffTop; ky = 0; kx = o / kCpHalfTap; local = o - kx * kCpHalfTap; row0 = 32 * rank; }
+        const int r = local >> 7, cpos = (local >> 4) & 7;       // row of the tile, physical 16-byte position
+        const int c = cpos ^ (r & 7);                            // logical chunk stored there
+        out[idx] = *reinterpret_cast<const uint4*>(w + ((size_t)(row0 + r) * 9 + (ky * 3 + kx)) * 64 + c * 8);
+    }
+}
+
+void launch_pretile_conv_pair(const uint16_t* w, uint16_t* out, cudaStream_t s) {
+    pretile_conv_pair_kernel<<<(2 * kConvPairWeightBytes / 16 + 255) / 256, 256, 0, s>>>(w, reinterpret_cast<uint4*>(out));
+}
+
+int conv_pair_smem_bytes(const ConvPlan& plan) {
+    return kConvPairWeightBytes + plan.n_stages * plan.stage_bytes + kCpOutStageBytes + kCpBarBytes + 1024;
+}
+
+cudaError_t configure_grouped_conv_pair() {
+    return cudaFuncSetAttribute(grouped_conv3x3_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+}
+
+// Cluster of two CTAs; grid = an even number of CTAs (one per SM).  a.tile_prefix counts (pair of images, strip) units.
+cudaError_t launch_grouped_conv_pair(const CUtensorMap& tmap_x, const CUtensorMap& tmap_y, const ConvArgs& a, int smem_bytes,
+                                     int sm_count, cudaStream_t s) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(sm_count & ~1);
+    cfg.blockDim = dim3(kCpThreads);
+    cfg.dynamicSmemBytes = (size_t)smem_bytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 2;
+    ++g_kernel_launches;
+    return cudaLaunchKernelEx(&cfg, grouped_conv3x3_pair_kernel, tmap_x, tmap_y, a);
+}
+
+}  // namespace mt

@@ -74,6 +74,7 @@ struct Ctx {
     int act_ld[MT_MAX_LAYERS + 1] = {0};
     CUtensorMap act_map[MT_MAX_LAYERS + 1];
     CUtensorMap act_map32[MT_MAX_LAYERS + 1];   // dense inputs again, as 32-row boxes
+    CUtensorMap act_store_map[MT_MAX_LAYERS + 1];   // conv activations as the store boxes of the CTA-pair executor
     float* d_out_b = nullptr;
     float* d_pool_partial = nullptr;     // per-strip channel sums of a conv layer that feeds a pool
     WorkItem* d_items[MT_MAX_LAYERS] = {nullptr};   // per dense layer
@@ -146,6 +147,7 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     CU_OK(configure_grouped_conv());
     CU_OK(configure_grouped_gemm_pair());
     CU_OK(configure_fused_mlp());
+    CU_OK(configure_grouped_conv_pair());
     g.T = 0;
     g.live = 0;
     g.has_family = false;
@@ -190,14 +192,16 @@ mt_status encode_weight_tiles(CUtensorMap* map, const void* ptr, size_t n_tiles_
     return r == CUDA_SUCCESS ? MT_OK : MT_ERR_CUDA;
 }
 
-mt_status encode_nhwc(CUtensorMap* map, const void* ptr, int C, int W, int H, int n_img, int box_w, int box_h) {
+mt_status encode_nhwc(CUtensorMap* map, const void* ptr, int C, int W, int H, int n_img, int box_w, int box_h,
+                      int box_c = 0) {
     cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)n_img};
     cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
-    cuuint32_t box[4] = {(cuuint32_t)C, (cuuint32_t)box_w, (cuuint32_t)box_h, 1};
+    cuuint32_t box[4] = {(cuuint32_t)(box_c ? box_c : C), (cuuint32_t)box_w, (cuuint32_t)box_h, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
+    // a box row of 64 channels is 128 bytes, of 32 channels 64 bytes: the swizzle span follows it
     CUresult r = g.encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, box[0] == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? MT_OK : MT_ERR_CUDA;
 }
 
@@ -232,6 +236,8 @@ mt_status ensure_workspace(int n) {
             CU_OK(cudaMemset(g.act[b], 0, bytes));
             if (f.kind == MT_CONV3X3) {
                 mt_status st = encode_nhwc(&g.act_map[b], g.act[b], f.in_ch, f.w, f.h, cap, g.conv.Wp, g.conv.R + 2);
+                if (st != MT_OK) return st;
+                st = encode_nhwc(&g.act_store_map[b], g.act[b], f.in_ch, f.w, f.h, cap, 32, 1, 32);
                 if (st != MT_OK) return st;
             }
         }
@@ -430,6 +436,10 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
     int tiles_per_image = 0;
     for (const HostLayer& f : g.family)
         if (f.kind == MT_CONV3X3) tiles_per_image = g.conv.strips_per_image;
+    // Conv layers run on CTA pairs (two images of a tenant per cluster) when the strip geometry allows the tap
+    // pairing; MT_CONV_PAIR=0 forces the one-CTA executor.
+    const char* cpair_env = getenv("MT_CONV_PAIR");
+    const bool conv_pair = tiles_per_image > 0 && g.conv.Wp == 64 && g.sm_count >= 2 && !(cpair_env && cpair_env[0] == '0');
 
     // Dense families: the payload rows move into bucketed order inside the scatter pass when the batch is spread over
     // enough CTAs and small enough for them; otherwise as a gather pass of its own over the whole GPU.
@@ -443,6 +453,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
         a.row_bytes = g.in_elems * 2; a.dst_ld_bytes = g.act_ld[0] * 2;
         for (int l = 0; l < 8; ++l) {
             a.tile_n[l] = g.tile_n[l]; a.tile_m[l] = pair_mode[l] ? 2 * BM : BM;
+            if (l < L && g.family[l].kind == MT_CONV3X3) a.tile_m[l] = conv_pair ? 2 : 1;
             a.items[l] = (l < MT_MAX_LAYERS) ? g.d_items[l] : nullptr;
         }
         a.item_grid = g.sm_count;
@@ -494,7 +505,10 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             a.stage_bytes = g.conv.stage_bytes; a.n_stages = g.conv.n_stages;
             a.strips_per_image = g.conv.strips_per_image; a.box_bytes = g.conv.box_bytes;
             a.status = g.d_status;
-            launch_grouped_conv(l == 0 ? in_map : g.act_map[l], a, g.conv.smem_bytes, g.sm_count, s);
+            // a layer that feeds the pool stores nothing: any valid map will do for it
+            if (conv_pair) CU_OK(launch_grouped_conv_pair(l == 0 ? in_map : g.act_map[l], feeds_pool ? (l == 0 ? in_map : g.act_map[l]) : g.act_store_map[l + 1],
+                                                          a, conv_pair_smem_bytes(g.conv), g.sm_count, s));
+            else launch_grouped_conv(l == 0 ? in_map : g.act_map[l], a, g.conv.smem_bytes, g.sm_count, s);
         } else {
             Timer t(K_POOL, s);
             // a pool always follows a conv (checked at registration), whose epilogue already reduced every strip
@@ -584,7 +598,7 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
         const size_t n_tiles = padded_weight_tiles(h);
         size_t wbytes, raw;
         if (h.kind == MT_DENSE) { wbytes = n_tiles * (size_t)(h.in_ch / BK) * TILE_BYTES; raw = (size_t)h.out_ch * h.in_ch * 2; }
-        else { wbytes = (size_t)9 * h.out_ch * h.in_ch * 2; raw = wbytes; }
+        else { raw = (size_t)9 * h.out_ch * h.in_ch * 2; wbytes = raw + 2 * (size_t)kConvPairWeightBytes; }   // one-CTA image + the pair's two
         w_off[l] = total; total += align_up(wbytes, 1024);
         b_off[l] = total; total += align_up(n_tiles * BN * sizeof(float), 1024);
         if (raw > raw_max) raw_max = raw;
@@ -615,7 +629,10 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
         }
         if (e != cudaSuccess) break;
         if (h.kind == MT_DENSE) launch_pretile_dense(src, h.out_ch, h.in_ch, (uint16_t*)(block + w_off[l]), 0);
-        else launch_pretile_conv(src, h.out_ch, h.in_ch, (uint16_t*)(block + w_off[l]), 0);
+        else {
+            launch_pretile_conv(src, h.out_ch, h.in_ch, (uint16_t*)(block + w_off[l]), 0);
+            launch_pretile_conv_pair(src, (uint16_t*)(block + w_off[l]) + kConvPairImageOffset, 0);
+        }
         e = cudaGetLastError();
         if (e == cudaSuccess && layers[l].bias)
             e = cudaMemcpy(block + b_off[l], layers[l].bias, sizeof(float) * h.out_ch, cudaMemcpyDefault);

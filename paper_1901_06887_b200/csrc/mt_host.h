@@ -37,7 +37,8 @@ struct BucketArgs {
     int n_layers;
     int rows_per_unit;        // conv: tiles per image
     int tile_n[8];            // dense: output columns per work item of each layer (128 or 256)
-    int tile_m[8];            // dense: rows per work item of each layer (128, or 256 for the CTA-pair executor)
+    int tile_m[8];            // dense: rows per work item of each layer (128, or 256 for the CTA-pair executor);
+                              // conv: images per work unit (1, or 2 for the CTA-pair executor)
     int32_t* block_hist;      // [ceil(n / kHistChunk)][T + 1]
     int32_t* counts;          // [T + 1]
     int32_t* offsets;         // [T + 2]
@@ -147,6 +148,19 @@ struct ConvArgs {
 };
 cudaError_t configure_grouped_conv();
 void launch_grouped_conv(const CUtensorMap& tmap_x, const ConvArgs& a, int smem_bytes, int sm_count, cudaStream_t s);
+
+// CTA-pair form of the conv executor (grouped_conv_pair.cu; padded row length 64 only).  Its weight images (two of
+// kConvPairWeightBytes, rank 0 first) follow the one-CTA image in the layer's weight block, kConvPairImageOffset
+// elements in.  ConvArgs::tile_prefix must count (pair of images, strip) units: BucketArgs::tile_m = 2 for the layer.
+constexpr int kConvPairWeightBytes = 60 * 1024;
+constexpr int kConvPairImageOffset = 9 * 64 * 64;          // bf16 elements of the one-CTA image
+void launch_pretile_conv_pair(const uint16_t* w, uint16_t* out, cudaStream_t s);
+int conv_pair_smem_bytes(const ConvPlan& plan);
+cudaError_t configure_grouped_conv_pair();
+// tmap_y: the layer's output (NHWC bf16) as boxes of 32 channels x 32 pixels x 1 row, 64-byte swizzle (unused by a
+// layer that feeds the pool)
+cudaError_t launch_grouped_conv_pair(const CUtensorMap& tmap_x, const CUtensorMap& tmap_y, const ConvArgs& a, int smem_bytes,
+                                     int sm_count, cudaStream_t s);
 
 // Second half of the fused pooling: sums the per-strip channel sums of each image and divides by H*W.
 void launch_pool_finalize(const float* partial, int n, int strips, int C, int HW, uint16_t* out, int ld_out,

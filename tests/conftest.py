@@ -26,3 +26,12 @@ def small_batch_path(request, monkeypatch):
     if request.param == "layered":
         monkeypatch.setenv("MT_FUSED", "0")
     return request.param
+
+
+@pytest.fixture(params=["pair", "single"])
+def conv_path(request, monkeypatch):
+    """Conv layers whose padded row length is 64 pixels run on CTA pairs (two images of a tenant per cluster);
+    MT_CONV_PAIR=0 sends them to the one-CTA executor.  Tests that take this fixture run once on each."""
+    if request.param == "single":
+        monkeypatch.setenv("MT_CONV_PAIR", "0")
+    return request.param

@@ -29,7 +29,7 @@ def test_config3_full():
     full(3, 4, max_models=1024)
 
 
-def test_config4_full():
+def test_config4_full(conv_path):
     full(4, 3)
 
 

@@ -90,13 +90,13 @@ def test_cta_pair_executor(n, tenants, widths, monkeypatch):
 
 
 @pytest.mark.parametrize("h,w", [(8, 8), (5, 7), (56, 56), (3, 126), (17, 20)])
-def test_config4_reduced_geometries(h, w):
+def test_config4_reduced_geometries(h, w, conv_path):
     wl = synth.make_workload(4, n=7, n_tenants=3, h=h, w=w, n_conv=2)
     run_and_check(wl.models, wl.model_ids, wl.inputs)
 
 
 @pytest.mark.parametrize("h,w,n,tenants", [(56, 56, 40, 5), (37, 40, 30, 4), (10, 33, 200, 3)])
-def test_conv_many_strips_per_cta(h, w, n, tenants):
+def test_conv_many_strips_per_cta(h, w, n, tenants, conv_path):
     # enough images that every CTA walks several strips: tap pairing across strip borders, the ring of TMEM
     # accumulators wrapping around, tenant changes (weight reloads) inside a CTA's range, ragged last strips
     wl = synth.make_workload(4, n=n, n_tenants=tenants, h=h, w=w, n_conv=3)
