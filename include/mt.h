@@ -100,6 +100,16 @@ mt_status mt_infer(const void* inputs, const int32_t* model_ids, int32_t n, void
 mt_status mt_infer_host(const void* inputs_host, const int32_t* model_ids_host, int32_t n,
                         void* outputs_host, void* stream);
 
+/* The same, without the final synchronisation, for callers that keep several batches in flight: everything is
+ * enqueued on `stream` (copy in, the pass, copy out) and the call returns at once; synchronise `stream` before
+ * reading outputs_host.  Host buffers must be pinned (cudaHostAlloc / cudaHostRegister) for the copies to be
+ * asynchronous, and must stay untouched until the stream has passed the call.  Two device staging slots are used
+ * in turn: a caller that alternates between TWO streams overlaps one batch's copies with its neighbours' kernels
+ * (the kernels themselves run one batch after the other, since they share one workspace; the library orders them
+ * with events).  mt_infer and mt_infer_host must not be in flight on other streams at the same time. */
+mt_status mt_infer_host_async(const void* inputs_host, const int32_t* model_ids_host, int32_t n,
+                              void* outputs_host, void* stream);
+
 /* Mark the id dead and free its weights.  Synchronises the device first, so it cannot race an
  * mt_infer in flight.  The id may be re-issued by a later mt_register_model. */
 mt_status mt_release(int32_t model_id);

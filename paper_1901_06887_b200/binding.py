@@ -20,7 +20,7 @@ STATUS_NAMES = {0: "MT_OK", 1: "MT_ERR_INVALID_ARG", 2: "MT_ERR_BAD_MODEL_ID", 3
                 4: "MT_ERR_UNSUPPORTED", 5: "MT_ERR_OOM", 6: "MT_ERR_CUDA", 7: "MT_ERR_ARCH",
                 8: "MT_ERR_TIMEOUT", 9: "MT_ERR_NOT_INIT"}
 
-EXPORTS = ["mt_init", "mt_shutdown", "mt_register_model", "mt_infer", "mt_infer_host", "mt_release",
+EXPORTS = ["mt_init", "mt_shutdown", "mt_register_model", "mt_infer", "mt_infer_host", "mt_infer_host_async", "mt_release",
            "mt_get_async_status", "mt_status_string", "mt_debug_last_bucketing", "mt_set_kernel_timing",
            "mt_get_kernel_times", "mt_bucket_noalloc", "mt_debug_wait_timeout", "mt_debug_launch_count"]
 
@@ -53,6 +53,7 @@ def lib() -> ctypes.CDLL:
         l.mt_register_model.argtypes = [ctypes.POINTER(LayerDesc), i32, ctypes.POINTER(i32)]
         l.mt_infer.argtypes = [vp, vp, i32, vp, vp]
         l.mt_infer_host.argtypes = [vp, vp, i32, vp, vp]
+        l.mt_infer_host_async.argtypes = [vp, vp, i32, vp, vp]
         l.mt_release.argtypes = [i32]
         l.mt_get_async_status.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32)]
         l.mt_status_string.argtypes = [i32]
@@ -133,6 +134,14 @@ def mt_infer_host(inputs, model_ids, n: int, outputs, stream=None) -> None:
     """Same with host buffers (pinned torch tensors or numpy arrays); returns after the outputs have landed."""
     _check(lib().mt_infer_host(_ptr(inputs), _ptr(model_ids), int(n), _ptr(outputs), _stream_handle(stream)),
            "mt_infer_host")
+
+
+def mt_infer_host_async(inputs, model_ids, n: int, outputs, stream=None) -> None:
+    """mt_infer_host without the final synchronisation: pinned host buffers, everything enqueued on `stream`.
+    Alternate between two streams to overlap one batch's copies with the next batch's kernels; synchronise the
+    stream before reading `outputs`."""
+    _check(lib().mt_infer_host_async(_ptr(inputs), _ptr(model_ids), int(n), _ptr(outputs), _stream_handle(stream)),
+           "mt_infer_host_async")
 
 
 def mt_get_async_status(stream=None) -> Tuple[int, int]:

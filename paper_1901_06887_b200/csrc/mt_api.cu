@@ -87,6 +87,18 @@ struct Ctx {
     float* st_out = nullptr;
     int st_cap = 0;
 
+    // staging for mt_infer_host_async: two slots used in turn, so that the copies of one call overlap the compute
+    // of its neighbours when the caller alternates between two streams
+    void* as_in[2] = {nullptr, nullptr};
+    int32_t* as_ids[2] = {nullptr, nullptr};
+    float* as_out[2] = {nullptr, nullptr};
+    int as_cap = 0;
+    int as_next = 0;
+    cudaEvent_t as_slot_done[2] = {nullptr, nullptr};   // the slot's device-to-host copy has finished
+    bool as_slot_used[2] = {false, false};
+    cudaEvent_t as_compute_done = nullptr;               // the previous call's kernels have finished (shared workspace)
+    bool as_have_compute = false;
+
     // timing
     int timing = 0;                      // 0 off, 1 every kernel, 2 only the layer executors
     std::vector<TimedLaunch> timed;
@@ -556,6 +568,15 @@ mt_status mt_shutdown(void) {
     cudaFree(g.st_ids); g.st_ids = nullptr;
     cudaFree(g.st_out); g.st_out = nullptr;
     g.st_cap = 0;
+    for (int k = 0; k < 2; ++k) {
+        cudaFree(g.as_in[k]); g.as_in[k] = nullptr;
+        cudaFree(g.as_ids[k]); g.as_ids[k] = nullptr;
+        cudaFree(g.as_out[k]); g.as_out[k] = nullptr;
+        if (g.as_slot_done[k]) { cudaEventDestroy(g.as_slot_done[k]); g.as_slot_done[k] = nullptr; }
+        g.as_slot_used[k] = false;
+    }
+    if (g.as_compute_done) { cudaEventDestroy(g.as_compute_done); g.as_compute_done = nullptr; }
+    g.as_cap = 0; g.as_next = 0; g.as_have_compute = false;
     for (TimedLaunch& t : g.timed) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
     g.timed.clear();
     for (cudaEvent_t e : g.event_pool) cudaEventDestroy(e);
@@ -729,6 +750,55 @@ mt_status mt_infer_host(const void* inputs_host, const int32_t* model_ids_host, 
     if (st != MT_OK) return st;
     CU_OK(cudaMemcpyAsync(outputs_host, g.st_out, (size_t)n * g.out_elems * sizeof(float), cudaMemcpyDeviceToHost, s));
     CU_OK(cudaStreamSynchronize(s));
+    return MT_OK;
+}
+
+mt_status mt_infer_host_async(const void* inputs_host, const int32_t* model_ids_host, int32_t n, void* outputs_host,
+                              void* stream) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g.init) return MT_ERR_NOT_INIT;
+    if (n < 0) return MT_ERR_INVALID_ARG;
+    if (n == 0) return MT_OK;
+    if (!inputs_host || !model_ids_host || !outputs_host) return MT_ERR_INVALID_ARG;
+    if (!g.has_family || g.live == 0) return MT_ERR_BAD_MODEL_ID;
+    CU_OK(cudaSetDevice(g.device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (n > g.as_cap) {
+        CU_OK(cudaDeviceSynchronize());
+        for (int k = 0; k < 2; ++k) {
+            cudaFree(g.as_in[k]); cudaFree(g.as_ids[k]); cudaFree(g.as_out[k]);
+            g.as_in[k] = nullptr; g.as_ids[k] = nullptr; g.as_out[k] = nullptr;
+            g.as_slot_used[k] = false;
+        }
+        g.as_cap = 0;
+        for (int k = 0; k < 2; ++k) {
+            CU_OK(cudaMalloc(&g.as_in[k], (size_t)n * g.in_elems * 2));
+            CU_OK(cudaMalloc(&g.as_ids[k], (size_t)n * sizeof(int32_t)));
+            CU_OK(cudaMalloc(&g.as_out[k], (size_t)n * g.out_elems * sizeof(float)));
+            if (!g.as_slot_done[k]) CU_OK(cudaEventCreateWithFlags(&g.as_slot_done[k], cudaEventDisableTiming));
+        }
+        if (!g.as_compute_done) CU_OK(cudaEventCreateWithFlags(&g.as_compute_done, cudaEventDisableTiming));
+        g.as_have_compute = false;
+        g.as_cap = n;
+    }
+    // grow the workspace (a device-wide synchronisation) before anything of this call is in flight
+    mt_status st = ensure_workspace(n);
+    if (st != MT_OK) return st;
+    const int k = g.as_next;
+    g.as_next ^= 1;
+    // the slot's previous user must have copied its outputs out
+    if (g.as_slot_used[k]) CU_OK(cudaStreamWaitEvent(s, g.as_slot_done[k], 0));
+    CU_OK(cudaMemcpyAsync(g.as_in[k], inputs_host, (size_t)n * g.in_elems * 2, cudaMemcpyHostToDevice, s));
+    CU_OK(cudaMemcpyAsync(g.as_ids[k], model_ids_host, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+    // the kernels of consecutive calls share one workspace: they run one call after the other, whatever the streams
+    if (g.as_have_compute) CU_OK(cudaStreamWaitEvent(s, g.as_compute_done, 0));
+    st = infer_device(g.as_in[k], g.as_ids[k], n, g.as_out[k], s);
+    if (st != MT_OK) return st;
+    CU_OK(cudaEventRecord(g.as_compute_done, s));
+    g.as_have_compute = true;
+    CU_OK(cudaMemcpyAsync(outputs_host, g.as_out[k], (size_t)n * g.out_elems * sizeof(float), cudaMemcpyDeviceToHost, s));
+    CU_OK(cudaEventRecord(g.as_slot_done[k], s));
+    g.as_slot_used[k] = true;
     return MT_OK;
 }
 

@@ -164,6 +164,27 @@ def test_repeat_runs_are_bitwise_identical_and_host_entry_matches():
     assert np.array_equal(harness.run_batch(wl.model_ids, wl.inputs, 64), got)
 
 
+def test_async_host_entry_on_two_streams_matches_device_entry():
+    # five different batches in flight on two alternating streams: every batch's outputs equal mt_infer's, bit for bit
+    wl = synth.make_workload(2, n=700, n_tenants=6, widths=(256, 512, 384, 64))
+    fresh()
+    harness.register_models(wl.models)
+    batches = [synth.make_requests(2, wl.models, n=n, salt=50 + k) for k, n in enumerate((700, 300, 700, 650, 1))]
+    want = [harness.run_batch(ids, x, 64) for ids, x in batches]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    h_in = [torch.from_numpy(x.view(np.int16)).pin_memory() for _, x in batches]
+    h_ids = [torch.from_numpy(ids).pin_memory() for ids, _ in batches]
+    h_out = [torch.full((len(ids), 64), float("nan"), dtype=torch.float32).pin_memory() for ids, _ in batches]
+    for rep in range(2):
+        for k in range(len(batches)):
+            mt.mt_infer_host_async(h_in[k], h_ids[k], len(batches[k][0]), h_out[k], streams[k % 2])
+        torch.cuda.synchronize()
+        assert mt.mt_get_async_status() == (0, -1)
+        for k in range(len(batches)):
+            assert np.array_equal(h_out[k].numpy(), want[k]), (rep, k)
+            h_out[k].fill_(float("nan"))
+
+
 def test_growing_batches_and_wider_models_reallocate_correctly(small_batch_path):
     rng = np.random.default_rng(9)
     mk = lambda h: synth.make_mlp(3, h, (128, h, 64))
