@@ -102,21 +102,33 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                 const int nbox = (cur.rows_valid + 31) >> 5;
                 // weight tile (nt, kb) of 128 rows x 64 columns starts at element (nt * kblocks + kb) * 8192
                 const uint16_t* wsrc = cur.w + (size_t)cur.n_tile * kWTiles * kblocks * (BN * BK);
+                // Only the 8-row groups of a weight tile that hold output features are fetched (a 64-wide last layer
+                // would otherwise stream as many zero rows as weights); what stays in the stage from earlier items
+                // only reaches accumulator columns (or, transposed, lanes) that are never stored.
+                uint32_t wbytes[kWTiles];
+                uint32_t wsum = 0;
+#pragma unroll
+                for (int wt = 0; wt < kWTiles; ++wt) {
+                    const int rows = min(BN, max(0, cur.N - (cur.n_tile * kWTiles + wt) * BN));
+                    wbytes[wt] = (uint32_t)((rows + 7) & ~7) * (BK * 2);
+                    wsum += wbytes[wt];
+                }
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { ok = false; break; }
                     const uint32_t a_dst = base + stage * kStageBytes;
                     if (swap) {          // only the 32-row boxes that hold the segment's requests
-                        mbar_expect_tx(full_bar(stage), (uint32_t)(nbox * 4096 + kWTiles * TILE_BYTES));
+                        mbar_expect_tx(full_bar(stage), (uint32_t)(nbox * 4096) + wsum);
                         for (int b = 0; b < nbox; ++b)
                             tma_load_2d(a_dst + b * 4096, &tmap_a32, kb * BK, cur.row0 + b * 32, full_bar(stage));
                     } else {
-                        mbar_expect_tx(full_bar(stage), kStageBytes);
+                        mbar_expect_tx(full_bar(stage), (uint32_t)TILE_BYTES + wsum);
                         tma_load_2d(a_dst, &tmap_a, kb * BK, cur.row0, full_bar(stage));
                     }
 #pragma unroll
                     for (int wt = 0; wt < kWTiles; ++wt)
-                        bulk_load(a_dst + (1 + wt) * TILE_BYTES, wsrc + ((size_t)wt * kblocks + kb) * (BN * BK),
-                                  TILE_BYTES, full_bar(stage));
+                        if (wbytes[wt])
+                            bulk_load(a_dst + (1 + wt) * TILE_BYTES, wsrc + ((size_t)wt * kblocks + kb) * (BN * BK),
+                                      wbytes[wt], full_bar(stage));
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
                 cur = nxt;
