@@ -248,14 +248,32 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
     int run = cta_excl_scan(sum, s_warp, &total);
     for (int t = lo; t < hi; ++t) { offsets[t] = run; s_next[t] = run; counts[t] = s_cnt[t]; run += s_cnt[t]; }
     if (threadIdx.x == 0) offsets[T1] = total;
-    for (int l = 0; l < n_layers; ++l) {
-        int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
+    {
         const int hi_t = min(hi, T);
-        int usum = 0;
-        for (int t = lo; t < hi_t; ++t) usum += layer_units(models, t, l, s_cnt[t], rows_per_unit, tn.v[l], tn.m[l]);
-        int urun = cta_excl_scan(usum, s_warp, &total);
-        for (int t = lo; t < hi_t; ++t) { prefix[t] = urun; urun += layer_units(models, t, l, s_cnt[t], rows_per_unit, tn.v[l], tn.m[l]); }
-        if (threadIdx.x == 0) prefix[T] = total;
+        if (per == 1) {
+            // one bucket per thread: the units of all layers first, so that the loads from the tenant table are in
+            // flight together instead of one round trip per layer
+            int units[MT_MAX_LAYERS];
+#pragma unroll
+            for (int l = 0; l < MT_MAX_LAYERS; ++l)
+                units[l] = (l < n_layers && lo < hi_t) ? layer_units(models, lo, l, s_cnt[lo], rows_per_unit, tn.v[l], tn.m[l]) : 0;
+#pragma unroll
+            for (int l = 0; l < MT_MAX_LAYERS; ++l) {
+                if (l >= n_layers) break;
+                const int urun = cta_excl_scan(units[l], s_warp, &total);
+                if (lo < hi_t) tile_prefix[(size_t)l * (T + 1) + lo] = urun;
+                if (threadIdx.x == 0) tile_prefix[(size_t)l * (T + 1) + T] = total;
+            }
+        } else {
+            for (int l = 0; l < n_layers; ++l) {
+                int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
+                int usum = 0;
+                for (int t = lo; t < hi_t; ++t) usum += layer_units(models, t, l, s_cnt[t], rows_per_unit, tn.v[l], tn.m[l]);
+                int urun = cta_excl_scan(usum, s_warp, &total);
+                for (int t = lo; t < hi_t; ++t) { prefix[t] = urun; urun += layer_units(models, t, l, s_cnt[t], rows_per_unit, tn.v[l], tn.m[l]); }
+                if (threadIdx.x == 0) prefix[T] = total;
+            }
+        }
     }
     __syncthreads();
     // rounds in order, and inside a round the warps take turns: positions inside a bucket ascend with arrival index
@@ -283,9 +301,13 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
     for (int l = 0; l < n_layers; ++l) {
         WorkItem* out = items.v[l];
         if (!out) continue;
+        // the layer's unit prefixes into shared memory (s_cnt is free by now): the search per item stays on the SM
         const int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
-        const int n_items = prefix[T];
-        for (int item = threadIdx.x; item < n_items; item += nthr) out[item] = make_work_item(item, l, T, models, offsets, prefix, tn.m[l]);
+        for (int t = threadIdx.x; t < T1; t += nthr) s_cnt[t] = prefix[t];
+        __syncthreads();
+        const int n_items = s_cnt[T];
+        for (int item = threadIdx.x; item < n_items; item += nthr) out[item] = make_work_item(item, l, T, models, offsets, s_cnt, tn.m[l]);
+        __syncthreads();
     }
 }
 
