@@ -59,21 +59,74 @@ __device__ __forceinline__ int cta_excl_scan(int v, int32_t* s_warp, int* total)
     return r;
 }
 
-// Work units (tiles / strips) tenant t contributes to layer l, given its request count c.
+// The same for MT_MAX_LAYERS values per thread at once (three barriers for all of them instead of three each).
+// s_vec: MT_MAX_LAYERS x 33 ints of shared memory.
+__device__ __forceinline__ void cta_excl_scan_vec(const int (&v)[MT_MAX_LAYERS], int (&excl)[MT_MAX_LAYERS],
+                                                  int (&total)[MT_MAX_LAYERS], int32_t* s_vec) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+    int incl[MT_MAX_LAYERS];
+#pragma unroll
+    for (int l = 0; l < MT_MAX_LAYERS; ++l) {
+        incl[l] = v[l];
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int u = __shfl_up_sync(0xffffffffu, incl[l], d);
+            if (lane >= d) incl[l] += u;
+        }
+        if (lane == 31) s_vec[l * 33 + warp] = incl[l];
+    }
+    __syncthreads();
+    if (warp == 0) {
+#pragma unroll
+        for (int l = 0; l < MT_MAX_LAYERS; ++l) {
+            const int w = (lane < n_warps) ? s_vec[l * 33 + lane] : 0;
+            int wi = w;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int u = __shfl_up_sync(0xffffffffu, wi, d);
+                if (lane >= d) wi += u;
+            }
+            s_vec[l * 33 + lane] = wi - w;
+            if (lane == 31) s_vec[l * 33 + 32] = wi;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int l = 0; l < MT_MAX_LAYERS; ++l) {
+        excl[l] = incl[l] - v[l] + s_vec[l * 33 + warp];
+        total[l] = s_vec[l * 33 + 32];
+    }
+    __syncthreads();
+}
+
+// What the unit count of a layer depends on, read from the tenant table without looking at the request count first:
+// callers fetch the heads of all layers back to back, so the loads are in flight together (a load behind a branch on
+// the count costs one memory round trip per layer on the single CTA's critical path).
+struct LayerHead { int kind, N; };
+__device__ __forceinline__ LayerHead load_head(const ModelDev* models, int t, int l) {
+    const LayerDev& L = models[t].layer[l];
+    LayerHead h;
+    h.kind = __ldg(&L.kind);
+    h.N = __ldg(&L.N);
+    return h;
+}
+// Work units (tiles / strips) a tenant with c requests contributes to a layer.
+__device__ __forceinline__ int units_of(LayerHead h, int c, int rows_per_unit, int tile_n, int tile_m) {
+    if (c <= 0) return 0;
+    if (h.kind == MT_DENSE) return ((c + tile_m - 1) / tile_m) * ((h.N + tile_n - 1) / tile_n);
+    if (h.kind == MT_CONV3X3) return ((c + tile_m - 1) / tile_m) * rows_per_unit;   // tile_m = images per unit
+    return 0;
+}
 __device__ __forceinline__ int layer_units(const ModelDev* models, int t, int l, int c, int rows_per_unit, int tile_n,
                                            int tile_m) {
-    if (c <= 0) return 0;
-    const LayerDev& L = models[t].layer[l];
-    if (L.kind == MT_DENSE) return ((c + tile_m - 1) / tile_m) * ((L.N + tile_n - 1) / tile_n);
-    if (L.kind == MT_CONV3X3) return ((c + tile_m - 1) / tile_m) * rows_per_unit;   // tile_m = images per unit
-    return 0;
+    return units_of(load_head(models, t, l), c, rows_per_unit, tile_n, tile_m);
 }
 
 // Offsets (exclusive scan of counts over the T + 1 buckets, offsets[T + 1] = n) and, per layer, the prefix sums of
 // the work units each tenant contributes.  Run by one CTA of any multiple of 32 threads; counts[] must be visible.
 __device__ __forceinline__ void scan_buckets(int T, const ModelDev* __restrict__ models, int n_layers, int rows_per_unit,
                                              const LayerTileN& tn, const int32_t* counts, int32_t* __restrict__ offsets,
-                                             int32_t* __restrict__ tile_prefix, int32_t* s_warp) {
+                                             int32_t* __restrict__ tile_prefix, int32_t* s_warp, int32_t* s_vec) {
     const int T1 = T + 1;
     const int per = (T1 + (int)blockDim.x - 1) / (int)blockDim.x;     // each thread owns `per` consecutive buckets
     const int lo = min((int)threadIdx.x * per, T1), hi = min(lo + per, T1);
@@ -87,16 +140,21 @@ __device__ __forceinline__ void scan_buckets(int T, const ModelDev* __restrict__
     if (per == 1) {
         // one bucket per thread (the usual case): the units of all layers first, so that the loads from the tenant
         // table are in flight together instead of one round trip per layer
+        LayerHead head[MT_MAX_LAYERS];
+        const int t_own = min(lo, T - 1);
+#pragma unroll
+        for (int l = 0; l < MT_MAX_LAYERS; ++l) head[l] = (l < n_layers) ? load_head(models, t_own, l) : LayerHead{-1, 0};
+        const int c_own = (lo < hi_t) ? counts[lo] : 0;
         int units[MT_MAX_LAYERS];
 #pragma unroll
-        for (int l = 0; l < MT_MAX_LAYERS; ++l)
-            units[l] = (l < n_layers && lo < hi_t) ? layer_units(models, lo, l, counts[lo], rows_per_unit, tn.v[l], tn.m[l]) : 0;
+        for (int l = 0; l < MT_MAX_LAYERS; ++l) units[l] = units_of(head[l], c_own, rows_per_unit, tn.v[l], tn.m[l]);
+        int urun[MT_MAX_LAYERS], utotal[MT_MAX_LAYERS];
+        cta_excl_scan_vec(units, urun, utotal, s_vec);
 #pragma unroll
         for (int l = 0; l < MT_MAX_LAYERS; ++l) {
             if (l >= n_layers) break;
-            const int urun = cta_excl_scan(units[l], s_warp, &total);
-            if (lo < hi_t) tile_prefix[(size_t)l * (T + 1) + lo] = urun;
-            if (threadIdx.x == 0) tile_prefix[(size_t)l * (T + 1) + T] = total;
+            if (lo < hi_t) tile_prefix[(size_t)l * (T + 1) + lo] = urun[l];
+            if (threadIdx.x == 0) tile_prefix[(size_t)l * (T + 1) + T] = utotal[l];
         }
         return;
     }
@@ -122,6 +180,7 @@ bucket_hist_scan(const int32_t* __restrict__ ids, int n, int T, const ModelDev* 
     pdl_wait();
     extern __shared__ int32_t s_hist[];   // T + 1
     __shared__ int32_t s_warp[33];
+    __shared__ int32_t s_vec[MT_MAX_LAYERS * 33];
     __shared__ int s_last;
     const int T1 = T + 1;
     for (int t = threadIdx.x; t < T1; t += blockDim.x) s_hist[t] = 0;
@@ -168,7 +227,7 @@ bucket_hist_scan(const int32_t* __restrict__ ids, int n, int T, const ModelDev* 
         counts[t] = run;
     }
     __syncthreads();
-    scan_buckets(T, models, n_layers, rows_per_unit, tn, counts, offsets, tile_prefix, s_warp);
+    scan_buckets(T, models, n_layers, rows_per_unit, tn, counts, offsets, tile_prefix, s_warp, s_vec);
 }
 
 struct ItemPtrs { WorkItem* v[8]; };
@@ -215,6 +274,7 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
     pdl_wait();
     extern __shared__ int32_t s_mem[];          // s_cnt[T + 1], s_next[T + 1]
     __shared__ int32_t s_warp[33];
+    __shared__ int32_t s_vec[MT_MAX_LAYERS * 33];
     const int T1 = T + 1;
     int32_t* s_cnt = s_mem;
     int32_t* s_next = s_mem + T1;
@@ -253,16 +313,21 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
         if (per == 1) {
             // one bucket per thread: the units of all layers first, so that the loads from the tenant table are in
             // flight together instead of one round trip per layer
+            LayerHead head[MT_MAX_LAYERS];
+            const int t_own = min(lo, T - 1);
+#pragma unroll
+            for (int l = 0; l < MT_MAX_LAYERS; ++l) head[l] = (l < n_layers) ? load_head(models, t_own, l) : LayerHead{-1, 0};
+            const int c_own = (lo < hi_t) ? s_cnt[lo] : 0;
             int units[MT_MAX_LAYERS];
 #pragma unroll
-            for (int l = 0; l < MT_MAX_LAYERS; ++l)
-                units[l] = (l < n_layers && lo < hi_t) ? layer_units(models, lo, l, s_cnt[lo], rows_per_unit, tn.v[l], tn.m[l]) : 0;
+            for (int l = 0; l < MT_MAX_LAYERS; ++l) units[l] = units_of(head[l], c_own, rows_per_unit, tn.v[l], tn.m[l]);
+            int urun[MT_MAX_LAYERS], utotal[MT_MAX_LAYERS];
+            cta_excl_scan_vec(units, urun, utotal, s_vec);
 #pragma unroll
             for (int l = 0; l < MT_MAX_LAYERS; ++l) {
                 if (l >= n_layers) break;
-                const int urun = cta_excl_scan(units[l], s_warp, &total);
-                if (lo < hi_t) tile_prefix[(size_t)l * (T + 1) + lo] = urun;
-                if (threadIdx.x == 0) tile_prefix[(size_t)l * (T + 1) + T] = total;
+                if (lo < hi_t) tile_prefix[(size_t)l * (T + 1) + lo] = urun[l];
+                if (threadIdx.x == 0) tile_prefix[(size_t)l * (T + 1) + T] = utotal[l];
             }
         } else {
             for (int l = 0; l < n_layers; ++l) {
