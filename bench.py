@@ -35,9 +35,9 @@ DEFAULT_STEPS = {1: 5000, 2: 1500, 3: 2500, 4: 1500, 5: 50}
 ORACLE_SAMPLE = {1: 64, 2: 2048, 3: 16384, 4: 24, 5: 96}      # requests of the batch the CPU baseline times
 N_INPUT_BUFFERS = 3
 # DRAM traffic of the dominant kernel from the ncu captures summarised under profiles/ (see there):
-#   config 2: measured on a reduced case, traffic / algorithmic bytes = 0.996, scaled to the full launch;
+#   config 2: measured on a reduced case, traffic / algorithmic bytes = 0.995, scaled to the full launch;
 #   config 4: measured at full size, bytes per step (four conv launches).  None = not captured.
-TRAFFIC_RATIO = {2: 0.996}
+TRAFFIC_RATIO = {2: 0.995}
 TRAFFIC_BYTES = {4: 615.7e6}
 
 
