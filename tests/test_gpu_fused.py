@@ -95,3 +95,50 @@ def test_layered_last_layer_writes_arrival_order_with_rejected_ids(n):
     assert np.isnan(got[~good]).all() and np.isfinite(got[good]).all()
     ref = oracle.forward(models, ids[good], x[good])
     assert harness.scaled_error(got[good], ref).max() <= TOL
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_families_against_the_oracle(seed):
+    # seeded random MLP families and batches: widths from 64 to 640 (inputs of a layer in multiples of 64, outputs
+    # arbitrary), 1 to 40 tenants some of which get no request, segment sizes straddling the 64-request
+    # (transposed items) and 128-request (row tile) borders, a few rejected ids; small draws take the one-launch
+    # path, the others the layer-by-layer path
+    rng = np.random.default_rng(1000 + seed)
+    T = int(rng.integers(1, 41))
+    depth = int(rng.integers(1, 5))
+    k_in = 64 * int(rng.integers(1, 6))
+    n_out = int(rng.integers(1, 300))
+    small = seed % 3 == 0
+    hid_choices = [64, 128, 192, 256] if small else [64, 128, 256, 320, 512, 640]
+    models = []
+    for t in range(T):
+        widths = (k_in,) + tuple(int(rng.choice(hid_choices)) for _ in range(depth - 1)) + (n_out,)
+        models.append(synth.make_mlp(8, 100 * seed + t, widths))
+    sizes = rng.choice([0, 1, 3, 63, 64, 65, 127, 128, 129, 200], size=T)
+    if small:
+        sizes = np.minimum(sizes, max(1, 500 // T))
+    ids = np.repeat(np.arange(T), sizes).astype(np.int32)
+    if len(ids) == 0:
+        ids = np.zeros(1, np.int32)
+    n_bad = int(rng.integers(0, 4))
+    ids = np.concatenate([ids, np.full(n_bad, T + 3, np.int32)])
+    rng.shuffle(ids)
+    n = len(ids)
+    x = bits(rng.standard_normal((n, k_in)))
+    fresh(max(64, T))
+    harness.register_models(models)
+    got = harness.run_batch(ids, x, n_out)
+    st, bad = mt.mt_get_async_status()
+    good = ids < T
+    if n_bad:
+        assert st == 2 and bad == int(np.flatnonzero(~good)[0])
+        assert np.isnan(got[~good]).all()
+    else:
+        assert (st, bad) == (0, -1)
+    counts, offsets, perm, inv = mt.mt_debug_last_bucketing(n)
+    oc, oo, op, oi = oracle.bucket(np.where(good, ids, T), T + 1)
+    assert np.array_equal(counts, oc[:T]) and np.array_equal(offsets, oo)
+    assert np.array_equal(perm, op) and np.array_equal(inv, oi)
+    ref = oracle.forward(models, ids[good], x[good])
+    assert np.isfinite(got[good]).all()
+    assert harness.scaled_error(got[good], ref).max() <= TOL
