@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the mixed-tenant inference hot path.
 
-One "step" = one mt_infer call: bucketing, one grouped launch per layer, un-permute, over one synthetic
+One "step" = one mt_infer call: bucketing, one grouped launch per layer (the last one returns the rows to arrival order), over one synthetic
 mixed batch.  Default workload: 64 tenants x MLP 1024-4096-4096-1024, 4096 requests, Zipf(1.1).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]

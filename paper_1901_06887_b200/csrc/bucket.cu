@@ -12,9 +12,7 @@
 //                                  bucketed order (128-bit copies), work items of the dense layers
 //           bucket_single_cta      both passes in one CTA for batches of at most 512 requests
 //           gather_rows            X_b[j, :] = X[perm[j], :] as a pass of its own (payloads too large for pass 2)
-//           unpermute_rows         out[perm[j], :] = out_b[j, :] (executors that cannot write arrival order themselves)
-#include <limits>
-
+//           (the return to arrival order, out[perm[j], :] = out_b[j, :], happens in the last layer's epilogue)
 #include "mt_device.cuh"
 #include "mt_host.h"
 
@@ -477,22 +475,6 @@ __global__ void gather_rows(const uint4* __restrict__ src, const int32_t* __rest
     }
 }
 
-// out[perm[j], :] = out_b[j, :] for j < n_valid; rows of rejected requests (j >= n_valid) become NaN.
-template <typename V>
-__global__ void unpermute_rows(const V* __restrict__ src, const int32_t* __restrict__ perm,
-                               const int32_t* __restrict__ offsets, int T, int n, int row_vec,
-                               V* __restrict__ dst, V nan_v) {
-    pdl_launch_dependents();
-    pdl_wait();
-    const int n_valid = offsets[T];
-    const long long total = (long long)n * row_vec;
-    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
-         idx += (long long)gridDim.x * blockDim.x) {
-        const int j = (int)(idx / row_vec), v = (int)(idx % row_vec);
-        dst[(size_t)perm[j] * row_vec + v] = (j < n_valid) ? src[idx] : nan_v;
-    }
-}
-
 // Self-test of the bounded wait every executor relies on: one thread waits on an mbarrier that nobody ever
 // completes; after limit_ns it must give up, raise the abort flag and report MT_ERR_TIMEOUT - and return.
 __global__ void wait_timeout_probe(int32_t* status, unsigned long long limit_ns, int32_t* gave_up) {
@@ -549,20 +531,6 @@ void launch_gather_rows(const void* src, const int32_t* perm, int n, int row_byt
     const int row_vec = row_bytes / 16;
     launch_pdl(gather_rows, dim3(grid_for((long long)n * row_vec, 256, sm_count)), dim3(256), 0, s,
         (const uint4*)src, perm, n, row_vec, (uint4*)dst, dst_ld_bytes / 16);
-}
-
-void launch_unpermute(const float* src, const int32_t* perm, const int32_t* offsets, int T, int n, int out_elems,
-                      float* dst, int sm_count, cudaStream_t s) {
-    const float qnan = std::numeric_limits<float>::quiet_NaN();
-    const bool vec_ok = (out_elems % 4 == 0) && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0);
-    if (vec_ok) {
-        const int row_vec = out_elems / 4;
-        launch_pdl(unpermute_rows<float4>, dim3(grid_for((long long)n * row_vec, 256, sm_count)), dim3(256), 0, s,
-            (const float4*)src, perm, offsets, T, n, row_vec, (float4*)dst, make_float4(qnan, qnan, qnan, qnan));
-    } else {
-        launch_pdl(unpermute_rows<float>, dim3(grid_for((long long)n * out_elems, 256, sm_count)), dim3(256), 0, s,
-            src, perm, offsets, T, n, out_elems, dst, qnan);
-    }
 }
 
 }  // namespace mt

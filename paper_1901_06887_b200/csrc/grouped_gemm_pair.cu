@@ -164,6 +164,17 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmA
         int it = 0;
         WorkItem cur = {};
         if (pair_id < total) cur = load_pair_item(p.items, pair_id);
+        // last layer: rows go straight to their arrival positions in the caller's buffer (see GemmArgs::perm)
+        const int32_t* const perm = p.out_fp32 ? p.perm : nullptr;
+        const bool out_vec_ok = (p.ld_out & 3) == 0 && (reinterpret_cast<uintptr_t>(p.out) & 15) == 0;
+        if (perm) {
+            // requests whose id was rejected sort behind every live segment and get no work item: NaN rows
+            const int n_valid = p.offsets[p.T], n_all = p.offsets[p.T + 1];
+            for (int j = n_valid + blockIdx.x; j < n_all; j += gridDim.x) {
+                float* dst = reinterpret_cast<float*>(p.out) + (size_t)perm[j] * p.ld_out;
+                for (int e = threadIdx.x - 64; e < p.ld_out; e += 128) dst[e] = __int_as_float(0x7fc00000);
+            }
+        }
         for (int item = pair_id; item < total; item += n_pairs, ++it) {
             WorkItem nxt = {};
             if (item + n_pairs < total) nxt = load_pair_item(p.items, item + n_pairs);
@@ -176,7 +187,8 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmA
             const int N = c.N, relu = c.relu;
             const int my_valid = min(BM, max(0, c.rows_valid - (int)rank * BM));
             const bool row_ok = r < my_valid;
-            const size_t grow = (size_t)(c.row0 + (int)rank * BM + r);
+            const size_t grow = (perm && row_ok) ? (size_t)__ldg(perm + c.row0 + (int)rank * BM + r)
+                                                 : (size_t)(c.row0 + (int)rank * BM + r);
 #pragma unroll 1
             for (int ch = 0; ch < kPairTN / 32; ++ch) {
                 uint32_t v[32];
@@ -204,7 +216,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmA
                     // rows past the tenant's segment belong to someone else: never stored
                 } else if (p.out_fp32) {
                     float* dst = reinterpret_cast<float*>(p.out) + grow * p.ld_out + n0;
-                    if (full_chunk && (p.ld_out & 3) == 0) {
+                    if (full_chunk && out_vec_ok) {
 #pragma unroll
                         for (int j = 0; j < 8; ++j)
                             reinterpret_cast<float4*>(dst)[j] = make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
@@ -271,6 +283,7 @@ cudaError_t launch_grouped_gemm_pair(const CUtensorMap& tmap_a, const GemmArgs& 
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 2;
+    ++g_kernel_launches;
     return cudaLaunchKernelEx(&cfg, grouped_gemm_pair_kernel, tmap_a, a);
 }
 

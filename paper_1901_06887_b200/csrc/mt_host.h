@@ -60,8 +60,6 @@ void launch_bucketing(const BucketArgs& a, cudaStream_t s);
 void launch_wait_timeout_probe(int32_t* status, unsigned long long limit_ns, int32_t* gave_up, cudaStream_t s);
 void launch_gather_rows(const void* src, const int32_t* perm, int n, int row_bytes, void* dst, int dst_ld_bytes,
                         int sm_count, cudaStream_t s);
-void launch_unpermute(const float* src, const int32_t* perm, const int32_t* offsets, int T, int n, int out_elems,
-                      float* dst, int sm_count, cudaStream_t s);
 
 // Re-lay a dense weight matrix W[N][K] (bf16, row-major) as ceil(N/128) x (K/64) tiles of 128 rows x 64
 // columns, each tile 16 KiB in the 128-byte-swizzled shared-memory image the tensor-core kernels consume;

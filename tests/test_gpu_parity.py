@@ -78,15 +78,32 @@ def test_config5_reduced():
 
 @pytest.mark.parametrize("n,tenants,widths", [(2500, 2, (256, 512, 256)), (3100, 3, (128, 768, 10)), (1024, 1, (64, 256, 256))])
 def test_cta_pair_executor(n, tenants, widths, monkeypatch):
-    # MT_PAIR=1, >= 1024 requests per tenant on average and layers >= 256 wide: the 256 x 256 CTA-pair executor runs
-    # those layers (ragged last row tiles, tiles whose second half is empty, bf16 and fp32 outputs); the result must
-    # also equal the one-CTA executor's bit for bit (same products, same accumulation order per output)
+    # >= 1024 requests per tenant on average and layers >= 256 wide: the 256 x 256 CTA-pair executor runs those
+    # layers (ragged last row tiles, tiles whose second half is empty, bf16 and fp32 outputs, the last layer writing
+    # arrival order); MT_PAIR=0 sends the same batch to the one-CTA executor, whose result must be equal bit for bit
+    # (same products, same accumulation order per output)
     wl = synth.make_workload(5, n=n, n_tenants=tenants, widths=widths)
-    monkeypatch.setenv("MT_PAIR", "1")
     got_pair, _ = run_and_check(wl.models, wl.model_ids, wl.inputs)
-    monkeypatch.delenv("MT_PAIR")
+    monkeypatch.setenv("MT_PAIR", "0")
     got_one, _ = run_and_check(wl.models, wl.model_ids, wl.inputs)
     assert np.array_equal(got_pair, got_one)
+
+
+def test_cta_pair_executor_rejected_ids_and_unaligned_output():
+    wl = synth.make_workload(5, n=2300, n_tenants=2, widths=(128, 256, 260))
+    ids = wl.model_ids.copy()
+    ids[[5, 900, 2299]] = 7                                   # never issued
+    fresh()
+    harness.register_models(wl.models)
+    buf = torch.full((2300 * 260 + 1,), float("nan"), dtype=torch.float32, device="cuda")
+    out = buf[1:].view(2300, 260)                            # 4-byte aligned only
+    mt.mt_infer(harness.bf16_bits_to_device(wl.inputs), torch.from_numpy(ids).cuda(), 2300, out)
+    assert mt.mt_get_async_status() == (2, 5)
+    got = out.cpu().numpy()
+    good = ids < 2
+    assert np.isnan(got[~good]).all()
+    ref = oracle.forward(wl.models, ids[good], wl.inputs[good])
+    assert harness.scaled_error(got[good], ref).max() <= TOL
 
 
 @pytest.mark.parametrize("h,w", [(8, 8), (5, 7), (56, 56), (3, 126), (17, 20)])
