@@ -13,18 +13,27 @@
 //           bucket_single_cta      both passes in one CTA for batches of at most 512 requests
 //           gather_rows            X_b[j, :] = X[perm[j], :] as a pass of its own (payloads too large for pass 2)
 //           (the return to arrival order, out[perm[j], :] = out_b[j, :], happens in the last layer's epilogue)
+#include <climits>
+
 #include "mt_device.cuh"
 #include "mt_host.h"
 
 namespace mt {
 
 
-struct LayerTileN { int v[8]; int m[8]; };   // per layer: columns (v) and rows (m) of one dense work item
+// Per layer: columns (v) and rows (m) of one dense work item, and the layer's kind (the same for every tenant of the
+// hosted family).
+struct LayerTileN { int v[8]; int m[8]; int kind[8]; };
+
+// Compact copy of what the bucketing passes need from the tenant table, one row of `ld` ints per field: row 0 =
+// alive flag, row 1 + l = out features of layer l.  (Reading these through the 328-byte ModelDev records costs one
+// memory sector per tenant and field; a thousand tenants' worth from a single CTA took several microseconds.)
+struct Brief { const int32_t* p; int ld; };
 
 // ids outside [0, T) or of dead models go to the extra bucket T, so they sort behind every live segment.
-__device__ __forceinline__ int classify(int id, int T, const ModelDev* models) {
+__device__ __forceinline__ int classify(int id, int T, Brief br) {
     if (id < 0 || id >= T) return T;
-    return models[id].alive ? id : T;
+    return __ldg(br.p + id) ? id : T;
 }
 
 // Exclusive scan across the threads of a CTA (any multiple of 32 threads up to 1024): returns the sum of `v` over
@@ -60,12 +69,13 @@ __device__ __forceinline__ int cta_excl_scan(int v, int32_t* s_warp, int* total)
 // The same for MT_MAX_LAYERS values per thread at once (three barriers for all of them instead of three each).
 // s_vec: MT_MAX_LAYERS x 33 ints of shared memory.
 __device__ __forceinline__ void cta_excl_scan_vec(const int (&v)[MT_MAX_LAYERS], int (&excl)[MT_MAX_LAYERS],
-                                                  int (&total)[MT_MAX_LAYERS], int32_t* s_vec) {
+                                                  int (&total)[MT_MAX_LAYERS], int32_t* s_vec, int n_used) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
     int incl[MT_MAX_LAYERS];
 #pragma unroll
     for (int l = 0; l < MT_MAX_LAYERS; ++l) {
         incl[l] = v[l];
+        if (l >= n_used) continue;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
             const int u = __shfl_up_sync(0xffffffffu, incl[l], d);
@@ -77,6 +87,7 @@ __device__ __forceinline__ void cta_excl_scan_vec(const int (&v)[MT_MAX_LAYERS],
     if (warp == 0) {
 #pragma unroll
         for (int l = 0; l < MT_MAX_LAYERS; ++l) {
+            if (l >= n_used) continue;
             const int w = (lane < n_warps) ? s_vec[l * 33 + lane] : 0;
             int wi = w;
 #pragma unroll
@@ -91,6 +102,7 @@ __device__ __forceinline__ void cta_excl_scan_vec(const int (&v)[MT_MAX_LAYERS],
     __syncthreads();
 #pragma unroll
     for (int l = 0; l < MT_MAX_LAYERS; ++l) {
+        if (l >= n_used) { excl[l] = 0; total[l] = 0; continue; }
         excl[l] = incl[l] - v[l] + s_vec[l * 33 + warp];
         total[l] = s_vec[l * 33 + 32];
     }
@@ -101,11 +113,10 @@ __device__ __forceinline__ void cta_excl_scan_vec(const int (&v)[MT_MAX_LAYERS],
 // callers fetch the heads of all layers back to back, so the loads are in flight together (a load behind a branch on
 // the count costs one memory round trip per layer on the single CTA's critical path).
 struct LayerHead { int kind, N; };
-__device__ __forceinline__ LayerHead load_head(const ModelDev* models, int t, int l) {
-    const LayerDev& L = models[t].layer[l];
+__device__ __forceinline__ LayerHead load_head(Brief br, const LayerTileN& tn, int t, int l) {
     LayerHead h;
-    h.kind = __ldg(&L.kind);
-    h.N = __ldg(&L.N);
+    h.kind = tn.kind[l];
+    h.N = __ldg(br.p + (size_t)(1 + l) * br.ld + t);
     return h;
 }
 // Work units (tiles / strips) a tenant with c requests contributes to a layer.
@@ -115,24 +126,28 @@ __device__ __forceinline__ int units_of(LayerHead h, int c, int rows_per_unit, i
     if (h.kind == MT_CONV3X3) return ((c + tile_m - 1) / tile_m) * rows_per_unit;   // tile_m = images per unit
     return 0;
 }
-__device__ __forceinline__ int layer_units(const ModelDev* models, int t, int l, int c, int rows_per_unit, int tile_n,
-                                           int tile_m) {
-    return units_of(load_head(models, t, l), c, rows_per_unit, tile_n, tile_m);
+__device__ __forceinline__ int layer_units(Brief br, const LayerTileN& tn, int t, int l, int c, int rows_per_unit) {
+    return units_of(load_head(br, tn, t, l), c, rows_per_unit, tn.v[l], tn.m[l]);
 }
 
 // Offsets (exclusive scan of counts over the T + 1 buckets, offsets[T + 1] = n) and, per layer, the prefix sums of
 // the work units each tenant contributes.  Run by one CTA of any multiple of 32 threads; counts[] must be visible.
-__device__ __forceinline__ void scan_buckets(int T, const ModelDev* __restrict__ models, int n_layers, int rows_per_unit,
+__device__ __forceinline__ void scan_buckets(int T, Brief br, int n_layers, int rows_per_unit,
                                              const LayerTileN& tn, const int32_t* counts, int32_t* __restrict__ offsets,
-                                             int32_t* __restrict__ tile_prefix, int32_t* s_warp, int32_t* s_vec) {
+                                             int32_t* __restrict__ tile_prefix, int32_t* s_warp, int32_t* s_vec,
+                                             int own_count = -1) {
+    // own_count >= 0: the caller has counts[threadIdx.x] in a register (one bucket per thread), no need to read it back
     const int T1 = T + 1;
     const int per = (T1 + (int)blockDim.x - 1) / (int)blockDim.x;     // each thread owns `per` consecutive buckets
     const int lo = min((int)threadIdx.x * per, T1), hi = min(lo + per, T1);
+    const bool have_own = own_count >= 0 && per == 1;
     int sum = 0;
-    for (int t = lo; t < hi; ++t) sum += counts[t];
+    if (have_own) sum = (lo < hi) ? own_count : 0;
+    else for (int t = lo; t < hi; ++t) sum += counts[t];
     int total;
     int run = cta_excl_scan(sum, s_warp, &total);
-    for (int t = lo; t < hi; ++t) { offsets[t] = run; run += counts[t]; }
+    if (have_own) { if (lo < hi) offsets[lo] = run; }
+    else for (int t = lo; t < hi; ++t) { offsets[t] = run; run += counts[t]; }
     if (threadIdx.x == 0) offsets[T1] = total;
     const int hi_t = min(hi, T);               // the extra bucket of rejected ids contributes no work
     if (per == 1) {
@@ -141,13 +156,13 @@ __device__ __forceinline__ void scan_buckets(int T, const ModelDev* __restrict__
         LayerHead head[MT_MAX_LAYERS];
         const int t_own = min(lo, T - 1);
 #pragma unroll
-        for (int l = 0; l < MT_MAX_LAYERS; ++l) head[l] = (l < n_layers) ? load_head(models, t_own, l) : LayerHead{-1, 0};
-        const int c_own = (lo < hi_t) ? counts[lo] : 0;
+        for (int l = 0; l < MT_MAX_LAYERS; ++l) head[l] = (l < n_layers) ? load_head(br, tn, t_own, l) : LayerHead{-1, 0};
+        const int c_own = (lo < hi_t) ? (have_own ? own_count : counts[lo]) : 0;
         int units[MT_MAX_LAYERS];
 #pragma unroll
         for (int l = 0; l < MT_MAX_LAYERS; ++l) units[l] = units_of(head[l], c_own, rows_per_unit, tn.v[l], tn.m[l]);
         int urun[MT_MAX_LAYERS], utotal[MT_MAX_LAYERS];
-        cta_excl_scan_vec(units, urun, utotal, s_vec);
+        cta_excl_scan_vec(units, urun, utotal, s_vec, n_layers);
 #pragma unroll
         for (int l = 0; l < MT_MAX_LAYERS; ++l) {
             if (l >= n_layers) break;
@@ -159,9 +174,9 @@ __device__ __forceinline__ void scan_buckets(int T, const ModelDev* __restrict__
     for (int l = 0; l < n_layers; ++l) {
         int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
         int usum = 0;
-        for (int t = lo; t < hi_t; ++t) usum += layer_units(models, t, l, counts[t], rows_per_unit, tn.v[l], tn.m[l]);
+        for (int t = lo; t < hi_t; ++t) usum += layer_units(br, tn, t, l, counts[t], rows_per_unit);
         int urun = cta_excl_scan(usum, s_warp, &total);
-        for (int t = lo; t < hi_t; ++t) { prefix[t] = urun; urun += layer_units(models, t, l, counts[t], rows_per_unit, tn.v[l], tn.m[l]); }
+        for (int t = lo; t < hi_t; ++t) { prefix[t] = urun; urun += layer_units(br, tn, t, l, counts[t], rows_per_unit); }
         if (threadIdx.x == 0) prefix[T] = total;
     }
 }
@@ -171,7 +186,7 @@ __device__ __forceinline__ void scan_buckets(int T, const ModelDev* __restrict__
 // turns the block histograms into per-tenant exclusive prefixes over the blocks, the counts, the offsets and the
 // per-layer unit prefixes.
 __global__ void __launch_bounds__(kHistChunk)
-bucket_hist_scan(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models, int n_layers,
+bucket_hist_scan(const int32_t* __restrict__ ids, int n, int T, Brief br, int n_layers,
                  int rows_per_unit, LayerTileN tn, int32_t* block_hist, int32_t* counts, int32_t* __restrict__ offsets,
                  int32_t* __restrict__ tile_prefix, int32_t* ticket, int32_t* __restrict__ status) {
     pdl_launch_dependents();
@@ -185,7 +200,7 @@ bucket_hist_scan(const int32_t* __restrict__ ids, int n, int T, const ModelDev* 
     __syncthreads();
     const int i = blockIdx.x * kHistChunk + threadIdx.x;
     if (i < n) {
-        const int b = classify(ids[i], T, models);
+        const int b = classify(ids[i], T, br);
         if (b == T) {
             atomicCAS(&status[ST_CODE], MT_OK, MT_ERR_BAD_MODEL_ID);
             atomicMin(&status[ST_BAD_INDEX], i);
@@ -207,6 +222,7 @@ bucket_hist_scan(const int32_t* __restrict__ ids, int n, int T, const ModelDev* 
     __threadfence();
     // per bucket (one thread each; neighbouring threads read neighbouring words): exclusive prefix over the blocks
     const int n_blocks = gridDim.x;
+    int own_count = -1;                        // counts[threadIdx.x] when every bucket has a thread of its own
     for (int t = threadIdx.x; t < T1; t += blockDim.x) {
         int run = 0;
         int b = 0;
@@ -223,9 +239,12 @@ bucket_hist_scan(const int32_t* __restrict__ ids, int n, int T, const ModelDev* 
             run += v;
         }
         counts[t] = run;
+        own_count = run;
     }
+    if (T1 > (int)blockDim.x) own_count = -1;
+    else if ((int)threadIdx.x >= T1) own_count = 0;
     __syncthreads();
-    scan_buckets(T, models, n_layers, rows_per_unit, tn, counts, offsets, tile_prefix, s_warp, s_vec);
+    scan_buckets(T, br, n_layers, rows_per_unit, tn, counts, offsets, tile_prefix, s_warp, s_vec, own_count);
 }
 
 struct ItemPtrs { WorkItem* v[8]; };
@@ -264,7 +283,7 @@ __device__ __forceinline__ WorkItem make_work_item(int item, int l, int T, const
 constexpr int kSingleCtaMax = 4096;
 
 __global__ void __launch_bounds__(1024)
-bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models, int n_layers,
+bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models, Brief br, int n_layers,
                   int rows_per_unit, LayerTileN tn, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
                   int32_t* __restrict__ tile_prefix, int32_t* __restrict__ perm, int32_t* __restrict__ inv,
                   ItemPtrs items, int32_t* __restrict__ status) {
@@ -287,7 +306,7 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
         bucket[r] = -1;
         const int i = r * nthr + threadIdx.x;
         if (r < rounds && i < n) {
-            const int b = classify(ids[i], T, models);
+            const int b = classify(ids[i], T, br);
             bucket[r] = b;
             if (b == T) {
                 atomicCAS(&status[ST_CODE], MT_OK, MT_ERR_BAD_MODEL_ID);
@@ -314,13 +333,13 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
             LayerHead head[MT_MAX_LAYERS];
             const int t_own = min(lo, T - 1);
 #pragma unroll
-            for (int l = 0; l < MT_MAX_LAYERS; ++l) head[l] = (l < n_layers) ? load_head(models, t_own, l) : LayerHead{-1, 0};
+            for (int l = 0; l < MT_MAX_LAYERS; ++l) head[l] = (l < n_layers) ? load_head(br, tn, t_own, l) : LayerHead{-1, 0};
             const int c_own = (lo < hi_t) ? s_cnt[lo] : 0;
             int units[MT_MAX_LAYERS];
 #pragma unroll
             for (int l = 0; l < MT_MAX_LAYERS; ++l) units[l] = units_of(head[l], c_own, rows_per_unit, tn.v[l], tn.m[l]);
             int urun[MT_MAX_LAYERS], utotal[MT_MAX_LAYERS];
-            cta_excl_scan_vec(units, urun, utotal, s_vec);
+            cta_excl_scan_vec(units, urun, utotal, s_vec, n_layers);
 #pragma unroll
             for (int l = 0; l < MT_MAX_LAYERS; ++l) {
                 if (l >= n_layers) break;
@@ -331,9 +350,9 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
             for (int l = 0; l < n_layers; ++l) {
                 int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
                 int usum = 0;
-                for (int t = lo; t < hi_t; ++t) usum += layer_units(models, t, l, s_cnt[t], rows_per_unit, tn.v[l], tn.m[l]);
+                for (int t = lo; t < hi_t; ++t) usum += layer_units(br, tn, t, l, s_cnt[t], rows_per_unit);
                 int urun = cta_excl_scan(usum, s_warp, &total);
-                for (int t = lo; t < hi_t; ++t) { prefix[t] = urun; urun += layer_units(models, t, l, s_cnt[t], rows_per_unit, tn.v[l], tn.m[l]); }
+                for (int t = lo; t < hi_t; ++t) { prefix[t] = urun; urun += layer_units(br, tn, t, l, s_cnt[t], rows_per_unit); }
                 if (threadIdx.x == 0) prefix[T] = total;
             }
         }
@@ -381,7 +400,7 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
 // A CTA takes kBucketChunk requests (small, so that the row move spreads over many SMs); CTAs beyond the last block
 // of requests only expand work items.
 __global__ void __launch_bounds__(kScatterThreads)
-bucket_scatter_expand(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models,
+bucket_scatter_expand(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models, Brief br,
                       const int32_t* __restrict__ block_hist, const int32_t* __restrict__ offsets,
                       int32_t* __restrict__ perm, int32_t* __restrict__ inv, const uint4* __restrict__ rows_src,
                       uint4* __restrict__ rows_dst, int row_vec, int dst_ld_vec, int n_layers, LayerTileN tn,
@@ -401,16 +420,29 @@ bucket_scatter_expand(const int32_t* __restrict__ ids, int n, int T, const Model
             s_next[t] = offsets[t] + block_hist[(size_t)hist_block * T1 + t];
         __syncthreads();
         // (chunk0 - first id of the pass-1 block) is a multiple of kBucketChunk = 64: whole warps only
-        for (int i = hist_block * kHistChunk + threadIdx.x; i < chunk0; i += blockDim.x) {
-            const int b = classify(ids[i], T, models);
-            const unsigned peers = __match_any_sync(0xffffffffu, b);
-            if ((__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&s_next[b], __popc(peers));
+        // (at most kHistChunk / kScatterThreads rounds; the ids of all rounds are fetched first, then the tenant
+        // table entries, so that each kind of load costs one round trip instead of one per round)
+        constexpr int kRounds = kHistChunk / kScatterThreads;
+        int pre_id[kRounds], pre_b[kRounds];
+#pragma unroll
+        for (int q = 0; q < kRounds; ++q) {
+            const int i = hist_block * kHistChunk + q * kScatterThreads + (int)threadIdx.x;
+            pre_id[q] = (i < chunk0) ? ids[i] : INT_MIN;
+        }
+#pragma unroll
+        for (int q = 0; q < kRounds; ++q) pre_b[q] = (pre_id[q] == INT_MIN) ? -1 : classify(pre_id[q], T, br);
+#pragma unroll
+        for (int q = 0; q < kRounds; ++q) {
+            if (pre_b[q] >= 0) {      // whole warps: the part before this CTA's requests is a multiple of 64 long
+                const unsigned peers = __match_any_sync(__activemask(), pre_b[q]);
+                if ((__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&s_next[pre_b[q]], __popc(peers));
+            }
         }
         __syncthreads();
         const int i = chunk0 + threadIdx.x;
         const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
         const bool mine = threadIdx.x < kBucketChunk && i < n;
-        const int b = mine ? classify(ids[i], T, models) : -1;
+        const int b = mine ? classify(ids[i], T, br) : -1;
         // warps take turns in arrival order, so positions inside a bucket ascend with the arrival index
         for (int w = 0; w < kBucketChunk / 32; ++w) {
             if (warp == w && mine) {
@@ -507,21 +539,22 @@ void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
     const int n_hist_blocks = (a.n + kHistChunk - 1) / kHistChunk;
     const size_t smem = sizeof(int32_t) * (size_t)(a.T + 1);
     LayerTileN tn;
-    for (int l = 0; l < 8; ++l) { tn.v[l] = a.tile_n[l] > 0 ? a.tile_n[l] : BN; tn.m[l] = a.tile_m[l] > 0 ? a.tile_m[l] : BM; }
+    for (int l = 0; l < 8; ++l) { tn.v[l] = a.tile_n[l] > 0 ? a.tile_n[l] : BN; tn.m[l] = a.tile_m[l] > 0 ? a.tile_m[l] : BM; tn.kind[l] = a.kind[l]; }
+    Brief br{a.brief, a.brief_ld};
     ItemPtrs ip;
     for (int l = 0; l < 8; ++l) ip.v[l] = a.items[l];
     // measured: one CTA wins up to a few hundred requests; beyond that its serial scatter and the item expansion
     // by a single CTA cost more than the extra launches of the multi-CTA path
     if (a.n <= 512 && a.T + 1 <= 4096) {
         const int threads = (a.n <= 256) ? 256 : 1024;
-        launch_pdl(bucket_single_cta, dim3(1), dim3(threads), 2 * smem, s, a.ids, a.n, a.T, a.models, a.n_layers, a.rows_per_unit, tn, a.counts,
+        launch_pdl(bucket_single_cta, dim3(1), dim3(threads), 2 * smem, s, a.ids, a.n, a.T, a.models, br, a.n_layers, a.rows_per_unit, tn, a.counts,
                                                       a.offsets, a.tile_prefix, a.perm, a.inv, ip, a.status);
         return;
     }
-    launch_pdl(bucket_hist_scan, dim3(n_hist_blocks), dim3(kHistChunk), smem, s, a.ids, a.n, a.T, a.models, a.n_layers, a.rows_per_unit, tn,
+    launch_pdl(bucket_hist_scan, dim3(n_hist_blocks), dim3(kHistChunk), smem, s, a.ids, a.n, a.T, br, a.n_layers, a.rows_per_unit, tn,
                a.block_hist, a.counts, a.offsets, a.tile_prefix, a.ticket, a.status);
     const int grid2 = n_blocks > a.item_grid ? n_blocks : a.item_grid;
-    launch_pdl(bucket_scatter_expand, dim3(grid2), dim3(kScatterThreads), smem + sizeof(int32_t) * kBucketChunk, s, a.ids, a.n, a.T, a.models,
+    launch_pdl(bucket_scatter_expand, dim3(grid2), dim3(kScatterThreads), smem + sizeof(int32_t) * kBucketChunk, s, a.ids, a.n, a.T, a.models, br,
                a.block_hist, a.offsets, a.perm, a.inv, (const uint4*)a.rows_src, (uint4*)a.rows_dst, a.row_bytes / 16,
                a.dst_ld_bytes / 16, a.n_layers, tn, a.tile_prefix, ip);
 }

@@ -52,6 +52,7 @@ struct Ctx {
     int T = 0;                           // id slots in use (highest issued id + 1)
     std::vector<HostModel> models;
     ModelDev* d_models = nullptr;
+    int32_t* d_brief = nullptr;          // [1 + MT_MAX_LAYERS][max_models]: alive, out features per layer (bucketing passes)
     CUtensorMap* d_wmaps = nullptr;      // [max_models][MT_MAX_LAYERS]: dense weights as 128 x 64 boxes of the tiled image
     EncodeTiledFn encode = nullptr;
 
@@ -138,6 +139,8 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     g.models.assign(max_models, HostModel());
     CU_OK(cudaMalloc(&g.d_models, sizeof(ModelDev) * (size_t)max_models));
     CU_OK(cudaMemset(g.d_models, 0, sizeof(ModelDev) * (size_t)max_models));
+    CU_OK(cudaMalloc(&g.d_brief, sizeof(int32_t) * (size_t)(1 + MT_MAX_LAYERS) * max_models));
+    CU_OK(cudaMemset(g.d_brief, 0, sizeof(int32_t) * (size_t)(1 + MT_MAX_LAYERS) * max_models));
     CU_OK(cudaMalloc(&g.d_wmaps, sizeof(CUtensorMap) * (size_t)max_models * MT_MAX_LAYERS));
     CU_OK(cudaMalloc(&g.d_status, sizeof(int32_t) * ST_WORDS));
     CU_OK(cudaMalloc(&g.d_ticket, sizeof(int32_t)));
@@ -456,6 +459,8 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
         Timer t(K_BUCKET, s);
         BucketArgs a;
         a.ids = ids; a.n = n; a.T = g.T; a.models = g.d_models; a.n_layers = L; a.rows_per_unit = tiles_per_image;
+        a.brief = g.d_brief; a.brief_ld = g.max_models;
+        for (int l = 0; l < 8; ++l) a.kind[l] = (l < L) ? g.family[l].kind : -1;
         a.ticket = g.d_ticket;
         a.rows_src = rows_in_scatter ? inputs : nullptr; a.rows_dst = g.act[0];
         a.row_bytes = g.in_elems * 2; a.dst_ld_bytes = g.act_ld[0] * 2;
@@ -550,6 +555,7 @@ mt_status mt_shutdown(void) {
     g.models.clear();
     free_workspace();
     cudaFree(g.d_models); g.d_models = nullptr;
+    cudaFree(g.d_brief); g.d_brief = nullptr;
     cudaFree(g.d_wmaps); g.d_wmaps = nullptr;
     cudaFree(g.d_status); g.d_status = nullptr;
     cudaFree(g.d_ticket); g.d_ticket = nullptr;
@@ -661,6 +667,10 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
         e = cudaMemcpy(g.d_wmaps + (size_t)id * MT_MAX_LAYERS + l, &wm, sizeof wm, cudaMemcpyHostToDevice);
     }
     if (e == cudaSuccess) e = cudaMemcpy(g.d_models + id, &md, sizeof md, cudaMemcpyHostToDevice);
+    for (int r = 0; r <= n_layers && e == cudaSuccess; ++r) {      // the compact copy: alive, then out features per layer
+        const int32_t v = (r == 0) ? 1 : hl[r - 1].out_ch;
+        e = cudaMemcpy(g.d_brief + (size_t)r * g.max_models + id, &v, sizeof v, cudaMemcpyHostToDevice);
+    }
     if (raw_dev) cudaFree(raw_dev);
     if (e != cudaSuccess) {
         cudaFree(block);
@@ -702,6 +712,8 @@ mt_status mt_release(int32_t model_id) {
     ModelDev md;
     memset(&md, 0, sizeof md);
     CU_OK(cudaMemcpy(g.d_models + model_id, &md, sizeof md, cudaMemcpyHostToDevice));
+    const int32_t dead = 0;
+    CU_OK(cudaMemcpy(g.d_brief + model_id, &dead, sizeof dead, cudaMemcpyHostToDevice));
     HostModel& hm = g.models[model_id];
     cudaFree(hm.dev_block);
     hm.dev_block = nullptr;

@@ -34,6 +34,9 @@ struct BucketArgs {
     int n;
     int T;                    // id slots in use (highest issued id + 1)
     const ModelDev* models;
+    const int32_t* brief;     // compact tenant fields, rows of brief_ld ints: row 0 alive, row 1 + l out features of layer l
+    int brief_ld;
+    int kind[8];              // layer kinds of the hosted family
     int n_layers;
     int rows_per_unit;        // conv: tiles per image
     int tile_n[8];            // dense: output columns per work item of each layer (128 or 256)
