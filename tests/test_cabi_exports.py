@@ -74,8 +74,11 @@ def test_register_validation_happens_on_the_host(lib):
 def test_calls_before_init_fail_cleanly(lib):
     mt.mt_shutdown()
     for fn, args in ((lib.mt_release, (0,)), (lib.mt_infer, (None, None, 4, None, None)),
-                     (lib.mt_infer_host, (None, None, 4, None, None)), (lib.mt_get_async_status, (None, None, None))):
+                     (lib.mt_infer_host, (None, None, 4, None, None)), (lib.mt_infer_host_async, (None, None, 4, None, None)),
+                     (lib.mt_get_async_status, (None, None, None)), (lib.mt_debug_wait_timeout, (20, None))):
         assert fn(*args) == 9                                             # MT_ERR_NOT_INIT
+    assert mt.mt_debug_launch_count() >= 0                                # a plain counter: no device needed
+    assert lib.mt_debug_launch_count(None) == 1                           # MT_ERR_INVALID_ARG
 
 
 def test_synth_workloads_match_their_descriptions():
