@@ -11,7 +11,8 @@
 // their arrival positions.  Weights stream through a four-stage ring of 32 KiB (both 128-row tiles of one K block),
 // fetched as bulk copies of the pre-swizzled images written at registration; the producer runs ahead across layers.
 //
-// Roles: warp 0 producer, warp 1 tcgen05.mma issuer, warps 2..5 gather / epilogue (one TMEM lane quarter each).
+// Roles: warp 0 producer, warp 1 tcgen05.mma issuer, warps 2..9 gather / epilogue (two warps per TMEM lane quarter,
+// which take the accumulator's 32-column chunks in turn: the drain of a layer is on the pass's critical path).
 // Same semantics as the layer-by-layer path: the paper's layer-by-layer evaluation of a DNN (Sec. 1.1) for many
 // co-resident models (Sec. 3).
 #include "mt_device.cuh"
@@ -19,7 +20,9 @@
 
 namespace mt {
 
-constexpr int kFusedThreads = 192;
+constexpr int kFusedThreads = 320;
+constexpr int kFusedWarps = kFusedThreads / 32;
+constexpr int kFusedEpiThreads = kFusedThreads - 64;   // 256
 constexpr int kFusedStages = 4;
 constexpr int kFusedStageBytes = 2 * TILE_BYTES;          // weight tiles (0, kb) and (1, kb)
 constexpr int kFusedABytes = 4 * TILE_BYTES;              // 128 rows x 256 features, four K blocks
@@ -66,7 +69,7 @@ fused_mlp_kernel(const FusedArgs p) {
     if (threadIdx.x == 0) {
         for (int s = 0; s < kFusedStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         mbar_init(acc_full_bar, 1);
-        mbar_init(act_ready_bar, 128);
+        mbar_init(act_ready_bar, kFusedEpiThreads);
         *abort_flag = 0;
         fence_mbar_init();
     }
@@ -83,12 +86,12 @@ fused_mlp_kernel(const FusedArgs p) {
     pdl_wait();
     // ---------------------------------------------------------------- stable counting sort, repeated by every CTA
     // chunk c = requests [32c, 32c + 32): rank inside the chunk from the warp's match mask, per-chunk histogram
-    constexpr int kMaxOwn = (512 / 32 + 5) / 6;       // chunks one warp may own (3)
+    constexpr int kMaxOwn = (512 / 32 + kFusedWarps - 1) / kFusedWarps;       // chunks one warp may own (2)
     int own_b[kMaxOwn], own_rank[kMaxOwn];
 #pragma unroll
     for (int q = 0; q < kMaxOwn; ++q) {
         own_b[q] = -1; own_rank[q] = 0;
-        const int c = warp + 6 * q;
+        const int c = warp + kFusedWarps * q;
         const int i = c * 32 + lane;
         if (c < n_chunks && i < n) {
             const int id = p.ids[i];
@@ -136,7 +139,7 @@ fused_mlp_kernel(const FusedArgs p) {
     __syncthreads();
 #pragma unroll
     for (int q = 0; q < kMaxOwn; ++q) {
-        const int c = warp + 6 * q;
+        const int c = warp + kFusedWarps * q;
         const int i = c * 32 + lane;
         if (own_b[q] >= 0) {
             const int pos = s_off[own_b[q]] + s_chist[c * T1 + own_b[q]] + own_rank[q];
@@ -225,9 +228,10 @@ fused_mlp_kernel(const FusedArgs p) {
                 if (ok && leader) umma_commit(acc_full_bar);
             }
         }
-    } else {                  // ------------------------------------------------ gather + epilogue (warps 2..5)
-        const int et = threadIdx.x - 64;            // 0..127
+    } else {                  // ------------------------------------------------ gather + epilogue (warps 2..9)
+        const int et = threadIdx.x - 64;            // 0..255
         const int q = warp & 3;                     // TMEM lane quarter this warp may read
+        const int turn = (warp - 2) >> 2;           // which of the quarter's two warps: it takes chunks turn, turn + 2, ...
         const int r = q * 32 + lane;                // accumulator row = request of the unit
         uint32_t acc_phase = 0;
         bool ok = true;
@@ -236,7 +240,7 @@ fused_mlp_kernel(const FusedArgs p) {
             // requests whose id was rejected sort behind every live segment and belong to no unit: NaN rows
             for (int j = s_off[T]; j < n; ++j) {
                 float* dst = p.out + (size_t)s_perm[j] * p.out_elems;
-                for (int e = et; e < p.out_elems; e += 128) dst[e] = __int_as_float(0x7fc00000);
+                for (int e = et; e < p.out_elems; e += kFusedEpiThreads) dst[e] = __int_as_float(0x7fc00000);
             }
         }
         const int cpr = p.K0 >> 3;                  // 16-byte chunks per input row
@@ -245,10 +249,27 @@ fused_mlp_kernel(const FusedArgs p) {
             // gather the unit's rows (arrival order -> bucketed rows) into the operand buffer: row rr, chunk ch of the
             // row goes to K block ch / 8, 16-byte position (ch % 8) ^ (rr % 8) of the 128-byte swizzle row
             const uint4* src = reinterpret_cast<const uint4*>(p.inputs);
-            for (int idx = et; idx < c.rows * cpr; idx += 128) {
-                const int rr = idx / cpr, ch = idx - rr * cpr;
-                const uint4 v = __ldg(src + (size_t)s_perm[c.j0 + rr] * cpr + ch);
-                *reinterpret_cast<uint4*>(smem + (ch >> 3) * TILE_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4)) = v;
+            {
+                const int total_ch = c.rows * cpr;
+                int idx = et;
+                for (; idx + 3 * kFusedEpiThreads < total_ch; idx += 4 * kFusedEpiThreads) {   // four loads in flight
+                    uint4 v[4];
+                    int rr[4], ch[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int e = idx + k * kFusedEpiThreads;
+                        rr[k] = e / cpr; ch[k] = e - rr[k] * cpr;
+                        v[k] = __ldg(src + (size_t)s_perm[c.j0 + rr[k]] * cpr + ch[k]);
+                    }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        *reinterpret_cast<uint4*>(smem + (ch[k] >> 3) * TILE_BYTES + rr[k] * 128 + (((ch[k] & 7) ^ (rr[k] & 7)) << 4)) = v[k];
+                }
+                for (; idx < total_ch; idx += kFusedEpiThreads) {
+                    const int rr = idx / cpr, ch = idx - rr * cpr;
+                    const uint4 v = __ldg(src + (size_t)s_perm[c.j0 + rr] * cpr + ch);
+                    *reinterpret_cast<uint4*>(smem + (ch >> 3) * TILE_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4)) = v;
+                }
             }
             fence_proxy_async_smem();
             mbar_arrive(act_ready_bar);
@@ -262,24 +283,22 @@ fused_mlp_kernel(const FusedArgs p) {
                 // complete: by then every epilogue thread has finished with the previous layer's bias (the MMAs could
                 // not start before all of them had handed over the layer's input).  The barrier that publishes it
                 // also makes the give-up decision of a timed-out wait unanimous.
-                const float bias_lo = Ld.bias[et];
-                const float bias_hi = (N > BN) ? Ld.bias[et + BN] : 0.0f;
+                const float bias_mine = (et < BN || N > BN) ? Ld.bias[et] : 0.0f;      // padded to whole 128-feature tiles
                 const bool got = mbar_wait(acc_full_bar, acc_phase, abort_flag, p.status, 44);
                 acc_phase ^= 1u;
-                s_bias[et] = bias_lo;
-                s_bias[et + BN] = bias_hi;
+                s_bias[et] = bias_mine;
                 int any_failed;
                 asm volatile(
                     "{\n\t"
                     ".reg .pred pi, po;\n\t"
                     "setp.ne.b32 pi, %1, 0;\n\t"
-                    "bar.red.or.pred po, 1, 128, pi;\n\t"
+                    "bar.red.or.pred po, 1, 256, pi;\n\t"
                     "selp.u32 %0, 1, 0, po;\n\t"
                     "}\n"
                     : "=r"(any_failed) : "r"(got ? 0 : 1) : "memory");
                 if (any_failed) { ok = false; break; }
                 tc_fence_after();
-                for (int n0 = 0; n0 < N; n0 += 32) {
+                for (int n0 = turn * 32; n0 < N; n0 += 64) {
                     uint32_t v[32];
                     __syncwarp();
                     tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + n0, v);
