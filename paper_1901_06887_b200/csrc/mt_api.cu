@@ -361,10 +361,12 @@ struct Timer {
     static int open_kernel;              // mode 2: executor whose group of launches is open (-1 none)
     static cudaEvent_t open_start;
     static int open_count;
+    static cudaStream_t open_stream;
     int kernel;
     cudaStream_t s;
     bool each;
     cudaEvent_t start = nullptr;
+    static void close_group() { close_group(open_stream); }
     static void close_group(cudaStream_t st) {
         if (open_kernel < 0) return;
         cudaEvent_t stop = pooled_event();
@@ -378,12 +380,13 @@ struct Timer {
             cudaEventRecord(start, s);
         } else if (g.timing == 2) {
             const bool executor = (k == K_GEMM || k == K_CONV || k == K_FUSED);
-            if (open_kernel >= 0 && open_kernel != k) close_group(s);
+            if (open_kernel >= 0 && (open_kernel != k || open_stream != s)) close_group();
             if (executor && open_kernel < 0) {
                 open_start = pooled_event();
                 cudaEventRecord(open_start, s);
                 open_kernel = k;
                 open_count = 0;
+                open_stream = s;
             }
             if (executor) ++open_count;
         }
@@ -398,6 +401,7 @@ struct Timer {
 int Timer::open_kernel = -1;
 cudaEvent_t Timer::open_start = nullptr;
 int Timer::open_count = 0;
+cudaStream_t Timer::open_stream = nullptr;
 
 mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outputs, cudaStream_t s) {
     if (!g.init) return MT_ERR_NOT_INIT;
@@ -431,7 +435,8 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             if (grid > n) grid = n;
             if (grid > g.sm_count) grid = g.sm_count;
             CU_OK(launch_fused_mlp(a, grid, s));
-            Timer::close_group(s);
+            // the group of launches stays open: a step of this path is ONE launch, and the next call's joins it (an
+            // event pair per launch costs more than the launch); it closes when the times are read or timing changes
             g.last_n = n;
             return MT_OK;
         }
@@ -575,6 +580,7 @@ mt_status mt_shutdown(void) {
     }
     if (g.as_compute_done) { cudaEventDestroy(g.as_compute_done); g.as_compute_done = nullptr; }
     g.as_cap = 0; g.as_next = 0; g.as_have_compute = false;
+    Timer::close_group();
     for (TimedLaunch& t : g.timed) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
     g.timed.clear();
     for (cudaEvent_t e : g.event_pool) cudaEventDestroy(e);
@@ -870,6 +876,7 @@ mt_status mt_debug_launch_count(int64_t* count_out) {
 
 mt_status mt_set_kernel_timing(int32_t enable) {
     std::lock_guard<std::mutex> lk(g_mu);
+    Timer::close_group();
     g.timing = enable < 0 ? 0 : (enable > 2 ? 1 : enable);
     return MT_OK;
 }
@@ -877,6 +884,7 @@ mt_status mt_set_kernel_timing(int32_t enable) {
 mt_status mt_get_kernel_times(const char** names, double* total_ms, int32_t* launches, int32_t cap, int32_t* n_out) {
     std::lock_guard<std::mutex> lk(g_mu);
     if (!names || !total_ms || !launches || !n_out || cap < 0) return MT_ERR_INVALID_ARG;
+    Timer::close_group();
     double ms[K_COUNT] = {0};
     int cnt[K_COUNT] = {0};
     for (TimedLaunch& t : g.timed) {
