@@ -267,7 +267,7 @@ def main():
     # ---- timed region: device-resident inputs, CUDA events on the launching stream, per-kernel events inside
     sampler = ClockSampler(local_rank)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    mt.mt_set_kernel_timing(2)          # events around the grouped layer executors only (the dominant kernel)
+    mt.mt_set_kernel_timing(3)          # events around the layer executors (the dominant kernel) on every 4th step
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
@@ -350,11 +350,14 @@ def main():
     if rank == 0:
         peaks, peaks_kind = load_peaks()
         per_kernel = {name: {"ms_per_step": t / bd_steps, "launches_per_step": c / bd_steps} for name, t, c in breakdown}
-        timed = dict((nm, t / args.steps) for nm, t, c in kernel_times)
+        # per step = per-launch average x launches per step (the executors are timed on every fourth step)
+        lps = {nm: c / bd_steps for nm, t, c in breakdown}
+        timed = dict((nm, t / max(c, 1) * lps.get(nm, 1.0)) for nm, t, c in kernel_times)
         dom = "grouped_conv3x3" if cfg == 4 else ("fused_mlp" if "fused_mlp" in timed else "grouped_gemm")
         dom_ms = timed.get(dom, 0.0)
         roof = gemm_roofline(wl, dom_ms, peaks, peaks_kind, cfg)
         roof["kernel"] = dom
+        roof["kernel_timing"] = "CUDA events around each run of the executor's launches, every 4th step of the timed region"
         flops = synth.workload_flops(wl.models, wl.model_ids)
         bytes_all = synth.workload_bytes(wl.models, wl.model_ids)
         t_roof = max(flops / (peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12),

@@ -141,7 +141,8 @@ mt_status mt_debug_launch_count(int64_t* count_out);
 /* Per-kernel device timing.  enable = 1: every kernel launch of mt_infer is bracketed by CUDA events on the
  * caller's stream; enable = 2: only the layer executors (dense / conv / the one-launch path) are, and consecutive
  * launches of the same executor (also across calls, when a call is a single launch) share one pair of events, so
- * that the launches still overlap as they do untimed;
+ * that the launches still overlap as they do untimed; enable = 3: as 2, on every fourth call only (an event between
+ * two kernels still costs the overlap at that boundary, a few microseconds per pair);
  * 0: off.  mt_get_kernel_times synchronises those events, then fills up to `cap`
  * entries: names[i] (static strings), total_ms[i], launches[i]; *n_out = number of kernels seen.
  * Reading resets the accumulators. */

@@ -176,7 +176,7 @@ def mt_debug_launch_count() -> int:
 
 
 def mt_set_kernel_timing(enable) -> None:
-    """0/False off, 1/True every kernel, 2 only the grouped layer executors."""
+    """0/False off, 1/True every kernel, 2 only the grouped layer executors, 3 the same on every fourth call."""
     _check(lib().mt_set_kernel_timing(int(enable)), "mt_set_kernel_timing")
 
 

@@ -99,7 +99,9 @@ struct Ctx {
     bool as_have_compute = false;
 
     // timing
-    int timing = 0;                      // 0 off, 1 every kernel, 2 only the layer executors
+    int timing = 0;                      // 0 off, 1 every kernel, 2 only the layer executors, 3 the same on every 4th call
+    int timing_now = 0;                  // the mode in force for the current call (0, 1 or 2)
+    unsigned timing_calls = 0;
     std::vector<TimedLaunch> timed;
     std::vector<cudaEvent_t> event_pool;
 };
@@ -374,11 +376,11 @@ struct Timer {
         g.timed.push_back({open_kernel, open_start, stop, open_count});
         open_kernel = -1;
     }
-    Timer(int k, cudaStream_t st) : kernel(k), s(st), each(g.timing == 1) {
+    Timer(int k, cudaStream_t st) : kernel(k), s(st), each(g.timing_now == 1) {
         if (each) {
             start = pooled_event();
             cudaEventRecord(start, s);
-        } else if (g.timing == 2) {
+        } else if (g.timing_now == 2) {
             const bool executor = (k == K_GEMM || k == K_CONV || k == K_FUSED);
             if (open_kernel >= 0 && (open_kernel != k || open_stream != s)) close_group();
             if (executor && open_kernel < 0) {
@@ -415,6 +417,9 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
     if (st != MT_OK) return st;
     const int L = (int)g.family.size();
     const HostLayer& f0 = g.family[0];
+    // mode 3 times the executors of every fourth call only (a call that is a single launch keeps its group open
+    // across calls instead, which costs nothing per call)
+    g.timing_now = (g.timing == 3) ? (((g.timing_calls++ & 3u) == 0) ? 2 : 0) : g.timing;
     // Small batch of narrow MLPs: the whole pass in one launch (MT_FUSED=0 forces the layer-by-layer path).
     {
         bool all_dense = true;
@@ -425,6 +430,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
         }
         const char* fused_env = getenv("MT_FUSED");
         if (all_dense && !(fused_env && fused_env[0] == '0') && fused_mlp_fits(n, g.T, max_w)) {
+            if (g.timing == 3) g.timing_now = 2;
             Timer t(K_FUSED, s);
             FusedArgs a;
             a.inputs = static_cast<const uint16_t*>(inputs); a.ids = ids; a.n = n; a.T = g.T; a.models = g.d_models;
@@ -877,7 +883,9 @@ mt_status mt_debug_launch_count(int64_t* count_out) {
 mt_status mt_set_kernel_timing(int32_t enable) {
     std::lock_guard<std::mutex> lk(g_mu);
     Timer::close_group();
-    g.timing = enable < 0 ? 0 : (enable > 2 ? 1 : enable);
+    g.timing = enable < 0 ? 0 : (enable > 3 ? 1 : enable);
+    g.timing_now = 0;
+    g.timing_calls = 0;
     return MT_OK;
 }
 
