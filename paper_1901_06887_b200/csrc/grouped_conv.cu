@@ -447,6 +447,81 @@ void launch_pool_finalize(const float* partial, int n, int strips, int C, int HW
     launch_pdl(pool_finalize_kernel, dim3((n * C + 255) / 256), dim3(256), 0, s, partial, n, strips, C, 1.0f / (float)HW, out, ld_out);
 }
 
+// Pool + narrow head in one launch: for every image, finish the global average pool (sum the strips' channel sums in
+// a fixed order, divide by H*W, round to bf16 - exactly what pool_finalize hands to a dense layer) and apply the
+// model's last dense layer (64 -> at most 64 outputs, fp32 accumulate, bias, optional ReLU), writing the fp32 row to
+// the request's arrival position.  One warp per image: lane c holds channels c and c + 32.  Rows of rejected requests
+// (bucketed rows at and after offsets[T]) become NaN.  The head's weights are read from the executor's tiled image
+// (128 rows x 64 columns per tile, 16-byte chunk c of row r at chunk c ^ (r & 7)); K = 64 is one tile column.
+__global__ void __launch_bounds__(256)
+pool_head_kernel(const float* __restrict__ partial, int n, int strips, float inv_hw, const ModelDev* __restrict__ models,
+                 int layer, const int32_t* __restrict__ offsets, int T, const int32_t* __restrict__ perm,
+                 float* __restrict__ out, int out_elems) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const int j = blockIdx.x * 8 + (threadIdx.x >> 5);          // bucketed row = image
+    if (j >= n) return;
+    float* dst = out + (size_t)perm[j] * out_elems;
+    if (j >= offsets[T]) {                                       // rejected id: no model
+        for (int o = lane; o < out_elems; o += 32) dst[o] = __int_as_float(0x7fc00000);
+        return;
+    }
+    int lo = 0, hi = T;                                          // tenant of row j: largest t with offsets[t] <= j
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (offsets[mid] <= j) lo = mid; else hi = mid;
+    }
+    const LayerDev& L = models[lo].layer[layer];
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll 4
+    for (int k = 0; k < strips; ++k) {      // fixed order: the pooled value does not depend on timing
+        const float* q = partial + ((size_t)j * strips + k) * 64;
+        s0 += __ldg(q + lane);
+        s1 += __ldg(q + lane + 32);
+    }
+    // the pooled activation as the dense executor would see it: rounded to bf16
+    const float p0 = __uint_as_float(pack_bf16x2(0.0f, s0 * inv_hw) & 0xFFFF0000u);
+    const float p1 = __uint_as_float(pack_bf16x2(0.0f, s1 * inv_hw) & 0xFFFF0000u);
+    const uint16_t* w = L.w;
+    const float* bias = L.bias;
+    const int N = L.N, relu = L.relu;
+    const int c0 = lane, c1 = lane + 32;
+    for (int o0 = 0; o0 < N; o0 += 8) {
+        // W[o][c] in the tiled image: row o of tile 0, chunk (c / 8) ^ (o & 7), element c % 8.  Eight outputs at a
+        // time, their weights fetched before any of the reductions.
+        float acc[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int o = min(o0 + e, N - 1);
+            const float w0 = __uint_as_float((uint32_t)__ldg(w + o * 64 + (((c0 >> 3) ^ (o & 7)) << 3) + (c0 & 7)) << 16);
+            const float w1 = __uint_as_float((uint32_t)__ldg(w + o * 64 + (((c1 >> 3) ^ (o & 7)) << 3) + (c1 & 7)) << 16);
+            acc[e] = p0 * w0 + p1 * w1;
+        }
+        const float b = (o0 + (lane & 7) < N) ? __ldg(bias + o0 + (lane & 7)) : 0.0f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], d);
+        }
+        // lane e (< 8) writes output o0 + e
+        float mine = acc[0];
+#pragma unroll
+        for (int e = 1; e < 8; ++e) mine = ((lane & 7) == e) ? acc[e] : mine;
+        if (lane < 8 && o0 + lane < N) {
+            float v = mine + b;
+            if (relu) v = fmaxf(v, 0.0f);
+            dst[o0 + lane] = v;
+        }
+    }
+}
+
+void launch_pool_head(const float* partial, int n, int strips, int HW, const ModelDev* models, int layer,
+                      const int32_t* offsets, int T, const int32_t* perm, float* out, int out_elems, cudaStream_t s) {
+    launch_pdl(pool_head_kernel, dim3((n + 7) / 8), dim3(256), 0, s, partial, n, strips, 1.0f / (float)HW, models, layer,
+               offsets, T, perm, out, out_elems);
+}
+
 cudaError_t configure_grouped_conv() {
     return cudaFuncSetAttribute(grouped_conv3x3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
 }

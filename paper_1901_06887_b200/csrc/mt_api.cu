@@ -38,7 +38,7 @@ struct HostModel {
 
 enum KernelId { K_BUCKET = 0, K_GATHER, K_GEMM, K_CONV, K_POOL, K_FUSED, K_COUNT };
 const char* const kKernelNames[K_COUNT] = {"bucketing (histogram, scans, scatter, row move, work items)", "gather_rows",
-                                           "grouped_gemm", "grouped_conv3x3", "pool_finalize", "fused_mlp"};
+                                           "grouped_gemm", "grouped_conv3x3", "pool (finalize, or pool + head)", "fused_mlp"};
 
 struct TimedLaunch {
     int kernel;
@@ -458,6 +458,11 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
     int tiles_per_image = 0;
     for (const HostLayer& f : g.family)
         if (f.kind == MT_CONV3X3) tiles_per_image = g.conv.strips_per_image;
+    // A global average pool followed by a narrow last dense layer (a classifier head) runs as one small launch.
+    const char* ph_env = getenv("MT_POOL_HEAD");
+    const bool pool_head = L >= 3 && g.family[L - 2].kind == MT_GLOBAL_AVG_POOL && g.family[L - 1].kind == MT_DENSE &&
+                           g.family[L - 2].in_ch == 64 && g.family[L - 1].in_ch == 64 && g.out_elems <= 64 &&
+                           !(ph_env && ph_env[0] == '0');
     // Conv layers run on CTA pairs (two images of a tenant per cluster) when the strip geometry allows the tap
     // pairing; MT_CONV_PAIR=0 forces the one-CTA executor.
     const char* cpair_env = getenv("MT_CONV_PAIR");
@@ -533,6 +538,12 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             if (conv_pair) CU_OK(launch_grouped_conv_pair(l == 0 ? in_map : g.act_map[l], feeds_pool ? (l == 0 ? in_map : g.act_map[l]) : g.act_store_map[l + 1],
                                                           a, conv_pair_smem_bytes(g.conv), g.sm_count, s));
             else launch_grouped_conv(l == 0 ? in_map : g.act_map[l], a, g.conv.smem_bytes, g.sm_count, s);
+        } else if (pool_head && l == L - 2) {
+            // pool + narrow last dense layer in one launch (the loop ends here: the head is done)
+            Timer t(K_POOL, s);
+            launch_pool_head(g.d_pool_partial, n, g.conv.strips_per_image, f.h * f.w, g.d_models, L - 1, g.d_offsets, g.T,
+                             g.d_perm, (float*)outputs, g.out_elems, s);
+            break;
         } else {
             Timer t(K_POOL, s);
             // a pool always follows a conv (checked at registration), whose epilogue already reduced every strip

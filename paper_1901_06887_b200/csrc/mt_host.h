@@ -167,4 +167,9 @@ cudaError_t launch_grouped_conv_pair(const CUtensorMap& tmap_x, const CUtensorMa
 void launch_pool_finalize(const float* partial, int n, int strips, int C, int HW, uint16_t* out, int ld_out,
                           cudaStream_t s);
 
+// The same fused with the model's last layer when that is a dense layer from the pooled 64 channels to at most 64
+// outputs: pooled values (rounded to bf16) x head weights, bias, optional ReLU, fp32 rows written to arrival order.
+void launch_pool_head(const float* partial, int n, int strips, int HW, const ModelDev* models, int layer,
+                      const int32_t* offsets, int T, const int32_t* perm, float* out, int out_elems, cudaStream_t s);
+
 }  // namespace mt

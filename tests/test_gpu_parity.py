@@ -120,6 +120,21 @@ def test_conv_many_strips_per_cta(h, w, n, tenants, conv_path):
     run_and_check(wl.models, wl.model_ids, wl.inputs)
 
 
+def test_pool_followed_by_head_both_ways(monkeypatch):
+    # a global average pool followed by a narrow last dense layer runs as one small launch; MT_POOL_HEAD=0 (and any
+    # head wider than 64) takes the pool_finalize + grouped dense path instead: both against the oracle
+    wl = synth.make_workload(4, n=23, n_tenants=4, h=12, w=40, n_conv=2)
+    got_fused, _ = run_and_check(wl.models, wl.model_ids, wl.inputs)
+    monkeypatch.setenv("MT_POOL_HEAD", "0")
+    got_split, _ = run_and_check(wl.models, wl.model_ids, wl.inputs)
+    assert np.abs(got_fused - got_split).max() <= 1e-4        # same bf16 pooled values and weights, other summation order
+    ids = wl.model_ids.copy(); ids[3] = 9                      # a rejected id on the fused pool + head path
+    monkeypatch.delenv("MT_POOL_HEAD")
+    got = harness.run_batch(ids, wl.inputs, 10)
+    assert mt.mt_get_async_status() == (2, 3)
+    assert np.isnan(got[3]).all() and np.array_equal(np.delete(got, 3, 0), np.delete(got_fused, 3, 0))
+
+
 def test_conv_single_tap_shift_closed_form_on_gpu():
     # tap (ky,kx) with weight 1 on the diagonal: Y = shifted X (zero outside), exact in bf16
     H, W = 6, 9
