@@ -484,6 +484,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             a.tile_n[l] = g.tile_n[l]; a.tile_m[l] = pair_mode[l] ? 2 * BM : BM;
             if (l < L && g.family[l].kind == MT_CONV3X3) a.tile_m[l] = conv_pair ? 2 : 1;
             a.items[l] = (l < MT_MAX_LAYERS) ? g.d_items[l] : nullptr;
+            if (pool_head && l == L - 1) a.items[l] = nullptr;     // the pool + head launch needs no work items
         }
         a.item_grid = g.sm_count;
         a.block_hist = g.d_block_hist; a.counts = g.d_counts; a.offsets = g.d_offsets; a.tile_prefix = g.d_tile_prefix;
