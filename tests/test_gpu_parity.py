@@ -135,6 +135,22 @@ def test_pool_followed_by_head_both_ways(monkeypatch):
     assert np.isnan(got[3]).all() and np.array_equal(np.delete(got, 3, 0), np.delete(got_fused, 3, 0))
 
 
+@pytest.mark.parametrize("n_out,relu", [(1, 0), (33, 1), (64, 0), (65, 0)])
+def test_pool_head_widths(n_out, relu):
+    # heads of 1..64 outputs go through the pool + head launch (also with a ReLU on the head), 65 through the
+    # pool_finalize + grouped dense path
+    rng = np.random.default_rng(n_out)
+    H, W = 9, 31
+    models = []
+    for t in range(3):
+        m = synth.make_conv_stack(4, 50 + t, 1, 64, H, W, n_out)
+        m[-1].relu = relu
+        models.append(m)
+    ids = rng.integers(0, 3, 11).astype(np.int32)
+    x = bits(rng.standard_normal((11, H * W * 64)))
+    run_and_check(models, ids, x)
+
+
 def test_conv_single_tap_shift_closed_form_on_gpu():
     # tap (ky,kx) with weight 1 on the diagonal: Y = shifted X (zero outside), exact in bf16
     H, W = 6, 9
