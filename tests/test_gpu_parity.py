@@ -233,6 +233,42 @@ def test_async_host_entry_on_two_streams_matches_device_entry():
             h_out[k].fill_(float("nan"))
 
 
+@pytest.mark.parametrize("family", ["conv", "mlp", "small_mlp"])
+def test_different_batches_back_to_back_without_synchronising(family):
+    # three different batches enqueued one after the other on one stream, no synchronisation in between (each
+    # launch's prologue overlaps its predecessor's tail; workspaces are reused): every batch must match the oracle
+    if family == "conv":
+        wl = synth.make_workload(4, n=20, n_tenants=4, h=56, w=56, n_conv=2)
+        mk = lambda k, n: synth.make_requests(4, wl.models, n=n, salt=70 + k)
+        sizes = (20, 9, 20)
+    elif family == "mlp":
+        wl = synth.make_workload(3, n=900, n_tenants=40)
+        mk = lambda k, n: synth.make_requests(3, wl.models, n=n, salt=70 + k)
+        sizes = (900, 700, 900)
+    else:
+        wl = synth.make_workload(1, n=64)
+        mk = lambda k, n: synth.make_requests(1, wl.models, n=n, salt=70 + k)
+        sizes = (64, 33, 64)
+    fresh(max(64, len(wl.models)))
+    harness.register_models(wl.models)
+    batches = [mk(k, n) for k, n in enumerate(sizes)]
+    mt.mt_infer(harness.bf16_bits_to_device(batches[0][1]), torch.from_numpy(batches[0][0]).cuda(), sizes[0],
+                torch.empty((sizes[0], wl.out_elems), device="cuda"))      # sizes the workspace
+    torch.cuda.synchronize()
+    xs = [harness.bf16_bits_to_device(x.reshape(len(i), -1)) for i, x in batches]
+    ids = [torch.from_numpy(i).cuda() for i, _ in batches]
+    outs = [torch.full((len(i), wl.out_elems), float("nan"), device="cuda") for i, _ in batches]
+    for rep in range(3):
+        for k in range(3):
+            mt.mt_infer(xs[k], ids[k], sizes[k], outs[k])
+    torch.cuda.synchronize()
+    assert mt.mt_get_async_status() == (0, -1)
+    for k, (i, x) in enumerate(batches):
+        ref = oracle.forward(wl.models, i, x)
+        got = outs[k].cpu().numpy()
+        assert np.isfinite(got).all() and harness.scaled_error(got, ref).max() <= TOL, k
+
+
 def test_growing_batches_and_wider_models_reallocate_correctly(small_batch_path):
     rng = np.random.default_rng(9)
     mk = lambda h: synth.make_mlp(3, h, (128, h, 64))
