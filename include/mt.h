@@ -12,7 +12,8 @@
  *
  * Threading: all calls are serialised by one internal mutex.  A context has
  * one workspace, so two mt_infer calls must not be in flight on different
- * streams at the same time (order them with events, or use one stream).
+ * streams at the same time (order them with events, or use one stream;
+ * mt_infer_host_async does that ordering itself and may be used on two streams).
  *
  * Every function returns an mt_status; MT_OK (0) is success.  No function
  * throws, traps or aborts.  There is no CPU fallback: on a device that is not
