@@ -1,5 +1,5 @@
 // Grouped 3x3 convolution executor, CTA-pair form (images whose padded row length is 64 pixels, i.e. the 56 x 56
-// workload): the same implicit GEMM, strip geometry and tap pairing as grouped_conv.cu,
+// workload): the same implicit GEMM and tap pairing as grouped_conv.cu,
 //     Y[r, y, x, o] = act(b_t[o] + sum_{ky,kx,c} X[r, y+ky-1, x+kx-1, c] * W_t[o, ky, kx, c]),
 // but two CTAs of a cluster (two SMs) work in lockstep on the same strip of TWO images of one tenant, and ONE
 // thread of the leader CTA issues tcgen05.mma.cta_group::2 (M = 256: 128 pixels of each image) for both.
@@ -12,12 +12,20 @@
 // W(2,kx), rank 1: W(0,kx)); 60 KiB per CTA instead of 72.
 //
 // Synchronisation inside the pair (every wait bounded, as everywhere):
-//   sfull[s]   in the leader: announces the bytes of BOTH CTAs' strip loads; both loads report there;
-//   sempty[s]  in each CTA: its own epilogue releases its own strip buffer;
+//   bfull[k]   in the leader: announces the bytes of BOTH CTAs' loads of a block of two image rows; both report there;
+//   bempty[k]  in each CTA: its own epilogue releases its own blocks;
 //   tfull[a]   in both CTAs, signalled together by a multicast commit: each CTA drains its own 128 accumulator rows;
 //   tempty[a]  in the leader: 16 arrivals (one per epilogue warp, 8 local and 8 remote);
 //   wfull      in each CTA for its own weight image; the peer then arrives on wpeer in the leader;
 //   wempty     in both CTAs, multicast commit once every MMA on the old weights is done.
+// Input staging.  The image is fetched in blocks of two padded rows (128 pixels, 16 KiB, zero fill outside the image
+// as the padding): block b of an image holds input rows 2b-1 and 2b, so the tile of output rows 2i, 2i+1 reads block
+// i (tap row 0), block i shifted by one row (tap row 1: second row of block i, first row of block i+1) and block i+1
+// (tap row 2).  Blocks go round a ring of eight slots in load order, so consecutive blocks are neighbours in shared
+// memory and a shifted operand simply runs on into the next slot; behind the last slot sits a copy of the first row
+// of the block in slot 0 for the operand that starts in the last slot.  Nothing is fetched twice (a strip with its
+// own halo re-read half of its rows), a block is released as soon as the tile below it has been issued and
+// completed, and loads run six tiles ahead of the tensor pipe instead of one or two strips.
 // The two CTAs meet at a cluster barrier before they exit.  A tenant with an odd number of images leaves the peer
 // of its last pair a copy of the leader's image, computed and not stored.
 //
@@ -37,11 +45,14 @@ constexpr int kOffPair = 3 * kCpHalfTap;                  // stacked pairs: rank
 constexpr int kOffBot = kOffPair + 3 * kCpFullTap;        // ky = 2 taps alone, this CTA's 32 output channels
 constexpr int kOffTop = kOffBot + 3 * kCpHalfTap;         // ky = 0 taps alone
 static_assert(kOffTop + 3 * kCpHalfTap == kConvPairWeightBytes, "weight image layout");
-constexpr int kCpMaxStages = 4;
+constexpr int kCpRing = 8;                                // slots of the block ring
+constexpr int kCpBlockBytes = 2 * 64 * 128;               // two padded rows of 64 pixels x 64 channels
+constexpr int kCpGhostBytes = 64 * 128 + 1024;            // first row of the block in slot 0, again, behind the last slot
 constexpr int kCpSlots = 8;                               // TMEM ring: 8 accumulators of 64 columns
 constexpr int kCpBarBytes = 2048;
 constexpr int kCpRecords = 16;
 constexpr int kCpOutStageBytes = 8 * 2048;                // per epilogue warp: 32 pixels x 64 bytes
+constexpr int kCpSmemBytes = kConvPairWeightBytes + kCpRing * kCpBlockBytes + kCpGhostBytes + kCpOutStageBytes + kCpBarBytes + 1024;
 
 __device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
                                                  uint32_t leader_bar) {
@@ -56,32 +67,34 @@ struct PairStrip {
 };
 
 __global__ void __launch_bounds__(kCpThreads, 1)
-grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_y,
-                            const ConvArgs p) {
+grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_x1,
+                            const __grid_constant__ CUtensorMap tmap_y, const ConvArgs p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw);
     const uint32_t w_smem = base;
-    const uint32_t strip0 = base + kConvPairWeightBytes;
+    const uint32_t ring0 = base + kConvPairWeightBytes;           // kCpRing blocks, then the ghost row
+    const uint32_t ghost0 = ring0 + kCpRing * kCpBlockBytes;
     // output staging: one 2 KiB region per epilogue warp (32 pixels x 32 channels), the source of its TMA stores
-    const uint32_t out_stage0 = strip0 + p.n_stages * p.stage_bytes;
-    uint8_t* out_stage_ptr = smem + kConvPairWeightBytes + p.n_stages * p.stage_bytes;
+    const uint32_t out_stage0 = ghost0 + kCpGhostBytes;
+    uint8_t* out_stage_ptr = smem + kConvPairWeightBytes + kCpRing * kCpBlockBytes + kCpGhostBytes;
     const uint32_t bar0 = out_stage0 + kCpOutStageBytes;
     uint8_t* bar_ptr = out_stage_ptr + kCpOutStageBytes;
-    auto sfull_bar = [&](int s) { return bar0 + 8u * s; };
-    auto sempty_bar = [&](int s) { return bar0 + 8u * (kCpMaxStages + s); };
-    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kCpMaxStages + a); };
-    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kCpMaxStages + kCpSlots + a); };
-    const uint32_t wfull_bar = bar0 + 8u * (2 * kCpMaxStages + 2 * kCpSlots);
+    auto bfull_bar = [&](int k) { return bar0 + 8u * k; };
+    auto bempty_bar = [&](int k) { return bar0 + 8u * (kCpRing + k); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kCpRing + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kCpRing + kCpSlots + a); };
+    const uint32_t wfull_bar = bar0 + 8u * (2 * kCpRing + 2 * kCpSlots);
     const uint32_t wempty_bar = wfull_bar + 8u;
     const uint32_t wpeer_bar = wfull_bar + 16u;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * (2 * kCpMaxStages + 2 * kCpSlots + 3));
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * (2 * kCpRing + 2 * kCpSlots + 3));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    float* s_bias = reinterpret_cast<float*>(bar_ptr + 256);          // 64 floats
-    // Per-strip record, producer -> epilogue of the same CTA: x = flags (1 new tenant, 8 copy of the leader's image:
-    // do not store, 4 the strip's last tile is finished by the next strip), y = image (bucketed index), z = first output row, w = tenant.
-    int4* s_rec = reinterpret_cast<int4*>(bar_ptr + 512);             // kCpRecords x 16 bytes
+    static_assert(8 * (2 * kCpRing + 2 * kCpSlots + 3) + 8 <= 512, "barriers, TMEM address and abort flag come before the bias");
+    float* s_bias = reinterpret_cast<float*>(bar_ptr + 512);          // 64 floats
+    // Per-strip record, producer -> epilogue of the same CTA: x = flags (1 new tenant, 2 the strip starts a segment, 8 copy
+    // of the leader's image: do not store), y = image (bucketed index), z = first output row, w = tenant.
+    int4* s_rec = reinterpret_cast<int4*>(bar_ptr + 768);             // kCpRecords x 16 bytes
     float* s_pool = reinterpret_cast<float*>(bar_ptr + 1024);         // 8 warps x 32 channel sums (fused pooling)
 
     pdl_launch_dependents();
@@ -89,7 +102,7 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     const uint32_t rank = cluster_ctarank();          // 0 = leader (issues the MMAs), 1 = peer
     const bool is_leader = (rank == 0);
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kCpMaxStages; ++s) { mbar_init(sfull_bar(s), 1); mbar_init(sempty_bar(s), 1); }
+        for (int k = 0; k < kCpRing; ++k) { mbar_init(bfull_bar(k), 1); mbar_init(bempty_bar(k), 1); }
         for (int a = 0; a < kCpSlots; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 2 * (kCpEpiThreads / 32)); }
         mbar_init(wfull_bar, 1);
         mbar_init(wempty_bar, 1);
@@ -97,10 +110,11 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tmap_x);
+        prefetch_tensormap(&tmap_x1);
         prefetch_tensormap(&tmap_y);
     }
-    // the last rows of every strip stage are read (for rows that are never stored) but not written by the TMA box
-    for (int i = threadIdx.x; i < (p.n_stages * p.stage_bytes) / 16; i += blockDim.x)
+    // operands shifted by one or two pixels read a little past what the copies wrote (for pad columns only)
+    for (int i = threadIdx.x; i < (kCpRing * kCpBlockBytes + kCpGhostBytes) / 16; i += blockDim.x)
         reinterpret_cast<uint4*>(smem + kConvPairWeightBytes)[i] = make_uint4(0, 0, 0, 0);
     fence_proxy_async_smem();
     if (warp == 1) {                                  // the same warp of both CTAs
@@ -148,22 +162,35 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
 
     if (warp == 0) {
         if (lane == 0) {   // ------------------------------------------------ TMA producer (both CTAs)
-            int stage = 0; uint32_t phase = 0;
             int w_loads = 0, w_tenant = -1;
             const uint32_t wpeer_leader = map_to_cta(wpeer_bar, 0);
-            for (int s = s_begin; s < s_end; ++s) {
+            const uint32_t bfull_leader0 = map_to_cta(bfull_bar(0), 0);
+            int nb = 0;                     // blocks armed so far; block b goes to slot b % kCpRing
+            bool ok = true;
+            for (int s = s_begin; ok && s < s_end; ++s) {
                 const PairStrip c = locate(s);
                 const bool new_tenant = (c.t != w_tenant);
-                if (!mbar_wait(sempty_bar(stage), phase ^ 1u, abort_flag, p.status, 52)) break;
                 const int img = p.perm ? p.perm[c.j] : c.j;
-                const bool defer_bottom = s + 1 < s_end && c.strip_in_image + 1 < p.strips_per_image;
+                const bool seg_start = (s == s_begin) || c.strip_in_image == 0;
+                // published to this CTA's epilogue with the strip's first block (the issuer starts the strip's first
+                // tile only after that block has landed)
                 s_rec[(s - s_begin) & (kCpRecords - 1)] =
-                    make_int4((new_tenant ? 1 : 0) | (defer_bottom ? 4 : 0) | (c.dummy ? 8 : 0), c.j, c.y0, c.t);
-                if (is_leader) mbar_expect_tx(sfull_bar(stage), 2u * (uint32_t)p.box_bytes);   // both CTAs' bytes
-                tma_load_4d_pair(strip0 + stage * p.stage_bytes, &tmap_x, 0, -1, c.y0 - 1, img, map_to_cta(sfull_bar(stage), 0));
+                    make_int4((new_tenant ? 1 : 0) | (seg_start ? 2 : 0) | (c.dummy ? 8 : 0), c.j, c.y0, c.t);
+                // blocks of the strip: kb = 0 is the block of its first tile (loaded by the strip above unless the strip
+                // starts a segment), kb = k the block of tile k, kb = TS the block under its last tile
+                for (int kb = seg_start ? 0 : 1; kb <= TS; ++kb) {
+                    const int slot = nb & (kCpRing - 1);
+                    if (!mbar_wait(bempty_bar(slot), (uint32_t)(((nb / kCpRing) & 1) ^ 1), abort_flag, p.status, 52)) { ok = false; break; }
+                    const int y_in = c.y0 + 2 * kb - 1;              // first input row of the block
+                    const uint32_t bytes = kCpBlockBytes + (slot == 0 ? 64u * 128u : 0u);
+                    if (is_leader) mbar_expect_tx(bfull_bar(slot), 2u * bytes);   // both CTAs' bytes
+                    tma_load_4d_pair(ring0 + slot * kCpBlockBytes, &tmap_x, 0, -1, y_in, img, bfull_leader0 + 8u * slot);
+                    if (slot == 0) tma_load_4d_pair(ghost0, &tmap_x1, 0, -1, y_in, img, bfull_leader0);
+                    ++nb;
+                }
+                if (!ok) break;
                 if (new_tenant) {
-                    // The issuer releases the old weights when it reaches this strip, i.e. after the strip has
-                    // landed in both CTAs: so the strip goes first.
+                    // The issuer releases the old weights when it reaches this strip in its own order.
                     if (w_loads > 0 && !mbar_wait_spin(wempty_bar, (uint32_t)((w_loads - 1) & 1), abort_flag, p.status, 51, 64)) break;
                     mbar_expect_tx(wfull_bar, kConvPairWeightBytes);
                     bulk_load(w_smem, p.models[c.t].layer[p.layer].w + kConvPairImageOffset + (size_t)rank * (kConvPairWeightBytes / 2),
@@ -175,7 +202,6 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                     w_tenant = c.t;
                     ++w_loads;
                 }
-                if (++stage == p.n_stages) { stage = 0; phase ^= 1u; }
             }
         }
     } else if (warp == 1) {
@@ -185,14 +211,16 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
             const uint32_t tb = __shfl_sync(0xffffffffu, *tmem_slot, 0);
             constexpr uint32_t idesc64 = make_idesc_bf16(2 * BM, kCpN);
             constexpr uint32_t idesc128 = make_idesc_bf16(2 * BM, 2 * kCpN);
-            int stage = 0; uint32_t phase = 0;
             int g = 0;                      // tiles started so far by this pair; tile g lives in TMEM slot g % kCpSlots
+            int bc = 0;                     // load-order number of the block with the current tile's first input rows
             int w_loads = 0;
             bool ok = true;
             const uint32_t w_lo = desc_lo(w_smem);
+            const uint32_t ring_lo = desc_lo(ring0);
             constexpr uint32_t kHalfLo = kCpHalfTap >> 4, kFullLo = kCpFullTap >> 4;
             constexpr uint32_t kMidLo = kOffMid >> 4, kPairLo = kOffPair >> 4, kBotLo = kOffBot >> 4, kTopLo = kOffTop >> 4;
             constexpr uint32_t kPixLo = 128 >> 4;                // one pixel (128 bytes) further
+            constexpr uint32_t kBlockLo = kCpBlockBytes >> 4;
             // four K steps of one 128-pixel block (of each CTA) against one tap operand
             auto issue = [&](uint32_t a_lo, uint32_t b_lo, uint32_t d_tmem, uint32_t idesc, bool overwrite) {
                 if (!leader) return;
@@ -202,9 +230,10 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                 umma_pair_lohi<true>(d_tmem, a_lo + 4, b_lo + 4, idesc);
                 umma_pair_lohi<true>(d_tmem, a_lo + 6, b_lo + 6, idesc);
             };
+            auto bfull_parity = [](int q) { return (uint32_t)((q / kCpRing) & 1); };
             int t_hi = -1;                  // units [.., t_hi) belong to the current tenant
             int in_image = 0;               // index of the current strip inside its image
-            uint32_t strip_ready = 0, slot_ready = 0;
+            uint32_t block_ready = 0, slot_ready = 0;
             for (int s = s_begin; ok && s < s_end; ++s) {
                 const bool new_tenant = (s >= t_hi);
                 if (new_tenant) {           // rare: a tenant border (or the first unit)
@@ -212,41 +241,42 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                     t_hi = cur_hi;
                     in_image = c.strip_in_image;
                 }
-                if (!strip_ready) {
-                    if (!mbar_wait_spin(sfull_bar(stage), phase, abort_flag, p.status, 55)) break;
+                // a segment = the tiles of one image that this pair computes one after the other
+                const bool seg_start = !(s > s_begin && in_image > 0);
+                const bool seg_end = !(s + 1 < s_end && in_image + 1 < p.strips_per_image);
+                if (seg_start) {
+                    if (!mbar_wait_spin(bfull_bar(bc & (kCpRing - 1)), bfull_parity(bc), abort_flag, p.status, 55)) break;
+                    block_ready = 0;
                 }
-                tc_fence_after();
                 if (new_tenant) {
                     if (w_loads > 0 && leader) umma_commit_pair(wempty_bar);     // fires when all MMAs on the old weights are done
                     if (!mbar_wait(wfull_bar, (uint32_t)(w_loads & 1), abort_flag, p.status, 56)) break;
                     if (!mbar_wait_spin(wpeer_bar, (uint32_t)(w_loads & 1), abort_flag, p.status, 57)) break;
                     ++w_loads;
                 }
-                const bool pair_top = s > s_begin && in_image > 0;
-                const bool defer_bottom = s + 1 < s_end && in_image + 1 < p.strips_per_image;
-                const uint32_t strip_lo = desc_lo(strip0 + stage * p.stage_bytes);
-                const int next_stage = (stage + 1 == p.n_stages) ? 0 : stage + 1;
-                const uint32_t next_phase = (stage + 1 == p.n_stages) ? (phase ^ 1u) : phase;
-                strip_ready = 0;
-                for (int i = 0; i < TS; ++i, ++g) {
+                for (int i = 0; i < TS; ++i, ++g, ++bc) {
                     const int slot = g % kCpSlots;
+                    // the block under the tile (its tap row 1 runs on into that block's first row)
+                    if (!block_ready) {
+                        if (!mbar_wait_spin(bfull_bar((bc + 1) & (kCpRing - 1)), bfull_parity(bc + 1), abort_flag, p.status, 59)) { ok = false; break; }
+                    }
                     if (!slot_ready) {   // the slot must have been drained by both CTAs' epilogues of tile g - kCpSlots
                         if (!mbar_wait_spin(tempty_bar(slot), (uint32_t)(((g / kCpSlots) & 1) ^ 1), abort_flag, p.status, 54)) { ok = false; break; }
                     }
                     tc_fence_after();
                     const uint32_t d_this = tb + slot * kCpN;
-                    const uint32_t blk = strip_lo + (uint32_t)(i * BM) * kPixLo;     // padded pixel i*128 of the strip
-                    const bool last_tile = (i == TS - 1);
-                    // ky = 1 first: these overwrite the fresh accumulator
+                    const uint32_t blk = ring_lo + (uint32_t)(bc & (kCpRing - 1)) * kBlockLo;
+                    const bool more_in_segment = !(i == TS - 1 && seg_end);
+                    // tap row 1 first: these overwrite the fresh accumulator
                     issue(blk + (uint32_t)(Wp + 0) * kPixLo, w_lo + kMidLo + 0 * kHalfLo, d_this, idesc64, true);
                     // look ahead: the answers are consumed after the rest of this tile has been queued
                     const uint32_t poll_slot = mbar_test_wait(tempty_bar((g + 1) % kCpSlots), (uint32_t)((((g + 1) / kCpSlots) & 1) ^ 1));
-                    uint32_t poll_strip = 0;
-                    if (last_tile) poll_strip = mbar_test_wait(sfull_bar(next_stage), next_phase);
+                    uint32_t poll_block = 0;
+                    if (more_in_segment) poll_block = mbar_test_wait(bfull_bar((bc + 2) & (kCpRing - 1)), bfull_parity(bc + 2));
                     issue(blk + (uint32_t)(Wp + 1) * kPixLo, w_lo + kMidLo + 1 * kHalfLo, d_this, idesc64, false);
                     issue(blk + (uint32_t)(Wp + 2) * kPixLo, w_lo + kMidLo + 2 * kHalfLo, d_this, idesc64, false);
-                    // block at the tile's first row: ky = 0 of this tile and ky = 2 of the tile above
-                    const bool have_above = (i > 0) || pair_top;
+                    // the tile's own block: tap row 0 of this tile and tap row 2 of the tile above
+                    const bool have_above = (i > 0) || !seg_start;
                     const bool adjacent = slot != 0;                              // slots g-1 and g contiguous in TMEM
                     if (have_above && adjacent) {
 #pragma unroll
@@ -261,18 +291,20 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                     }
                     if (have_above && leader) umma_commit_pair(tfull_bar((g - 1) % kCpSlots));    // tile above is complete
                     slot_ready = poll_slot;
-                    if (last_tile) strip_ready = (s + 1 < s_end) ? poll_strip : 0;
+                    block_ready = poll_block;
                 }
                 if (!ok) break;
-                if (!defer_bottom) {
-                    // nobody below will finish the strip's last tile: its ky = 2 taps from the block under it
-                    const uint32_t blk = strip_lo + (uint32_t)(TS * BM) * kPixLo;
+                if (seg_end) {
+                    // no tile below finishes the segment's last tile: its tap row 2 from the block under it (landed:
+                    // the tile waited for it)
+                    const uint32_t blk = ring_lo + (uint32_t)(bc & (kCpRing - 1)) * kBlockLo;
                     const int last = (g - 1) % kCpSlots;
                     for (int kx = 0; kx < 3; ++kx)
                         issue(blk + kx * kPixLo, w_lo + kBotLo + kx * kHalfLo, tb + last * kCpN, idesc64, false);
                     if (leader) umma_commit_pair(tfull_bar(last));
+                    ++bc;
+                    block_ready = 0;
                 }
-                stage = next_stage; phase = next_phase;
                 if (++in_image == p.strips_per_image) in_image = 0;
             }
         }
@@ -285,7 +317,8 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
         constexpr int rows_per_tile = BM / Wp;
         int g = 0, relu = 0;
         bool ok = true;
-        int img_j = 0, y0 = 0, store = 1, release_at = 0;
+        int img_j = 0, y0 = 0, store = 1;
+        int rel = 0;                                // blocks released so far (load order), kept by the releasing thread
         const bool pooling = (p.pool_partial != nullptr);
         const uint32_t tempty_leader0 = map_to_cta(tempty_bar(0), 0);   // the leader's tempty barriers, 8 bytes apart
         for (int s = s_begin; ok && s < s_end; ++s) {
@@ -303,10 +336,10 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                     // the strip's record was published (with the strip's data) before any of its MMAs were issued
                     const int4 rec = s_rec[(s - s_begin) & (kCpRecords - 1)];
                     img_j = rec.y; y0 = rec.z; store = (rec.x & 8) ? 0 : 1;
-                    // Which completion tells that no MMA will read the strip's buffer again: the strip's last tile
-                    // when the strip finishes it itself; when its ky = 2 taps are left to the next strip (which reads
-                    // its own buffer for them), already the tile before - that commit follows the last tile's other taps.
-                    release_at = ((rec.x & 4) && TS >= 2) ? TS - 2 : TS - 1;
+                    // This completion (tile g) follows every read of the block under tile g (by tile g and, if the
+                    // segment goes on, by the first two tap rows of tile g + 1, which are queued before the commit);
+                    // the segment's first tile also hands back its own block.
+                    if (threadIdx.x == 64 && (rec.x & 2)) { mbar_arrive(bempty_bar(rel & (kCpRing - 1))); ++rel; }
                     if (rec.x & 1) {                // new tenant: its bias into shared memory, ReLU flag into a register
                         const LayerDev& L = p.models[rec.w].layer[p.layer];
                         asm volatile("bar.sync 1, %0;" ::"n"(kCpEpiThreads) : "memory");   // everyone done with the old bias
@@ -315,7 +348,7 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                         asm volatile("bar.sync 1, %0;" ::"n"(kCpEpiThreads) : "memory");
                     }
                 }
-                if (i == release_at && threadIdx.x == 64) mbar_arrive(sempty_bar((s - s_begin) % p.n_stages));
+                if (threadIdx.x == 64) { mbar_arrive(bempty_bar(rel & (kCpRing - 1))); ++rel; }
                 tc_fence_after();
                 uint32_t v[32];
                 tmem_ld32(tmem_base + (static_cast<uint32_t>(q4 * 32) << 16) + slot * kCpN + half * 32, v);
@@ -446,21 +479,20 @@ void launch_pretile_conv_pair(const uint16_t* w, uint16_t* out, cudaStream_t s) 
     pretile_conv_pair_kernel<<<(2 * kConvPairWeightBytes / 16 + 255) / 256, 256, 0, s>>>(w, reinterpret_cast<uint4*>(out));
 }
 
-int conv_pair_smem_bytes(const ConvPlan& plan) {
-    return kConvPairWeightBytes + plan.n_stages * plan.stage_bytes + kCpOutStageBytes + kCpBarBytes + 1024;
-}
+int conv_pair_smem_bytes() { return kCpSmemBytes; }
 
 cudaError_t configure_grouped_conv_pair() {
     return cudaFuncSetAttribute(grouped_conv3x3_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
 }
 
 // Cluster of two CTAs; grid = an even number of CTAs (one per SM).  a.tile_prefix counts (pair of images, strip) units.
-cudaError_t launch_grouped_conv_pair(const CUtensorMap& tmap_x, const CUtensorMap& tmap_y, const ConvArgs& a, int smem_bytes,
-                                     int sm_count, cudaStream_t s) {
+// tmap_x2 / tmap_x1: the layer's input with boxes of 64 pixels x 2 rows / x 1 row; tmap_y: its output, 32 x 32 store boxes.
+cudaError_t launch_grouped_conv_pair(const CUtensorMap& tmap_x2, const CUtensorMap& tmap_x1, const CUtensorMap& tmap_y,
+                                     const ConvArgs& a, int sm_count, cudaStream_t s) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(sm_count & ~1);
     cfg.blockDim = dim3(kCpThreads);
-    cfg.dynamicSmemBytes = (size_t)smem_bytes;
+    cfg.dynamicSmemBytes = (size_t)kCpSmemBytes;
     cfg.stream = s;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -469,7 +501,7 @@ cudaError_t launch_grouped_conv_pair(const CUtensorMap& tmap_x, const CUtensorMa
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 2;
     ++g_kernel_launches;
-    return cudaLaunchKernelEx(&cfg, grouped_conv3x3_pair_kernel, tmap_x, tmap_y, a);
+    return cudaLaunchKernelEx(&cfg, grouped_conv3x3_pair_kernel, tmap_x2, tmap_x1, tmap_y, a);
 }
 
 }  // namespace mt

@@ -75,6 +75,8 @@ struct Ctx {
     CUtensorMap act_map[MT_MAX_LAYERS + 1];
     CUtensorMap act_map32[MT_MAX_LAYERS + 1];   // dense inputs again, as 32-row boxes
     CUtensorMap act_store_map[MT_MAX_LAYERS + 1];   // conv activations as the store boxes of the CTA-pair executor
+    CUtensorMap act_rows2_map[MT_MAX_LAYERS + 1];   // ... and as its load boxes of two rows and of one row
+    CUtensorMap act_rows1_map[MT_MAX_LAYERS + 1];
     float* d_pool_partial = nullptr;     // per-strip channel sums of a conv layer that feeds a pool
     WorkItem* d_items[MT_MAX_LAYERS] = {nullptr};   // per dense layer
     size_t items_cap[MT_MAX_LAYERS] = {0};
@@ -252,6 +254,12 @@ mt_status ensure_workspace(int n) {
                 if (st != MT_OK) return st;
                 st = encode_nhwc(&g.act_store_map[b], g.act[b], f.in_ch, f.w, f.h, cap, 32, 1, 32);
                 if (st != MT_OK) return st;
+                if (g.conv.Wp == 64) {
+                    st = encode_nhwc(&g.act_rows2_map[b], g.act[b], f.in_ch, f.w, f.h, cap, 64, 2);
+                    if (st != MT_OK) return st;
+                    st = encode_nhwc(&g.act_rows1_map[b], g.act[b], f.in_ch, f.w, f.h, cap, 64, 1);
+                    if (st != MT_OK) return st;
+                }
             }
         }
     }
@@ -491,7 +499,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
         a.perm = g.d_perm; a.inv = g.d_inv; a.status = g.d_status;
         launch_bucketing(a, s);
     }
-    CUtensorMap in_map;
+    CUtensorMap in_map, in_rows2_map, in_rows1_map;
     if (f0.kind == MT_DENSE) {
         if (!rows_in_scatter) {
             Timer t(K_GATHER, s);
@@ -500,6 +508,12 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
     } else {
         st = encode_nhwc(&in_map, inputs, f0.in_ch, f0.w, f0.h, n, g.conv.Wp, g.conv.R + 2);
         if (st != MT_OK) return st;
+        if (conv_pair) {
+            st = encode_nhwc(&in_rows2_map, inputs, f0.in_ch, f0.w, f0.h, n, 64, 2);
+            if (st != MT_OK) return st;
+            st = encode_nhwc(&in_rows1_map, inputs, f0.in_ch, f0.w, f0.h, n, 64, 1);
+            if (st != MT_OK) return st;
+        }
     }
     for (int l = 0; l < L; ++l) {
         const HostLayer& f = g.family[l];
@@ -536,8 +550,9 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             a.strips_per_image = g.conv.strips_per_image; a.box_bytes = g.conv.box_bytes;
             a.status = g.d_status;
             // a layer that feeds the pool stores nothing: any valid map will do for it
-            if (conv_pair) CU_OK(launch_grouped_conv_pair(l == 0 ? in_map : g.act_map[l], feeds_pool ? (l == 0 ? in_map : g.act_map[l]) : g.act_store_map[l + 1],
-                                                          a, conv_pair_smem_bytes(g.conv), g.sm_count, s));
+            if (conv_pair) CU_OK(launch_grouped_conv_pair(l == 0 ? in_rows2_map : g.act_rows2_map[l], l == 0 ? in_rows1_map : g.act_rows1_map[l],
+                                                          feeds_pool ? (l == 0 ? in_map : g.act_map[l]) : g.act_store_map[l + 1],
+                                                          a, g.sm_count, s));
             else launch_grouped_conv(l == 0 ? in_map : g.act_map[l], a, g.conv.smem_bytes, g.sm_count, s);
         } else if (pool_head && l == L - 2) {
             // pool + narrow last dense layer in one launch (the loop ends here: the head is done)

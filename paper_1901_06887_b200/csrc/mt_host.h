@@ -156,12 +156,13 @@ void launch_grouped_conv(const CUtensorMap& tmap_x, const ConvArgs& a, int smem_
 constexpr int kConvPairWeightBytes = 60 * 1024;
 constexpr int kConvPairImageOffset = 9 * 64 * 64;          // bf16 elements of the one-CTA image
 void launch_pretile_conv_pair(const uint16_t* w, uint16_t* out, cudaStream_t s);
-int conv_pair_smem_bytes(const ConvPlan& plan);
+int conv_pair_smem_bytes();
 cudaError_t configure_grouped_conv_pair();
-// tmap_y: the layer's output (NHWC bf16) as boxes of 32 channels x 32 pixels x 1 row, 64-byte swizzle (unused by a
-// layer that feeds the pool)
-cudaError_t launch_grouped_conv_pair(const CUtensorMap& tmap_x, const CUtensorMap& tmap_y, const ConvArgs& a, int smem_bytes,
-                                     int sm_count, cudaStream_t s);
+// tmap_x2, tmap_x1: the layer's input (NHWC bf16) as boxes of 64 channels x 64 pixels x 2 rows and x 1 row (the executor
+// fetches the image in blocks of two rows, whatever ConvArgs says about strip stages); tmap_y: the layer's output as
+// boxes of 32 channels x 32 pixels x 1 row, 64-byte swizzle (unused by a layer that feeds the pool)
+cudaError_t launch_grouped_conv_pair(const CUtensorMap& tmap_x2, const CUtensorMap& tmap_x1, const CUtensorMap& tmap_y,
+                                     const ConvArgs& a, int sm_count, cudaStream_t s);
 
 // Second half of the fused pooling: sums the per-strip channel sums of each image and divides by H*W.
 void launch_pool_finalize(const float* partial, int n, int strips, int C, int HW, uint16_t* out, int ld_out,
