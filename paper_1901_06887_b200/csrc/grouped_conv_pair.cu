@@ -90,12 +90,14 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     const uint32_t wpeer_bar = wfull_bar + 16u;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_ptr + 8 * (2 * kCpRing + 2 * kCpSlots + 3));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    static_assert(8 * (2 * kCpRing + 2 * kCpSlots + 3) + 8 <= 512, "barriers, TMEM address and abort flag come before the bias");
+    static_assert(8 * (2 * kCpRing + 2 * kCpSlots + 3) + 8 <= 320, "barriers, TMEM address and abort flag come before the bias");
     float* s_bias = reinterpret_cast<float*>(bar_ptr + 512);          // 64 floats
     // Per-strip record, producer -> epilogue of the same CTA: x = flags (1 new tenant, 2 the strip starts a segment, 8 copy
     // of the leader's image: do not store), y = image (bucketed index), z = first output row, w = tenant.
     int4* s_rec = reinterpret_cast<int4*>(bar_ptr + 768);             // kCpRecords x 16 bytes
     float* s_pool = reinterpret_cast<float*>(bar_ptr + 1024);         // 8 warps x 32 channel sums (fused pooling)
+    int* s_first = reinterpret_cast<int*>(bar_ptr + 320);             // the first unit's tenant: id, units, requests
+    const uint16_t** s_first_w = reinterpret_cast<const uint16_t**>(bar_ptr + 352);   // ... and its weight block
 
     pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -113,10 +115,8 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
         prefetch_tensormap(&tmap_x1);
         prefetch_tensormap(&tmap_y);
     }
-    // operands shifted by one or two pixels read a little past what the copies wrote (for pad columns only)
-    for (int i = threadIdx.x; i < (kCpRing * kCpBlockBytes + kCpGhostBytes) / 16; i += blockDim.x)
-        reinterpret_cast<uint4*>(smem + kConvPairWeightBytes)[i] = make_uint4(0, 0, 0, 0);
-    fence_proxy_async_smem();
+    // Operands shifted by one or two pixels read a little past what the copies wrote, whatever the previous kernel left
+    // there: rows of the product that belong to pad columns, which are neither stored nor pooled.
     if (warp == 1) {                                  // the same warp of both CTAs
         tmem_alloc_pair(smem_u32(tmem_slot), kCpSlots * kCpN);
         tmem_relinquish_pair();
@@ -136,8 +136,25 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     constexpr int Wp = 64;
     const int TS = p.tiles_per_strip;
 
+    // The first unit's tenant, its range of units and requests and its weight image: every thread looks at a few
+    // tenants, all loads independent of one another, instead of a binary search of dependent loads by each role -
+    // this sits between the previous layer's end and the first MMA.
+    if (s_begin < s_end) {
+        for (int i = threadIdx.x; i < p.T; i += blockDim.x) {
+            const int lo = p.tile_prefix[i], hi = p.tile_prefix[i + 1];
+            const int seg = p.offsets[i], seg_hi = p.offsets[i + 1];
+            const uint16_t* w = p.models[i].layer[p.layer].w;
+            if (lo <= s_begin && s_begin < hi) {
+                s_first[0] = i; s_first[1] = lo; s_first[2] = hi; s_first[3] = seg; s_first[4] = seg_hi - seg;
+                *s_first_w = w;
+            }
+        }
+    }
+    __syncthreads();
+
     // pair-strip -> (tenant, this CTA's image, first row); units of one tenant are consecutive: its range is cached
     int cur_t = -1, cur_lo = 0, cur_hi = 0, cur_seg = 0, cur_n = 0;
+    if (s_begin < s_end) { cur_t = s_first[0]; cur_lo = s_first[1]; cur_hi = s_first[2]; cur_seg = s_first[3]; cur_n = s_first[4]; }
     auto locate = [&](int s) {
         if (s < cur_lo || s >= cur_hi) {
             int lo = 0, hi = p.T;
@@ -167,11 +184,31 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
             const uint32_t bfull_leader0 = map_to_cta(bfull_bar(0), 0);
             int nb = 0;                     // blocks armed so far; block b goes to slot b % kCpRing
             bool ok = true;
+            auto start_weights = [&](int t, const uint16_t* w) {
+                // The issuer releases the old weights when it reaches the tenant's first strip in its own order.
+                if (w_loads > 0 && !mbar_wait_spin(wempty_bar, (uint32_t)((w_loads - 1) & 1), abort_flag, p.status, 51, 64)) return false;
+                mbar_expect_tx(wfull_bar, kConvPairWeightBytes);
+                bulk_load(w_smem, w + kConvPairImageOffset + (size_t)rank * (kConvPairWeightBytes / 2), kConvPairWeightBytes, wfull_bar);
+                w_tenant = t;
+                return true;
+            };
+            auto announce_weights = [&]() {
+                if (!is_leader) {      // tell the leader's issuer once this CTA's share has landed
+                    if (!mbar_wait(wfull_bar, (uint32_t)(w_loads & 1), abort_flag, p.status, 53)) return false;
+                    mbar_arrive_remote(wpeer_leader);
+                }
+                ++w_loads;
+                return true;
+            };
             for (int s = s_begin; ok && s < s_end; ++s) {
                 const PairStrip c = locate(s);
                 const bool new_tenant = (c.t != w_tenant);
                 const int img = p.perm ? p.perm[c.j] : c.j;
                 const bool seg_start = (s == s_begin) || c.strip_in_image == 0;
+                // the very first weights go out before the first blocks: the first MMA needs both, and this is the
+                // larger copy (later ones must wait for the issuer to let go of the old weights, so the blocks go first)
+                const bool weights_first = new_tenant && w_loads == 0;
+                if (weights_first && !start_weights(c.t, *s_first_w)) break;
                 // published to this CTA's epilogue with the strip's first block (the issuer starts the strip's first
                 // tile only after that block has landed)
                 s_rec[(s - s_begin) & (kCpRecords - 1)] =
@@ -189,19 +226,8 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                     ++nb;
                 }
                 if (!ok) break;
-                if (new_tenant) {
-                    // The issuer releases the old weights when it reaches this strip in its own order.
-                    if (w_loads > 0 && !mbar_wait_spin(wempty_bar, (uint32_t)((w_loads - 1) & 1), abort_flag, p.status, 51, 64)) break;
-                    mbar_expect_tx(wfull_bar, kConvPairWeightBytes);
-                    bulk_load(w_smem, p.models[c.t].layer[p.layer].w + kConvPairImageOffset + (size_t)rank * (kConvPairWeightBytes / 2),
-                              kConvPairWeightBytes, wfull_bar);
-                    if (!is_leader) {      // tell the leader's issuer once this CTA's share has landed
-                        if (!mbar_wait(wfull_bar, (uint32_t)(w_loads & 1), abort_flag, p.status, 53)) break;
-                        mbar_arrive_remote(wpeer_leader);
-                    }
-                    w_tenant = c.t;
-                    ++w_loads;
-                }
+                if (new_tenant && !weights_first && !start_weights(c.t, p.models[c.t].layer[p.layer].w)) break;
+                if (new_tenant && !announce_weights()) break;
             }
         }
     } else if (warp == 1) {
