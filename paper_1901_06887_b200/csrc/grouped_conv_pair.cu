@@ -4,12 +4,12 @@
 // but two CTAs of a cluster (two SMs) work in lockstep on the same strip of TWO images of one tenant, and ONE
 // thread of the leader CTA issues tcgen05.mma.cta_group::2 (M = 256: 128 pixels of each image) for both.
 //
-// Why: with 64 output channels an instruction is short, and the one-CTA executor is bound by what its single
-// issuing thread can feed (measured: the thread spends about 1850 cycles per 128-pixel tile, of which the tensor
-// pipe is busy about 1150).  A pair instruction costs the issuing thread the same and keeps two tensor pipes busy,
-// so the issue cost per tile halves.  Each CTA holds only its share of the B operand: for the N = 64 instructions
-// its 32 output channels of the tap, for the paired N = 128 instructions one of the two stacked tap tiles (rank 0:
-// W(2,kx), rank 1: W(0,kx)); 60 KiB per CTA instead of 72.
+// Why: with 64 output channels an instruction is short and bound by the operand reads from shared memory (an
+// M = 128 x N = 64 x K = 16 step reads 4 KiB of pixels for 32 cycles of tensor work).  A pair instruction lets each CTA
+// hold only its share of the B operand: for the N = 64 instructions its 32 output channels of the tap, for the paired
+// N = 128 instructions one of the two stacked tap tiles (rank 0: W(2,kx), rank 1: W(0,kx)); 60 KiB per CTA instead of
+// 72, which is what makes room for the ring of input blocks below, and half the B bytes per instruction.  The issuing
+// thread's cost per instruction is the same as in the one-CTA form (half as many threads issue half as many each).
 //
 // Synchronisation inside the pair (every wait bounded, as everywhere):
 //   bfull[k]   in the leader: announces the bytes of BOTH CTAs' loads of a block of two image rows; both report there;

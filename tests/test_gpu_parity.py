@@ -120,6 +120,16 @@ def test_conv_many_strips_per_cta(h, w, n, tenants, conv_path):
     run_and_check(wl.models, wl.model_ids, wl.inputs)
 
 
+@pytest.mark.parametrize("h,w,n,tenants", [(1, 62, 9, 2), (2, 31, 11, 3), (57, 56, 37, 3), (3, 33, 300, 2), (112, 40, 24, 2)])
+def test_conv_row_block_ring_edges(h, w, n, tenants, conv_path):
+    # padded rows of 64 pixels (the CTA-pair executor's geometry; the one-CTA path runs the same cases): images of one
+    # and of an odd number of rows (a last block that is all padding), the widest and the narrowest image of that
+    # geometry, tenants with an odd number of images, and CTAs that walk through far more than eight two-row blocks
+    # (the shared-memory ring wraps several times, within an image and across images and tenants)
+    wl = synth.make_workload(4, n=n, n_tenants=tenants, h=h, w=w, n_conv=2)
+    run_and_check(wl.models, wl.model_ids, wl.inputs)
+
+
 def test_pool_followed_by_head_both_ways(monkeypatch):
     # a global average pool followed by a narrow last dense layer runs as one small launch; MT_POOL_HEAD=0 (and any
     # head wider than 64) takes the pool_finalize + grouped dense path instead: both against the oracle
