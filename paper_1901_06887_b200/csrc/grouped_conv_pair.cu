@@ -99,7 +99,7 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     int* s_first = reinterpret_cast<int*>(bar_ptr + 320);             // the first unit's tenant: id, units, requests
     const uint16_t** s_first_w = reinterpret_cast<const uint16_t**>(bar_ptr + 352);   // ... and its weight block
 
-    pdl_launch_dependents();
+    if (!p.late_trigger) pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();          // 0 = leader (issues the MMAs), 1 = peer
     const bool is_leader = (rank == 0);
@@ -127,7 +127,10 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    pdl_wait();   // everything above overlapped the previous kernel's tail; its results are needed from here on
+    // Everything above overlapped the previous kernel's tail; its results are needed from here on.  Behind another conv
+    // layer of the same call (early_lookup) the wait comes a little later: the bucketing results read next are older
+    // than that layer's own dependency, which it let pass before it allowed this launch to start.
+    if (!p.early_lookup) pdl_wait();
     // contiguous range of pair-strips for this cluster: unit = (tenant, pair of images, strip of 2 tiles)
     const int total = p.tile_prefix[p.T];
     const int n_pairs = gridDim.x >> 1, pair_id = blockIdx.x >> 1;
@@ -151,6 +154,16 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
         }
     }
     __syncthreads();
+    if (p.early_lookup) {
+        // the first weights (unchanged since registration) are on their way while the previous layer drains: at the
+        // start of a launch they are what the first MMA waits for longest
+        if (threadIdx.x == 0 && s_begin < s_end) {
+            mbar_expect_tx(wfull_bar, kConvPairWeightBytes);
+            bulk_load(w_smem, *s_first_w + kConvPairImageOffset + (size_t)rank * (kConvPairWeightBytes / 2), kConvPairWeightBytes, wfull_bar);
+        }
+        pdl_wait();
+    }
+    if (p.late_trigger) pdl_launch_dependents();
 
     // pair-strip -> (tenant, this CTA's image, first row); units of one tenant are consecutive: its range is cached
     int cur_t = -1, cur_lo = 0, cur_hi = 0, cur_seg = 0, cur_n = 0;
@@ -208,7 +221,10 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                 // the very first weights go out before the first blocks: the first MMA needs both, and this is the
                 // larger copy (later ones must wait for the issuer to let go of the old weights, so the blocks go first)
                 const bool weights_first = new_tenant && w_loads == 0;
-                if (weights_first && !start_weights(c.t, *s_first_w)) break;
+                if (weights_first) {
+                    if (p.early_lookup) w_tenant = c.t;                      // requested before the dependency wait
+                    else if (!start_weights(c.t, *s_first_w)) break;
+                }
                 // published to this CTA's epilogue with the strip's first block (the issuer starts the strip's first
                 // tile only after that block has landed)
                 s_rec[(s - s_begin) & (kCpRecords - 1)] =

@@ -544,6 +544,8 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             a.out = (uint16_t*)g.act[l + 1];
             const bool feeds_pool = (l + 1 < L) && g.family[l + 1].kind == MT_GLOBAL_AVG_POOL;
             a.pool_partial = feeds_pool ? g.d_pool_partial : nullptr;
+            a.late_trigger = (conv_pair && l + 1 < L && g.family[l + 1].kind == MT_CONV3X3) ? 1 : 0;
+            a.early_lookup = (conv_pair && l > 0 && g.family[l - 1].kind == MT_CONV3X3) ? 1 : 0;
             a.H = f.h; a.W = f.w;
             a.Wp = g.conv.Wp; a.R = g.conv.R; a.tiles_per_strip = g.conv.tiles_per_strip;
             a.stage_bytes = g.conv.stage_bytes; a.n_stages = g.conv.n_stages;

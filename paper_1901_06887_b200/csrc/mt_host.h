@@ -145,6 +145,11 @@ struct ConvArgs {
     float* pool_partial;          // non-null: the layer feeds a global average pool; [n][strips_per_image][64] sums
     int H, W;
     int Wp, R, tiles_per_strip, stage_bytes, n_stages, strips_per_image, box_bytes;
+    // CTA-pair executor, consecutive conv layers of one call (programmatic dependent launch).  late_trigger: let the next
+    // launch start only after this one's dependency wait has returned, so that everything older than this launch's
+    // predecessor is complete when the next one starts.  early_lookup (only behind a launch with late_trigger, which is
+    // not the bucketing itself): read the bucketing results and request the first weights BEFORE the dependency wait.
+    int late_trigger = 0, early_lookup = 0;
     int32_t* status;
 };
 cudaError_t configure_grouped_conv();
