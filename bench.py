@@ -1,18 +1,29 @@
 #!/usr/bin/env python
 """Benchmark of the mixed-tenant inference hot path.
 
-One "step" = one mt_infer call: bucketing, one grouped launch per layer (the last one returns the rows to arrival order), over one synthetic
-mixed batch.  Default workload: 64 tenants x MLP 1024-4096-4096-1024, 4096 requests, Zipf(1.1).
+One "step" = one mt_infer call: bucketing, one grouped launch per layer (the last one returns the rows to arrival
+order), over one synthetic mixed batch.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
 
-With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank hosts all tenants and runs its
-own batch (requests of different batches are independent; no collective on the data path): weak scaling.
+Without --config the headline (`value`, `roofline`, `e2e`, ...) is workload 2 (64 tenants x MLP 1024-4096-4096-1024,
+4096 requests, Zipf 1.1) and `per_config` carries the same measurements for all five workloads.  With --config C only
+that workload runs.
+
+Timing: after W warm-up steps, EXACTLY K steps between two CUDA events on the launching stream (a synchronisation and,
+with several ranks, a barrier on both sides): that block gives `value` and `ms_per_step`.  A block of K steps may last
+only milliseconds, in which the GPU neither reaches its power cap nor gives the clock sampler a sample; so (one rank
+only) the same block is repeated until about two seconds of device time have passed, and `sustained` reports the
+per-step time of the blocks (min / median / max / first / last) with the SM clock sampled during each.
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank hosts all tenants and runs its own batch
+(requests of different batches are independent; no collective on the data path): weak scaling.
 Prints ONE JSON line on rank 0.
 """
 from __future__ import annotations
 
 import argparse
+import datetime
 import json
 import os
 import subprocess
@@ -31,14 +42,24 @@ from paper_1901_06887_b200 import synth  # noqa: E402
 METRIC = "mixed-tenant requests/sec"
 UNIT = "requests/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-DEFAULT_STEPS = {1: 20000, 2: 1500, 3: 2500, 4: 1500, 5: 50}
-ORACLE_SAMPLE = {1: 64, 2: 2048, 3: 16384, 4: 24, 5: 96}      # requests of the batch the CPU baseline times
+HEADLINE_CONFIG = 2
+DEFAULT_STEPS = {1: 2000, 2: 200, 3: 400, 4: 400, 5: 20}
+SUSTAIN_MS = 2000.0          # repeat the timed block until this much device time has passed ...
+MAX_BLOCKS = 400             # ... or this many blocks
 N_INPUT_BUFFERS = 3
-# DRAM traffic of the dominant kernel from the ncu captures summarised under profiles/ (see there):
-#   config 2: measured on a reduced case, traffic / algorithmic bytes = 0.995, scaled to the full launch;
-#   config 4: measured at full size, bytes per step (four conv launches).  None = not captured.
-TRAFFIC_RATIO = {2: 0.995}
-TRAFFIC_BYTES = {4: 608.5e6}
+# Requests of the batch the reference arm (--impl reference) times per step.
+REFERENCE_SAMPLE = {1: 64, 2: 512, 3: 4096, 4: 6, 5: 24}
+# DRAM traffic of the dominant kernel, from the ncu captures summarised under profiles/.  "ratio": traffic over
+# algorithmic bytes measured on a reduced case of the same kernel, scaled to the full launch (traffic grows with the
+# weights of the tenants that have requests, as the algorithmic bytes do); "bytes": measured at full size, per step.
+# An entry is deleted when its kernel changes and comes back with the next capture.
+TRAFFIC = {
+    2: {"ratio": 0.995, "source": "profiles/grouped_gemm_c2_reduced_ncu_full.md (16 tenants, 1024 requests: 841.5 MB "
+                                  "measured / 845.8 MB algorithmic), scaled by algorithmic bytes"},
+    3: {"ratio": 1.02, "source": "profiles/grouped_gemm128_c3_reduced_ncu_full.md (250 tenants, 4096 requests), scaled "
+                                 "by algorithmic bytes"},
+    4: {"bytes": 608.5e6, "source": "profiles/grouped_conv3x3_pair_c4_full_ncu_full.md (full size, four conv launches)"},
+}
 
 
 def load_peaks():
@@ -78,126 +99,164 @@ def result_line(metric_units: float, ms_total: float, n_steps: int, **extra):
     return d
 
 
+def gpu_selector(local_rank: int) -> str:
+    """What `nvidia-smi -i` needs to find THIS process's GPU: its UUID (nvidia-smi counts physical devices and knows
+    nothing of CUDA_VISIBLE_DEVICES, so the CUDA index would name another GPU on a shared host)."""
+    try:
+        import torch
+        u = str(torch.cuda.get_device_properties(local_rank).uuid)
+        return u if u.startswith("GPU-") else "GPU-" + u
+    except Exception:
+        return str(local_rank)
+
+
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons sampled while the timed region runs (read-only queries)."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    """nvidia-smi clocks and throttle reasons sampled while the timed region runs (read-only queries), with time
+    stamps so that samples can be assigned to the timed blocks."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    REASONS = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
-    def __init__(self, gpu_index: int):
-        self.gpu = gpu_index
+    def __init__(self, selector: str, period_ms: int = 20):
+        self.selector = selector
+        self.period_ms = period_ms
         self.proc = None
         self.path = None
+        self.samples = []          # (unix time, sm MHz, max MHz, watts, [reasons])
 
     def start(self):
         try:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
-                 "-lms", "50"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+                ["nvidia-smi", "-i", self.selector, "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", str(self.period_ms)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
-            return out
+            return
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         try:
             for line in open(self.path):
                 parts = [p.strip() for p in line.split(",")]
-                if len(parts) < 7:
+                if len(parts) < 8:
                     continue
                 try:
-                    sm.append(float(parts[0])); mx.append(float(parts[1]))
+                    ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    sm, mx = float(parts[1]), float(parts[2])
+                    watts = float(parts[3])
                 except ValueError:
                     continue
-                for nm, v in zip(names, parts[3:7]):
-                    if v.lower().startswith("active"):
-                        reasons.add(nm)
+                reasons = [nm for nm, v in zip(self.REASONS, parts[4:8]) if v.lower().startswith("active")]
+                self.samples.append((ts, sm, mx, watts, reasons))
             os.unlink(self.path)
         except Exception:
             pass
-        if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        self.proc = None
+
+    def summary(self, t0=None, t1=None):
+        """Median SM clock, maximum, reasons seen and sample count over [t0, t1] (all samples by default)."""
+        sel = [s for s in self.samples if (t0 is None or s[0] >= t0) and (t1 is None or s[0] <= t1)]
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": len(sel)}
+        if sel:
+            out.update(sm_mhz=float(np.median([s[1] for s in sel])), sm_max_mhz=float(max(s[2] for s in sel)),
+                       power_w=float(np.median([s[3] for s in sel])),
+                       reasons=sorted({r for s in sel for r in s[4]}))
         return out
 
 
-def gemm_roofline(wl, kernel_ms_per_launch_sum, peaks, peaks_kind, config):
+def dominant_roofline(wl, kernel_ms_per_step, peaks, peaks_kind, config, long_run):
     """Roofline of the dominant kernel (the grouped layer executor), all its launches of one step together:
-    algorithmic bytes (weights + bias of tenants with requests once, activations in, activations out) and
-    flops of those layers, against the measured HBM and bf16 peaks; the larger time bounds it."""
+    algorithmic bytes (weights + bias of tenants with requests once, activations in, activations out) and flops of
+    those layers, against the measured HBM and bf16 peaks; the larger time bounds it.  A tensor-bound kernel is held
+    against the burst cuBLAS figure when its timed region was short and against the sustained one when the region
+    lasted long enough for the power cap to act (long_run); the fraction of the other peak is given beside it."""
     per_layer_bytes = synth.workload_bytes(wl.models, wl.model_ids, per_layer=True)
     kinds = [l.kind for l in wl.models[0]]
     dom_kind = synth.CONV3X3 if synth.CONV3X3 in kinds else synth.DENSE
     counts = np.bincount(wl.model_ids, minlength=len(wl.models))
     byts = sum(b for b, k in zip(per_layer_bytes, kinds) if k == dom_kind)
     flops = sum(int(c) * sum(synth.layer_flops(l) for l in m if l.kind == dom_kind) for c, m in zip(counts, wl.models))
-    # tensor peak: the kernel is timed inside a seconds-long loop (power cap active), so the sustained cuBLAS
-    # figure is the matching denominator; the burst figure is reported beside it
-    tc_peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+    burst = peaks["bf16_tflops"]
+    sustained = peaks.get("bf16_tflops_sustained", burst)
     t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
-    t_tc = flops / (tc_peak * 1e12)
-    sec = kernel_ms_per_launch_sum * 1e-3
+    t_tc = flops / (burst * 1e12)
+    sec = kernel_ms_per_step * 1e-3
     if t_hbm >= t_tc:
         ach = byts / sec / 1e9 if sec > 0 else 0.0
         roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"]}
     else:
         ach = flops / sec / 1e12 if sec > 0 else 0.0
+        tc_peak = sustained if long_run else burst
         roof = {"bound": "tensor", "achieved": ach, "peak": tc_peak, "unit": "TFLOP/s", "frac": ach / tc_peak,
-                "peak_kind": "sustained (kernel timed inside a long loop)", "burst_peak": peaks["bf16_tflops"],
-                "frac_of_burst_peak": ach / peaks["bf16_tflops"]}
-    traffic = None
-    if config in TRAFFIC_RATIO:
-        traffic = int(TRAFFIC_RATIO[config] * byts)
-    elif config in TRAFFIC_BYTES:
-        traffic = int(TRAFFIC_BYTES[config])
-    roof.update(traffic=traffic, peak_source="of " + peaks_kind, kernel="grouped_conv3x3" if dom_kind == synth.CONV3X3 else "grouped_gemm",
-                algorithmic_bytes_per_step=int(byts), flops_per_step=int(flops), kernel_ms_per_step=kernel_ms_per_launch_sum)
+                "peak_kind": "sustained (timed inside a seconds-long loop)" if long_run else "burst (timed region under a second)",
+                "frac_of_burst_peak": ach / burst, "frac_of_sustained_peak": ach / sustained}
+    traffic, source = None, None
+    t = TRAFFIC.get(config)
+    if t is not None:
+        traffic = int(t["ratio"] * byts) if "ratio" in t else int(t["bytes"])
+        source = t["source"]
+    roof.update(traffic=traffic, traffic_source=source, peak_source="of " + peaks_kind,
+                algorithmic_bytes_per_step=int(byts), flops_per_step=int(flops), kernel_ms_per_step=kernel_ms_per_step)
     return roof
 
 
-def time_oracle(wl, config, n_sample=None, repeats=1):
+def oracle_sample(wl, config):
+    """Requests the CPU baseline times: the whole batch for workloads 1-4; for workload 5 the first 128 requests of
+    every tenant (at least 1024 in all), whose time is extrapolated linearly since every request of a tenant costs the same."""
+    if config != 5:
+        return np.arange(wl.n), "the whole batch of %d requests" % wl.n
+    pick = []
+    for t in range(len(wl.models)):
+        pick.append(np.flatnonzero(wl.model_ids == t)[:128])
+    idx = np.sort(np.concatenate(pick))
+    return idx, "%d of %d requests (the first 128 of every tenant); extrapolated from %d requests" % (len(idx), wl.n, len(idx))
+
+
+def time_oracle(wl, config, repeats=3):
     import oracle
     oracle.build()
-    n_s = min(wl.n, n_sample or ORACLE_SAMPLE[config])
-    ids, x = wl.model_ids[:n_s], wl.inputs[:n_s]
+    idx, what = oracle_sample(wl, config)
+    ids, x = wl.model_ids[idx], wl.inputs[idx]
     best = None
     for _ in range(repeats):
         t0 = time.perf_counter()
         oracle.forward(wl.models, ids, x)
         dt = time.perf_counter() - t0
         best = dt if best is None else min(best, dt)
-    return {"value": n_s / best, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
-            "sample": "first %d of %d requests of the batch, all tenants resident, wall clock %.2f s" % (n_s, wl.n, best)}
+    flops = synth.workload_flops(wl.models, ids)
+    return {"value": len(idx) / best, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
+            "gflops": flops / best / 1e9,
+            "sample": "%s, all tenants resident, best of %d, wall clock %.2f s" % (what, repeats, best)}
 
 
 def run_reference(args, rank, world):
     """The reference arm: the fp64 CPU oracle as it stands, on the host cores, rank 0 only."""
     if rank != 0:
         return
-    wl = synth.make_workload(args.config)
-    n_s = min(wl.n, max(1, ORACLE_SAMPLE[args.config] // 4))
+    cfg = args.config or HEADLINE_CONFIG
+    wl = synth.make_workload(cfg)
+    n_s = min(wl.n, REFERENCE_SAMPLE[cfg])
     import oracle
     oracle.build()
     ids, x = wl.model_ids[:n_s], wl.inputs[:n_s]
     for _ in range(min(args.warmup, 1)):
         oracle.forward(wl.models, ids, x)
-    steps = min(args.steps, 8)
+    steps = min(args.steps or 8, 8)
     t0 = time.perf_counter()
     for _ in range(steps):
         oracle.forward(wl.models, ids, x)
     ms = (time.perf_counter() - t0) * 1e3
     line = result_line(n_s * steps, ms, steps, n_gpus=args.gpus, steps=steps, warmup=min(args.warmup, 1), scaling="weak",
                        vs_baseline=None, dtype="f64", data="synthetic", impl="reference",
-                       config={"workload": synth.CONFIG_NAMES[args.config],
+                       config={"workload": synth.CONFIG_NAMES[cfg],
                                "sample": "each step = first %d of %d requests" % (n_s, wl.n)})
     line["cpu_baseline"] = {"value": line["value"], "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
                             "sample": "first %d of %d requests per step, %d steps" % (n_s, wl.n, steps)}
@@ -205,40 +264,17 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=None)
-    ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--e2e-steps", type=int, default=None)
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--tenants", type=int, default=None, help="reduced case: number of tenants (profiling captures)")
-    ap.add_argument("--requests", type=int, default=None, help="reduced case: requests per batch")
-    ap.add_argument("--profile", action="store_true", help="timed loop only (no e2e, CPU baseline or clock sampler)")
-    args = ap.parse_args()
-    if args.steps is None:
-        args.steps = DEFAULT_STEPS[args.config]
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+def median(xs):
+    return float(np.median(xs)) if len(xs) else None
 
-    rank, world, local_rank = env_int("RANK", 0), env_int("WORLD_SIZE", 1), env_int("LOCAL_RANK", 0)
-    if args.impl == "reference":
-        run_reference(args, rank, world)
-        return
 
-    import torch
-    import torch.distributed as dist
-    from paper_1901_06887_b200 import binding as mt, harness
+def measure_config(cfg, args, ctx):
+    """Everything the bench reports for one workload, as a dict in the layout of the JSON line."""
+    torch, dist, mt, harness = ctx["torch"], ctx["dist"], ctx["mt"], ctx["harness"]
+    rank, world, local_rank = ctx["rank"], ctx["world"], ctx["local_rank"]
+    peaks, peaks_kind = ctx["peaks"], ctx["peaks_kind"]
+    steps = args.steps if args.steps is not None else DEFAULT_STEPS[cfg]
 
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the CUDA library is the only implementation")
-    torch.cuda.set_device(local_rank)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-
-    cfg = args.config
     over = {"n_tenants": args.tenants} if args.tenants else {}
     models = synth.make_models(cfg, **over)
     batches = [synth.make_requests(cfg, models, n=args.requests, salt=1000 * rank + b) for b in range(N_INPUT_BUFFERS)]
@@ -264,52 +300,72 @@ def main():
     if st != (0, -1):
         raise SystemExit("device status after warm-up: %r" % (st,))
 
-    # ---- timed region: device-resident inputs, CUDA events on the launching stream, per-kernel events inside
-    sampler = ClockSampler(local_rank)
+    # ---- timed region: device-resident inputs, CUDA events on the launching stream, executor events inside
+    sampler = ClockSampler(gpu_selector(local_rank))
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    mt.mt_set_kernel_timing(3)          # events around the layer executors (the dominant kernel) on every 4th step
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
     if not args.profile:
         sampler.start()
-    launches_before = mt.mt_debug_launch_count()
-    e0.record(stream)
-    for i in range(args.steps):
-        step(i)
-    mt.mt_set_kernel_timing(0)          # closes the last group of executor launches: its stop event goes in here
-    e1.record(stream)
-    torch.cuda.synchronize()
-    launches = mt.mt_debug_launch_count() - launches_before      # kernels the library enqueued in the timed region
-    if world > 1:
-        dist.barrier()
-    clocks = sampler.stop()
-    local_ms = e0.elapsed_time(e1)
-    kernel_times = mt.mt_get_kernel_times()
+        time.sleep(0.05)
+    blocks = []                         # (ms, executor kernel times, wall start, wall end)
+    launches = 0
+    total_ms = 0.0
+    max_blocks = 1 if (world > 1 or args.profile) else MAX_BLOCKS
+    for b in range(max_blocks):
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        mt.mt_set_kernel_timing(3)      # events around the layer executors (the dominant kernel) on every 4th step
+        w0 = time.time()
+        before = mt.mt_debug_launch_count()
+        e0.record(stream)
+        for i in range(steps):
+            step(i)
+        mt.mt_set_kernel_timing(0)      # closes the last group of executor launches: its stop event goes in here
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        w1 = time.time()
+        if b == 0:
+            launches = mt.mt_debug_launch_count() - before      # kernels the library enqueued in the timed region
+        ms = e0.elapsed_time(e1)
+        blocks.append((ms, mt.mt_get_kernel_times(), w0, w1))
+        total_ms += ms
+        if total_ms >= SUSTAIN_MS:
+            break
+    sampler.stop()
+    local_ms = blocks[0][0]
+
     # per-kernel breakdown of every launch of the path: a short separate pass (its events perturb small batches)
     mt.mt_set_kernel_timing(1)
-    bd_steps = max(3, min(args.steps, 50))
+    bd_steps = max(3, min(steps, 50))
     for i in range(bd_steps):
         step(i)
     torch.cuda.synchronize()
     mt.mt_set_kernel_timing(0)
     breakdown = mt.mt_get_kernel_times()
-    units, ms = aggregate(n * args.steps, local_ms, world)
+    units, ms = aggregate(n * steps, local_ms, world)
 
     if args.profile:
-        if rank == 0:
-            print(json.dumps({"profile_run": True, "ms_per_step": ms / args.steps,
-                              "kernels": {nm: t / max(c, 1) for nm, t, c in breakdown}}), flush=True)
         mt.mt_shutdown()
-        if world > 1:
-            dist.destroy_process_group()
-        return
+        return {"profile_run": True, "ms_per_step": ms / steps, "kernels": {nm: t / max(c, 1) for nm, t, c in breakdown}}
+
+    # launch floor: a chain of empty kernels launched like the kernels of the path
+    floor_us = None
+    if world == 1:
+        mt.mt_debug_empty_launches(200, stream)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        mt.mt_debug_empty_launches(2000, stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        floor_us = e0.elapsed_time(e1) / 2000 * 1e3
 
     # ---- end to end: host buffers in, host buffers out, through the public entry points.  Every step copies its
     # inputs and ids from pinned host memory and its outputs back.  Primary figure: mt_infer_host_async on two
     # alternating streams (a batch's copies overlap its neighbours' kernels); beside it the synchronous
     # mt_infer_host, which returns only when the outputs have landed.
-    e2e_steps = args.e2e_steps or max(4, min(args.steps, 50))
+    e2e_steps = args.e2e_steps or max(4, min(steps, 50))
     h_in = [torch.from_numpy(x.view(np.int16)).pin_memory() for _, x in batches]
     h_ids = [torch.from_numpy(i).pin_memory() for i, _ in batches]
     h_outs = [torch.empty((n, out_elems), dtype=torch.float32).pin_memory() for _ in range(2)]
@@ -346,48 +402,145 @@ def main():
     st = mt.mt_get_async_status()
     if st != (0, -1):
         raise SystemExit("device status after the timed region: %r" % (st,))
-
-    if rank == 0:
-        peaks, peaks_kind = load_peaks()
-        per_kernel = {name: {"ms_per_step": t / bd_steps, "launches_per_step": c / bd_steps} for name, t, c in breakdown}
-        # per step = per-launch average x launches per step (the executors are timed on every fourth step)
-        lps = {nm: c / bd_steps for nm, t, c in breakdown}
-        timed = dict((nm, t / max(c, 1) * lps.get(nm, 1.0)) for nm, t, c in kernel_times)
-        dom = "grouped_conv3x3" if cfg == 4 else ("fused_mlp" if "fused_mlp" in timed else "grouped_gemm")
-        dom_ms = timed.get(dom, 0.0)
-        roof = gemm_roofline(wl, dom_ms, peaks, peaks_kind, cfg)
-        roof["kernel"] = dom
-        roof["kernel_timing"] = "CUDA events around each run of the executor's launches, every 4th step of the timed region"
-        flops = synth.workload_flops(wl.models, wl.model_ids)
-        bytes_all = synth.workload_bytes(wl.models, wl.model_ids)
-        t_roof = max(flops / (peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12),
-                     bytes_all / (peaks["hbm_gbs"] * 1e9))
-        line = result_line(units, ms, args.steps, n_gpus=world, steps=args.steps, warmup=args.warmup, scaling="weak",
-                           vs_baseline=None, dtype="bf16", data="synthetic")
-        line["config"] = {"workload": synth.CONFIG_NAMES[cfg], "requests_per_step_per_gpu": n, "tenants": len(models),
-                          "reduced": bool(args.tenants or args.requests),
-                          "l2": "weights streamed per step exceed the 126 MB L2 only for c2/c3/c5; inputs rotate over "
-                                "%d device buffers" % N_INPUT_BUFFERS,
-                          "parallelism": "replicas x%d (each GPU hosts all tenants, own batch)" % world}
-        line["tflops"] = flops * args.steps * world / (ms * 1e-3) / 1e12
-        line["whole_pass_roofline"] = {"roofline_ms": t_roof * 1e3, "measured_ms": line["ms_per_step"],
-                                       "frac": t_roof * 1e3 / line["ms_per_step"], "peaks": "of " + peaks_kind,
-                                       "flops_per_step": int(flops), "algorithmic_bytes_per_step": int(bytes_all)}
-        line["roofline"] = roof
-        line["kernels"] = per_kernel
-        line["gpu_launches"] = int(launches)
-        line["e2e"] = dict(result_line(e2e_units, e2e_ms, e2e_steps), steps=e2e_steps,
-                           h2d_bytes_per_step=int(n * wl.in_elems * 2 + n * 4), d2h_bytes_per_step=int(n * out_elems * 4))
-        line["e2e"]["call"] = "mt_infer_host_async, two streams in turn"
-        line["e2e"]["synchronous_call"] = {"value": sync_units / (sync_ms * 1e-3), "unit": UNIT, "ms_per_step": sync_ms / e2e_steps,
-                                           "call": "mt_infer_host"}
-        for k in ("metric", "higher_is_better"):
-            line["e2e"].pop(k, None)
-        line["clocks"] = clocks
-        if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = time_oracle(wl, cfg)
-        print(json.dumps(line), flush=True)
     mt.mt_shutdown()
+    del dev_in, dev_ids, dev_out, h_in, h_ids, h_outs
+    torch.cuda.empty_cache()
+    if rank != 0:
+        return None
+
+    per_kernel = {name: {"ms_per_step": t / bd_steps, "launches_per_step": c / bd_steps} for name, t, c in breakdown}
+    lps = {nm: c / bd_steps for nm, t, c in breakdown}
+    dom = "grouped_conv3x3" if cfg == 4 else ("fused_mlp" if "fused_mlp" in lps else "grouped_gemm")
+
+    def dom_ms(kernel_times):
+        # per step = per-launch average x launches per step (the executors are timed on every fourth step)
+        for nm, t, c in kernel_times:
+            if nm == dom:
+                return t / max(c, 1) * lps.get(nm, 1.0)
+        return 0.0
+
+    block_ms = [b[0] / steps for b in blocks]
+    block_clk = [sampler.summary(b[2], b[3]) for b in blocks]
+    block_dom = [dom_ms(b[1]) for b in blocks]
+    long_first = blocks[0][0] >= 1000.0
+    roof = dominant_roofline(wl, block_dom[0], peaks, peaks_kind, cfg, long_first)
+    roof["kernel"] = dom
+    roof["kernel_timing"] = "CUDA events around each run of the executor's launches, every 4th step of the timed region"
+    line = result_line(units, ms, steps, n_gpus=world, steps=steps, warmup=args.warmup, scaling="weak",
+                       vs_baseline=None, dtype="bf16", data="synthetic")
+    line["config"] = {"workload": synth.CONFIG_NAMES[cfg], "requests_per_step_per_gpu": n, "tenants": len(models),
+                      "reduced": bool(args.tenants or args.requests),
+                      "l2": "weights streamed per step exceed the 126 MB L2 only for c2/c3/c5; inputs rotate over "
+                            "%d device buffers" % N_INPUT_BUFFERS,
+                      "parallelism": "replicas x%d (each GPU hosts all tenants, own batch)" % world}
+    flops = synth.workload_flops(wl.models, wl.model_ids)
+    bytes_all = synth.workload_bytes(wl.models, wl.model_ids)
+    line["tflops"] = flops * steps * world / (ms * 1e-3) / 1e12
+
+    def whole_pass(ms_per_step, long_run):
+        tc = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) if long_run else peaks["bf16_tflops"]
+        t_roof = max(flops / (tc * 1e12), bytes_all / (peaks["hbm_gbs"] * 1e9))
+        return {"roofline_ms": t_roof * 1e3, "measured_ms": ms_per_step, "frac": t_roof * 1e3 / ms_per_step,
+                "peaks": "of " + peaks_kind + (", tensor peak sustained" if long_run else ", tensor peak burst"),
+                "flops_per_step": int(flops), "algorithmic_bytes_per_step": int(bytes_all)}
+
+    line["whole_pass_roofline"] = whole_pass(line["ms_per_step"], long_first)
+    line["roofline"] = roof
+    if len(blocks) > 1 or blocks[0][0] >= SUSTAIN_MS:
+        # the later half of the blocks: the GPU has been busy for at least a second by then
+        tail = list(range(len(blocks) // 2, len(blocks)))
+        tail_ms = median([block_ms[i] for i in tail])
+        tail_dom = median([block_dom[i] for i in tail])
+        tail_clk = sampler.summary(blocks[tail[0]][2], blocks[tail[-1]][3])
+        first_clk = block_clk[0]
+        sus = {"blocks": len(blocks), "steps_per_block": steps, "device_seconds": total_ms * 1e-3,
+               "ms_per_step": {"min": min(block_ms), "median": median(block_ms), "max": max(block_ms),
+                               "first": block_ms[0], "last": block_ms[-1], "later_half_median": tail_ms},
+               "value_later_half": n * world / (tail_ms * 1e-3),
+               "sm_mhz": {"first_block": first_clk["sm_mhz"], "later_half": tail_clk["sm_mhz"]},
+               "ms_x_mhz": {"first_block": (block_ms[0] * first_clk["sm_mhz"]) if first_clk["sm_mhz"] else None,
+                            "later_half": (tail_ms * tail_clk["sm_mhz"]) if tail_clk["sm_mhz"] else None},
+               "reasons_later_half": tail_clk["reasons"],
+               "roofline_later_half": dominant_roofline(wl, tail_dom, peaks, peaks_kind, cfg, True),
+               "whole_pass_roofline_later_half": whole_pass(tail_ms, True)}
+        for k in ("traffic", "traffic_source", "algorithmic_bytes_per_step", "flops_per_step"):
+            sus["roofline_later_half"].pop(k, None)
+        line["sustained"] = sus
+    line["kernels"] = per_kernel
+    line["gpu_launches"] = int(launches)
+    if floor_us is not None:
+        line["launch_floor_us"] = floor_us
+        line["launch_floor"] = ("one link of a chain of 2000 empty kernels launched like the kernels of the path "
+                                "(programmatic dependent launch); this step has %d launches" % round(launches / steps))
+    line["e2e"] = dict(result_line(e2e_units, e2e_ms, e2e_steps), steps=e2e_steps,
+                       h2d_bytes_per_step=int(n * wl.in_elems * 2 + n * 4), d2h_bytes_per_step=int(n * out_elems * 4))
+    line["e2e"]["call"] = "mt_infer_host_async, two streams in turn"
+    line["e2e"]["synchronous_call"] = {"value": sync_units / (sync_ms * 1e-3), "unit": UNIT, "ms_per_step": sync_ms / e2e_steps,
+                                       "call": "mt_infer_host"}
+    for k in ("metric", "higher_is_better"):
+        line["e2e"].pop(k, None)
+    clocks = sampler.summary()
+    clocks["timed_block"] = block_clk[0]
+    clocks["period_ms"] = sampler.period_ms
+    line["clocks"] = clocks
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = time_oracle(wl, cfg)
+    return line
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=None, choices=[1, 2, 3, 4, 5],
+                    help="only this workload (default: workload 2 as the headline and all five under per_config)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true", help="headline workload only")
+    ap.add_argument("--tenants", type=int, default=None, help="reduced case: number of tenants (profiling captures)")
+    ap.add_argument("--requests", type=int, default=None, help="reduced case: requests per batch")
+    ap.add_argument("--profile", action="store_true", help="timed loop only (no e2e, CPU baseline or clock sampler)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank, world, local_rank = env_int("RANK", 0), env_int("WORLD_SIZE", 1), env_int("LOCAL_RANK", 0)
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_1901_06887_b200 import binding as mt, harness
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library is the only implementation")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    peaks, peaks_kind = load_peaks()
+    ctx = dict(torch=torch, dist=dist, mt=mt, harness=harness, rank=rank, world=world, local_rank=local_rank,
+               peaks=peaks, peaks_kind=peaks_kind)
+
+    head_cfg = args.config or HEADLINE_CONFIG
+    line = measure_config(head_cfg, args, ctx)
+    reduced = bool(args.tenants or args.requests or args.profile)
+    if args.config is None and world == 1 and not reduced and not args.no_per_config and line is not None:
+        # the same measurements for all five workloads; --steps applies to the headline only
+        per = {"c%d" % head_cfg: {k: v for k, v in line.items() if k not in ("metric", "unit", "higher_is_better", "n_gpus",
+                                                                              "scaling", "vs_baseline", "data")}}
+        sub = argparse.Namespace(**vars(args))
+        sub.steps = None
+        sub.e2e_steps = None
+        for cfg in (1, 3, 4, 5):
+            r = measure_config(cfg, sub, ctx)
+            per["c%d" % cfg] = {k: v for k, v in r.items() if k not in ("metric", "unit", "higher_is_better", "n_gpus",
+                                                                         "scaling", "vs_baseline", "data")}
+        line["per_config"] = {k: per[k] for k in sorted(per)}
+    if rank == 0 and line is not None:
+        print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 

@@ -62,7 +62,8 @@ typedef struct {
     const void* bias;      /* fp32 [out_ch] */
 } mt_layer_desc;
 
-/* Create the context on CUDA device `device`.  max_models bounds the id space (<= 8192), max_batch is
+/* Set-up and tear-down of the worker's context (no passage of the paper: it describes the service, not a library).
+ * Create the context on CUDA device `device`.  max_models bounds the id space (<= 8192), max_batch is
  * a hint for the first workspace allocation (the workspace grows on demand, see mt_infer).  Calling
  * mt_register_model before mt_init initialises device 0 with defaults (1024 models).
  * Errors: MT_ERR_ARCH, MT_ERR_CUDA, MT_ERR_OOM, MT_ERR_INVALID_ARG (already initialised with other
@@ -111,8 +112,9 @@ mt_status mt_infer_host(const void* inputs_host, const int32_t* model_ids_host, 
 mt_status mt_infer_host_async(const void* inputs_host, const int32_t* model_ids_host, int32_t n,
                               void* outputs_host, void* stream);
 
-/* Mark the id dead and free its weights.  Synchronises the device first, so it cannot race an
- * mt_infer in flight.  The id may be re-issued by a later mt_register_model. */
+/* A tenant withdraws its model (Sec. 3: tenants upload models to the service and may remove them again; the paper
+ * names no call for it).  Marks the id dead and frees its weights.  Synchronises the device first, so it cannot race
+ * an mt_infer in flight.  The id may be re-issued by a later mt_register_model. */
 mt_status mt_release(int32_t model_id);
 
 /* Synchronise `stream`, then report and clear the sticky device-side status of the calls so far:
@@ -139,6 +141,20 @@ mt_status mt_debug_wait_timeout(int32_t limit_ms, void* stream);
  * mt_infer_host since it was loaded (registration and the no-allocation call are not counted). */
 mt_status mt_debug_launch_count(int64_t* count_out);
 
+/* Bench hook: enqueue `count` (0..100000) kernels that do nothing, chained on `stream` by programmatic dependent
+ * launch exactly like the kernels of the path.  Timing a long chain gives the least a launch of the path can cost
+ * (the launch floor that bounds a batch as small as 64 requests); not counted by mt_debug_launch_count. */
+mt_status mt_debug_empty_launches(int32_t count, void* stream);
+
+/* Test / A-B timing hook: which executor a batch takes.  Each switch starts from the environment variable read ONCE
+ * by mt_init ("0" = off) and can be changed afterwards with this call; nothing reads the environment per batch.
+ *   "fused"      (MT_FUSED)      one launch for a small batch of narrow MLPs; off: the layer-by-layer path
+ *   "pair"       (MT_PAIR)       CTA-pair dense executor for batches with >= 1024 requests per tenant
+ *   "conv_pair"  (MT_CONV_PAIR)  CTA-pair conv executor for padded rows of 64 pixels; off: the one-CTA executor
+ *   "pool_head"  (MT_POOL_HEAD)  pool + narrow head as one launch; off: pool_finalize + a grouped dense launch
+ * Unknown name: MT_ERR_INVALID_ARG.  Results agree with the oracle on every setting. */
+mt_status mt_debug_set_option(const char* name, int32_t value);
+
 /* Per-kernel device timing.  enable = 1: every kernel launch of mt_infer is bracketed by CUDA events on the
  * caller's stream; enable = 2: only the layer executors (dense / conv / the one-launch path) are, and consecutive
  * launches of the same executor (also across calls, when a call is a single launch) share one pair of events, so
@@ -159,8 +175,11 @@ mt_status mt_get_kernel_times(const char** names, double* total_ms, int32_t* lau
  * in a process whose device memory belongs wholly to a different allocator.  mt_infer cannot serve them,
  * because its workspace is allocated (and grown) with cudaMalloc.  This call does the same stable counting
  * sort of a batch by model id, using a fixed scratch array that is part of the library image: each GPU that
- * loads the library holds about 1.03 MiB for it until the process exits.  It never calls cudaMalloc,
- * cudaFree or any allocating routine, and needs no mt_init.
+ * loads the library holds 1,057,804 bytes (1.01 MiB) for it until the process exits.  It never calls cudaMalloc,
+ * cudaFree or any allocating routine, and needs no mt_init.  One caveat: the FIRST call on each device is where the
+ * driver loads this part of the library (kernels and the scratch array itself, under lazy module loading) and where
+ * the array's address is looked up, so that one call may allocate inside the driver.  Make it at start-up, outside
+ * any allocator hook or frozen-memory phase - a call with n = 0 is enough; later calls allocate nothing.
  *
  *   model_ids   device, int32 [n]
  *   n           0 .. MT_NOALLOC_MAX_BATCH        (larger: MT_ERR_UNSUPPORTED, nothing enqueued)

@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "MT_OK", 1: "MT_ERR_INVALID_ARG", 2: "MT_ERR_BAD_MODEL_ID", 3
 
 EXPORTS = ["mt_init", "mt_shutdown", "mt_register_model", "mt_infer", "mt_infer_host", "mt_infer_host_async", "mt_release",
            "mt_get_async_status", "mt_status_string", "mt_debug_last_bucketing", "mt_set_kernel_timing",
-           "mt_get_kernel_times", "mt_bucket_noalloc", "mt_debug_wait_timeout", "mt_debug_launch_count"]
+           "mt_get_kernel_times", "mt_bucket_noalloc", "mt_debug_wait_timeout", "mt_debug_launch_count", "mt_debug_set_option", "mt_debug_empty_launches"]
 
 
 class MtError(RuntimeError):
@@ -65,6 +65,8 @@ def lib() -> ctypes.CDLL:
         l.mt_bucket_noalloc.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
         l.mt_debug_wait_timeout.argtypes = [i32, vp]
         l.mt_debug_launch_count.argtypes = [ctypes.POINTER(ctypes.c_int64)]
+        l.mt_debug_set_option.argtypes = [ctypes.c_char_p, i32]
+        l.mt_debug_empty_launches.argtypes = [i32, vp]
         for name in EXPORTS:
             if name != "mt_status_string":
                 getattr(l, name).restype = ctypes.c_int
@@ -173,6 +175,16 @@ def mt_debug_launch_count() -> int:
     c = ctypes.c_int64(0)
     _check(lib().mt_debug_launch_count(ctypes.byref(c)), "mt_debug_launch_count")
     return int(c.value)
+
+
+def mt_debug_empty_launches(count: int, stream=None) -> None:
+    """Enqueue `count` empty kernels chained like the kernels of the path (to time the launch floor)."""
+    _check(lib().mt_debug_empty_launches(int(count), _stream_handle(stream)), "mt_debug_empty_launches")
+
+
+def mt_debug_set_option(name: str, value: int) -> None:
+    """Switch an executor choice ("fused", "pair", "conv_pair", "pool_head") on or off for the calls that follow."""
+    _check(lib().mt_debug_set_option(name.encode(), int(value)), "mt_debug_set_option")
 
 
 def mt_set_kernel_timing(enable) -> None:

@@ -373,12 +373,15 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
         if (r >= rounds) break;
         const int i = r * nthr + threadIdx.x;
         const int b = bucket[r];
+        // the lanes that hold a request, agreed on by the whole warp BEFORE the divergent branch: the ranks below
+        // are only right if every such lane takes part in the match, which __activemask() would not promise
+        const unsigned live = __ballot_sync(0xffffffffu, i < n);
         for (int w = 0; w < n_warps; ++w) {
             if (warp == w && i < n) {
-                const unsigned peers = __match_any_sync(__activemask(), b);
+                const unsigned peers = __match_any_sync(live, b);
                 const int rank = __popc(peers & ((1u << lane) - 1u));
                 const int pos = s_next[b] + rank;
-                __syncwarp(__activemask());
+                __syncwarp(live);
                 if (rank == 0) s_next[b] += __popc(peers);
                 perm[pos] = i;
                 inv[i] = pos;
@@ -453,12 +456,14 @@ bucket_scatter_expand(const int32_t* __restrict__ ids, int n, int T, const Model
         const bool mine = threadIdx.x < kBucketChunk && i < n;
         const int b = mine ? classify(ids[i], T, br) : -1;
         // warps take turns in arrival order, so positions inside a bucket ascend with the arrival index
+        // (the participating lanes are agreed on before the divergent branch; see bucket_single_cta)
+        const unsigned live = __ballot_sync(0xffffffffu, mine);
         for (int w = 0; w < kBucketChunk / 32; ++w) {
             if (warp == w && mine) {
-                const unsigned peers = __match_any_sync(__activemask(), b);
+                const unsigned peers = __match_any_sync(live, b);
                 const int rank = __popc(peers & ((1u << lane) - 1u));
                 const int pos = s_next[b] + rank;
-                __syncwarp(__activemask());
+                __syncwarp(live);
                 if (rank == 0) s_next[b] += __popc(peers);
                 perm[pos] = i;
                 inv[i] = pos;
@@ -532,6 +537,18 @@ __global__ void wait_timeout_probe(int32_t* status, unsigned long long limit_ns,
 
 void launch_wait_timeout_probe(int32_t* status, unsigned long long limit_ns, int32_t* gave_up, cudaStream_t s) {
     wait_timeout_probe<<<1, 32, 0, s>>>(status, limit_ns, gave_up);
+}
+
+// A kernel that does nothing but take part in the programmatic dependent launch chain like every kernel of the path:
+// `count` of them back to back measure what one link of such a chain costs at least (the launch floor).
+__global__ void empty_chain_kernel() {
+    pdl_launch_dependents();
+    pdl_wait();
+}
+
+void launch_empty_chain(int count, cudaStream_t s) {
+    for (int i = 0; i < count; ++i) launch_pdl(empty_chain_kernel, dim3(1), dim3(32), 0, s);
+    g_kernel_launches -= (unsigned long long)count;    // not kernels of the inference path
 }
 
 // ------------------------------------------------------------------------------------------ launchers

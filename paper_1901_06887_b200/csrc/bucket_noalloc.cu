@@ -6,7 +6,10 @@
 // process whose device memory is entirely owned by another allocator, or a library called while the CUDA
 // context's allocator lock must not be taken.  mt_bucket_noalloc gives them the same stable counting sort
 // (counts, offsets, perm, inv) with the scratch held in a fixed array that is part of the library image:
-// every GPU that loads the library carries kScratchInts * 4 bytes (about 1.03 MiB) until the process exits.
+// every GPU that loads the library carries kScratchInts * 4 = 1,057,804 bytes (1.01 MiB) until the process exits.
+// The FIRST call on a device may still allocate inside the driver: with lazy module loading that call loads this
+// file's kernels and places the scratch array.  Make it once at start-up (n = 0 is enough), outside any allocator
+// hook or frozen-memory phase; every later call on that device allocates nothing.
 //
 // The kernels below are separate copies of the bucketing passes, without the model table: an id is valid iff
 // it lies in [0, n_models).
@@ -112,12 +115,15 @@ na_scatter(const int32_t* __restrict__ ids, int n, int T, const int32_t* __restr
     const int i = blockIdx.x * kChunk + threadIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = (i < n) ? bucket_of(ids[i], T) : -1;
+    // lanes that hold a request, agreed on by the whole warp before the divergent branch (the ranks are only right
+    // if every such lane takes part in the match)
+    const unsigned live = __ballot_sync(0xffffffffu, i < n);
     for (int w = 0; w < kChunk / 32; ++w) {                   // warps take turns, so the sort is stable
         if (warp == w && i < n) {
-            const unsigned peers = __match_any_sync(__activemask(), b);
+            const unsigned peers = __match_any_sync(live, b);
             const int rank = __popc(peers & ((1u << lane) - 1u));
             const int pos = s_next[b] + rank;
-            __syncwarp(__activemask());
+            __syncwarp(live);
             if (rank == 0) s_next[b] += __popc(peers);
             perm[pos] = i;
             inv[i] = pos;

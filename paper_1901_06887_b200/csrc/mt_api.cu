@@ -86,19 +86,28 @@ struct Ctx {
     void* st_in = nullptr;
     int32_t* st_ids = nullptr;
     float* st_out = nullptr;
-    int st_cap = 0;
+    size_t st_cap_in = 0, st_cap_ids = 0, st_cap_out = 0;   // bytes: a new family changes the row sizes, not only n
 
     // staging for mt_infer_host_async: two slots used in turn, so that the copies of one call overlap the compute
     // of its neighbours when the caller alternates between two streams
     void* as_in[2] = {nullptr, nullptr};
     int32_t* as_ids[2] = {nullptr, nullptr};
     float* as_out[2] = {nullptr, nullptr};
-    int as_cap = 0;
+    size_t as_cap_in = 0, as_cap_ids = 0, as_cap_out = 0;   // bytes, per slot
     int as_next = 0;
     cudaEvent_t as_slot_done[2] = {nullptr, nullptr};   // the slot's device-to-host copy has finished
     bool as_slot_used[2] = {false, false};
     cudaEvent_t as_compute_done = nullptr;               // the previous call's kernels have finished (shared workspace)
     bool as_have_compute = false;
+
+    // switches for tests and A/B timing: read from the environment once, at mt_init (MT_FUSED, MT_PAIR, MT_CONV_PAIR,
+    // MT_POOL_HEAD; "0" turns the path off), changed afterwards only through mt_debug_set_option
+    bool opt_fused = true, opt_pair = true, opt_conv_pair = true, opt_pool_head = true;
+
+    // tensor maps over the caller's images (first conv layer), kept while pointer and batch size stay the same
+    const void* in_map_ptr = nullptr;
+    int in_map_n = 0;
+    CUtensorMap in_map, in_rows2_map, in_rows1_map;
 
     // timing
     int timing = 0;                      // 0 off, 1 every kernel, 2 only the layer executors, 3 the same on every 4th call
@@ -170,6 +179,12 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     g.has_family = false;
     g.cap_n = 0;
     g.ws_dirty = true;
+    g.in_map_ptr = nullptr;
+    auto env_on = [](const char* name) { const char* v = getenv(name); return !(v && v[0] == '0'); };
+    g.opt_fused = env_on("MT_FUSED");
+    g.opt_pair = env_on("MT_PAIR");
+    g.opt_conv_pair = env_on("MT_CONV_PAIR");
+    g.opt_pool_head = env_on("MT_POOL_HEAD");
     g.init = true;
     return MT_OK;
 }
@@ -182,6 +197,21 @@ void free_workspace() {
     for (int b = 0; b <= MT_MAX_LAYERS; ++b) { cudaFree(g.act[b]); g.act[b] = nullptr; }
     for (int l = 0; l < MT_MAX_LAYERS; ++l) { cudaFree(g.d_items[l]); g.d_items[l] = nullptr; g.items_cap[l] = 0; }
     g.cap_n = 0;
+}
+
+// The host-buffer entry points' device staging.  Sized in bytes for the family's rows at the time; released when
+// the context adopts another family (the caller has synchronised the device).
+void free_staging() {
+    cudaFree(g.st_in); cudaFree(g.st_ids); cudaFree(g.st_out);
+    g.st_in = nullptr; g.st_ids = nullptr; g.st_out = nullptr;
+    g.st_cap_in = g.st_cap_ids = g.st_cap_out = 0;
+    for (int k = 0; k < 2; ++k) {
+        cudaFree(g.as_in[k]); cudaFree(g.as_ids[k]); cudaFree(g.as_out[k]);
+        g.as_in[k] = nullptr; g.as_ids[k] = nullptr; g.as_out[k] = nullptr;
+        g.as_slot_used[k] = false;
+    }
+    g.as_cap_in = g.as_cap_ids = g.as_cap_out = 0;
+    g.as_have_compute = false;
 }
 
 mt_status encode_2d(CUtensorMap* map, void* ptr, int ld, int rows, int box_rows = BM) {
@@ -436,8 +466,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             all_dense = all_dense && g.family[l].kind == MT_DENSE;
             if (g.width[l] > max_w) max_w = g.width[l];
         }
-        const char* fused_env = getenv("MT_FUSED");
-        if (all_dense && !(fused_env && fused_env[0] == '0') && fused_mlp_fits(n, g.T, max_w)) {
+        if (all_dense && g.opt_fused && fused_mlp_fits(n, g.T, max_w)) {
             if (g.timing == 3) g.timing_now = 2;
             Timer t(K_FUSED, s);
             FusedArgs a;
@@ -460,21 +489,18 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
     // There it moves half the weight bytes per SM from L2 and runs about 4 % faster under the power cap (at a lower
     // clock).  MT_PAIR=0 keeps the one-CTA executor.
     bool pair_mode[MT_MAX_LAYERS] = {false};
-    const char* pair_env = getenv("MT_PAIR");
-    const bool pair_ok = !(pair_env && pair_env[0] == '0') && (g.sm_count >= 2) && (n / (g.live > 0 ? g.live : 1) >= 1024);
+    const bool pair_ok = g.opt_pair && (g.sm_count >= 2) && (n / (g.live > 0 ? g.live : 1) >= 1024);
     for (int l = 0; l < L; ++l) pair_mode[l] = pair_ok && g.family[l].kind == MT_DENSE && g.tile_n[l] == 256;
     int tiles_per_image = 0;
     for (const HostLayer& f : g.family)
         if (f.kind == MT_CONV3X3) tiles_per_image = g.conv.strips_per_image;
     // A global average pool followed by a narrow last dense layer (a classifier head) runs as one small launch.
-    const char* ph_env = getenv("MT_POOL_HEAD");
     const bool pool_head = L >= 3 && g.family[L - 2].kind == MT_GLOBAL_AVG_POOL && g.family[L - 1].kind == MT_DENSE &&
                            g.family[L - 2].in_ch == 64 && g.family[L - 1].in_ch == 64 && g.out_elems <= 64 &&
-                           !(ph_env && ph_env[0] == '0');
+                           g.opt_pool_head;
     // Conv layers run on CTA pairs (two images of a tenant per cluster) when the strip geometry allows the tap
     // pairing; MT_CONV_PAIR=0 forces the one-CTA executor.
-    const char* cpair_env = getenv("MT_CONV_PAIR");
-    const bool conv_pair = tiles_per_image > 0 && g.conv.Wp == 64 && g.sm_count >= 2 && !(cpair_env && cpair_env[0] == '0');
+    const bool conv_pair = tiles_per_image > 0 && g.conv.Wp == 64 && g.sm_count >= 2 && g.opt_conv_pair;
 
     // Dense families: the payload rows move into bucketed order inside the scatter pass when the batch is spread over
     // enough CTAs and small enough for them; otherwise as a gather pass of its own over the whole GPU.
@@ -499,21 +525,24 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
         a.perm = g.d_perm; a.inv = g.d_inv; a.status = g.d_status;
         launch_bucketing(a, s);
     }
-    CUtensorMap in_map, in_rows2_map, in_rows1_map;
+    CUtensorMap &in_map = g.in_map, &in_rows2_map = g.in_rows2_map, &in_rows1_map = g.in_rows1_map;
     if (f0.kind == MT_DENSE) {
         if (!rows_in_scatter) {
             Timer t(K_GATHER, s);
             launch_gather_rows(inputs, g.d_perm, n, g.in_elems * 2, g.act[0], g.act_ld[0] * 2, g.sm_count, s);
         }
-    } else {
+    } else if (g.in_map_ptr != inputs || g.in_map_n != n) {
+        g.in_map_ptr = nullptr;
         st = encode_nhwc(&in_map, inputs, f0.in_ch, f0.w, f0.h, n, g.conv.Wp, g.conv.R + 2);
         if (st != MT_OK) return st;
-        if (conv_pair) {
+        if (g.conv.Wp == 64) {
             st = encode_nhwc(&in_rows2_map, inputs, f0.in_ch, f0.w, f0.h, n, 64, 2);
             if (st != MT_OK) return st;
             st = encode_nhwc(&in_rows1_map, inputs, f0.in_ch, f0.w, f0.h, n, 64, 1);
             if (st != MT_OK) return st;
         }
+        g.in_map_ptr = inputs;
+        g.in_map_n = n;
     }
     for (int l = 0; l < L; ++l) {
         const HostLayer& f = g.family[l];
@@ -604,17 +633,11 @@ mt_status mt_shutdown(void) {
     cudaFree(g.d_tile_prefix); g.d_tile_prefix = nullptr;
     cudaFree(g.st_in); g.st_in = nullptr;
     cudaFree(g.st_ids); g.st_ids = nullptr;
-    cudaFree(g.st_out); g.st_out = nullptr;
-    g.st_cap = 0;
-    for (int k = 0; k < 2; ++k) {
-        cudaFree(g.as_in[k]); g.as_in[k] = nullptr;
-        cudaFree(g.as_ids[k]); g.as_ids[k] = nullptr;
-        cudaFree(g.as_out[k]); g.as_out[k] = nullptr;
+    free_staging();
+    for (int k = 0; k < 2; ++k)
         if (g.as_slot_done[k]) { cudaEventDestroy(g.as_slot_done[k]); g.as_slot_done[k] = nullptr; }
-        g.as_slot_used[k] = false;
-    }
     if (g.as_compute_done) { cudaEventDestroy(g.as_compute_done); g.as_compute_done = nullptr; }
-    g.as_cap = 0; g.as_next = 0; g.as_have_compute = false;
+    g.as_next = 0;
     Timer::close_group();
     for (TimedLaunch& t : g.timed) { cudaEventDestroy(t.start); cudaEventDestroy(t.stop); }
     g.timed.clear();
@@ -728,6 +751,8 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
             if (f.kind == MT_CONV3X3) plan_conv(f.h, f.w, &g.conv);   // cannot fail: validate_layers bounds w
         for (int b = 0; b <= MT_MAX_LAYERS; ++b) g.width[b] = 0;
         g.ws_dirty = true;
+        g.in_map_ptr = nullptr;
+        free_staging();   // sized for the previous family's rows (no model is live: nothing is in flight)
     }
     for (int l = 0; l < n_layers; ++l) {
         const int wd = layer_in_elems(hl[l]);
@@ -780,20 +805,23 @@ mt_status mt_infer_host(const void* inputs_host, const int32_t* model_ids_host, 
     if (!g.has_family || g.live == 0) return MT_ERR_BAD_MODEL_ID;
     CU_OK(cudaSetDevice(g.device));
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (n > g.st_cap) {
+    const size_t in_bytes = (size_t)n * g.in_elems * 2, id_bytes = (size_t)n * sizeof(int32_t),
+                 out_bytes = (size_t)n * g.out_elems * sizeof(float);
+    if (in_bytes > g.st_cap_in || id_bytes > g.st_cap_ids || out_bytes > g.st_cap_out) {
         CU_OK(cudaDeviceSynchronize());
         cudaFree(g.st_in); cudaFree(g.st_ids); cudaFree(g.st_out);
-        g.st_in = nullptr; g.st_ids = nullptr; g.st_out = nullptr; g.st_cap = 0;
-        CU_OK(cudaMalloc(&g.st_in, (size_t)n * g.in_elems * 2));
-        CU_OK(cudaMalloc(&g.st_ids, (size_t)n * sizeof(int32_t)));
-        CU_OK(cudaMalloc(&g.st_out, (size_t)n * g.out_elems * sizeof(float)));
-        g.st_cap = n;
+        g.st_in = nullptr; g.st_ids = nullptr; g.st_out = nullptr;
+        g.st_cap_in = g.st_cap_ids = g.st_cap_out = 0;
+        CU_OK(cudaMalloc(&g.st_in, in_bytes));
+        CU_OK(cudaMalloc(&g.st_ids, id_bytes));
+        CU_OK(cudaMalloc(&g.st_out, out_bytes));
+        g.st_cap_in = in_bytes; g.st_cap_ids = id_bytes; g.st_cap_out = out_bytes;
     }
-    CU_OK(cudaMemcpyAsync(g.st_in, inputs_host, (size_t)n * g.in_elems * 2, cudaMemcpyHostToDevice, s));
-    CU_OK(cudaMemcpyAsync(g.st_ids, model_ids_host, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+    CU_OK(cudaMemcpyAsync(g.st_in, inputs_host, in_bytes, cudaMemcpyHostToDevice, s));
+    CU_OK(cudaMemcpyAsync(g.st_ids, model_ids_host, id_bytes, cudaMemcpyHostToDevice, s));
     mt_status st = infer_device(g.st_in, g.st_ids, n, g.st_out, s);
     if (st != MT_OK) return st;
-    CU_OK(cudaMemcpyAsync(outputs_host, g.st_out, (size_t)n * g.out_elems * sizeof(float), cudaMemcpyDeviceToHost, s));
+    CU_OK(cudaMemcpyAsync(outputs_host, g.st_out, out_bytes, cudaMemcpyDeviceToHost, s));
     CU_OK(cudaStreamSynchronize(s));
     return MT_OK;
 }
@@ -808,23 +836,25 @@ mt_status mt_infer_host_async(const void* inputs_host, const int32_t* model_ids_
     if (!g.has_family || g.live == 0) return MT_ERR_BAD_MODEL_ID;
     CU_OK(cudaSetDevice(g.device));
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (n > g.as_cap) {
+    const size_t in_bytes = (size_t)n * g.in_elems * 2, id_bytes = (size_t)n * sizeof(int32_t),
+                 out_bytes = (size_t)n * g.out_elems * sizeof(float);
+    if (in_bytes > g.as_cap_in || id_bytes > g.as_cap_ids || out_bytes > g.as_cap_out) {
         CU_OK(cudaDeviceSynchronize());
         for (int k = 0; k < 2; ++k) {
             cudaFree(g.as_in[k]); cudaFree(g.as_ids[k]); cudaFree(g.as_out[k]);
             g.as_in[k] = nullptr; g.as_ids[k] = nullptr; g.as_out[k] = nullptr;
             g.as_slot_used[k] = false;
         }
-        g.as_cap = 0;
+        g.as_cap_in = g.as_cap_ids = g.as_cap_out = 0;
         for (int k = 0; k < 2; ++k) {
-            CU_OK(cudaMalloc(&g.as_in[k], (size_t)n * g.in_elems * 2));
-            CU_OK(cudaMalloc(&g.as_ids[k], (size_t)n * sizeof(int32_t)));
-            CU_OK(cudaMalloc(&g.as_out[k], (size_t)n * g.out_elems * sizeof(float)));
+            CU_OK(cudaMalloc(&g.as_in[k], in_bytes));
+            CU_OK(cudaMalloc(&g.as_ids[k], id_bytes));
+            CU_OK(cudaMalloc(&g.as_out[k], out_bytes));
             if (!g.as_slot_done[k]) CU_OK(cudaEventCreateWithFlags(&g.as_slot_done[k], cudaEventDisableTiming));
         }
         if (!g.as_compute_done) CU_OK(cudaEventCreateWithFlags(&g.as_compute_done, cudaEventDisableTiming));
         g.as_have_compute = false;
-        g.as_cap = n;
+        g.as_cap_in = in_bytes; g.as_cap_ids = id_bytes; g.as_cap_out = out_bytes;
     }
     // grow the workspace (a device-wide synchronisation) before anything of this call is in flight
     mt_status st = ensure_workspace(n);
@@ -833,15 +863,15 @@ mt_status mt_infer_host_async(const void* inputs_host, const int32_t* model_ids_
     g.as_next ^= 1;
     // the slot's previous user must have copied its outputs out
     if (g.as_slot_used[k]) CU_OK(cudaStreamWaitEvent(s, g.as_slot_done[k], 0));
-    CU_OK(cudaMemcpyAsync(g.as_in[k], inputs_host, (size_t)n * g.in_elems * 2, cudaMemcpyHostToDevice, s));
-    CU_OK(cudaMemcpyAsync(g.as_ids[k], model_ids_host, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+    CU_OK(cudaMemcpyAsync(g.as_in[k], inputs_host, in_bytes, cudaMemcpyHostToDevice, s));
+    CU_OK(cudaMemcpyAsync(g.as_ids[k], model_ids_host, id_bytes, cudaMemcpyHostToDevice, s));
     // the kernels of consecutive calls share one workspace: they run one call after the other, whatever the streams
     if (g.as_have_compute) CU_OK(cudaStreamWaitEvent(s, g.as_compute_done, 0));
     st = infer_device(g.as_in[k], g.as_ids[k], n, g.as_out[k], s);
     if (st != MT_OK) return st;
     CU_OK(cudaEventRecord(g.as_compute_done, s));
     g.as_have_compute = true;
-    CU_OK(cudaMemcpyAsync(outputs_host, g.as_out[k], (size_t)n * g.out_elems * sizeof(float), cudaMemcpyDeviceToHost, s));
+    CU_OK(cudaMemcpyAsync(outputs_host, g.as_out[k], out_bytes, cudaMemcpyDeviceToHost, s));
     CU_OK(cudaEventRecord(g.as_slot_done[k], s));
     g.as_slot_used[k] = true;
     return MT_OK;
@@ -902,10 +932,33 @@ mt_status mt_debug_wait_timeout(int32_t limit_ms, void* stream) {
     return MT_OK;
 }
 
+mt_status mt_debug_empty_launches(int32_t count, void* stream) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g.init) return MT_ERR_NOT_INIT;
+    if (count < 0 || count > 100000) return MT_ERR_INVALID_ARG;
+    CU_OK(cudaSetDevice(g.device));
+    launch_empty_chain(count, static_cast<cudaStream_t>(stream));
+    CU_OK(cudaGetLastError());
+    return MT_OK;
+}
+
 mt_status mt_debug_launch_count(int64_t* count_out) {
     std::lock_guard<std::mutex> lk(g_mu);
     if (!count_out) return MT_ERR_INVALID_ARG;
     *count_out = (int64_t)mt::g_kernel_launches;
+    return MT_OK;
+}
+
+mt_status mt_debug_set_option(const char* name, int32_t value) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g.init) return MT_ERR_NOT_INIT;
+    if (!name) return MT_ERR_INVALID_ARG;
+    const bool on = value != 0;
+    if (!strcmp(name, "fused")) g.opt_fused = on;
+    else if (!strcmp(name, "pair")) g.opt_pair = on;
+    else if (!strcmp(name, "conv_pair")) g.opt_conv_pair = on;
+    else if (!strcmp(name, "pool_head")) g.opt_pool_head = on;
+    else return MT_ERR_INVALID_ARG;
     return MT_OK;
 }
 

@@ -61,6 +61,8 @@ struct BucketArgs {
 void launch_bucketing(const BucketArgs& a, cudaStream_t s);
 // One thread waits (bounded by limit_ns) on a barrier nobody completes; *gave_up = 1 and the status word is set.
 void launch_wait_timeout_probe(int32_t* status, unsigned long long limit_ns, int32_t* gave_up, cudaStream_t s);
+// `count` empty kernels chained by programmatic dependent launch (the launch floor of the path).
+void launch_empty_chain(int count, cudaStream_t s);
 void launch_gather_rows(const void* src, const int32_t* perm, int n, int row_bytes, void* dst, int dst_ld_bytes,
                         int sm_count, cudaStream_t s);
 

@@ -23,9 +23,10 @@ def check_bucketing(model_ids, n_tenants):
     assert np.array_equal(inv, oi)
 
 
-def run_and_check(models, model_ids, inputs, sample=None, max_models=None, tol=TOL, register=True):
+def run_and_check(models, model_ids, inputs, sample=None, max_models=None, tol=TOL, register=True, stats=None):
     """Register (optionally), run one batch through the C-ABI, compare with the oracle.
-    sample: arrival indices to check against the oracle (None = all).  Returns (gpu_out, max_scaled_err)."""
+    sample: arrival indices to check against the oracle (None = all).  Returns (gpu_out, max_scaled_err);
+    a dict passed as `stats` also receives the 99.99th percentile and the number of compared elements."""
     if register:
         fresh(max_models or max(64, len(models)))
         ids = harness.register_models(models)
@@ -42,13 +43,49 @@ def run_and_check(models, model_ids, inputs, sample=None, max_models=None, tol=T
         sample = np.asarray(sample)
         ref = oracle.forward(models, model_ids[sample], inputs[sample])
         err = harness.scaled_error(got[sample], ref)
-    assert err.max() <= tol, "max scaled error %.3e (99.99th pct %.3e)" % (err.max(), np.quantile(err, 0.9999))
+    p9999 = float(np.quantile(err, 0.9999))
+    if stats is not None:
+        stats.update(max=float(err.max()), p9999=p9999, elements=int(err.size))
+    assert err.max() <= tol, "max scaled error %.3e (99.99th pct %.3e)" % (err.max(), p9999)
     return got, float(err.max())
 
 
-def stratified_sample(model_ids, n_tenants, per_tenant, tile=128, seed=0):
-    """Arrival indices covering, per tenant: first and last request of its segment, the neighbours of every
-    multiple of `tile` in bucketed order, plus random ones up to per_tenant."""
+def sample_positions(lo, hi, per_tenant, tiles, rng):
+    """Bucketed positions to check inside one segment [lo, hi).  Always the first and the last row; then both
+    neighbours of row-tile boundaries (multiples of every width in `tiles`, widest first), spread evenly over the
+    WHOLE segment when there are more of them than the budget allows, the last boundary (the one in front of the
+    ragged tail tile) always among them; the rest of the budget is filled with random rows."""
+    budget = max(int(per_tenant), 2)
+    chosen = [lo] if hi - lo == 1 else [lo, hi - 1]
+    seen = set(chosen)
+
+    def take(p):
+        if lo <= p < hi and p not in seen and len(chosen) < budget:
+            seen.add(p)
+            chosen.append(p)
+
+    for tile in sorted(tiles, reverse=True):
+        bounds = [b for b in range(lo + tile, hi, tile) if not (b in seen and b - 1 in seen)]   # not those a wider tile already gave
+        room = (budget - len(chosen)) // 2
+        if room <= 0 or not bounds:
+            continue
+        if len(bounds) > room:       # evenly spaced over the segment, ending with the last boundary
+            idx = np.unique(np.round(np.linspace(0, len(bounds) - 1, room)).astype(int))
+            bounds = [bounds[i] for i in idx]
+        for b in reversed(bounds):   # the last boundary first: it survives whatever the budget
+            take(b - 1)
+            take(b)
+    extra = min(budget - len(chosen), (hi - lo) - len(chosen))
+    if extra > 0:
+        rest = np.setdiff1d(np.arange(lo, hi), np.fromiter(seen, dtype=np.int64))
+        for p in rng.choice(rest, size=extra, replace=False).tolist():
+            take(int(p))
+    return chosen
+
+
+def stratified_sample(model_ids, n_tenants, per_tenant, tiles=(128, 256), seed=0):
+    """Arrival indices covering, per tenant, the positions of sample_positions (at most per_tenant of them;
+    128- and 256-row boundaries, since the CTA-pair executors work on 256-row tiles)."""
     rng = np.random.default_rng(seed)
     _, offsets, perm, _ = oracle.bucket(model_ids, n_tenants)
     picked = []
@@ -56,12 +93,5 @@ def stratified_sample(model_ids, n_tenants, per_tenant, tile=128, seed=0):
         lo, hi = int(offsets[t]), int(offsets[t + 1])
         if hi == lo:
             continue
-        pos = {lo, hi - 1}
-        for b in range(lo + tile, hi, tile):
-            pos.update((b - 1, b))
-        pos = sorted(pos)[:max(per_tenant, 2)]
-        extra = per_tenant - len(pos)
-        if extra > 0 and hi - lo > len(pos):
-            pos += rng.choice(np.arange(lo, hi), size=min(extra, hi - lo), replace=False).tolist()
-        picked += [int(perm[p]) for p in set(pos)]
+        picked += [int(perm[p]) for p in sample_positions(lo, hi, per_tenant, tiles, rng)]
     return np.array(sorted(set(picked)), dtype=np.int64)

@@ -26,7 +26,7 @@ def test_config1_is_one_launch_and_layered_path_agrees(monkeypatch):
     wl = synth.make_workload(1)
     (got, _), k = launches_of(lambda: run_and_check(wl.models, wl.model_ids, wl.inputs))
     assert k == 1
-    monkeypatch.setenv("MT_FUSED", "0")
+    mt.mt_debug_set_option("fused", 0)
     layered, k = launches_of(lambda: harness.run_batch(wl.model_ids, wl.inputs, 10))
     assert k == 5                                     # bucketing, gather, three layers (the last one un-permutes)
     ref = oracle.forward(wl.models, wl.model_ids, wl.inputs)

@@ -135,11 +135,11 @@ def test_pool_followed_by_head_both_ways(monkeypatch):
     # head wider than 64) takes the pool_finalize + grouped dense path instead: both against the oracle
     wl = synth.make_workload(4, n=23, n_tenants=4, h=12, w=40, n_conv=2)
     got_fused, _ = run_and_check(wl.models, wl.model_ids, wl.inputs)
-    monkeypatch.setenv("MT_POOL_HEAD", "0")
+    monkeypatch.setenv("MT_POOL_HEAD", "0")                    # read by mt_init inside run_and_check
     got_split, _ = run_and_check(wl.models, wl.model_ids, wl.inputs)
     assert np.abs(got_fused - got_split).max() <= 1e-4        # same bf16 pooled values and weights, other summation order
     ids = wl.model_ids.copy(); ids[3] = 9                      # a rejected id on the fused pool + head path
-    monkeypatch.delenv("MT_POOL_HEAD")
+    mt.mt_debug_set_option("pool_head", 1)
     got = harness.run_batch(ids, wl.inputs, 10)
     assert mt.mt_get_async_status() == (2, 3)
     assert np.isnan(got[3]).all() and np.array_equal(np.delete(got, 3, 0), np.delete(got_fused, 3, 0))
@@ -305,3 +305,36 @@ def test_family_mismatch_is_rejected():
     with pytest.raises(mt.MtError) as e:
         mt.mt_release(5)
     assert e.value.code == 2
+
+
+@pytest.mark.parametrize("entry", ["sync", "async"])
+def test_host_entries_after_a_wider_family_replaces_a_narrow_one(entry):
+    # the host-buffer entry points keep device staging sized for the family's rows: when every model has been released
+    # and a family with wider inputs and outputs is registered, a batch of the SAME size must get new staging
+    def host_call(models, ids, x, out_elems):
+        n = len(ids)
+        h_x = torch.from_numpy(x.view(np.int16)).pin_memory()
+        h_ids = torch.from_numpy(ids).pin_memory()
+        h_out = torch.full((n, out_elems), float("nan"), dtype=torch.float32).pin_memory()
+        if entry == "sync":
+            mt.mt_infer_host(h_x, h_ids, n, h_out)
+        else:
+            for _ in range(3):                                   # both staging slots
+                mt.mt_infer_host_async(h_x, h_ids, n, h_out)
+            torch.cuda.synchronize()
+        assert mt.mt_get_async_status() == (0, -1)
+        got = h_out.numpy()
+        ref = oracle.forward(models, ids, x)
+        assert np.isfinite(got).all() and harness.scaled_error(got, ref).max() <= TOL
+
+    rng = np.random.default_rng(21)
+    n = 600
+    fresh()
+    narrow = [synth.make_mlp(2, t, (64, 128, 8)) for t in range(3)]
+    ids = harness.register_models(narrow)
+    host_call(narrow, rng.integers(0, 3, n).astype(np.int32), bits(rng.standard_normal((n, 64))), 8)
+    for i in ids:
+        mt.mt_release(i)
+    wide = [synth.make_mlp(2, 10 + t, (512, 256, 200)) for t in range(2)]
+    assert harness.register_models(wide) == [0, 1]
+    host_call(wide, rng.integers(0, 2, n).astype(np.int32), bits(rng.standard_normal((n, 512))), 200)
