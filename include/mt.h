@@ -152,6 +152,8 @@ mt_status mt_debug_empty_launches(int32_t count, void* stream);
  *   "pair"       (MT_PAIR)       CTA-pair dense executor for batches with >= 1024 requests per tenant
  *   "conv_pair"  (MT_CONV_PAIR)  CTA-pair conv executor for padded rows of 64 pixels; off: the one-CTA executor
  *   "pool_head"  (MT_POOL_HEAD)  pool + narrow head as one launch; off: pool_finalize + a grouped dense launch
+ *   "perm_gather" (MT_PERM_GATHER) first dense layer reads the caller's rows through the permutation with TMA gathers
+ *                instead of a row-move pass: 0 never, 1 (default) for batches of at most 256 requests, 2 always
  * Unknown name: MT_ERR_INVALID_ARG.  Results agree with the oracle on every setting. */
 mt_status mt_debug_set_option(const char* name, int32_t value);
 

@@ -88,7 +88,58 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     pdl_wait();   // everything above overlapped the previous kernel's tail; its results are needed from here on
     const int total = p.tile_prefix[p.T];
 
-    if (warp == 0) {
+    if (warp == 0 && p.gather_perm) {
+        // ---------------------------------------------------------------- TMA producer, rows through the permutation
+        // The whole warp walks the loop: lane 0 waits for the stage, announces the bytes and fetches the weights, then
+        // lane l fetches rows 4l .. 4l + 3 of the tile with ONE gather of four rows named by perm (32 gathers build
+        // the same 16 KiB swizzled image as one 128-row box; a transposed item needs only its 8 or 16).
+        int stage = 0; uint32_t phase = 0;
+        bool ok = true;
+        WorkItem cur = {};
+        if ((int)blockIdx.x < total) cur = load_item(p.items, blockIdx.x);
+        for (int item = blockIdx.x; ok && item < total; item += gridDim.x) {
+            WorkItem nxt = {};
+            if (item + (int)gridDim.x < total) nxt = load_item(p.items, item + gridDim.x);
+            const int kblocks = cur.k_blocks;
+            const bool swap = kSwapOk && cur.rows_valid <= kSwapRows;
+            const int n_g4 = swap ? ((cur.rows_valid + 31) >> 5) * 8 : 32;       // gathers (= lanes) per stage
+            // rows past the segment are computed and never stored: any valid row will do for them
+            int rr[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int r = 4 * lane + j;
+                rr[j] = __ldg(p.gather_perm + cur.row0 + (r < cur.rows_valid ? r : 0));
+            }
+            const uint16_t* wsrc = cur.w + (size_t)cur.n_tile * kWTiles * kblocks * (BN * BK);
+            uint32_t wbytes[kWTiles];
+            uint32_t wsum = 0;
+#pragma unroll
+            for (int wt = 0; wt < kWTiles; ++wt) {
+                const int rows = min(BN, max(0, cur.N - (cur.n_tile * kWTiles + wt) * BN));
+                wbytes[wt] = (uint32_t)((rows + 7) & ~7) * (BK * 2);
+                wsum += wbytes[wt];
+            }
+            for (int kb = 0; kb < kblocks; ++kb) {
+                const uint32_t a_dst = base + stage * kStageBytes;
+                if (lane == 0) {
+                    ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1);
+                    if (ok) {
+                        mbar_expect_tx(full_bar(stage), (uint32_t)(n_g4 * 512) + wsum);
+#pragma unroll
+                        for (int wt = 0; wt < kWTiles; ++wt)
+                            if (wbytes[wt])
+                                bulk_load(a_dst + (1 + wt) * TILE_BYTES, wsrc + ((size_t)wt * kblocks + kb) * (BN * BK),
+                                          wbytes[wt], full_bar(stage));
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                if (lane < n_g4) tma_gather4(a_dst + lane * 512, &tmap_a, kb * BK, rr[0], rr[1], rr[2], rr[3], full_bar(stage));
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            }
+            cur = nxt;
+        }
+    } else if (warp == 0) {
         if (lane == 0) {   // ------------------------------------------------ TMA producer
             int stage = 0; uint32_t phase = 0;
             bool ok = true;

@@ -91,7 +91,43 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmA
     const int n_pairs = gridDim.x >> 1;
     const int pair_id = blockIdx.x >> 1;
 
-    if (warp == 0) {
+    if (warp == 0 && p.gather_perm) {
+        // ------------------------------------------------ TMA producer (both CTAs), rows through the permutation: the
+        // whole warp walks the loop, lane 0 waits, announces and fetches the weights, lane l gathers rows 4l .. 4l + 3
+        int stage = 0; uint32_t phase = 0;
+        bool ok = true;
+        WorkItem cur = {};
+        if (pair_id < total) cur = load_pair_item(p.items, pair_id);
+        for (int item = pair_id; ok && item < total; item += n_pairs) {
+            WorkItem nxt = {};
+            if (item + n_pairs < total) nxt = load_pair_item(p.items, item + n_pairs);
+            const int kblocks = cur.k_blocks;
+            const CUtensorMap* wmap = p.wmaps + (size_t)cur.t * MT_MAX_LAYERS + p.layer;
+            const int wrow0 = (cur.n_tile * 2 + (int)rank) * kblocks * BN;
+            int rr[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int r = (int)rank * BM + 4 * lane + j;         // rows past the segment: any valid row
+                rr[j] = __ldg(p.gather_perm + cur.row0 + (r < cur.rows_valid ? r : 0));
+            }
+            for (int kb = 0; kb < kblocks; ++kb) {
+                const uint32_t a_dst = base + stage * kPairStageBytes;
+                const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
+                if (lane == 0) {
+                    ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 31);
+                    if (ok) {
+                        if (is_leader) mbar_expect_tx(full_bar(stage), 2 * kPairStageBytes);   // both CTAs' bytes
+                        tma_load_2d_pair(a_dst + TILE_BYTES, wmap, 0, wrow0 + kb * BN, leader_full);
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                tma_gather4_pair(a_dst + lane * 512, &tmap_a, kb * BK, rr[0], rr[1], rr[2], rr[3], leader_full);
+                if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+            }
+            cur = nxt;
+        }
+    } else if (warp == 0) {
         if (lane == 0) {   // ------------------------------------------------ TMA producer (both CTAs)
             int stage = 0; uint32_t phase = 0;
             bool ok = true;

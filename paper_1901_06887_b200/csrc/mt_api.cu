@@ -103,6 +103,7 @@ struct Ctx {
     // switches for tests and A/B timing: read from the environment once, at mt_init (MT_FUSED, MT_PAIR, MT_CONV_PAIR,
     // MT_POOL_HEAD; "0" turns the path off), changed afterwards only through mt_debug_set_option
     bool opt_fused = true, opt_pair = true, opt_conv_pair = true, opt_pool_head = true;
+    int opt_gather = 1;                  // 0 never, 1 small batches, 2 always
 
     // tensor maps over the caller's images (first conv layer), kept while pointer and batch size stay the same
     const void* in_map_ptr = nullptr;
@@ -185,6 +186,7 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     g.opt_pair = env_on("MT_PAIR");
     g.opt_conv_pair = env_on("MT_CONV_PAIR");
     g.opt_pool_head = env_on("MT_POOL_HEAD");
+    { const char* v = getenv("MT_PERM_GATHER"); g.opt_gather = (v && v[0] >= '0' && v[0] <= '2') ? v[0] - '0' : 1; }
     g.init = true;
     return MT_OK;
 }
@@ -504,7 +506,14 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
 
     // Dense families: the payload rows move into bucketed order inside the scatter pass when the batch is spread over
     // enough CTAs and small enough for them; otherwise as a gather pass of its own over the whole GPU.
-    const bool rows_in_scatter = f0.kind == MT_DENSE && n > 512 && (size_t)n * g.in_elems * 2 <= ((size_t)64 << 20);
+    // Small batches (one bucketing CTA, which cannot move rows): the first dense layer reads the caller's rows through
+    // perm, four rows per TMA gather, and no row pass runs at all.  Measured: a gather costs the producer about 130
+    // cycles against one box load per 128 rows, and a tile is fetched once per column tile, so beyond a few hundred
+    // requests moving each row once is cheaper (config 3: +57 us, config 5: +10 ms with gathers; at 512 requests the
+    // two are level).  "perm_gather" = 2
+    // forces the gather for any batch size (tests).
+    const bool perm_gather = f0.kind == MT_DENSE && (g.opt_gather == 2 || (g.opt_gather == 1 && n <= 256));
+    const bool rows_in_scatter = f0.kind == MT_DENSE && !perm_gather && n > 512 && (size_t)n * g.in_elems * 2 <= ((size_t)64 << 20);
     {
         Timer t(K_BUCKET, s);
         BucketArgs a;
@@ -527,7 +536,15 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
     }
     CUtensorMap &in_map = g.in_map, &in_rows2_map = g.in_rows2_map, &in_rows1_map = g.in_rows1_map;
     if (f0.kind == MT_DENSE) {
-        if (!rows_in_scatter) {
+        if (perm_gather) {
+            if (g.in_map_ptr != inputs || g.in_map_n != n) {
+                g.in_map_ptr = nullptr;
+                st = encode_2d(&in_map, const_cast<void*>(inputs), g.in_elems, n, 1);   // one-row boxes: the gather form
+                if (st != MT_OK) return st;
+                g.in_map_ptr = inputs;
+                g.in_map_n = n;
+            }
+        } else if (!rows_in_scatter) {
             Timer t(K_GATHER, s);
             launch_gather_rows(inputs, g.d_perm, n, g.in_elems * 2, g.act[0], g.act_ld[0] * 2, g.sm_count, s);
         }
@@ -562,8 +579,10 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             a.perm = direct ? g.d_perm : nullptr;
             a.offsets = g.d_offsets;
             a.status = g.d_status;
-            if (pair_mode[l]) CU_OK(launch_grouped_gemm_pair(g.act_map[l], a, g.sm_count, s));
-            else launch_grouped_gemm(g.act_map[l], g.act_map32[l], a, g.tile_n[l], g.sm_count, s);
+            const bool gather = (l == 0) && perm_gather;
+            a.gather_perm = gather ? g.d_perm : nullptr;
+            if (pair_mode[l]) CU_OK(launch_grouped_gemm_pair(gather ? in_map : g.act_map[l], a, g.sm_count, s));
+            else launch_grouped_gemm(gather ? in_map : g.act_map[l], g.act_map32[l], a, g.tile_n[l], g.sm_count, s);
         } else if (f.kind == MT_CONV3X3) {
             Timer t(K_CONV, s);
             ConvArgs a;
@@ -958,6 +977,7 @@ mt_status mt_debug_set_option(const char* name, int32_t value) {
     else if (!strcmp(name, "pair")) g.opt_pair = on;
     else if (!strcmp(name, "conv_pair")) g.opt_conv_pair = on;
     else if (!strcmp(name, "pool_head")) g.opt_pool_head = on;
+    else if (!strcmp(name, "perm_gather")) g.opt_gather = value < 0 ? 0 : (value > 2 ? 2 : value);
     else return MT_ERR_INVALID_ARG;
     return MT_OK;
 }

@@ -188,6 +188,25 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
+// TMA gather: four rows of a 2-D tensor, picked by index, land as four consecutive 128-byte rows (the tensor map's box
+// is one row of 64 bf16 high; the 128-byte swizzle follows the shared-memory address, so four-row groups written one
+// after the other form the same image as one tiled box).  c0 = first column, r0..r3 = row indices.
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* map, int c0, int r0, int r1, int r2, int r3,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar)
+        : "memory");
+}
+// The same from a CTA of a pair, completion bytes reported to a barrier of the pair's leader.
+__device__ __forceinline__ void tma_gather4_pair(uint32_t dst, const CUtensorMap* map, int c0, int r0, int r1, int r2, int r3,
+                                                 uint32_t leader_bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(leader_bar)
+        : "memory");
+}
+
 // TMA: tiled tensor store shared -> global (elements outside the tensor are dropped), tracked by bulk async-groups.
 __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t src) {
     asm volatile(

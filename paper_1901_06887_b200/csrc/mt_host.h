@@ -88,11 +88,16 @@ struct GemmArgs {
     // filled with NaN by the same launch - no separate un-permute pass.
     const int32_t* perm;
     const int32_t* offsets;       // [T + 2]
+    // First layer only: non-null gather_perm makes the executor read its input rows from the caller's buffer (arrival
+    // order) through the permutation - bucketed row j is row gather_perm[j] of the tensor behind the gather map (boxes
+    // of one row x 64 columns), fetched four rows per TMA gather - so the payload is never moved into bucketed order.
+    const int32_t* gather_perm;
     int32_t* status;
 };
 cudaError_t configure_grouped_gemm();
 // tile_n: 128 or 256 output columns per work item; must match BucketArgs::tile_n of that layer.
 // tmap_a: 128-row boxes of the layer's input; tmap_a32: 32-row boxes of the same buffer (transposed small items).
+// With GemmArgs::gather_perm set, tmap_a is the gather map over the caller's rows (tmap_a32 is then unused).
 void launch_grouped_gemm(const CUtensorMap& tmap_a, const CUtensorMap& tmap_a32, const GemmArgs& a, int tile_n,
                          int sm_count, cudaStream_t s);
 

@@ -28,7 +28,7 @@ def test_config1_is_one_launch_and_layered_path_agrees(monkeypatch):
     assert k == 1
     mt.mt_debug_set_option("fused", 0)
     layered, k = launches_of(lambda: harness.run_batch(wl.model_ids, wl.inputs, 10))
-    assert k == 5                                     # bucketing, gather, three layers (the last one un-permutes)
+    assert k == 4                                     # bucketing, three layers (the first reads through perm, the last writes through it)
     ref = oracle.forward(wl.models, wl.model_ids, wl.inputs)
     assert harness.scaled_error(layered, ref).max() <= TOL
     assert np.abs(layered - got).max() <= 1e-4        # same products; only the accumulation grouping may differ
@@ -142,3 +142,29 @@ def test_random_families_against_the_oracle(seed):
     ref = oracle.forward(models, ids[good], x[good])
     assert np.isfinite(got[good]).all()
     assert harness.scaled_error(got[good], ref).max() <= TOL
+
+
+@pytest.mark.parametrize("case", ["c2_reduced", "c3_reduced", "pair", "ragged_single", "tiny_layered"])
+def test_first_layer_reads_rows_through_perm(case, monkeypatch):
+    # MT_PERM_GATHER=2: the first dense layer fetches its rows from the caller's buffer through the permutation (four
+    # rows per TMA gather) at every batch size - 128-row tiles, transposed small segments, the CTA-pair executor - and
+    # no row pass runs; results must equal the row-move path's bit for bit (same operands, same order of products)
+    if case == "c2_reduced":
+        wl = synth.make_workload(2, n=900, n_tenants=7, widths=(1024, 512, 640, 256))
+    elif case == "c3_reduced":
+        wl = synth.make_workload(3, n=1500, n_tenants=120)
+    elif case == "pair":
+        wl = synth.make_workload(5, n=2500, n_tenants=2, widths=(256, 512, 256))
+    elif case == "ragged_single":
+        wl = synth.make_workload(5, n=385, n_tenants=1, widths=(128, 320, 130))
+    else:
+        wl = synth.make_workload(1)
+        monkeypatch.setenv("MT_FUSED", "0")
+    T = len(wl.models)
+    monkeypatch.setenv("MT_PERM_GATHER", "2")
+    (got, _), k = launches_of(lambda: run_and_check(wl.models, wl.model_ids, wl.inputs, max_models=max(64, T)))
+    n_layers = len(wl.models[0])
+    assert k == (1 if wl.n <= 512 else 2) + n_layers          # bucketing and the layers, nothing else
+    monkeypatch.setenv("MT_PERM_GATHER", "0")
+    moved, _ = run_and_check(wl.models, wl.model_ids, wl.inputs, max_models=max(64, T))
+    assert np.array_equal(got, moved)
