@@ -141,6 +141,17 @@ mt_status mt_debug_wait_timeout(int32_t limit_ms, void* stream);
  * mt_infer_host since it was loaded (registration and the no-allocation call are not counted). */
 mt_status mt_debug_launch_count(int64_t* count_out);
 
+/* Cost-aware scheduling (Sec. 3.2: a DNN's work per layer is fixed by its shape, so the cost of every work item is
+ * known before a request arrives).  Each dense layer's work items are laid out heaviest first - tenants ranked on the
+ * host, at registration, by the modelled cost of one of their items - and dealt back and forth over the CTAs.
+ * mt_debug_item_cost: the model itself (pure host code, usable without a GPU): SM cycles of an item with k_blocks
+ * K blocks of 64, n_cols output columns and `rows` requests (<= 64: transposed form); 0 for an empty item.
+ * mt_debug_schedule_balance: for dense layer `layer` of the LAST mt_infer (layer-by-layer path), the heaviest CTA's
+ * modelled cost over the mean (*max_over_mean_out; 1.0 = perfectly even), the number of work items and of CTAs (or
+ * CTA pairs) they were dealt to.  Synchronises the device. */
+mt_status mt_debug_item_cost(int32_t k_blocks, int32_t n_cols, int32_t rows, double* cycles_out);
+mt_status mt_debug_schedule_balance(int32_t layer, double* max_over_mean_out, int32_t* n_items_out, int32_t* n_ctas_out);
+
 /* Bench hook: enqueue `count` (0..100000) kernels that do nothing, chained on `stream` by programmatic dependent
  * launch exactly like the kernels of the path.  Timing a long chain gives the least a launch of the path can cost
  * (the launch floor that bounds a batch as small as 64 requests); not counted by mt_debug_launch_count. */

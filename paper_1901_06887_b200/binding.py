@@ -22,7 +22,8 @@ STATUS_NAMES = {0: "MT_OK", 1: "MT_ERR_INVALID_ARG", 2: "MT_ERR_BAD_MODEL_ID", 3
 
 EXPORTS = ["mt_init", "mt_shutdown", "mt_register_model", "mt_infer", "mt_infer_host", "mt_infer_host_async", "mt_release",
            "mt_get_async_status", "mt_status_string", "mt_debug_last_bucketing", "mt_set_kernel_timing",
-           "mt_get_kernel_times", "mt_bucket_noalloc", "mt_debug_wait_timeout", "mt_debug_launch_count", "mt_debug_set_option", "mt_debug_empty_launches"]
+           "mt_get_kernel_times", "mt_bucket_noalloc", "mt_debug_wait_timeout", "mt_debug_launch_count", "mt_debug_set_option", "mt_debug_empty_launches", "mt_debug_item_cost",
+           "mt_debug_schedule_balance"]
 
 
 class MtError(RuntimeError):
@@ -67,6 +68,8 @@ def lib() -> ctypes.CDLL:
         l.mt_debug_launch_count.argtypes = [ctypes.POINTER(ctypes.c_int64)]
         l.mt_debug_set_option.argtypes = [ctypes.c_char_p, i32]
         l.mt_debug_empty_launches.argtypes = [i32, vp]
+        l.mt_debug_item_cost.argtypes = [i32, i32, i32, ctypes.POINTER(ctypes.c_double)]
+        l.mt_debug_schedule_balance.argtypes = [i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i32), ctypes.POINTER(i32)]
         for name in EXPORTS:
             if name != "mt_status_string":
                 getattr(l, name).restype = ctypes.c_int
@@ -175,6 +178,21 @@ def mt_debug_launch_count() -> int:
     c = ctypes.c_int64(0)
     _check(lib().mt_debug_launch_count(ctypes.byref(c)), "mt_debug_launch_count")
     return int(c.value)
+
+
+def mt_debug_item_cost(k_blocks: int, n_cols: int, rows: int) -> float:
+    """Modelled SM cycles of one dense work item (host code only; needs no GPU)."""
+    c = ctypes.c_double(0.0)
+    _check(lib().mt_debug_item_cost(int(k_blocks), int(n_cols), int(rows), ctypes.byref(c)), "mt_debug_item_cost")
+    return float(c.value)
+
+
+def mt_debug_schedule_balance(layer: int) -> Tuple[float, int, int]:
+    """(heaviest CTA's modelled cost / mean, work items, CTAs) of a dense layer of the last mt_infer."""
+    r, n, g = ctypes.c_double(0.0), ctypes.c_int32(0), ctypes.c_int32(0)
+    _check(lib().mt_debug_schedule_balance(int(layer), ctypes.byref(r), ctypes.byref(n), ctypes.byref(g)),
+           "mt_debug_schedule_balance")
+    return float(r.value), int(n.value), int(g.value)
 
 
 def mt_debug_empty_launches(count: int, stream=None) -> None:

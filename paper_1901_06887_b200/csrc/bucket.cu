@@ -28,7 +28,10 @@ struct LayerTileN { int v[8]; int m[8]; int kind[8]; };
 // Compact copy of what the bucketing passes need from the tenant table, one row of `ld` ints per field: row 0 =
 // alive flag, row 1 + l = out features of layer l.  (Reading these through the 328-byte ModelDev records costs one
 // memory sector per tenant and field; a thousand tenants' worth from a single CTA took several microseconds.)
-struct Brief { const int32_t* p; int ld; };
+// `order` (rows of `ld` ints, one per layer) lists the tenants of a layer in the order their work items are laid out:
+// heaviest per-item cost first, as ranked on the host from the layer shapes (known before any request arrives).
+struct Brief { const int32_t* p; int ld; const int32_t* order; };
+__device__ __forceinline__ int tenant_at(Brief br, int l, int rank) { return __ldg(br.order + (size_t)l * br.ld + rank); }
 
 // ids outside [0, T) or of dead models go to the extra bucket T, so they sort behind every live segment.
 __device__ __forceinline__ int classify(int id, int T, Brief br) {
@@ -131,9 +134,10 @@ __device__ __forceinline__ int layer_units(Brief br, const LayerTileN& tn, int t
 }
 
 // Offsets (exclusive scan of counts over the T + 1 buckets, offsets[T + 1] = n) and, per layer, the prefix sums of
-// the work units each tenant contributes.  Run by one CTA of any multiple of 32 threads; counts[] must be visible.
+// the work units each tenant contributes, taken in the layer's cost order (tile_prefix[l][r] belongs to the tenant of
+// rank r).  Run by one CTA of any multiple of 32 threads; counts[] must be visible (cnt may be a shared-memory copy).
 __device__ __forceinline__ void scan_buckets(int T, Brief br, int n_layers, int rows_per_unit,
-                                             const LayerTileN& tn, const int32_t* counts, int32_t* __restrict__ offsets,
+                                             const LayerTileN& tn, const int32_t* cnt, int32_t* __restrict__ offsets,
                                              int32_t* __restrict__ tile_prefix, int32_t* s_warp, int32_t* s_vec,
                                              int own_count = -1) {
     // own_count >= 0: the caller has counts[threadIdx.x] in a register (one bucket per thread), no need to read it back
@@ -143,24 +147,27 @@ __device__ __forceinline__ void scan_buckets(int T, Brief br, int n_layers, int 
     const bool have_own = own_count >= 0 && per == 1;
     int sum = 0;
     if (have_own) sum = (lo < hi) ? own_count : 0;
-    else for (int t = lo; t < hi; ++t) sum += counts[t];
+    else for (int t = lo; t < hi; ++t) sum += cnt[t];
     int total;
     int run = cta_excl_scan(sum, s_warp, &total);
     if (have_own) { if (lo < hi) offsets[lo] = run; }
-    else for (int t = lo; t < hi; ++t) { offsets[t] = run; run += counts[t]; }
+    else for (int t = lo; t < hi; ++t) { offsets[t] = run; run += cnt[t]; }
     if (threadIdx.x == 0) offsets[T1] = total;
     const int hi_t = min(hi, T);               // the extra bucket of rejected ids contributes no work
     if (per == 1) {
-        // one bucket per thread (the usual case): the units of all layers first, so that the loads from the tenant
-        // table are in flight together instead of one round trip per layer
-        LayerHead head[MT_MAX_LAYERS];
-        const int t_own = min(lo, T - 1);
+        // one rank per thread (the usual case): the tenants of that rank in every layer first, then their shapes, then
+        // their counts, so that each kind of load is in flight for all layers together
+        const int r_own = min(lo, T - 1);
+        int t_l[MT_MAX_LAYERS];
 #pragma unroll
-        for (int l = 0; l < MT_MAX_LAYERS; ++l) head[l] = (l < n_layers) ? load_head(br, tn, t_own, l) : LayerHead{-1, 0};
-        const int c_own = (lo < hi_t) ? (have_own ? own_count : counts[lo]) : 0;
+        for (int l = 0; l < MT_MAX_LAYERS; ++l) t_l[l] = (l < n_layers) ? tenant_at(br, l, r_own) : 0;
+        LayerHead head[MT_MAX_LAYERS];
+#pragma unroll
+        for (int l = 0; l < MT_MAX_LAYERS; ++l) head[l] = (l < n_layers) ? load_head(br, tn, t_l[l], l) : LayerHead{-1, 0};
         int units[MT_MAX_LAYERS];
 #pragma unroll
-        for (int l = 0; l < MT_MAX_LAYERS; ++l) units[l] = units_of(head[l], c_own, rows_per_unit, tn.v[l], tn.m[l]);
+        for (int l = 0; l < MT_MAX_LAYERS; ++l)
+            units[l] = (l < n_layers && lo < hi_t) ? units_of(head[l], cnt[t_l[l]], rows_per_unit, tn.v[l], tn.m[l]) : 0;
         int urun[MT_MAX_LAYERS], utotal[MT_MAX_LAYERS];
         cta_excl_scan_vec(units, urun, utotal, s_vec, n_layers);
 #pragma unroll
@@ -174,9 +181,13 @@ __device__ __forceinline__ void scan_buckets(int T, Brief br, int n_layers, int 
     for (int l = 0; l < n_layers; ++l) {
         int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
         int usum = 0;
-        for (int t = lo; t < hi_t; ++t) usum += layer_units(br, tn, t, l, counts[t], rows_per_unit);
+        for (int r = lo; r < hi_t; ++r) { const int t = tenant_at(br, l, r); usum += layer_units(br, tn, t, l, cnt[t], rows_per_unit); }
         int urun = cta_excl_scan(usum, s_warp, &total);
-        for (int t = lo; t < hi_t; ++t) { prefix[t] = urun; urun += layer_units(br, tn, t, l, counts[t], rows_per_unit); }
+        for (int r = lo; r < hi_t; ++r) {
+            const int t = tenant_at(br, l, r);
+            prefix[r] = urun;
+            urun += layer_units(br, tn, t, l, cnt[t], rows_per_unit);
+        }
         if (threadIdx.x == 0) prefix[T] = total;
     }
 }
@@ -239,27 +250,29 @@ bucket_hist_scan(const int32_t* __restrict__ ids, int n, int T, Brief br, int n_
             run += v;
         }
         counts[t] = run;
+        s_hist[t] = run;                       // the scan below reads counts by tenant rank: keep them on the SM
         own_count = run;
     }
     if (T1 > (int)blockDim.x) own_count = -1;
     else if ((int)threadIdx.x >= T1) own_count = 0;
     __syncthreads();
-    scan_buckets(T, br, n_layers, rows_per_unit, tn, counts, offsets, tile_prefix, s_warp, s_vec, own_count);
+    scan_buckets(T, br, n_layers, rows_per_unit, tn, s_hist, offsets, tile_prefix, s_warp, s_vec, own_count);
 }
 
 struct ItemPtrs { WorkItem* v[8]; };
 
 // Work item `item` of dense layer l: (tenant, row tile, column tile) and what the executor needs to know about it.
-__device__ __forceinline__ WorkItem make_work_item(int item, int l, int T, const ModelDev* __restrict__ models,
+__device__ __forceinline__ WorkItem make_work_item(int item, int l, int T, const ModelDev* __restrict__ models, Brief br,
                                                    const int32_t* __restrict__ offsets,
                                                    const int32_t* __restrict__ prefix, int tile_m) {
-    int lo = 0, hi = T;   // largest t with prefix[t] <= item
+    int lo = 0, hi = T;   // largest rank r with prefix[r] <= item
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
         if (prefix[mid] <= item) lo = mid; else hi = mid;
     }
-    const LayerDev& L = models[lo].layer[l];
-    const int seg0 = offsets[lo], n_t = offsets[lo + 1] - seg0;
+    const int t = tenant_at(br, l, lo);        // lo is a rank in the layer's cost order
+    const LayerDev& L = models[t].layer[l];
+    const int seg0 = offsets[t], n_t = offsets[t + 1] - seg0;
     const int m_tiles = (n_t + tile_m - 1) / tile_m;
     const int local = item - prefix[lo];
     // Order of a tenant's items: column tiles in groups of kColGroup, inside a group row tile by row tile.  Items in
@@ -281,7 +294,7 @@ __device__ __forceinline__ WorkItem make_work_item(int item, int l, int T, const
     w.bias = L.bias;
     w.N = L.N;
     w.relu = L.relu;
-    w.t = lo;
+    w.t = t;
     w.pad = 0;
     return w;
 }
@@ -337,16 +350,18 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
     {
         const int hi_t = min(hi, T);
         if (per == 1) {
-            // one bucket per thread: the units of all layers first, so that the loads from the tenant table are in
-            // flight together instead of one round trip per layer
-            LayerHead head[MT_MAX_LAYERS];
-            const int t_own = min(lo, T - 1);
+            // one rank per thread: tenants of that rank, their shapes and their counts for all layers together
+            const int r_own = min(lo, T - 1);
+            int t_l[MT_MAX_LAYERS];
 #pragma unroll
-            for (int l = 0; l < MT_MAX_LAYERS; ++l) head[l] = (l < n_layers) ? load_head(br, tn, t_own, l) : LayerHead{-1, 0};
-            const int c_own = (lo < hi_t) ? s_cnt[lo] : 0;
+            for (int l = 0; l < MT_MAX_LAYERS; ++l) t_l[l] = (l < n_layers) ? tenant_at(br, l, r_own) : 0;
+            LayerHead head[MT_MAX_LAYERS];
+#pragma unroll
+            for (int l = 0; l < MT_MAX_LAYERS; ++l) head[l] = (l < n_layers) ? load_head(br, tn, t_l[l], l) : LayerHead{-1, 0};
             int units[MT_MAX_LAYERS];
 #pragma unroll
-            for (int l = 0; l < MT_MAX_LAYERS; ++l) units[l] = units_of(head[l], c_own, rows_per_unit, tn.v[l], tn.m[l]);
+            for (int l = 0; l < MT_MAX_LAYERS; ++l)
+                units[l] = (l < n_layers && lo < hi_t) ? units_of(head[l], s_cnt[t_l[l]], rows_per_unit, tn.v[l], tn.m[l]) : 0;
             int urun[MT_MAX_LAYERS], utotal[MT_MAX_LAYERS];
             cta_excl_scan_vec(units, urun, utotal, s_vec, n_layers);
 #pragma unroll
@@ -359,9 +374,13 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
             for (int l = 0; l < n_layers; ++l) {
                 int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
                 int usum = 0;
-                for (int t = lo; t < hi_t; ++t) usum += layer_units(br, tn, t, l, s_cnt[t], rows_per_unit);
+                for (int r = lo; r < hi_t; ++r) { const int t = tenant_at(br, l, r); usum += layer_units(br, tn, t, l, s_cnt[t], rows_per_unit); }
                 int urun = cta_excl_scan(usum, s_warp, &total);
-                for (int t = lo; t < hi_t; ++t) { prefix[t] = urun; urun += layer_units(br, tn, t, l, s_cnt[t], rows_per_unit); }
+                for (int r = lo; r < hi_t; ++r) {
+                    const int t = tenant_at(br, l, r);
+                    prefix[r] = urun;
+                    urun += layer_units(br, tn, t, l, s_cnt[t], rows_per_unit);
+                }
                 if (threadIdx.x == 0) prefix[T] = total;
             }
         }
@@ -400,7 +419,7 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
         for (int t = threadIdx.x; t < T1; t += nthr) s_cnt[t] = prefix[t];
         __syncthreads();
         const int n_items = s_cnt[T];
-        for (int item = threadIdx.x; item < n_items; item += nthr) out[item] = make_work_item(item, l, T, models, offsets, s_cnt, tn.m[l]);
+        for (int item = threadIdx.x; item < n_items; item += nthr) out[item] = make_work_item(item, l, T, models, br, offsets, s_cnt, tn.m[l]);
         __syncthreads();
     }
 }
@@ -503,7 +522,7 @@ bucket_scatter_expand(const int32_t* __restrict__ ids, int n, int T, const Model
         __syncthreads();
         const int total = s_next[T];
         for (int item = blockIdx.x * blockDim.x + threadIdx.x; item < total; item += gridDim.x * blockDim.x)
-            out[item] = make_work_item(item, l, T, models, offsets, s_next, tn.m[l]);
+            out[item] = make_work_item(item, l, T, models, br, offsets, s_next, tn.m[l]);
         __syncthreads();
     }
 }
@@ -566,7 +585,7 @@ void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
     const size_t smem = sizeof(int32_t) * (size_t)(a.T + 1);
     LayerTileN tn;
     for (int l = 0; l < 8; ++l) { tn.v[l] = a.tile_n[l] > 0 ? a.tile_n[l] : BN; tn.m[l] = a.tile_m[l] > 0 ? a.tile_m[l] : BM; tn.kind[l] = a.kind[l]; }
-    Brief br{a.brief, a.brief_ld};
+    Brief br{a.brief, a.brief_ld, a.order};
     ItemPtrs ip;
     for (int l = 0; l < 8; ++l) ip.v[l] = a.items[l];
     // measured: one CTA wins up to a few hundred requests; beyond that its serial scatter and the item expansion

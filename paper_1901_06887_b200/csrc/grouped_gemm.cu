@@ -97,9 +97,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         bool ok = true;
         WorkItem cur = {};
         if ((int)blockIdx.x < total) cur = load_item(p.items, blockIdx.x);
-        for (int item = blockIdx.x; ok && item < total; item += gridDim.x) {
+        for (int k = 0, item = blockIdx.x; ok && item < total; ++k) {
+            const int item_next = dealt_item(k + 1, blockIdx.x, gridDim.x);
             WorkItem nxt = {};
-            if (item + (int)gridDim.x < total) nxt = load_item(p.items, item + gridDim.x);
+            if (item_next < total) nxt = load_item(p.items, item_next);
             const int kblocks = cur.k_blocks;
             const bool swap = kSwapOk && cur.rows_valid <= kSwapRows;
             const int n_g4 = swap ? ((cur.rows_valid + 31) >> 5) * 8 : 32;       // gathers (= lanes) per stage
@@ -138,6 +139,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                 if (++stage == kStages) { stage = 0; phase ^= 1u; }
             }
             cur = nxt;
+            item = item_next;
         }
     } else if (warp == 0) {
         if (lane == 0) {   // ------------------------------------------------ TMA producer
@@ -145,9 +147,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             bool ok = true;
             WorkItem cur = {};
             if ((int)blockIdx.x < total) cur = load_item(p.items, blockIdx.x);
-            for (int item = blockIdx.x; ok && item < total; item += gridDim.x) {
+            for (int k = 0, item = blockIdx.x; ok && item < total; ++k) {
+                const int item_next = dealt_item(k + 1, blockIdx.x, gridDim.x);
                 WorkItem nxt = {};
-                if (item + (int)gridDim.x < total) nxt = load_item(p.items, item + gridDim.x);   // in flight during this item
+                if (item_next < total) nxt = load_item(p.items, item_next);   // in flight during this item
                 const int kblocks = cur.k_blocks;
                 const bool swap = kSwapOk && cur.rows_valid <= kSwapRows;
                 const int nbox = (cur.rows_valid + 31) >> 5;
@@ -183,6 +186,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
                 cur = nxt;
+                item = item_next;
             }
         }
     } else if (warp == 1) {
@@ -203,9 +207,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             bool ok = true;
             int4 head = ((int)blockIdx.x < total) ? __ldg(reinterpret_cast<const int4*>(p.items + blockIdx.x)) : make_int4(0, 0, 0, 0);
             uint32_t ready = 0;
-            for (int item = blockIdx.x; ok && item < total; item += gridDim.x, ++it) {
-                const int4 next_head = (item + (int)gridDim.x < total)
-                                           ? __ldg(reinterpret_cast<const int4*>(p.items + item + gridDim.x)) : make_int4(0, 0, 0, 0);
+            for (int item = blockIdx.x; ok && item < total; ++it) {
+                const int item_next = dealt_item(it + 1, blockIdx.x, gridDim.x);
+                const int4 next_head = (item_next < total)
+                                           ? __ldg(reinterpret_cast<const int4*>(p.items + item_next)) : make_int4(0, 0, 0, 0);
                 const int kblocks = head.w;          // (row0, rows_valid, n_tile, k_blocks)
                 const bool swap = kSwapOk && head.y <= kSwapRows;
                 // transposed items: M = 128 weight rows, N = 32 or 64 request columns
@@ -248,6 +253,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                 }
                 if (ok && leader) umma_commit(tfull_bar(acc));
                 head = next_head;
+                item = item_next;
             }
         }
     } else {               // ---------------------------------------------------- epilogue (warps 2..5)
@@ -266,9 +272,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                 for (int e = threadIdx.x - 64; e < p.ld_out; e += 128) dst[e] = __int_as_float(0x7fc00000);
             }
         }
-        for (int item = blockIdx.x; item < total; item += gridDim.x, ++it) {
+        for (int item = blockIdx.x; item < total; item = dealt_item(++it, blockIdx.x, gridDim.x)) {
             WorkItem nxt = {};
-            if (item + (int)gridDim.x < total) nxt = load_item(p.items, item + gridDim.x);
+            const int item_next = dealt_item(it + 1, blockIdx.x, gridDim.x);
+            if (item_next < total) nxt = load_item(p.items, item_next);
             const WorkItem c = cur;
             cur = nxt;
             const int acc = it & 1;

@@ -98,9 +98,10 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmA
         bool ok = true;
         WorkItem cur = {};
         if (pair_id < total) cur = load_pair_item(p.items, pair_id);
-        for (int item = pair_id; ok && item < total; item += n_pairs) {
+        for (int k = 0, item = pair_id; ok && item < total; ++k) {
+            const int item_next = dealt_item(k + 1, pair_id, n_pairs);
             WorkItem nxt = {};
-            if (item + n_pairs < total) nxt = load_pair_item(p.items, item + n_pairs);
+            if (item_next < total) nxt = load_pair_item(p.items, item_next);
             const int kblocks = cur.k_blocks;
             const CUtensorMap* wmap = p.wmaps + (size_t)cur.t * MT_MAX_LAYERS + p.layer;
             const int wrow0 = (cur.n_tile * 2 + (int)rank) * kblocks * BN;
@@ -126,6 +127,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmA
                 if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
             }
             cur = nxt;
+            item = item_next;
         }
     } else if (warp == 0) {
         if (lane == 0) {   // ------------------------------------------------ TMA producer (both CTAs)
@@ -133,9 +135,10 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmA
             bool ok = true;
             WorkItem cur = {};
             if (pair_id < total) cur = load_pair_item(p.items, pair_id);
-            for (int item = pair_id; ok && item < total; item += n_pairs) {
+            for (int k = 0, item = pair_id; ok && item < total; ++k) {
+                const int item_next = dealt_item(k + 1, pair_id, n_pairs);
                 WorkItem nxt = {};
-                if (item + n_pairs < total) nxt = load_pair_item(p.items, item + n_pairs);
+                if (item_next < total) nxt = load_pair_item(p.items, item_next);
                 const int kblocks = cur.k_blocks;
                 // this CTA's half of the 256 columns: weight tile 2 * n_tile + rank, rows of the tiled image
                 const CUtensorMap* wmap = p.wmaps + (size_t)cur.t * MT_MAX_LAYERS + p.layer;
@@ -151,6 +154,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmA
                     if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
                 }
                 cur = nxt;
+                item = item_next;
             }
         }
     } else if (warp == 1) {
@@ -165,8 +169,9 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmA
             bool ok = true;
             int kblocks = (pair_id < total) ? __ldg(&p.items[pair_id].k_blocks) : 0;
             uint32_t ready = 0;
-            for (int item = pair_id; ok && item < total; item += n_pairs, ++it) {
-                const int next_kblocks = (item + n_pairs < total) ? __ldg(&p.items[item + n_pairs].k_blocks) : 0;
+            for (int item = pair_id; ok && item < total; ++it) {
+                const int item_next = dealt_item(it + 1, pair_id, n_pairs);
+                const int next_kblocks = (item_next < total) ? __ldg(&p.items[item_next].k_blocks) : 0;
                 const int acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
                 if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, 32)) break;
@@ -191,6 +196,7 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmA
                 }
                 if (ok && leader_lane) umma_commit_pair(tfull_bar(acc));   // both CTAs' epilogues may drain
                 kblocks = next_kblocks;
+                item = item_next;
             }
         }
     } else {               // ---------------------------------------------------- epilogue (warps 2..5, both CTAs)
@@ -211,9 +217,10 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmA
                 for (int e = threadIdx.x - 64; e < p.ld_out; e += 128) dst[e] = __int_as_float(0x7fc00000);
             }
         }
-        for (int item = pair_id; item < total; item += n_pairs, ++it) {
+        for (int item = pair_id; item < total; item = dealt_item(++it, pair_id, n_pairs)) {
             WorkItem nxt = {};
-            if (item + n_pairs < total) nxt = load_pair_item(p.items, item + n_pairs);
+            const int item_next = dealt_item(it + 1, pair_id, n_pairs);
+            if (item_next < total) nxt = load_pair_item(p.items, item_next);
             const WorkItem c = cur;
             cur = nxt;
             const int acc = it & 1;

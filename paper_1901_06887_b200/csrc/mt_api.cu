@@ -4,6 +4,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <climits>
 #include <cstdio>
 #include <cstring>
@@ -53,6 +54,8 @@ struct Ctx {
     std::vector<HostModel> models;
     ModelDev* d_models = nullptr;
     int32_t* d_brief = nullptr;          // [1 + MT_MAX_LAYERS][max_models]: alive, out features per layer (bucketing passes)
+    int32_t* d_order = nullptr;          // [MT_MAX_LAYERS][max_models]: per layer, tenants by descending a-priori item cost
+    bool last_pair[MT_MAX_LAYERS] = {false};   // executor form of each dense layer in the last mt_infer (balance report)
     CUtensorMap* d_wmaps = nullptr;      // [max_models][MT_MAX_LAYERS]: dense weights as 128 x 64 boxes of the tiled image
     EncodeTiledFn encode = nullptr;
 
@@ -155,6 +158,12 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     CU_OK(cudaMemset(g.d_models, 0, sizeof(ModelDev) * (size_t)max_models));
     CU_OK(cudaMalloc(&g.d_brief, sizeof(int32_t) * (size_t)(1 + MT_MAX_LAYERS) * max_models));
     CU_OK(cudaMemset(g.d_brief, 0, sizeof(int32_t) * (size_t)(1 + MT_MAX_LAYERS) * max_models));
+    CU_OK(cudaMalloc(&g.d_order, sizeof(int32_t) * (size_t)MT_MAX_LAYERS * max_models));
+    {
+        std::vector<int32_t> ident((size_t)MT_MAX_LAYERS * max_models);
+        for (size_t i = 0; i < ident.size(); ++i) ident[i] = (int32_t)(i % (size_t)max_models);
+        CU_OK(cudaMemcpy(g.d_order, ident.data(), sizeof(int32_t) * ident.size(), cudaMemcpyHostToDevice));
+    }
     CU_OK(cudaMalloc(&g.d_wmaps, sizeof(CUtensorMap) * (size_t)max_models * MT_MAX_LAYERS));
     CU_OK(cudaMalloc(&g.d_status, sizeof(int32_t) * ST_WORDS));
     CU_OK(cudaMalloc(&g.d_ticket, sizeof(int32_t)));
@@ -343,6 +352,50 @@ void recompute_tile_n() {
     }
 }
 
+// A-priori cost of one dense work item in SM cycles (Sec. 3.2: the work of a layer is fixed by its shape and known
+// before any request arrives).  Per K block of 64 the item either waits for its bytes - the rows of the weight tile
+// that hold output features plus the activation rows it fetches, at one SM's share of the HBM stream - or for the
+// tensor pipe; the larger of the two counts.  A fixed part per item covers the hand-over of the accumulator and the
+// epilogue's tail.  rows <= 64 is the transposed form (32-row activation boxes, weights on M).
+double item_cost_cycles(int k_blocks, int n_cols, int rows) {
+    if (k_blocks <= 0 || n_cols <= 0 || rows <= 0) return 0.0;
+    const double kBytesPerClk = 23.0;                 // 6.5 TB/s over 148 SMs at 1.9 GHz
+    const double kFixed = 700.0;
+    const int w_rows = (n_cols + 7) & ~7;
+    const bool swap = rows <= 64;
+    const double a_bytes = swap ? ((rows + 31) / 32) * 4096.0 : 16384.0;
+    const double bytes = w_rows * 128.0 + a_bytes;
+    const int w_tiles = (n_cols + 127) / 128;
+    // four K = 16 instructions per weight tile: N = 32/64 columns of requests when transposed, else N = 128 or 256
+    const double mma = swap ? w_tiles * 4 * (rows <= 32 ? 36.0 : 43.0) : (n_cols <= 128 ? 4 * 62.0 : 4 * 120.0);
+    const double per_kb = bytes / kBytesPerClk > mma ? bytes / kBytesPerClk : mma;
+    return kFixed + k_blocks * per_kb;
+}
+
+// Per dense layer: id slots 0 .. T-1 by descending cost of one full work item (dead slots last), ties in id order; the
+// other layers keep id order.  The bucketing passes lay the work items out in this order and the executors deal them
+// back and forth over their CTAs (longest-processing-time-first list scheduling with costs known a priori).
+mt_status recompute_order() {
+    if (!g.has_family || g.T == 0) return MT_OK;
+    std::vector<int32_t> row(g.T);
+    std::vector<double> cost(g.T);
+    for (size_t l = 0; l < g.family.size(); ++l) {
+        for (int t = 0; t < g.T; ++t) {
+            row[t] = t;
+            cost[t] = -1.0;
+            const HostModel& m = g.models[t];
+            if (g.family[l].kind == MT_DENSE && m.alive) {
+                const HostLayer& h = m.layers[l];
+                cost[t] = item_cost_cycles(h.in_ch / BK, h.out_ch < g.tile_n[l] ? h.out_ch : g.tile_n[l], BM);
+            }
+        }
+        if (g.family[l].kind == MT_DENSE)
+            std::stable_sort(row.begin(), row.end(), [&](int32_t a, int32_t b) { return cost[a] > cost[b]; });
+        CU_OK(cudaMemcpy(g.d_order + l * (size_t)g.max_models, row.data(), sizeof(int32_t) * g.T, cudaMemcpyHostToDevice));
+    }
+    return MT_OK;
+}
+
 mt_status validate_layers(const mt_layer_desc* layers, int n_layers) {
     if (!layers || n_layers < 1 || n_layers > MT_MAX_LAYERS) return n_layers > MT_MAX_LAYERS ? MT_ERR_UNSUPPORTED : MT_ERR_INVALID_ARG;
     for (int l = 0; l < n_layers; ++l) {
@@ -493,6 +546,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
     bool pair_mode[MT_MAX_LAYERS] = {false};
     const bool pair_ok = g.opt_pair && (g.sm_count >= 2) && (n / (g.live > 0 ? g.live : 1) >= 1024);
     for (int l = 0; l < L; ++l) pair_mode[l] = pair_ok && g.family[l].kind == MT_DENSE && g.tile_n[l] == 256;
+    for (int l = 0; l < MT_MAX_LAYERS; ++l) g.last_pair[l] = l < L && pair_mode[l];
     int tiles_per_image = 0;
     for (const HostLayer& f : g.family)
         if (f.kind == MT_CONV3X3) tiles_per_image = g.conv.strips_per_image;
@@ -518,7 +572,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
         Timer t(K_BUCKET, s);
         BucketArgs a;
         a.ids = ids; a.n = n; a.T = g.T; a.models = g.d_models; a.n_layers = L; a.rows_per_unit = tiles_per_image;
-        a.brief = g.d_brief; a.brief_ld = g.max_models;
+        a.brief = g.d_brief; a.brief_ld = g.max_models; a.order = g.d_order;
         for (int l = 0; l < 8; ++l) a.kind[l] = (l < L) ? g.family[l].kind : -1;
         a.ticket = g.d_ticket;
         a.rows_src = rows_in_scatter ? inputs : nullptr; a.rows_dst = g.act[0];
@@ -644,6 +698,7 @@ mt_status mt_shutdown(void) {
     free_workspace();
     cudaFree(g.d_models); g.d_models = nullptr;
     cudaFree(g.d_brief); g.d_brief = nullptr;
+    cudaFree(g.d_order); g.d_order = nullptr;
     cudaFree(g.d_wmaps); g.d_wmaps = nullptr;
     cudaFree(g.d_status); g.d_status = nullptr;
     cudaFree(g.d_ticket); g.d_ticket = nullptr;
@@ -784,6 +839,8 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
     g.live += 1;
     if (id + 1 > g.T) g.T = id + 1;
     recompute_tile_n();
+    st = recompute_order();
+    if (st != MT_OK) return st;
     *model_id_out = id;
     return MT_OK;
 }
@@ -806,7 +863,7 @@ mt_status mt_release(int32_t model_id) {
     hm.layers.clear();
     g.live -= 1;
     recompute_tile_n();
-    return MT_OK;
+    return recompute_order();
 }
 
 mt_status mt_infer(const void* inputs, const int32_t* model_ids, int32_t n, void* outputs, void* stream) {
@@ -948,6 +1005,45 @@ mt_status mt_debug_wait_timeout(int32_t limit_ms, void* stream) {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     launch_wait_timeout_probe(g.d_status, (unsigned long long)limit_ms * 1000000ull, g.d_status + 3, s);
     CU_OK(cudaGetLastError());
+    return MT_OK;
+}
+
+mt_status mt_debug_item_cost(int32_t k_blocks, int32_t n_cols, int32_t rows, double* cycles_out) {
+    if (!cycles_out || k_blocks < 0 || n_cols < 0 || rows < 0) return MT_ERR_INVALID_ARG;
+    *cycles_out = item_cost_cycles(k_blocks, n_cols, rows);
+    return MT_OK;
+}
+
+mt_status mt_debug_schedule_balance(int32_t layer, double* max_over_mean_out, int32_t* n_items_out, int32_t* n_ctas_out) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g.init) return MT_ERR_NOT_INIT;
+    if (!max_over_mean_out || layer < 0 || layer >= (int)g.family.size() || g.family[layer].kind != MT_DENSE || !g.d_items[layer])
+        return MT_ERR_INVALID_ARG;
+    CU_OK(cudaSetDevice(g.device));
+    CU_OK(cudaDeviceSynchronize());
+    int32_t n_items = 0;
+    CU_OK(cudaMemcpy(&n_items, g.d_tile_prefix + (size_t)layer * (g.T + 1) + g.T, sizeof n_items, cudaMemcpyDeviceToHost));
+    if (n_items < 0 || (size_t)n_items > g.items_cap[layer]) return MT_ERR_CUDA;
+    std::vector<WorkItem> items(n_items);
+    if (n_items) CU_OK(cudaMemcpy(items.data(), g.d_items[layer], sizeof(WorkItem) * (size_t)n_items, cudaMemcpyDeviceToHost));
+    const bool pair = g.last_pair[layer];
+    const int grid = pair ? (g.sm_count & ~1) / 2 : g.sm_count;
+    const int tn = pair ? 256 : g.tile_n[layer];
+    std::vector<double> per(grid, 0.0);
+    double sum = 0.0;
+    for (int i = 0; i < n_items; ++i) {
+        const WorkItem& w = items[i];
+        const int cols = w.N - w.n_tile * tn < tn ? w.N - w.n_tile * tn : tn;
+        const double c = item_cost_cycles(w.k_blocks, cols, w.rows_valid < BM ? w.rows_valid : BM);
+        const int k = i / grid, r = i % grid;
+        per[(k & 1) ? grid - 1 - r : r] += c;     // the executors' dealing (dealt_item)
+        sum += c;
+    }
+    double mx = 0.0;
+    for (double v : per) mx = v > mx ? v : mx;
+    *max_over_mean_out = sum > 0 ? mx / (sum / grid) : 1.0;
+    if (n_items_out) *n_items_out = n_items;
+    if (n_ctas_out) *n_ctas_out = grid;
     return MT_OK;
 }
 

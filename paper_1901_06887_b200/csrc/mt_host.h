@@ -25,6 +25,11 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 struct ModelDev;
 struct WorkItem;
 
+// Dealing of a layer's work items to the CTAs (or CTA pairs) of a persistent launch: rounds of `grid` consecutive
+// items, forwards in even rounds and backwards in odd ones.  The list is laid out heaviest items first, so a plain
+// round-robin would hand CTA 0 the largest item of every round; the back-and-forth order evens the sums out.
+__host__ __device__ inline int dealt_item(int k, int b, int grid) { return k * grid + ((k & 1) ? grid - 1 - b : b); }
+
 constexpr int kBucketChunk = 64;    // requests per CTA in the scatter pass (kHistChunk is a multiple of it)
 constexpr int kScatterThreads = 256;
 constexpr int kHistChunk = 1024;    // requests per CTA (and per row of block_hist) in the histogram pass
@@ -36,6 +41,8 @@ struct BucketArgs {
     const ModelDev* models;
     const int32_t* brief;     // compact tenant fields, rows of brief_ld ints: row 0 alive, row 1 + l out features of layer l
     int brief_ld;
+    const int32_t* order;     // rows of brief_ld ints, one per layer: tenants in the order their work items are laid out
+                              // (heaviest a-priori cost per item first for dense layers; id order for the others)
     int kind[8];              // layer kinds of the hosted family
     int n_layers;
     int rows_per_unit;        // conv: tiles per image

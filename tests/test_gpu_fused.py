@@ -168,3 +168,40 @@ def test_first_layer_reads_rows_through_perm(case, monkeypatch):
     monkeypatch.setenv("MT_PERM_GATHER", "0")
     moved, _ = run_and_check(wl.models, wl.model_ids, wl.inputs, max_models=max(64, T))
     assert np.array_equal(got, moved)
+
+
+def test_skewed_family_is_scheduled_evenly_and_matches_the_oracle():
+    # one tenant with 1024-wide layers and a quarter of the requests among thirty 128-wide ones: its work items cost
+    # eight times the others'.  Laid out heaviest first and dealt back and forth, every CTA's modelled share of a layer
+    # stays within 1.2x of the mean; the results are the oracle's whatever the order
+    rng = np.random.default_rng(77)
+    T = 31
+    models = [synth.make_mlp(9, 0, (512, 1024, 1024, 64))] + [synth.make_mlp(9, t, (512, 128, 128, 64)) for t in range(1, T)]
+    n = 30000                                          # about 4.5 work items per CTA: below that the item size itself bounds the balance
+    ids = np.where(rng.random(n) < 0.25, 0, rng.integers(1, T, n)).astype(np.int32)
+    x = bits(rng.standard_normal((n, 512)))
+    run_and_check(models, ids, x)
+    for layer, least_items in ((0, 400), (1, 400)):
+        ratio, n_items, n_ctas = mt.mt_debug_schedule_balance(layer)
+        assert n_items >= least_items and n_ctas == 148
+        assert ratio <= 1.2, (layer, ratio, n_items)
+
+
+def test_work_item_order_follows_cost_after_release_and_reregistration():
+    # ranks are recomputed whenever the set of models changes: release the heavy tenant, run, register it again
+    # under the freed id, run again - both batches match the oracle
+    rng = np.random.default_rng(78)
+    models = [synth.make_mlp(9, 100 + t, (128, 640 if t == 3 else 128, 40)) for t in range(6)]
+    fresh()
+    harness.register_models(models)
+    n = 1500
+    x = bits(rng.standard_normal((n, 128)))
+    ids = rng.integers(0, 6, n).astype(np.int32)
+    run_and_check(models, ids, x, register=False)
+    mt.mt_release(3)
+    live = ids != 3
+    got = harness.run_batch(ids, x, 40)
+    assert mt.mt_get_async_status()[0] == 2 and np.isnan(got[~live]).all()
+    assert harness.scaled_error(got[live], oracle.forward(models, ids[live], x[live])).max() <= TOL
+    assert mt.mt_register_model(models[3]) == 3
+    run_and_check(models, ids, x, register=False)
