@@ -295,7 +295,7 @@ __device__ __forceinline__ WorkItem make_work_item(int item, int l, int T, const
     w.N = L.N;
     w.relu = L.relu;
     w.t = t;
-    w.pad = 0;
+    w.flags = (l == models[t].n_layers - 1) ? kItemFinal : 0;    // models of one family may differ in depth
     return w;
 }
 

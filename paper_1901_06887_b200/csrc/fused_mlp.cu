@@ -100,7 +100,9 @@ fused_mlp_kernel(const FusedArgs p) {
                 atomicCAS(&p.status[ST_CODE], MT_OK, MT_ERR_BAD_MODEL_ID);
                 atomicMin(&p.status[ST_BAD_INDEX], i);
             }
-            const unsigned peers = __match_any_sync(__activemask(), b);
+            // (chunks are whole warps up to the batch's ragged end: the lanes with a request are lanes 0 .. n - 32c - 1)
+            const unsigned live = (n - c * 32 >= 32) ? 0xffffffffu : ((1u << (n - c * 32)) - 1u);
+            const unsigned peers = __match_any_sync(live, b);
             const int rank = __popc(peers & ((1u << lane) - 1u));
             if (rank == 0) s_chist[c * T1 + b] = __popc(peers);
             own_b[q] = b; own_rank[q] = rank;
@@ -167,7 +169,7 @@ fused_mlp_kernel(const FusedArgs p) {
         c.rows = min(BM, s_off[lo + 1] - c.j0);
         return c;
     };
-    const int L = p.n_layers;
+    // (models of one family may differ in depth: every unit runs its own tenant's number of layers)
 
     if (warp == 0) {
         if (lane == 0) {   // ------------------------------------------------ producer: weight tiles of every layer
@@ -175,6 +177,7 @@ fused_mlp_kernel(const FusedArgs p) {
             bool ok = true;
             for (int u = blockIdx.x; ok && u < total_units; u += gridDim.x) {
                 const UnitCoord c = locate(u);
+                const int L = p.models[c.t].n_layers;
                 for (int l = 0; ok && l < L; ++l) {
                     const LayerDev& Ld = p.models[c.t].layer[l];
                     const int kblocks = Ld.k_blocks, N = Ld.N;
@@ -202,6 +205,7 @@ fused_mlp_kernel(const FusedArgs p) {
         bool ok = true;
         for (int u = blockIdx.x; ok && u < total_units; u += gridDim.x) {
             const UnitCoord c = locate(u);
+            const int L = p.models[c.t].n_layers;
             for (int l = 0; ok && l < L; ++l) {
                 const LayerDev& Ld = p.models[c.t].layer[l];
                 const int kblocks = Ld.k_blocks;
@@ -246,6 +250,7 @@ fused_mlp_kernel(const FusedArgs p) {
         const int cpr = p.K0 >> 3;                  // 16-byte chunks per input row
         for (int u = blockIdx.x; ok && u < total_units; u += gridDim.x) {
             const UnitCoord c = locate(u);
+            const int L = p.models[c.t].n_layers;
             // gather the unit's rows (arrival order -> bucketed rows) into the operand buffer: row rr, chunk ch of the
             // row goes to K block ch / 8, 16-byte position (ch % 8) ^ (rr % 8) of the 128-byte swizzle row
             const uint4* src = reinterpret_cast<const uint4*>(p.inputs);

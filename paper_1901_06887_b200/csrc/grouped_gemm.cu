@@ -262,14 +262,14 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         int it = 0;
         WorkItem cur = {};
         if ((int)blockIdx.x < total) cur = load_item(p.items, blockIdx.x);
-        const int32_t* const perm = p.out_fp32 ? p.perm : nullptr;
-        const bool out_vec_ok = (p.ld_out & 3) == 0 && (reinterpret_cast<uintptr_t>(p.out) & 15) == 0;
-        if (perm) {
+        const int32_t* const perm = p.perm;
+        const bool out_vec_ok = (p.ld_final & 3) == 0 && (reinterpret_cast<uintptr_t>(p.final_out) & 15) == 0;
+        if (p.nan_fill) {
             // requests whose id was rejected sort behind every live segment and get no work item: NaN rows
             const int n_valid = p.offsets[p.T], n_all = p.offsets[p.T + 1];
             for (int j = n_valid + blockIdx.x; j < n_all; j += gridDim.x) {
-                float* dst = reinterpret_cast<float*>(p.out) + (size_t)perm[j] * p.ld_out;
-                for (int e = threadIdx.x - 64; e < p.ld_out; e += 128) dst[e] = __int_as_float(0x7fc00000);
+                float* dst = p.final_out + (size_t)perm[j] * p.ld_final;
+                for (int e = threadIdx.x - 64; e < p.ld_final; e += 128) dst[e] = __int_as_float(0x7fc00000);
             }
         }
         for (int item = blockIdx.x; item < total; item = dealt_item(++it, blockIdx.x, gridDim.x)) {
@@ -283,6 +283,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 4)) break;
             tc_fence_after();
             const int N = c.N, relu = c.relu;
+            const bool fin = (c.flags & kItemFinal) != 0;      // this tenant's last layer: fp32 rows to arrival order
             if (kSwapOk && c.rows_valid <= kSwapRows) {
                 // Transposed item: this thread owns output feature f, the accumulator columns are the requests.
                 // For one request the 32 lanes of a warp write 32 neighbouring features: a 64- or 128-byte run.
@@ -300,7 +301,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                         // output row of request j: its bucketed row, or (last layer) its arrival index - fetched by
                         // lane j once and handed round by shuffle
                         int my_row = row_b + lane;
-                        if (perm && lane < n_req) my_row = __ldg(perm + row_b + lane);
+                        if (fin && lane < n_req) my_row = __ldg(perm + row_b + lane);
                         tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccCols + wt * kSwapRows + b * 32, v);
                         tmem_ld_wait();
 #pragma unroll
@@ -309,7 +310,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                             if (f_ok && j < n_req) {
                                 float val = __uint_as_float(v[j]) + bias_f;
                                 if (relu) val = fmaxf(val, 0.0f);
-                                if (p.out_fp32) reinterpret_cast<float*>(p.out)[orow * p.ld_out + f] = val;
+                                if (fin) p.final_out[orow * p.ld_final + f] = val;
                                 else reinterpret_cast<uint16_t*>(p.out)[orow * p.ld_out + f] =
                                          static_cast<uint16_t>(pack_bf16x2(val, 0.0f) & 0xFFFFu);
                             }
@@ -322,7 +323,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                 continue;
             }
             const bool row_ok = r < c.rows_valid;
-            const size_t grow = (perm && row_ok) ? (size_t)__ldg(perm + c.row0 + r) : (size_t)(c.row0 + r);
+            const size_t grow = (fin && row_ok) ? (size_t)__ldg(perm + c.row0 + r) : (size_t)(c.row0 + r);
 #pragma unroll 1
             for (int ch = 0; ch < TN / 32; ++ch) {
                 uint32_t v[32];
@@ -348,8 +349,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                 const bool full_chunk = (n0 + 32 <= N);
                 if (!row_ok) {
                     // rows past the tenant's segment belong to someone else: never stored
-                } else if (p.out_fp32) {
-                    float* dst = reinterpret_cast<float*>(p.out) + grow * p.ld_out + n0;
+                } else if (fin) {
+                    float* dst = p.final_out + grow * p.ld_final + n0;
                     if (full_chunk && out_vec_ok) {
 #pragma unroll
                         for (int j = 0; j < 8; ++j)

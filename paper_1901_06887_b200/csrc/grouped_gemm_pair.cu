@@ -207,14 +207,14 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmA
         WorkItem cur = {};
         if (pair_id < total) cur = load_pair_item(p.items, pair_id);
         // last layer: rows go straight to their arrival positions in the caller's buffer (see GemmArgs::perm)
-        const int32_t* const perm = p.out_fp32 ? p.perm : nullptr;
-        const bool out_vec_ok = (p.ld_out & 3) == 0 && (reinterpret_cast<uintptr_t>(p.out) & 15) == 0;
-        if (perm) {
+        const int32_t* const perm = p.perm;
+        const bool out_vec_ok = (p.ld_final & 3) == 0 && (reinterpret_cast<uintptr_t>(p.final_out) & 15) == 0;
+        if (p.nan_fill) {
             // requests whose id was rejected sort behind every live segment and get no work item: NaN rows
             const int n_valid = p.offsets[p.T], n_all = p.offsets[p.T + 1];
             for (int j = n_valid + blockIdx.x; j < n_all; j += gridDim.x) {
-                float* dst = reinterpret_cast<float*>(p.out) + (size_t)perm[j] * p.ld_out;
-                for (int e = threadIdx.x - 64; e < p.ld_out; e += 128) dst[e] = __int_as_float(0x7fc00000);
+                float* dst = p.final_out + (size_t)perm[j] * p.ld_final;
+                for (int e = threadIdx.x - 64; e < p.ld_final; e += 128) dst[e] = __int_as_float(0x7fc00000);
             }
         }
         for (int item = pair_id; item < total; item = dealt_item(++it, pair_id, n_pairs)) {
@@ -228,9 +228,10 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmA
             if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 35)) break;
             tc_fence_after();
             const int N = c.N, relu = c.relu;
+            const bool fin = (c.flags & kItemFinal) != 0;      // this tenant's last layer: fp32 rows to arrival order
             const int my_valid = min(BM, max(0, c.rows_valid - (int)rank * BM));
             const bool row_ok = r < my_valid;
-            const size_t grow = (perm && row_ok) ? (size_t)__ldg(perm + c.row0 + (int)rank * BM + r)
+            const size_t grow = (fin && row_ok) ? (size_t)__ldg(perm + c.row0 + (int)rank * BM + r)
                                                  : (size_t)(c.row0 + (int)rank * BM + r);
 #pragma unroll 1
             for (int ch = 0; ch < kPairTN / 32; ++ch) {
@@ -257,8 +258,8 @@ grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const GemmA
                 const bool full_chunk = (n0 + 32 <= N);
                 if (!row_ok) {
                     // rows past the tenant's segment belong to someone else: never stored
-                } else if (p.out_fp32) {
-                    float* dst = reinterpret_cast<float*>(p.out) + grow * p.ld_out + n0;
+                } else if (fin) {
+                    float* dst = p.final_out + grow * p.ld_final + n0;
                     if (full_chunk && out_vec_ok) {
 #pragma unroll
                         for (int j = 0; j < 8; ++j)

@@ -310,7 +310,7 @@ mt_status ensure_workspace(int n) {
     // work items of the dense layers: at most (row tiles + one ragged tile per tenant) x column tiles of the widest model
     for (int l = 0; l < L; ++l) {
         if (g.family[l].kind != MT_DENSE) continue;
-        const int out_w = (l + 1 < L) ? g.width[l + 1] : g.out_elems;
+        const int out_w = std::max((l + 1 < L) ? g.width[l + 1] : 0, g.out_elems);   // hidden, or some tenant's last layer
         const size_t col_tiles = (size_t)(out_w + BN - 1) / BN;    // bound for either tile width
         g.items_cap[l] = ((size_t)cap / BM + (size_t)g.max_models + 1) * col_tiles;
         CU_OK(cudaMalloc(&g.d_items[l], sizeof(WorkItem) * g.items_cap[l]));
@@ -347,7 +347,7 @@ void recompute_tile_n() {
         if (g.family[l].kind != MT_DENSE) continue;
         int min_n = INT_MAX;
         for (const HostModel& m : g.models)
-            if (m.alive && m.layers[l].out_ch < min_n) min_n = m.layers[l].out_ch;
+            if (m.alive && l < m.layers.size() && m.layers[l].out_ch < min_n) min_n = m.layers[l].out_ch;
         g.tile_n[l] = (min_n != INT_MAX && min_n >= 256) ? 256 : BN;
     }
 }
@@ -384,7 +384,7 @@ mt_status recompute_order() {
             row[t] = t;
             cost[t] = -1.0;
             const HostModel& m = g.models[t];
-            if (g.family[l].kind == MT_DENSE && m.alive) {
+            if (g.family[l].kind == MT_DENSE && m.alive && l < m.layers.size()) {
                 const HostLayer& h = m.layers[l];
                 cost[t] = item_cost_cycles(h.in_ch / BK, h.out_ch < g.tile_n[l] ? h.out_ch : g.tile_n[l], BM);
             }
@@ -429,15 +429,25 @@ mt_status validate_layers(const mt_layer_desc* layers, int n_layers) {
 
 int layer_in_elems(const HostLayer& l) { return l.kind == MT_DENSE ? l.in_ch : l.in_ch * l.h * l.w; }
 
+bool all_dense(const std::vector<HostLayer>& m) {
+    for (const HostLayer& l : m)
+        if (l.kind != MT_DENSE) return false;
+    return true;
+}
+
+// What the models of one context share: input and output element counts, and the layer kinds index by index.  MLPs
+// (dense layers only) may differ in depth and in hidden widths; a tenant's layer j runs in the family's j-th launch
+// and its last layer, whichever launch that is, writes the output.  Conv families keep one depth and geometry.
 mt_status check_family(const std::vector<HostLayer>& m) {
     if (!g.has_family || g.live == 0) return MT_OK;
+    if (layer_in_elems(m[0]) != g.in_elems || m.back().out_ch != g.out_elems) return MT_ERR_SHAPE;
+    if (all_dense(m) && all_dense(g.family)) return MT_OK;
     if (m.size() != g.family.size()) return MT_ERR_SHAPE;
     for (size_t l = 0; l < m.size(); ++l) {
         const HostLayer &a = m[l], &f = g.family[l];
         if (a.kind != f.kind) return MT_ERR_SHAPE;
         if (a.kind != MT_DENSE && (a.in_ch != f.in_ch || a.out_ch != f.out_ch || a.h != f.h || a.w != f.w)) return MT_ERR_SHAPE;
     }
-    if (layer_in_elems(m[0]) != g.in_elems || m.back().out_ch != g.out_elems) return MT_ERR_SHAPE;
     return MT_OK;
 }
 
@@ -625,12 +635,14 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             a.tile_prefix = g.d_tile_prefix + (size_t)l * (g.T + 1);
             a.items = g.d_items[l];
             a.wmaps = g.d_wmaps; a.layer = l;
-            // the last layer writes straight into the caller's buffer in arrival order
-            const bool direct = last;
-            a.out = last ? outputs : g.act[l + 1];
-            a.ld_out = last ? g.out_elems : g.act_ld[l + 1];
-            a.out_fp32 = last ? 1 : 0;
-            a.perm = direct ? g.d_perm : nullptr;
+            // a tenant's last layer (any launch, for a family of mixed depths) writes straight into the caller's buffer in
+            // arrival order; the family's deepest launch also fills the rows of rejected requests
+            a.out = last ? nullptr : g.act[l + 1];
+            a.ld_out = last ? 0 : g.act_ld[l + 1];
+            a.final_out = static_cast<float*>(outputs);
+            a.ld_final = g.out_elems;
+            a.nan_fill = last ? 1 : 0;
+            a.perm = g.d_perm;
             a.offsets = g.d_offsets;
             a.status = g.d_status;
             const bool gather = (l == 0) && perm_gather;
@@ -805,8 +817,8 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
         e = cudaMemcpy(g.d_wmaps + (size_t)id * MT_MAX_LAYERS + l, &wm, sizeof wm, cudaMemcpyHostToDevice);
     }
     if (e == cudaSuccess) e = cudaMemcpy(g.d_models + id, &md, sizeof md, cudaMemcpyHostToDevice);
-    for (int r = 0; r <= n_layers && e == cudaSuccess; ++r) {      // the compact copy: alive, then out features per layer
-        const int32_t v = (r == 0) ? 1 : hl[r - 1].out_ch;
+    for (int r = 0; r <= MT_MAX_LAYERS && e == cudaSuccess; ++r) {   // the compact copy: alive, then out features per layer
+        const int32_t v = (r == 0) ? 1 : (r <= n_layers ? hl[r - 1].out_ch : 0);   // 0: the model has no such layer
         e = cudaMemcpy(g.d_brief + (size_t)r * g.max_models + id, &v, sizeof v, cudaMemcpyHostToDevice);
     }
     if (raw_dev) cudaFree(raw_dev);
@@ -827,6 +839,10 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
         g.ws_dirty = true;
         g.in_map_ptr = nullptr;
         free_staging();   // sized for the previous family's rows (no model is live: nothing is in flight)
+    }
+    if ((size_t)n_layers > g.family.size()) {      // a deeper MLP joins: the family gains launches
+        for (size_t l = g.family.size(); l < (size_t)n_layers; ++l) g.family.push_back(hl[l]);
+        g.ws_dirty = true;
     }
     for (int l = 0; l < n_layers; ++l) {
         const int wd = layer_in_elems(hl[l]);

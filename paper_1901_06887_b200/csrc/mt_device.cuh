@@ -43,8 +43,9 @@ struct __align__(16) WorkItem {
     int32_t N;           // tenant's out features
     int32_t relu;
     int32_t t;           // tenant (model id)
-    int32_t pad;
+    int32_t flags;       // bit 0: this is the tenant's LAST layer - fp32 rows go to the caller's buffer in arrival order
 };
+constexpr int32_t kItemFinal = 1;
 
 // Sticky status word written by kernels: [0] status code, [1] first bad arrival index, [2] where a wait gave up.
 enum { ST_CODE = 0, ST_BAD_INDEX = 1, ST_WHERE = 2, ST_WORDS = 4 };

@@ -87,12 +87,16 @@ struct GemmArgs {
     const WorkItem* items;        // the layer's work items
     const CUtensorMap* wmaps;     // [model][MT_MAX_LAYERS] tensor maps of the tiled dense weights (CTA-pair executor)
     int layer;
-    void* out;                    // bf16 or fp32, rows in bucketed order
-    int ld_out;                   // elements between output rows
-    int out_fp32;
-    // Last layer only (out_fp32): non-null perm sends bucketed row j straight to row perm[j] of `out` (the caller's
-    // buffer, arrival order), and the rows of rejected requests, bucketed rows [offsets[T], offsets[T + 1]), are
-    // filled with NaN by the same launch - no separate un-permute pass.
+    void* out;                    // bf16 hidden activations of the next layer, rows in bucketed order (may be null
+                                  // when every item of the launch is a tenant's last layer)
+    int ld_out;                   // elements between rows of `out`
+    // Items flagged kItemFinal (the tenant's last layer; models of a family may differ in depth, so any launch can
+    // hold some) write fp32 rows straight to row perm[j] of final_out, the caller's buffer in arrival order - there
+    // is no separate un-permute pass.  The launch with nan_fill set (the family's deepest layer) also fills the rows of
+    // rejected requests, bucketed rows [offsets[T], offsets[T + 1]), with NaN.
+    float* final_out;
+    int ld_final;
+    int nan_fill;
     const int32_t* perm;
     const int32_t* offsets;       // [T + 2]
     // First layer only: non-null gather_perm makes the executor read its input rows from the caller's buffer (arrival

@@ -1,0 +1,92 @@
+"""Families of mixed depth: MLP tenants with two, three and four layers (and differing hidden widths) share one
+context and one batch (the paper's catalogue of models is not uniform: Sec. 3.1 describes models as lists of
+standard layers of any length).  A tenant's layer j runs in the family's j-th launch; its last layer - whichever
+launch that is - writes the fp32 output in arrival order.  Checked against the per-request oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1901_06887_b200 import binding as mt, harness, synth
+
+from gpu_util import TOL, fresh, run_and_check
+
+pytestmark = pytest.mark.gpu
+
+
+def bits(a):
+    return synth.f32_to_bf16_bits(np.asarray(a, np.float32))
+
+
+def mixed_models(k_in, n_out, hidden_choices, T, seed, depths=(2, 3, 4, 1)):
+    rng = np.random.default_rng(seed)
+    models = []
+    for t in range(T):
+        d = depths[t % len(depths)]
+        widths = (k_in,) + tuple(int(rng.choice(hidden_choices)) for _ in range(d - 1)) + (n_out,)
+        models.append(synth.make_mlp(11, 1000 * seed + t, widths))
+    return models
+
+
+def test_mixed_depths_small_batch_both_paths(small_batch_path):
+    # at most 512 requests, layers at most 256 wide: one fused launch (or, with MT_FUSED=0, the layer-by-layer path)
+    models = mixed_models(128, 24, [64, 128, 192, 256], 9, 1)
+    assert sorted({len(m) for m in models}) == [1, 2, 3, 4]
+    rng = np.random.default_rng(5)
+    n = 400
+    ids = rng.integers(0, 9, n).astype(np.int32)
+    run_and_check(models, ids, bits(rng.standard_normal((n, 128))))
+
+
+@pytest.mark.parametrize("n,T,hidden", [(3000, 12, [128, 320, 512]), (9000, 5, [256, 512]), (700, 40, [64, 640])])
+def test_mixed_depths_layered_path(n, T, hidden):
+    # segments from a handful of requests (transposed items) to thousands (full tiles); 128- and 256-column work items
+    models = mixed_models(256, 72, hidden, T, 2 + T)
+    ids = synth.zipf_ids(3, n, T, 1.0, salt=T)
+    rng = np.random.default_rng(n)
+    got, _ = run_and_check(models, ids, bits(rng.standard_normal((n, 256))))
+    # the order of registration must not matter: deepest model last, so the family grows while models are added
+    order = np.argsort([len(m) for m in models], kind="stable")
+    remap = np.empty(T, np.int32)
+    remap[order] = np.arange(T, dtype=np.int32)
+    got2, _ = run_and_check([models[i] for i in order], remap[ids], bits(np.random.default_rng(n).standard_normal((n, 256))))
+    assert np.array_equal(got, got2)
+
+
+def test_mixed_depths_cta_pair_executor_and_rejected_ids():
+    # two tenants with thousands of requests each and layers at least 256 wide: the 256 x 256 CTA-pair executor; one
+    # tenant stops after two layers, the other after three; two ids are never issued
+    m2 = synth.make_mlp(11, 50, (256, 512, 256))
+    m3 = synth.make_mlp(11, 51, (256, 512, 256, 256))
+    rng = np.random.default_rng(8)
+    n = 2600
+    ids = rng.integers(0, 2, n).astype(np.int32)
+    ids[[7, 2000]] = 5
+    x = bits(rng.standard_normal((n, 256)))
+    fresh()
+    harness.register_models([m2, m3])
+    got = harness.run_batch(ids, x, 256)
+    assert mt.mt_get_async_status() == (2, 7)
+    good = ids < 2
+    assert np.isnan(got[~good]).all()
+    ref = oracle.forward([m2, m3], ids[good], x[good])
+    assert np.isfinite(got[good]).all() and harness.scaled_error(got[good], ref).max() <= TOL
+
+
+def test_a_family_still_needs_one_input_and_output_shape():
+    fresh()
+    assert mt.mt_register_model(synth.make_mlp(11, 0, (64, 128, 10))) == 0
+    assert mt.mt_register_model(synth.make_mlp(11, 1, (64, 10))) == 1                  # shallower: accepted
+    assert mt.mt_register_model(synth.make_mlp(11, 2, (64, 64, 64, 64, 10))) == 2      # deeper: accepted
+    for widths in ((128, 128, 10), (64, 128, 12)):
+        with pytest.raises(mt.MtError) as e:
+            mt.mt_register_model(synth.make_mlp(11, 3, widths))
+        assert e.value.code == 3
+    # conv families keep one depth
+    fresh()
+    wl = synth.make_workload(4, n=4, n_tenants=1, h=8, w=8, n_conv=2)
+    assert mt.mt_register_model(wl.models[0]) == 0
+    deeper = synth.make_workload(4, n=4, n_tenants=1, h=8, w=8, n_conv=3).models[0]
+    with pytest.raises(mt.MtError) as e:
+        mt.mt_register_model(deeper)
+    assert e.value.code == 3
