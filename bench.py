@@ -54,10 +54,6 @@ REFERENCE_SAMPLE = {1: 64, 2: 512, 3: 4096, 4: 6, 5: 24}
 # weights of the tenants that have requests, as the algorithmic bytes do); "bytes": measured at full size, per step.
 # An entry is deleted when its kernel changes and comes back with the next capture.
 TRAFFIC = {
-    2: {"ratio": 0.995, "source": "profiles/grouped_gemm_c2_reduced_ncu_full.md (16 tenants, 1024 requests: 841.5 MB "
-                                  "measured / 845.8 MB algorithmic), scaled by algorithmic bytes"},
-    3: {"ratio": 1.02, "source": "profiles/grouped_gemm128_c3_reduced_ncu_full.md (250 tenants, 4096 requests), scaled "
-                                 "by algorithmic bytes"},
     4: {"bytes": 608.5e6, "source": "profiles/grouped_conv3x3_pair_c4_full_ncu_full.md (full size, four conv launches)"},
 }
 
@@ -261,6 +257,86 @@ def run_reference(args, rank, world):
     line["cpu_baseline"] = {"value": line["value"], "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
                             "sample": "first %d of %d requests per step, %d steps" % (n_s, wl.n, steps)}
     line["e2e"] = {"value": line["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+    print(json.dumps(line), flush=True)
+
+
+def run_cache_sweep(args, ctx):
+    """Weight-residency leg (the paper's Sec. 3.3 argument with this machine's numbers): workload 2's 64 tenants behind a
+    device cache of a fraction of their total size, small batches through mt_infer_host_async on two streams; per
+    fraction the request-level hit ratio, requests/s, bytes copied per step, and the time the copies alone would take
+    at the PCIe rate measured in the same run."""
+    torch, mt, harness = ctx["torch"], ctx["mt"], ctx["harness"]
+    cfg = 2
+    nb = args.requests or 64
+    models = synth.make_models(cfg)
+    n_batches = 48
+    batches = [synth.make_requests(cfg, models, n=nb, salt=500 + b) for b in range(n_batches)]
+    out_elems = models[0][-1].out_ch
+    h_in = [torch.from_numpy(x.view(np.int16)).pin_memory() for _, x in batches]
+    h_ids = [torch.from_numpy(i).pin_memory() for i, _ in batches]
+    h_outs = [torch.empty((nb, out_elems), dtype=torch.float32).pin_memory() for _ in range(2)]
+    two = [torch.cuda.Stream(), torch.cuda.Stream()]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # PCIe rate of this box: one 256 MB pinned host -> device copy, best of 5
+    probe_h = torch.empty(256 << 20, dtype=torch.uint8).pin_memory()
+    probe_d = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    pcie = 0.0
+    for _ in range(5):
+        e0.record(); probe_d.copy_(probe_h, non_blocking=True); e1.record(); torch.cuda.synchronize()
+        pcie = max(pcie, (256 << 20) / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    del probe_h, probe_d
+    rows = []
+    block = None
+    for frac in (1.0, 0.97, 0.94, 0.9, 0.8, 0.7, 0.6, 0.5):
+        mt.mt_shutdown()
+        mt.mt_init(ctx["local_rank"], 64, nb)
+        if block is None:      # size of one tenant's block: register one model under a generous cache and read the counter
+            mt.mt_set_cache_bytes(1 << 30)
+            mt.mt_register_model(models[0])
+            block = mt.mt_get_cache_stats()["bytes_loaded"]
+            mt.mt_shutdown()
+            mt.mt_init(ctx["local_rank"], 64, nb)
+        cap = int(frac * len(models) * block) + (1 << 20)
+        mt.mt_set_cache_bytes(cap)
+        harness.register_models(models)
+
+        def step(i):
+            b = i % n_batches
+            mt.mt_infer_host_async(h_in[b], h_ids[b], nb, h_outs[i % 2], two[i % 2])
+
+        try:
+            for i in range(n_batches):       # one pass over all batches warms the cache into its steady state
+                step(i)
+            torch.cuda.synchronize()
+            mt.mt_get_cache_stats(reset=True)
+            steps = 4 * n_batches
+            e0.record(two[0])
+            for i in range(steps):
+                step(i)
+            two[0].wait_stream(two[1])
+            e1.record(two[0])
+            torch.cuda.synchronize()
+        except mt.MtError as err:
+            rows.append({"cache_fraction": frac, "error": str(err)})
+            continue
+        ms = e0.elapsed_time(e1)
+        st = mt.mt_get_cache_stats()
+        if mt.mt_get_async_status() != (0, -1):
+            raise SystemExit("device status in the cache sweep")
+        req = st["request_hits"] + st["request_misses"]
+        ten = st["tenant_hits"] + st["tenant_misses"]
+        rows.append({"cache_fraction": frac, "cache_bytes": cap,
+                     "request_hit_ratio": st["request_hits"] / max(req, 1), "tenant_hit_ratio": st["tenant_hits"] / max(ten, 1),
+                     "requests_per_s": nb * steps / (ms * 1e-3), "ms_per_step": ms / steps,
+                     "h2d_weight_bytes_per_step": st["bytes_loaded"] / steps,
+                     "pcie_ms_per_step_for_the_misses": st["bytes_loaded"] / steps / (pcie * 1e9) * 1e3,
+                     "evictions_per_step": st["evictions"] / steps})
+    mt.mt_shutdown()
+    full = rows[0]
+    line = {"cache_sweep": rows, "workload": synth.CONFIG_NAMES[cfg] + ", batches of %d requests" % nb,
+            "tenant_block_bytes": block, "pcie_h2d_gbs": pcie,
+            "note": "a miss copies one tenant's %.1f MB block: %.2f ms at the PCIe rate, against %.3f ms for a whole batch "
+                    "with every tenant resident" % (block / 1e6, block / (pcie * 1e9) * 1e3, full.get("ms_per_step", 0.0))}
     print(json.dumps(line), flush=True)
 
 
@@ -502,6 +578,8 @@ def main():
     ap.add_argument("--tenants", type=int, default=None, help="reduced case: number of tenants (profiling captures)")
     ap.add_argument("--requests", type=int, default=None, help="reduced case: requests per batch")
     ap.add_argument("--profile", action="store_true", help="timed loop only (no e2e, CPU baseline or clock sampler)")
+    ap.add_argument("--cache-sweep", action="store_true", help="weight-residency leg: workload 2 behind a device cache "
+                    "of 40-100 %% of its weights (prints its own JSON line)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -524,6 +602,10 @@ def main():
     ctx = dict(torch=torch, dist=dist, mt=mt, harness=harness, rank=rank, world=world, local_rank=local_rank,
                peaks=peaks, peaks_kind=peaks_kind)
 
+    if args.cache_sweep:
+        if rank == 0:
+            run_cache_sweep(args, ctx)
+        return
     head_cfg = args.config or HEADLINE_CONFIG
     line = measure_config(head_cfg, args, ctx)
     reduced = bool(args.tenants or args.requests or args.profile)

@@ -39,7 +39,8 @@ typedef enum {
     MT_ERR_CUDA = 6,          /* a CUDA runtime/driver call failed */
     MT_ERR_ARCH = 7,          /* device is not sm_100 */
     MT_ERR_TIMEOUT = 8,       /* (async) a bounded device-side wait gave up */
-    MT_ERR_NOT_INIT = 9
+    MT_ERR_NOT_INIT = 9,
+    MT_ERR_NOT_RESIDENT = 10  /* (async) a request names a registered model whose weights are not on the device now */
 } mt_status;
 
 typedef enum { MT_DENSE = 0, MT_CONV3X3 = 1, MT_GLOBAL_AVG_POOL = 2 } mt_layer_kind;
@@ -117,9 +118,50 @@ mt_status mt_infer_host_async(const void* inputs_host, const int32_t* model_ids_
  * an mt_infer in flight.  The id may be re-issued by a later mt_register_model. */
 mt_status mt_release(int32_t model_id);
 
+/* Weight residency (Sec. 3.3: weights are cached at every level of the memory hierarchy; a model's footprint is fixed,
+ * so the time to bring it in is predictable, and GPU memory need only hold the models in demand).  By default every
+ * registered model stays on the device.  mt_set_cache_bytes(B), called after mt_init while no model is registered,
+ * switches to a cache of B device bytes (one arena, allocated once; 0 switches back): registration then also keeps the
+ * model's block - weights in the executor's layout and biases - in pinned host memory, and the device holds the least
+ * recently used subset that fits.  MT_ERR_OOM: the arena cannot be allocated; a model larger than B is refused at
+ * registration with MT_ERR_OOM.
+ *
+ * Who decides what is resident:
+ *   mt_infer_host / mt_infer_host_async  read the batch's ids on the host and bring in exactly its tenants: blocks
+ *       missing on the device are copied from their host images on an internal stream (over least-recently-used
+ *       blocks if need be; blocks of this batch are never victims), the batch waits for the copies only, and copies
+ *       for the next batch run under the kernels of the current one.  MT_ERR_OOM (nothing enqueued) if the batch's
+ *       tenants do not fit the cache together.
+ *   mt_prefetch(ids, count, stream)       the same for a caller that keeps ids on the device: name the tenants of the
+ *       coming batch(es) (host array, duplicates allowed); work later enqueued on `stream` sees them resident.
+ *       MT_ERR_BAD_MODEL_ID for an id that is not live, MT_ERR_OOM if the set does not fit.
+ *   mt_infer                              never loads: a request for a registered but evicted model gets a NaN row and
+ *       the sticky status MT_ERR_NOT_RESIDENT (see mt_get_async_status); all other requests complete.
+ * A block that comes back is the same bytes as before, so outputs are bit-identical across evictions.
+ * mt_get_cache_stats fills the counters since the cache was set up (or since the last call with reset != 0). */
+typedef struct {
+    uint64_t capacity_bytes, resident_bytes;
+    uint64_t tenant_hits, tenant_misses;       /* per (batch or prefetch, tenant): block already there / had to be copied */
+    uint64_t request_hits, request_misses;     /* the same weighted by the tenant's requests in the batch (host-id entry points) */
+    uint64_t evictions, bytes_loaded;          /* blocks displaced; bytes copied host -> device for misses (registration included) */
+} mt_cache_stats;
+mt_status mt_set_cache_bytes(size_t device_bytes);
+mt_status mt_prefetch(const int32_t* model_ids_host, int32_t count, void* stream);
+mt_status mt_get_cache_stats(mt_cache_stats* out, int32_t reset);
+
+/* The cache's policy by itself - first-fit arena, least-recently-used eviction on a clock the caller makes up - for
+ * tests without a GPU.  access: result 0 = hit, 1 = placed (ids evicted to make room in evicted_out, at most
+ * evicted_cap of them, their number in *n_evicted_out), -1 = does not fit beside the blocks touched at `tick`. */
+mt_status mt_cache_sim_create(size_t capacity_bytes, void** sim_out);
+mt_status mt_cache_sim_access(void* sim, int32_t id, size_t bytes, uint64_t tick, int32_t* result_out, int64_t* offset_out,
+                              int32_t* evicted_out, int32_t evicted_cap, int32_t* n_evicted_out);
+mt_status mt_cache_sim_release(void* sim, int32_t id);
+mt_status mt_cache_sim_stats(void* sim, mt_cache_stats* out);
+mt_status mt_cache_sim_destroy(void* sim);
+
 /* Synchronise `stream`, then report and clear the sticky device-side status of the calls so far:
- * *status_out is MT_OK, MT_ERR_BAD_MODEL_ID (with the smallest offending arrival index of the first
- * such batch in *bad_request_index_out, else -1) or MT_ERR_TIMEOUT.  Either out pointer may be NULL. */
+ * *status_out is MT_OK, MT_ERR_BAD_MODEL_ID or MT_ERR_NOT_RESIDENT (with the smallest offending arrival index of the
+ * first such batch in *bad_request_index_out, else -1) or MT_ERR_TIMEOUT.  Either out pointer may be NULL. */
 mt_status mt_get_async_status(void* stream, int32_t* status_out, int32_t* bad_request_index_out);
 
 const char* mt_status_string(mt_status s);

@@ -18,18 +18,27 @@ LIB_PATH = os.path.join(_HERE, "libmt.so")
 MT_OK = 0
 STATUS_NAMES = {0: "MT_OK", 1: "MT_ERR_INVALID_ARG", 2: "MT_ERR_BAD_MODEL_ID", 3: "MT_ERR_SHAPE",
                 4: "MT_ERR_UNSUPPORTED", 5: "MT_ERR_OOM", 6: "MT_ERR_CUDA", 7: "MT_ERR_ARCH",
-                8: "MT_ERR_TIMEOUT", 9: "MT_ERR_NOT_INIT"}
+                8: "MT_ERR_TIMEOUT", 9: "MT_ERR_NOT_INIT", 10: "MT_ERR_NOT_RESIDENT"}
 
 EXPORTS = ["mt_init", "mt_shutdown", "mt_register_model", "mt_infer", "mt_infer_host", "mt_infer_host_async", "mt_release",
            "mt_get_async_status", "mt_status_string", "mt_debug_last_bucketing", "mt_set_kernel_timing",
            "mt_get_kernel_times", "mt_bucket_noalloc", "mt_debug_wait_timeout", "mt_debug_launch_count", "mt_debug_set_option", "mt_debug_empty_launches", "mt_debug_item_cost",
-           "mt_debug_schedule_balance"]
+           "mt_debug_schedule_balance", "mt_set_cache_bytes", "mt_prefetch", "mt_get_cache_stats", "mt_cache_sim_create",
+           "mt_cache_sim_access", "mt_cache_sim_release", "mt_cache_sim_stats", "mt_cache_sim_destroy"]
 
 
 class MtError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = int(code)
         super().__init__("%s failed: %s (%d)" % (where, STATUS_NAMES.get(int(code), "?"), int(code)))
+
+
+class CacheStats(ctypes.Structure):
+    _fields_ = [(k, ctypes.c_uint64) for k in ("capacity_bytes", "resident_bytes", "tenant_hits", "tenant_misses",
+                                               "request_hits", "request_misses", "evictions", "bytes_loaded")]
+
+    def as_dict(self):
+        return {k: int(getattr(self, k)) for k, _ in self._fields_}
 
 
 class LayerDesc(ctypes.Structure):
@@ -68,6 +77,15 @@ def lib() -> ctypes.CDLL:
         l.mt_debug_launch_count.argtypes = [ctypes.POINTER(ctypes.c_int64)]
         l.mt_debug_set_option.argtypes = [ctypes.c_char_p, i32]
         l.mt_debug_empty_launches.argtypes = [i32, vp]
+        l.mt_set_cache_bytes.argtypes = [ctypes.c_size_t]
+        l.mt_prefetch.argtypes = [vp, i32, vp]
+        l.mt_get_cache_stats.argtypes = [ctypes.POINTER(CacheStats), i32]
+        l.mt_cache_sim_create.argtypes = [ctypes.c_size_t, ctypes.POINTER(vp)]
+        l.mt_cache_sim_access.argtypes = [vp, i32, ctypes.c_size_t, ctypes.c_uint64, ctypes.POINTER(i32),
+                                          ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(i32), i32, ctypes.POINTER(i32)]
+        l.mt_cache_sim_release.argtypes = [vp, i32]
+        l.mt_cache_sim_stats.argtypes = [vp, ctypes.POINTER(CacheStats)]
+        l.mt_cache_sim_destroy.argtypes = [vp]
         l.mt_debug_item_cost.argtypes = [i32, i32, i32, ctypes.POINTER(ctypes.c_double)]
         l.mt_debug_schedule_balance.argtypes = [i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i32), ctypes.POINTER(i32)]
         for name in EXPORTS:
@@ -178,6 +196,53 @@ def mt_debug_launch_count() -> int:
     c = ctypes.c_int64(0)
     _check(lib().mt_debug_launch_count(ctypes.byref(c)), "mt_debug_launch_count")
     return int(c.value)
+
+
+def mt_set_cache_bytes(device_bytes: int) -> None:
+    """Switch to a weight cache of this many device bytes (0: every model resident).  Only while no model is registered."""
+    _check(lib().mt_set_cache_bytes(int(device_bytes)), "mt_set_cache_bytes")
+
+
+def mt_prefetch(model_ids, stream=None) -> None:
+    """Make these tenants (host ints) resident for work enqueued on `stream` afterwards."""
+    ids = np.ascontiguousarray(model_ids, dtype=np.int32)
+    _check(lib().mt_prefetch(ids.ctypes.data, int(ids.size), _stream_handle(stream)), "mt_prefetch")
+
+
+def mt_get_cache_stats(reset: bool = False) -> dict:
+    st = CacheStats()
+    _check(lib().mt_get_cache_stats(ctypes.byref(st), int(bool(reset))), "mt_get_cache_stats")
+    return st.as_dict()
+
+
+def mt_cache_sim_create(capacity_bytes: int):
+    """A stand-alone instance of the cache's policy (host code of the library; needs no GPU).  Returns its handle."""
+    h = ctypes.c_void_p()
+    _check(lib().mt_cache_sim_create(int(capacity_bytes), ctypes.byref(h)), "mt_cache_sim_create")
+    return h
+
+
+def mt_cache_sim_access(sim, model_id: int, nbytes: int, tick: int):
+    """Returns (result, offset, evicted ids): result 0 hit, 1 placed, -1 no room."""
+    res, off, n = ctypes.c_int32(0), ctypes.c_int64(0), ctypes.c_int32(0)
+    ev = (ctypes.c_int32 * 4096)()
+    _check(lib().mt_cache_sim_access(sim, int(model_id), int(nbytes), int(tick), ctypes.byref(res), ctypes.byref(off),
+                                     ev, 4096, ctypes.byref(n)), "mt_cache_sim_access")
+    return int(res.value), int(off.value), [int(ev[i]) for i in range(min(n.value, 4096))]
+
+
+def mt_cache_sim_release(sim, model_id: int) -> None:
+    _check(lib().mt_cache_sim_release(sim, int(model_id)), "mt_cache_sim_release")
+
+
+def mt_cache_sim_stats(sim) -> dict:
+    st = CacheStats()
+    _check(lib().mt_cache_sim_stats(sim, ctypes.byref(st)), "mt_cache_sim_stats")
+    return st.as_dict()
+
+
+def mt_cache_sim_destroy(sim) -> None:
+    _check(lib().mt_cache_sim_destroy(sim), "mt_cache_sim_destroy")
 
 
 def mt_debug_item_cost(k_blocks: int, n_cols: int, rows: int) -> float:

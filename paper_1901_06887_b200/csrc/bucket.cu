@@ -34,9 +34,16 @@ struct Brief { const int32_t* p; int ld; const int32_t* order; };
 __device__ __forceinline__ int tenant_at(Brief br, int l, int rank) { return __ldg(br.order + (size_t)l * br.ld + rank); }
 
 // ids outside [0, T) or of dead models go to the extra bucket T, so they sort behind every live segment.
+// (Row 0 of the compact table: 0 = no model, 1 = live and resident, 2 = registered but evicted from the device.)
 __device__ __forceinline__ int classify(int id, int T, Brief br) {
     if (id < 0 || id >= T) return T;
-    return __ldg(br.p + id) ? id : T;
+    return __ldg(br.p + id) == 1 ? id : T;
+}
+// Sticky status of a rejected request: its model is unknown, or known but not resident right now.
+__device__ __forceinline__ void report_rejected(int id, int i, int T, Brief br, int32_t* status) {
+    const bool evicted = id >= 0 && id < T && __ldg(br.p + id) == 2;
+    atomicCAS(&status[ST_CODE], MT_OK, evicted ? MT_ERR_NOT_RESIDENT : MT_ERR_BAD_MODEL_ID);
+    atomicMin(&status[ST_BAD_INDEX], i);
 }
 
 // Exclusive scan across the threads of a CTA (any multiple of 32 threads up to 1024): returns the sum of `v` over
@@ -212,10 +219,7 @@ bucket_hist_scan(const int32_t* __restrict__ ids, int n, int T, Brief br, int n_
     const int i = blockIdx.x * kHistChunk + threadIdx.x;
     if (i < n) {
         const int b = classify(ids[i], T, br);
-        if (b == T) {
-            atomicCAS(&status[ST_CODE], MT_OK, MT_ERR_BAD_MODEL_ID);
-            atomicMin(&status[ST_BAD_INDEX], i);
-        }
+        if (b == T) report_rejected(ids[i], i, T, br, status);
         const unsigned peers = __match_any_sync(__activemask(), b);
         if ((__ffs(peers) - 1) == (threadIdx.x & 31)) atomicAdd(&s_hist[b], __popc(peers));
     }
@@ -330,10 +334,7 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
         if (r < rounds && i < n) {
             const int b = classify(ids[i], T, br);
             bucket[r] = b;
-            if (b == T) {
-                atomicCAS(&status[ST_CODE], MT_OK, MT_ERR_BAD_MODEL_ID);
-                atomicMin(&status[ST_BAD_INDEX], i);
-            }
+            if (b == T) report_rejected(ids[i], i, T, br, status);
             const unsigned peers = __match_any_sync(__activemask(), b);
             if ((__ffs(peers) - 1) == lane) atomicAdd(&s_cnt[b], __popc(peers));
         }

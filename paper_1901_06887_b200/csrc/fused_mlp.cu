@@ -95,9 +95,10 @@ fused_mlp_kernel(const FusedArgs p) {
         const int i = c * 32 + lane;
         if (c < n_chunks && i < n) {
             const int id = p.ids[i];
-            const int b = (id < 0 || id >= T) ? T : (p.models[id].alive ? id : T);
+            const int alive = (id < 0 || id >= T) ? 0 : p.models[id].alive;     // 1 resident, 2 registered but evicted
+            const int b = alive == 1 ? id : T;
             if (b == T && blockIdx.x == 0) {
-                atomicCAS(&p.status[ST_CODE], MT_OK, MT_ERR_BAD_MODEL_ID);
+                atomicCAS(&p.status[ST_CODE], MT_OK, alive == 2 ? MT_ERR_NOT_RESIDENT : MT_ERR_BAD_MODEL_ID);
                 atomicMin(&p.status[ST_BAD_INDEX], i);
             }
             // (chunks are whole warps up to the batch's ragged end: the lanes with a request are lanes 0 .. n - 32c - 1)

@@ -11,6 +11,8 @@
 // epilogue of tile i overlaps the main loop of tile i+1.  Rows of a tile beyond the tenant's segment are
 // computed on whatever follows in memory and never stored (rows of a GEMM are independent).  The work list is
 // an array of 48-byte records expanded on the device after bucketing; CTA b takes items b, b + grid, ...
+#include <type_traits>
+
 #include "mt_device.cuh"
 #include "mt_host.h"
 
@@ -280,41 +282,72 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             cur = nxt;
             const int acc = it & 1;
             const uint32_t acc_phase = (it >> 1) & 1;
-            if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 4)) break;
-            tc_fence_after();
+            // Everything the drain needs besides the accumulator is fetched BEFORE the wait for it (the item's record
+            // is known one item ahead): output rows, through perm for a tenant's last layer, and the bias.  For short
+            // items - a few K blocks of a 64-wide layer - the drain is as long as the main loop, so its memory round
+            // trips must not come on top of it.
             const int N = c.N, relu = c.relu;
             const bool fin = (c.flags & kItemFinal) != 0;      // this tenant's last layer: fp32 rows to arrival order
-            if (kSwapOk && c.rows_valid <= kSwapRows) {
+            const bool swap_item = kSwapOk && c.rows_valid <= kSwapRows;
+            int my_row[2] = {c.row0 + lane, c.row0 + 32 + lane};
+            float bias_f[kWTiles];
+            size_t grow = (size_t)(c.row0 + r);
+            if (swap_item) {
+                if (fin) {
+                    if (lane < c.rows_valid) my_row[0] = __ldg(perm + c.row0 + lane);
+                    if (lane + 32 < c.rows_valid) my_row[1] = __ldg(perm + c.row0 + 32 + lane);
+                }
+#pragma unroll
+                for (int wt = 0; wt < kWTiles; ++wt) {
+                    const int f = c.n_tile * TN + wt * BN + r;
+                    bias_f[wt] = f < N ? __ldg(c.bias + f) : 0.0f;
+                }
+            } else if (fin && r < c.rows_valid) {
+                grow = (size_t)__ldg(perm + c.row0 + r);
+            }
+            if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 4)) break;
+            tc_fence_after();
+            if (swap_item) {
                 // Transposed item: this thread owns output feature f, the accumulator columns are the requests.
                 // For one request the 32 lanes of a warp write 32 neighbouring features: a 64- or 128-byte run.
+                // Requests are taken eight at a time and only as far as the segment goes (most segments of a
+                // long-tailed batch hold a handful); the output row of request j is handed round by shuffle.
                 const int nbox = (c.rows_valid + 31) >> 5;
+                auto store_box = [&](auto fin_c, const uint32_t (&v)[32], const int rows_of_box, const int n_req, const int f,
+                                     const float bias) {
+                    constexpr bool kFin = decltype(fin_c)::value;
+                    const bool f_ok = f < N;
+#pragma unroll
+                    for (int j0 = 0; j0 < 32; j0 += 8) {
+                        if (j0 < n_req) {                       // warp-uniform
+#pragma unroll
+                            for (int jj = 0; jj < 8; ++jj) {
+                                const int j = j0 + jj;
+                                const size_t orow = (size_t)__shfl_sync(0xffffffffu, rows_of_box, j);
+                                if (f_ok && j < n_req) {
+                                    float val = __uint_as_float(v[j]) + bias;
+                                    if (relu) val = fmaxf(val, 0.0f);
+                                    if (kFin) p.final_out[orow * p.ld_final + f] = val;
+                                    else reinterpret_cast<uint16_t*>(p.out)[orow * p.ld_out + f] =
+                                             static_cast<uint16_t>(pack_bf16x2(val, 0.0f) & 0xFFFFu);
+                                }
+                            }
+                        }
+                    }
+                };
 #pragma unroll 1
                 for (int wt = 0; wt < kWTiles; ++wt) {
                     const int f = c.n_tile * TN + wt * BN + r;
-                    const bool f_ok = f < N;
-                    const float bias_f = f_ok ? __ldg(c.bias + f) : 0.0f;
                     for (int b = 0; b < nbox; ++b) {
                         uint32_t v[32];
                         __syncwarp();
                         const int n_req = min(32, c.rows_valid - b * 32);
-                        const int row_b = c.row0 + b * 32;
-                        // output row of request j: its bucketed row, or (last layer) its arrival index - fetched by
-                        // lane j once and handed round by shuffle
-                        int my_row = row_b + lane;
-                        if (fin && lane < n_req) my_row = __ldg(perm + row_b + lane);
                         tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccCols + wt * kSwapRows + b * 32, v);
                         tmem_ld_wait();
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const size_t orow = (size_t)__shfl_sync(0xffffffffu, my_row, j);
-                            if (f_ok && j < n_req) {
-                                float val = __uint_as_float(v[j]) + bias_f;
-                                if (relu) val = fmaxf(val, 0.0f);
-                                if (fin) p.final_out[orow * p.ld_final + f] = val;
-                                else reinterpret_cast<uint16_t*>(p.out)[orow * p.ld_out + f] =
-                                         static_cast<uint16_t>(pack_bf16x2(val, 0.0f) & 0xFFFFu);
-                            }
-                        }
+                        const int rows_of_box = b == 0 ? my_row[0] : my_row[1];
+                        const float bias = wt == 0 ? bias_f[0] : bias_f[kWTiles - 1];
+                        if (fin) store_box(std::true_type{}, v, rows_of_box, n_req, f, bias);
+                        else store_box(std::false_type{}, v, rows_of_box, n_req, f, bias);
                     }
                 }
                 __syncwarp();
@@ -323,7 +356,6 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                 continue;
             }
             const bool row_ok = r < c.rows_valid;
-            const size_t grow = (fin && row_ok) ? (size_t)__ldg(perm + c.row0 + r) : (size_t)(c.row0 + r);
 #pragma unroll 1
             for (int ch = 0; ch < TN / 32; ++ch) {
                 uint32_t v[32];

@@ -14,6 +14,7 @@
 #include "../../include/mt.h"
 #include "mt_device.cuh"
 #include "mt_host.h"
+#include "weight_cache.h"
 
 namespace mt {
 unsigned long long g_kernel_launches = 0;
@@ -34,8 +35,42 @@ struct HostLayer {
 struct HostModel {
     bool alive = false;
     std::vector<HostLayer> layers;
-    void* dev_block = nullptr;
+    void* dev_block = nullptr;             // without the weight cache: the model's own allocation
+    // with the weight cache: the block lives in the arena while resident; its image is kept in pinned host memory
+    size_t block_bytes = 0;
+    void* host_image = nullptr;
+    std::vector<size_t> w_off, b_off;      // per layer: offsets of weights and bias inside the block
+    uint64_t last_batch = 0;               // number of the last batch that may have read the block
 };
+
+// What a tenant's entry in the device tables becomes when its block is (re)loaded or evicted: passed BY VALUE to a
+// one-CTA kernel on the caller's stream, so the change is ordered with the batches before and after it and no host
+// buffer has to outlive the call.
+struct TableUpdate {
+    ModelDev md;
+    CUtensorMap wmaps[MT_MAX_LAYERS];
+    int32_t alive;                         // 1 resident, 2 registered but not resident
+    int32_t id, n_wmaps;
+};
+
+__global__ void table_update_kernel(const __grid_constant__ TableUpdate u, ModelDev* models, int32_t* brief, CUtensorMap* wmaps) {
+    const int t = threadIdx.x;
+    if (u.alive == 1) {
+        const int n_words = sizeof(ModelDev) / 4;
+        const int32_t* src = reinterpret_cast<const int32_t*>(&u.md);
+        int32_t* dst = reinterpret_cast<int32_t*>(models + u.id);
+        for (int i = t; i < n_words; i += blockDim.x) dst[i] = src[i];
+        const int map_words = sizeof(CUtensorMap) / 4;
+        for (int l = 0; l < u.n_wmaps; ++l) {
+            const int32_t* ms = reinterpret_cast<const int32_t*>(&u.wmaps[l]);
+            int32_t* md = reinterpret_cast<int32_t*>(wmaps + (size_t)u.id * MT_MAX_LAYERS + l);
+            for (int i = t; i < map_words; i += blockDim.x) md[i] = ms[i];
+        }
+    } else if (t == 0) {
+        models[u.id].alive = u.alive;
+    }
+    if (t == 0) brief[u.id] = u.alive;
+}
 
 enum KernelId { K_BUCKET = 0, K_GATHER, K_GEMM, K_CONV, K_POOL, K_FUSED, K_COUNT };
 const char* const kKernelNames[K_COUNT] = {"bucketing (histogram, scans, scatter, row move, work items)", "gather_rows",
@@ -112,6 +147,19 @@ struct Ctx {
     const void* in_map_ptr = nullptr;
     int in_map_n = 0;
     CUtensorMap in_map, in_rows2_map, in_rows1_map;
+
+    // weight cache (off while cache_bytes == 0: every registered model stays resident in its own allocation)
+    size_t cache_bytes = 0;
+    uint8_t* arena = nullptr;
+    WeightCache cache;
+    cudaStream_t load_stream = nullptr;
+    uint64_t batch_no = 0;                              // batches enqueued so far (with the cache on)
+    uint64_t synced_batch = 0;                          // batches up to this one are known to have finished
+    uint64_t cache_tick = 0;                            // logical clock of the eviction policy
+    static constexpr int kBatchEvents = 8;
+    cudaEvent_t batch_done[kBatchEvents] = {nullptr};   // batch b's kernels have finished: batch_done[b % kBatchEvents]
+    cudaEvent_t loads_done = nullptr;
+    uint64_t request_hits = 0, request_misses = 0;
 
     // timing
     int timing = 0;                      // 0 off, 1 every kernel, 2 only the layer executors, 3 the same on every 4th call
@@ -350,6 +398,115 @@ void recompute_tile_n() {
             if (m.alive && l < m.layers.size() && m.layers[l].out_ch < min_n) min_n = m.layers[l].out_ch;
         g.tile_n[l] = (min_n != INT_MAX && min_n >= 256) ? 256 : BN;
     }
+}
+
+// ---------------------------------------------------------------------------------------------- weight cache
+// Device-table entry of model `id` for a block that starts at `base`.
+mt_status fill_table_update(int id, uint8_t* base, TableUpdate* u) {
+    const HostModel& hm = g.models[id];
+    memset(u, 0, sizeof *u);
+    u->id = id;
+    u->alive = 1;
+    u->md.alive = 1;
+    u->md.n_layers = (int)hm.layers.size();
+    for (size_t l = 0; l < hm.layers.size(); ++l) {
+        const HostLayer& h = hm.layers[l];
+        LayerDev& d = u->md.layer[l];
+        d.kind = h.kind; d.K = h.in_ch; d.N = h.out_ch; d.relu = h.relu;
+        d.n_tiles = (int)padded_weight_tiles(h);
+        d.k_blocks = h.kind == MT_DENSE ? h.in_ch / BK : 9;
+        if (h.kind == MT_GLOBAL_AVG_POOL) continue;
+        d.w = reinterpret_cast<const uint16_t*>(base + hm.w_off[l]);
+        d.bias = reinterpret_cast<const float*>(base + hm.b_off[l]);
+        if (h.kind == MT_DENSE) {
+            mt_status st = encode_weight_tiles(&u->wmaps[l], base + hm.w_off[l], padded_weight_tiles(h) * (size_t)(h.in_ch / BK));
+            if (st != MT_OK) return st;
+            u->n_wmaps = (int)l + 1;
+        }
+    }
+    return MT_OK;
+}
+
+void launch_table_update(const TableUpdate& u, cudaStream_t s) {
+    table_update_kernel<<<1, 128, 0, s>>>(u, g.d_models, g.d_brief, g.d_wmaps);
+}
+
+// Make the given tenants resident for the batch that is about to be enqueued on `s` (ids unique and live; reqs[i] =
+// requests of ids[i] in the batch, for the request-level hit count).  Blocks that are missing are copied from their
+// pinned host images on the load stream, into free arena space or over least-recently-used blocks; `s` waits for the
+// copies, then the device tables are switched by small kernels on `s`.  A victim's bytes may still be read by
+// batches in flight, so the copies wait for the youngest batch that could have used one.  MT_ERR_OOM: the set does
+// not fit the cache (nothing of this batch has been enqueued; tenants evicted on the way stay evicted).
+mt_status ensure_resident(const std::vector<int>& ids, const std::vector<int>& reqs, cudaStream_t s) {
+    if (!g.cache_bytes || ids.empty()) return MT_OK;
+    const uint64_t tick = ++g.cache_tick;
+    struct Load { int id; size_t off; };
+    std::vector<Load> loads;
+    std::vector<int> evicted;
+    mt_status result = MT_OK;
+    for (size_t i = 0; i < ids.size(); ++i) {
+        HostModel& hm = g.models[ids[i]];
+        size_t off = 0;
+        const WeightCache::Result r = g.cache.acquire(ids[i], hm.block_bytes, tick, &off, &evicted);
+        if (r == WeightCache::kNoRoom) { result = MT_ERR_OOM; break; }
+        if (r == WeightCache::kLoaded) { loads.push_back({ids[i], off}); g.request_misses += reqs[i]; }
+        else g.request_hits += reqs[i];
+        hm.last_batch = g.batch_no + 1;          // the batch being prepared
+    }
+    uint64_t youngest = 0;
+    for (int e : evicted) {
+        TableUpdate u;
+        memset(&u, 0, sizeof u);
+        u.id = e; u.alive = 2;
+        launch_table_update(u, s);
+        if (g.models[e].last_batch > youngest) youngest = g.models[e].last_batch;
+    }
+    if (!loads.empty()) {
+        if (youngest > g.synced_batch && youngest <= g.batch_no)
+            CU_OK(cudaStreamWaitEvent(g.load_stream, g.batch_done[youngest % Ctx::kBatchEvents], 0));
+        for (const Load& l : loads) {
+            const HostModel& hm = g.models[l.id];
+            CU_OK(cudaMemcpyAsync(g.arena + l.off, hm.host_image, hm.block_bytes, cudaMemcpyHostToDevice, g.load_stream));
+        }
+        CU_OK(cudaEventRecord(g.loads_done, g.load_stream));
+        CU_OK(cudaStreamWaitEvent(s, g.loads_done, 0));
+        for (const Load& l : loads) {
+            TableUpdate u;
+            mt_status st = fill_table_update(l.id, g.arena + l.off, &u);
+            if (st != MT_OK) return st;
+            launch_table_update(u, s);
+        }
+    }
+    CU_OK(cudaGetLastError());
+    return result;
+}
+
+// Tenant set of a batch whose ids the host can read: unique live ids and their request counts.
+void tenant_set_of(const int32_t* ids_host, int n, std::vector<int>* ids, std::vector<int>* reqs) {
+    std::vector<int> count(g.T, 0);
+    for (int i = 0; i < n; ++i) {
+        const int t = ids_host[i];
+        if (t >= 0 && t < g.T && g.models[t].alive) count[t] += 1;
+    }
+    for (int t = 0; t < g.T; ++t)
+        if (count[t]) { ids->push_back(t); reqs->push_back(count[t]); }
+}
+
+// Book-keeping around one batch when the cache is on: the batch number is the clock of "who may still be reading
+// which block"; a batch whose ids live on the device may read any resident block.
+void cache_begin_batch(bool ids_unknown) {
+    if (!g.cache_bytes) return;
+    if (ids_unknown) {
+        g.cache.touch_all(++g.cache_tick);
+        for (int t = 0; t < g.T; ++t)
+            if (g.models[t].alive && g.cache.resident(t)) g.models[t].last_batch = g.batch_no + 1;
+    }
+}
+mt_status cache_end_batch(cudaStream_t s) {
+    if (!g.cache_bytes) return MT_OK;
+    g.batch_no += 1;
+    CU_OK(cudaEventRecord(g.batch_done[g.batch_no % Ctx::kBatchEvents], s));
+    return MT_OK;
 }
 
 // A-priori cost of one dense work item in SM cycles (Sec. 3.2: the work of a layer is fixed by its shape and known
@@ -704,9 +861,20 @@ mt_status mt_shutdown(void) {
     if (!g.init) return MT_OK;
     cudaSetDevice(g.device);
     cudaDeviceSynchronize();
-    for (HostModel& m : g.models)
+    for (HostModel& m : g.models) {
         if (m.dev_block) { cudaFree(m.dev_block); m.dev_block = nullptr; }
+        if (m.host_image) { cudaFreeHost(m.host_image); m.host_image = nullptr; }
+    }
     g.models.clear();
+    cudaFree(g.arena); g.arena = nullptr;
+    g.cache.reset(0);
+    g.cache_bytes = 0;
+    if (g.load_stream) { cudaStreamDestroy(g.load_stream); g.load_stream = nullptr; }
+    for (cudaEvent_t& ev : g.batch_done)
+        if (ev) { cudaEventDestroy(ev); ev = nullptr; }
+    if (g.loads_done) { cudaEventDestroy(g.loads_done); g.loads_done = nullptr; }
+    g.batch_no = g.synced_batch = g.cache_tick = 0;
+    g.request_hits = g.request_misses = 0;
     free_workspace();
     cudaFree(g.d_models); g.d_models = nullptr;
     cudaFree(g.d_brief); g.d_brief = nullptr;
@@ -773,7 +941,23 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
         if (raw > raw_max) raw_max = raw;
     }
     uint8_t* block = nullptr;
-    CU_OK(cudaMalloc(&block, total));
+    if (g.cache_bytes) {
+        // a place in the arena, over least-recently-used tenants if need be (registration is synchronous: nothing is
+        // in flight once the device has been synchronised, so the victims' table entries are switched directly)
+        std::vector<int> evicted;
+        size_t off = 0;
+        if (g.cache.acquire(id, total, ++g.cache_tick, &off, &evicted) == WeightCache::kNoRoom) return MT_ERR_OOM;
+        CU_OK(cudaDeviceSynchronize());
+        g.synced_batch = g.batch_no;
+        for (int v : evicted) {
+            const int32_t two = 2;
+            CU_OK(cudaMemcpy(g.d_brief + v, &two, sizeof two, cudaMemcpyHostToDevice));
+            CU_OK(cudaMemcpy(&g.d_models[v].alive, &two, sizeof two, cudaMemcpyHostToDevice));
+        }
+        block = g.arena + off;
+    } else {
+        CU_OK(cudaMalloc(&block, total));
+    }
     cudaError_t e = cudaMemset(block, 0, total);
     void* raw_dev = nullptr;
     ModelDev md;
@@ -822,8 +1006,14 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
         e = cudaMemcpy(g.d_brief + (size_t)r * g.max_models + id, &v, sizeof v, cudaMemcpyHostToDevice);
     }
     if (raw_dev) cudaFree(raw_dev);
+    void* host_image = nullptr;
+    if (e == cudaSuccess && g.cache_bytes) {        // the host tier: the block's image in pinned memory
+        e = cudaMallocHost(&host_image, total);
+        if (e == cudaSuccess) e = cudaMemcpy(host_image, block, total, cudaMemcpyDeviceToHost);
+    }
     if (e != cudaSuccess) {
-        cudaFree(block);
+        if (g.cache_bytes) g.cache.release(id); else cudaFree(block);
+        if (host_image) cudaFreeHost(host_image);
         cudaGetLastError();
         return e == cudaErrorMemoryAllocation ? MT_ERR_OOM : MT_ERR_CUDA;
     }
@@ -851,7 +1041,12 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
     HostModel& hm = g.models[id];
     hm.alive = true;
     hm.layers = hl;
-    hm.dev_block = block;
+    hm.dev_block = g.cache_bytes ? nullptr : block;
+    hm.block_bytes = total;
+    hm.host_image = host_image;
+    hm.w_off = w_off;
+    hm.b_off = b_off;
+    hm.last_batch = 0;
     g.live += 1;
     if (id + 1 > g.T) g.T = id + 1;
     recompute_tile_n();
@@ -873,6 +1068,9 @@ mt_status mt_release(int32_t model_id) {
     const int32_t dead = 0;
     CU_OK(cudaMemcpy(g.d_brief + model_id, &dead, sizeof dead, cudaMemcpyHostToDevice));
     HostModel& hm = g.models[model_id];
+    g.synced_batch = g.batch_no;
+    if (g.cache_bytes) g.cache.release(model_id);
+    if (hm.host_image) { cudaFreeHost(hm.host_image); hm.host_image = nullptr; }
     cudaFree(hm.dev_block);
     hm.dev_block = nullptr;
     hm.alive = false;
@@ -884,7 +1082,10 @@ mt_status mt_release(int32_t model_id) {
 
 mt_status mt_infer(const void* inputs, const int32_t* model_ids, int32_t n, void* outputs, void* stream) {
     std::lock_guard<std::mutex> lk(g_mu);
-    return infer_device(inputs, model_ids, n, outputs, static_cast<cudaStream_t>(stream));
+    cache_begin_batch(true);      // ids on the device: the batch may read any resident tenant
+    mt_status st = infer_device(inputs, model_ids, n, outputs, static_cast<cudaStream_t>(stream));
+    if (st != MT_OK || n == 0) return st;
+    return cache_end_batch(static_cast<cudaStream_t>(stream));
 }
 
 mt_status mt_infer_host(const void* inputs_host, const int32_t* model_ids_host, int32_t n, void* outputs_host,
@@ -909,9 +1110,17 @@ mt_status mt_infer_host(const void* inputs_host, const int32_t* model_ids_host, 
         CU_OK(cudaMalloc(&g.st_out, out_bytes));
         g.st_cap_in = in_bytes; g.st_cap_ids = id_bytes; g.st_cap_out = out_bytes;
     }
+    if (g.cache_bytes) {          // the host sees the ids: bring exactly this batch's tenants in
+        std::vector<int> set, reqs;
+        tenant_set_of(model_ids_host, n, &set, &reqs);
+        mt_status rs = ensure_resident(set, reqs, s);
+        if (rs != MT_OK) return rs;
+    }
     CU_OK(cudaMemcpyAsync(g.st_in, inputs_host, in_bytes, cudaMemcpyHostToDevice, s));
     CU_OK(cudaMemcpyAsync(g.st_ids, model_ids_host, id_bytes, cudaMemcpyHostToDevice, s));
     mt_status st = infer_device(g.st_in, g.st_ids, n, g.st_out, s);
+    if (st != MT_OK) return st;
+    st = cache_end_batch(s);
     if (st != MT_OK) return st;
     CU_OK(cudaMemcpyAsync(outputs_host, g.st_out, out_bytes, cudaMemcpyDeviceToHost, s));
     CU_OK(cudaStreamSynchronize(s));
@@ -959,13 +1168,116 @@ mt_status mt_infer_host_async(const void* inputs_host, const int32_t* model_ids_
     CU_OK(cudaMemcpyAsync(g.as_ids[k], model_ids_host, id_bytes, cudaMemcpyHostToDevice, s));
     // the kernels of consecutive calls share one workspace: they run one call after the other, whatever the streams
     if (g.as_have_compute) CU_OK(cudaStreamWaitEvent(s, g.as_compute_done, 0));
+    if (g.cache_bytes) {          // after the wait: the table switches are ordered behind the previous batch's kernels
+        std::vector<int> set, reqs;
+        tenant_set_of(model_ids_host, n, &set, &reqs);
+        mt_status rs = ensure_resident(set, reqs, s);
+        if (rs != MT_OK) return rs;
+    }
     st = infer_device(g.as_in[k], g.as_ids[k], n, g.as_out[k], s);
+    if (st != MT_OK) return st;
+    st = cache_end_batch(s);
     if (st != MT_OK) return st;
     CU_OK(cudaEventRecord(g.as_compute_done, s));
     g.as_have_compute = true;
     CU_OK(cudaMemcpyAsync(outputs_host, g.as_out[k], out_bytes, cudaMemcpyDeviceToHost, s));
     CU_OK(cudaEventRecord(g.as_slot_done[k], s));
     g.as_slot_used[k] = true;
+    return MT_OK;
+}
+
+mt_status mt_set_cache_bytes(size_t device_bytes) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g.init) return MT_ERR_NOT_INIT;
+    if (g.live != 0) return MT_ERR_INVALID_ARG;          // only while no model is registered
+    CU_OK(cudaSetDevice(g.device));
+    CU_OK(cudaDeviceSynchronize());
+    cudaFree(g.arena); g.arena = nullptr;
+    g.cache.reset(0);
+    g.cache_bytes = 0;
+    if (device_bytes == 0) return MT_OK;
+    const size_t cap = device_bytes / 1024 * 1024;
+    if (cap == 0) return MT_ERR_INVALID_ARG;
+    cudaError_t e = cudaMalloc(&g.arena, cap);
+    if (e != cudaSuccess) { cudaGetLastError(); g.arena = nullptr; return e == cudaErrorMemoryAllocation ? MT_ERR_OOM : MT_ERR_CUDA; }
+    if (!g.load_stream) CU_OK(cudaStreamCreateWithFlags(&g.load_stream, cudaStreamNonBlocking));
+    for (cudaEvent_t& ev : g.batch_done)
+        if (!ev) CU_OK(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+    if (!g.loads_done) CU_OK(cudaEventCreateWithFlags(&g.loads_done, cudaEventDisableTiming));
+    g.cache.reset(cap);
+    g.cache_bytes = cap;
+    g.batch_no = g.synced_batch = g.cache_tick = 0;
+    g.request_hits = g.request_misses = 0;
+    return MT_OK;
+}
+
+mt_status mt_prefetch(const int32_t* model_ids_host, int32_t count, void* stream) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g.init) return MT_ERR_NOT_INIT;
+    if (count < 0 || (count > 0 && !model_ids_host)) return MT_ERR_INVALID_ARG;
+    if (!g.cache_bytes || count == 0) return MT_OK;       // without the cache every model is resident
+    for (int i = 0; i < count; ++i) {
+        const int t = model_ids_host[i];
+        if (t < 0 || t >= g.max_models || !g.models[t].alive) return MT_ERR_BAD_MODEL_ID;
+    }
+    CU_OK(cudaSetDevice(g.device));
+    std::vector<int> set, reqs;
+    tenant_set_of(model_ids_host, count, &set, &reqs);
+    for (int& r : reqs) r = 0;                            // a prefetch serves no request yet
+    return ensure_resident(set, reqs, static_cast<cudaStream_t>(stream));
+}
+
+mt_status mt_get_cache_stats(mt_cache_stats* out, int32_t reset) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g.init) return MT_ERR_NOT_INIT;
+    if (!out) return MT_ERR_INVALID_ARG;
+    const WeightCache::Stats& cs = g.cache.stats();
+    out->capacity_bytes = g.cache_bytes;
+    out->resident_bytes = g.cache.resident_bytes();
+    out->tenant_hits = cs.hits; out->tenant_misses = cs.misses;
+    out->evictions = cs.evictions; out->bytes_loaded = cs.bytes_loaded;
+    out->request_hits = g.request_hits; out->request_misses = g.request_misses;
+    if (reset) { g.cache.clear_stats(); g.request_hits = g.request_misses = 0; }
+    return MT_OK;
+}
+
+// The eviction policy by itself, on a made-up clock (host code only: usable without a GPU).
+struct CacheSim { mt::WeightCache c; };
+mt_status mt_cache_sim_create(size_t capacity_bytes, void** sim_out) {
+    if (!sim_out) return MT_ERR_INVALID_ARG;
+    CacheSim* s = new CacheSim();
+    s->c.reset(capacity_bytes);
+    *sim_out = s;
+    return MT_OK;
+}
+mt_status mt_cache_sim_access(void* sim, int32_t id, size_t bytes, uint64_t tick, int32_t* result_out, int64_t* offset_out,
+                              int32_t* evicted_out, int32_t evicted_cap, int32_t* n_evicted_out) {
+    if (!sim || !result_out) return MT_ERR_INVALID_ARG;
+    std::vector<int> ev;
+    size_t off = 0;
+    const mt::WeightCache::Result r = static_cast<CacheSim*>(sim)->c.acquire(id, bytes, tick, &off, &ev);
+    *result_out = (int32_t)r;
+    if (offset_out) *offset_out = r == mt::WeightCache::kNoRoom ? -1 : (int64_t)off;
+    if (n_evicted_out) *n_evicted_out = (int32_t)ev.size();
+    for (size_t i = 0; i < ev.size() && evicted_out && (int)i < evicted_cap; ++i) evicted_out[i] = ev[i];
+    return MT_OK;
+}
+mt_status mt_cache_sim_release(void* sim, int32_t id) {
+    if (!sim) return MT_ERR_INVALID_ARG;
+    static_cast<CacheSim*>(sim)->c.release(id);
+    return MT_OK;
+}
+mt_status mt_cache_sim_stats(void* sim, mt_cache_stats* out) {
+    if (!sim || !out) return MT_ERR_INVALID_ARG;
+    const mt::WeightCache& c = static_cast<CacheSim*>(sim)->c;
+    memset(out, 0, sizeof *out);
+    out->capacity_bytes = c.capacity(); out->resident_bytes = c.resident_bytes();
+    out->tenant_hits = c.stats().hits; out->tenant_misses = c.stats().misses;
+    out->evictions = c.stats().evictions; out->bytes_loaded = c.stats().bytes_loaded;
+    return MT_OK;
+}
+mt_status mt_cache_sim_destroy(void* sim) {
+    delete static_cast<CacheSim*>(sim);
     return MT_OK;
 }
 
@@ -994,6 +1306,7 @@ const char* mt_status_string(mt_status s) {
         case MT_ERR_ARCH: return "device is not sm_100";
         case MT_ERR_TIMEOUT: return "device-side wait timed out";
         case MT_ERR_NOT_INIT: return "not initialised";
+        case MT_ERR_NOT_RESIDENT: return "model registered but not resident on the device";
     }
     return "unknown status";
 }
