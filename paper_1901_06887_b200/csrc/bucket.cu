@@ -206,9 +206,10 @@ __device__ __forceinline__ void scan_buckets(int T, Brief br, int n_layers, int 
 __global__ void __launch_bounds__(kHistChunk)
 bucket_hist_scan(const int32_t* __restrict__ ids, int n, int T, Brief br, int n_layers,
                  int rows_per_unit, LayerTileN tn, int32_t* block_hist, int32_t* counts, int32_t* __restrict__ offsets,
-                 int32_t* __restrict__ tile_prefix, int32_t* ticket, int32_t* __restrict__ status) {
+                 int32_t* __restrict__ tile_prefix, int32_t* ticket, int32_t* __restrict__ status, unsigned* grid_bar) {
     pdl_launch_dependents();
     pdl_wait();
+    if (grid_bar && blockIdx.x == 0 && threadIdx.x < 8) grid_bar[threadIdx.x] = 0u;   // barrier counters of this call's conv launches
     extern __shared__ int32_t s_hist[];   // T + 1
     __shared__ int32_t s_warp[33];
     __shared__ int32_t s_vec[MT_MAX_LAYERS * 33];
@@ -312,9 +313,10 @@ __global__ void __launch_bounds__(1024)
 bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev* __restrict__ models, Brief br, int n_layers,
                   int rows_per_unit, LayerTileN tn, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
                   int32_t* __restrict__ tile_prefix, int32_t* __restrict__ perm, int32_t* __restrict__ inv,
-                  ItemPtrs items, int32_t* __restrict__ status) {
+                  ItemPtrs items, int32_t* __restrict__ status, unsigned* grid_bar) {
     pdl_launch_dependents();
     pdl_wait();
+    if (grid_bar && threadIdx.x < 8) grid_bar[threadIdx.x] = 0u;   // barrier counters of this call's conv launches
     extern __shared__ int32_t s_mem[];          // s_cnt[T + 1], s_next[T + 1]
     __shared__ int32_t s_warp[33];
     __shared__ int32_t s_vec[MT_MAX_LAYERS * 33];
@@ -594,11 +596,11 @@ void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
     if (a.n <= 512 && a.T + 1 <= 4096) {
         const int threads = (a.n <= 256) ? 256 : 1024;
         launch_pdl(bucket_single_cta, dim3(1), dim3(threads), 2 * smem, s, a.ids, a.n, a.T, a.models, br, a.n_layers, a.rows_per_unit, tn, a.counts,
-                                                      a.offsets, a.tile_prefix, a.perm, a.inv, ip, a.status);
+                                                      a.offsets, a.tile_prefix, a.perm, a.inv, ip, a.status, a.grid_bar);
         return;
     }
     launch_pdl(bucket_hist_scan, dim3(n_hist_blocks), dim3(kHistChunk), smem, s, a.ids, a.n, a.T, br, a.n_layers, a.rows_per_unit, tn,
-               a.block_hist, a.counts, a.offsets, a.tile_prefix, a.ticket, a.status);
+               a.block_hist, a.counts, a.offsets, a.tile_prefix, a.ticket, a.status, a.grid_bar);
     const int grid2 = n_blocks > a.item_grid ? n_blocks : a.item_grid;
     launch_pdl(bucket_scatter_expand, dim3(grid2), dim3(kScatterThreads), smem + sizeof(int32_t) * kBucketChunk, s, a.ids, a.n, a.T, a.models, br,
                a.block_hist, a.offsets, a.perm, a.inv, (const uint4*)a.rows_src, (uint4*)a.rows_dst, a.row_bytes / 16,

@@ -66,9 +66,13 @@ struct PairStrip {
     int t, j, y0, strip_in_image, dummy;
 };
 
+// Consecutive conv layers of one geometry run in ONE launch (p.n_stack of them, from layer p.layer on): every cluster
+// keeps its range of units through all layers, and between two layers all CTAs meet at a grid-wide barrier (a counter
+// in global memory, every wait bounded) - a layer boundary inside a launch costs a few microseconds, one between two
+// launches about three times that, since no CTA of the next launch can start while one of this launch holds its SM's
+// shared memory.  The next layer's first weights are requested before the barrier.
 __global__ void __launch_bounds__(kCpThreads, 1)
-grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_x1,
-                            const __grid_constant__ CUtensorMap tmap_y, const ConvArgs p) {
+grouped_conv3x3_pair_kernel(const __grid_constant__ ConvStackMaps maps, const ConvArgs p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -111,9 +115,11 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
         mbar_init(wpeer_bar, 1);
         *abort_flag = 0;
         fence_mbar_init();
-        prefetch_tensormap(&tmap_x);
-        prefetch_tensormap(&tmap_x1);
-        prefetch_tensormap(&tmap_y);
+        for (int k = 0; k < p.n_stack; ++k) {
+            prefetch_tensormap(&maps.x2[k]);
+            prefetch_tensormap(&maps.x1[k]);
+            prefetch_tensormap(&maps.y[k]);
+        }
     }
     // Operands shifted by one or two pixels read a little past what the copies wrote, whatever the previous kernel left
     // there: rows of the product that belong to pad columns, which are neither stored nor pooled.
@@ -190,13 +196,57 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
         return c;
     };
 
+    // End of layer k of the stack, called by every thread of the CTA at a converged point: this CTA's outputs are
+    // complete and visible (the storing lanes have waited for their tensor stores), then one thread arrives at the
+    // grid-wide counter and waits, for a bounded time, until all CTAs of the launch have (p.grid_bar was zeroed by the
+    // bucketing kernel of this call).  Afterwards the layer's outputs may be read by anyone, also through TMA.
+    auto layer_sync = [&](int k) {
+        asm volatile("fence.proxy.async;" ::: "memory");
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            atomicAdd(p.grid_bar, 1u);
+            const unsigned want = (unsigned)(k + 1) * gridDim.x;
+            const uint64_t t0 = global_timer_ns();
+            unsigned seen;
+            uint32_t it = 0;
+            while (true) {
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(p.grid_bar) : "memory");
+                if (seen >= want) break;
+                if ((++it & 0xFF) == 0) {
+                    if (*abort_flag) break;
+                    if (global_timer_ns() - t0 > kWaitLimitNs) {
+                        *abort_flag = 1;
+                        if (atomicCAS(&p.status[ST_CODE], MT_OK, MT_ERR_TIMEOUT) == MT_OK) p.status[ST_WHERE] = 60;
+                        break;
+                    }
+                }
+            }
+            __threadfence();
+            asm volatile("fence.proxy.async;" ::: "memory");
+        }
+        __syncthreads();
+    };
+    const int n_stack = p.n_stack;
+
     if (warp == 0) {
-        if (lane == 0) {   // ------------------------------------------------ TMA producer (both CTAs)
-            int w_loads = 0, w_tenant = -1;
+        // ------------------------------------------------------------------- TMA producer (lane 0 of both CTAs)
+        int w_loads = 0, w_tenant = -1;
+        int nb = 0;                     // blocks armed so far; block b goes to slot b % kCpRing
+        bool ok = true;
+        bool first_weights_out = p.early_lookup != 0;      // the stack's first weights were requested before the wait
+        for (int k = 0; k < n_stack; ++k) {
+          if (lane == 0 && ok && !*abort_flag) {
+            const int layer = p.layer + k;
+            const CUtensorMap* const tmap_x = &maps.x2[k];
+            const CUtensorMap* const tmap_x1 = &maps.x1[k];
+            const int32_t* const perm = (k == 0) ? p.perm : nullptr;
+            if (k > 0) w_tenant = -1;   // same tenants, other weights
+            {
+            // (indentation kept from the single-layer form)
+            
             const uint32_t wpeer_leader = map_to_cta(wpeer_bar, 0);
             const uint32_t bfull_leader0 = map_to_cta(bfull_bar(0), 0);
-            int nb = 0;                     // blocks armed so far; block b goes to slot b % kCpRing
-            bool ok = true;
             auto start_weights = [&](int t, const uint16_t* w) {
                 // The issuer releases the old weights when it reaches the tenant's first strip in its own order.
                 if (w_loads > 0 && !mbar_wait_spin(wempty_bar, (uint32_t)((w_loads - 1) & 1), abort_flag, p.status, 51, 64)) return false;
@@ -216,14 +266,14 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
             for (int s = s_begin; ok && s < s_end; ++s) {
                 const PairStrip c = locate(s);
                 const bool new_tenant = (c.t != w_tenant);
-                const int img = p.perm ? p.perm[c.j] : c.j;
+                const int img = perm ? perm[c.j] : c.j;
                 const bool seg_start = (s == s_begin) || c.strip_in_image == 0;
                 // the very first weights go out before the first blocks: the first MMA needs both, and this is the
                 // larger copy (later ones must wait for the issuer to let go of the old weights, so the blocks go first)
-                const bool weights_first = new_tenant && w_loads == 0;
+                const bool weights_first = new_tenant && s == s_begin;
                 if (weights_first) {
-                    if (p.early_lookup) w_tenant = c.t;                      // requested before the dependency wait
-                    else if (!start_weights(c.t, *s_first_w)) break;
+                    if (first_weights_out) w_tenant = c.t;     // requested before the dependency wait / the layer barrier
+                    else if (!start_weights(c.t, k == 0 ? *s_first_w : p.models[c.t].layer[layer].w)) { ok = false; break; }
                 }
                 // published to this CTA's epilogue with the strip's first block (the issuer starts the strip's first
                 // tile only after that block has landed)
@@ -237,25 +287,37 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                     const int y_in = c.y0 + 2 * kb - 1;              // first input row of the block
                     const uint32_t bytes = kCpBlockBytes + (slot == 0 ? 64u * 128u : 0u);
                     if (is_leader) mbar_expect_tx(bfull_bar(slot), 2u * bytes);   // both CTAs' bytes
-                    tma_load_4d_pair(ring0 + slot * kCpBlockBytes, &tmap_x, 0, -1, y_in, img, bfull_leader0 + 8u * slot);
-                    if (slot == 0) tma_load_4d_pair(ghost0, &tmap_x1, 0, -1, y_in, img, bfull_leader0);
+                    tma_load_4d_pair(ring0 + slot * kCpBlockBytes, tmap_x, 0, -1, y_in, img, bfull_leader0 + 8u * slot);
+                    if (slot == 0) tma_load_4d_pair(ghost0, tmap_x1, 0, -1, y_in, img, bfull_leader0);
                     ++nb;
                 }
                 if (!ok) break;
-                if (new_tenant && !weights_first && !start_weights(c.t, p.models[c.t].layer[p.layer].w)) break;
-                if (new_tenant && !announce_weights()) break;
+                if (new_tenant && !weights_first && !start_weights(c.t, p.models[c.t].layer[layer].w)) { ok = false; break; }
+                if (new_tenant && !announce_weights()) { ok = false; break; }
             }
+            // the next layer's first weights (they do not depend on this layer's results) go out before the barrier
+            first_weights_out = false;
+            if (ok && k + 1 < n_stack && s_begin < s_end) {
+                const int t0 = s_first[0];
+                if (start_weights(t0, p.models[t0].layer[layer + 1].w)) first_weights_out = true; else ok = false;
+            }
+            }
+          }
+          __syncwarp();
+          if (k + 1 < n_stack) layer_sync(k);
         }
     } else if (warp == 1) {
-        if (is_leader) {   // ------------------------------------------------ MMA issuer (leader CTA)
-            // The whole warp walks the loop (addresses and descriptors stay warp-uniform); one elected lane issues.
-            const bool leader = elect_one();
+        // ------------------------------------------------------------------- MMA issuer (leader CTA; the peer's warp 1
+        // only takes part in the layer barriers).  The whole warp walks the loop (addresses and descriptors stay
+        // warp-uniform); one elected lane issues.
+        const bool leader = elect_one();
             const uint32_t tb = __shfl_sync(0xffffffffu, *tmem_slot, 0);
             constexpr uint32_t idesc64 = make_idesc_bf16(2 * BM, kCpN);
             constexpr uint32_t idesc128 = make_idesc_bf16(2 * BM, 2 * kCpN);
             int g = 0;                      // tiles started so far by this pair; tile g lives in TMEM slot g % kCpSlots
             int bc = 0;                     // load-order number of the block with the current tile's first input rows
             int w_loads = 0;
+            bool w_released = false;        // the current weights were handed back at the end of a layer
             bool ok = true;
             const uint32_t w_lo = desc_lo(w_smem);
             const uint32_t ring_lo = desc_lo(ring0);
@@ -273,9 +335,12 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                 umma_pair_lohi<true>(d_tmem, a_lo + 6, b_lo + 6, idesc);
             };
             auto bfull_parity = [](int q) { return (uint32_t)((q / kCpRing) & 1); };
-            int t_hi = -1;                  // units [.., t_hi) belong to the current tenant
-            int in_image = 0;               // index of the current strip inside its image
             uint32_t block_ready = 0, slot_ready = 0;
+        for (int k = 0; k < n_stack; ++k) {
+          if (is_leader && ok && !*abort_flag) {
+            int t_hi = -1;                  // units [.., t_hi) belong to the current tenant (every layer starts over)
+            int in_image = 0;               // index of the current strip inside its image
+            block_ready = 0;
             for (int s = s_begin; ok && s < s_end; ++s) {
                 const bool new_tenant = (s >= t_hi);
                 if (new_tenant) {           // rare: a tenant border (or the first unit)
@@ -287,13 +352,14 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                 const bool seg_start = !(s > s_begin && in_image > 0);
                 const bool seg_end = !(s + 1 < s_end && in_image + 1 < p.strips_per_image);
                 if (seg_start) {
-                    if (!mbar_wait_spin(bfull_bar(bc & (kCpRing - 1)), bfull_parity(bc), abort_flag, p.status, 55)) break;
+                    if (!mbar_wait_spin(bfull_bar(bc & (kCpRing - 1)), bfull_parity(bc), abort_flag, p.status, 55)) { ok = false; break; }
                     block_ready = 0;
                 }
                 if (new_tenant) {
-                    if (w_loads > 0 && leader) umma_commit_pair(wempty_bar);     // fires when all MMAs on the old weights are done
-                    if (!mbar_wait(wfull_bar, (uint32_t)(w_loads & 1), abort_flag, p.status, 56)) break;
-                    if (!mbar_wait_spin(wpeer_bar, (uint32_t)(w_loads & 1), abort_flag, p.status, 57)) break;
+                    if (w_loads > 0 && !w_released && leader) umma_commit_pair(wempty_bar);   // fires when all MMAs on the old weights are done
+                    w_released = false;
+                    if (!mbar_wait(wfull_bar, (uint32_t)(w_loads & 1), abort_flag, p.status, 56)) { ok = false; break; }
+                    if (!mbar_wait_spin(wpeer_bar, (uint32_t)(w_loads & 1), abort_flag, p.status, 57)) { ok = false; break; }
                     ++w_loads;
                 }
                 for (int i = 0; i < TS; ++i, ++g, ++bc) {
@@ -349,6 +415,14 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                 }
                 if (++in_image == p.strips_per_image) in_image = 0;
             }
+            // the layer's weights go back to the producer, which requests the next layer's before the barrier
+            if (ok && k + 1 < n_stack && s_begin < s_end && w_loads > 0) {
+                if (leader) umma_commit_pair(wempty_bar);
+                w_released = true;
+            }
+          }
+          __syncwarp();
+          if (k + 1 < n_stack) layer_sync(k);
         }
     } else {               // ---------------------------------------------------- epilogue (warps 2..9, both CTAs)
         const int ew = warp - 2;
@@ -361,8 +435,12 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
         bool ok = true;
         int img_j = 0, y0 = 0, store = 1;
         int rel = 0;                                // blocks released so far (load order), kept by the releasing thread
-        const bool pooling = (p.pool_partial != nullptr);
         const uint32_t tempty_leader0 = map_to_cta(tempty_bar(0), 0);   // the leader's tempty barriers, 8 bytes apart
+      for (int k = 0; k < n_stack; ++k) {
+        const int layer = p.layer + k;
+        const bool pooling = (p.pool_partial != nullptr) && k == n_stack - 1;   // only the stack's last layer feeds the pool
+        const CUtensorMap* const tmap_y = &maps.y[k];
+        if (*abort_flag) ok = false;
         for (int s = s_begin; ok && s < s_end; ++s) {
             float psum[32];
 #pragma unroll
@@ -383,7 +461,7 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                     // the segment's first tile also hands back its own block.
                     if (threadIdx.x == 64 && (rec.x & 2)) { mbar_arrive(bempty_bar(rel & (kCpRing - 1))); ++rel; }
                     if (rec.x & 1) {                // new tenant: its bias into shared memory, ReLU flag into a register
-                        const LayerDev& L = p.models[rec.w].layer[p.layer];
+                        const LayerDev& L = p.models[rec.w].layer[layer];
                         asm volatile("bar.sync 1, %0;" ::"n"(kCpEpiThreads) : "memory");   // everyone done with the old bias
                         if (threadIdx.x - 64 < kCpN) s_bias[threadIdx.x - 64] = L.bias[threadIdx.x - 64];
                         relu = L.relu;
@@ -447,7 +525,7 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                     __syncwarp();
                     const int yw = y0 + i * rows_per_tile + (q4 >> 1);       // the warp's image row (warp-uniform)
                     if (lane == 0 && store && yw < p.H && (q4 & 1) * 32 < p.W) {
-                        tma_store_4d(&tmap_y, half * 32, (q4 & 1) * 32, yw, img_j, out_stage0 + ew * 2048);
+                        tma_store_4d(tmap_y, half * 32, (q4 & 1) * 32, yw, img_j, out_stage0 + ew * 2048);
                         bulk_commit_group();
                     }
                 }
@@ -480,6 +558,13 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __
                 asm volatile("bar.sync 1, %0;" ::"n"(kCpEpiThreads) : "memory");
             }
         }
+        if (k + 1 < n_stack) {
+            // this layer's outputs must have reached memory before anyone passes the barrier
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+            __syncwarp();
+            layer_sync(k);
+        }
+      }
     }
 
     // ---- tear-down: every thread of both CTAs gets here, also after an abandoned wait
@@ -528,9 +613,9 @@ cudaError_t configure_grouped_conv_pair() {
 }
 
 // Cluster of two CTAs; grid = an even number of CTAs (one per SM).  a.tile_prefix counts (pair of images, strip) units.
-// tmap_x2 / tmap_x1: the layer's input with boxes of 64 pixels x 2 rows / x 1 row; tmap_y: its output, 32 x 32 store boxes.
-cudaError_t launch_grouped_conv_pair(const CUtensorMap& tmap_x2, const CUtensorMap& tmap_x1, const CUtensorMap& tmap_y,
-                                     const ConvArgs& a, int sm_count, cudaStream_t s) {
+// maps: per layer of the stack (a.n_stack layers from a.layer on) the input as boxes of 64 pixels x 2 rows and x 1 row
+// and the output as 32 x 32 store boxes.
+cudaError_t launch_grouped_conv_pair(const ConvStackMaps& maps, const ConvArgs& a, int sm_count, cudaStream_t s) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(sm_count & ~1);
     cfg.blockDim = dim3(kCpThreads);
@@ -543,7 +628,7 @@ cudaError_t launch_grouped_conv_pair(const CUtensorMap& tmap_x2, const CUtensorM
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 2;
     ++g_kernel_launches;
-    return cudaLaunchKernelEx(&cfg, grouped_conv3x3_pair_kernel, tmap_x2, tmap_x1, tmap_y, a);
+    return cudaLaunchKernelEx(&cfg, grouped_conv3x3_pair_kernel, maps, a);
 }
 
 }  // namespace mt

@@ -89,6 +89,7 @@ struct Ctx {
     std::vector<HostModel> models;
     ModelDev* d_models = nullptr;
     int32_t* d_brief = nullptr;          // [1 + MT_MAX_LAYERS][max_models]: alive, out features per layer (bucketing passes)
+    unsigned* d_grid_bar = nullptr;      // [8] barrier counters of a call's multi-layer conv launches (zeroed by the bucketing kernel)
     int32_t* d_order = nullptr;          // [MT_MAX_LAYERS][max_models]: per layer, tenants by descending a-priori item cost
     bool last_pair[MT_MAX_LAYERS] = {false};   // executor form of each dense layer in the last mt_infer (balance report)
     CUtensorMap* d_wmaps = nullptr;      // [max_models][MT_MAX_LAYERS]: dense weights as 128 x 64 boxes of the tiled image
@@ -140,7 +141,7 @@ struct Ctx {
 
     // switches for tests and A/B timing: read from the environment once, at mt_init (MT_FUSED, MT_PAIR, MT_CONV_PAIR,
     // MT_POOL_HEAD; "0" turns the path off), changed afterwards only through mt_debug_set_option
-    bool opt_fused = true, opt_pair = true, opt_conv_pair = true, opt_pool_head = true;
+    bool opt_fused = true, opt_pair = true, opt_conv_pair = true, opt_pool_head = true, opt_conv_stack = true;
     int opt_gather = 1;                  // 0 never, 1 small batches, 2 always
 
     // tensor maps over the caller's images (first conv layer), kept while pointer and batch size stay the same
@@ -206,6 +207,8 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     CU_OK(cudaMemset(g.d_models, 0, sizeof(ModelDev) * (size_t)max_models));
     CU_OK(cudaMalloc(&g.d_brief, sizeof(int32_t) * (size_t)(1 + MT_MAX_LAYERS) * max_models));
     CU_OK(cudaMemset(g.d_brief, 0, sizeof(int32_t) * (size_t)(1 + MT_MAX_LAYERS) * max_models));
+    CU_OK(cudaMalloc(&g.d_grid_bar, sizeof(unsigned) * 8));
+    CU_OK(cudaMemset(g.d_grid_bar, 0, sizeof(unsigned) * 8));
     CU_OK(cudaMalloc(&g.d_order, sizeof(int32_t) * (size_t)MT_MAX_LAYERS * max_models));
     {
         std::vector<int32_t> ident((size_t)MT_MAX_LAYERS * max_models);
@@ -243,6 +246,7 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     g.opt_pair = env_on("MT_PAIR");
     g.opt_conv_pair = env_on("MT_CONV_PAIR");
     g.opt_pool_head = env_on("MT_POOL_HEAD");
+    g.opt_conv_stack = env_on("MT_CONV_STACK");
     { const char* v = getenv("MT_PERM_GATHER"); g.opt_gather = (v && v[0] >= '0' && v[0] <= '2') ? v[0] - '0' : 1; }
     g.init = true;
     return MT_OK;
@@ -740,6 +744,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
         BucketArgs a;
         a.ids = ids; a.n = n; a.T = g.T; a.models = g.d_models; a.n_layers = L; a.rows_per_unit = tiles_per_image;
         a.brief = g.d_brief; a.brief_ld = g.max_models; a.order = g.d_order;
+        a.grid_bar = conv_pair ? g.d_grid_bar : nullptr;
         for (int l = 0; l < 8; ++l) a.kind[l] = (l < L) ? g.family[l].kind : -1;
         a.ticket = g.d_ticket;
         a.rows_src = rows_in_scatter ? inputs : nullptr; a.rows_dst = g.act[0];
@@ -782,6 +787,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
         g.in_map_ptr = inputs;
         g.in_map_n = n;
     }
+    int n_conv_launch = 0;
     for (int l = 0; l < L; ++l) {
         const HostLayer& f = g.family[l];
         const bool last = (l == L - 1);
@@ -812,21 +818,39 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             a.models = g.d_models; a.layer = l; a.T = g.T; a.offsets = g.d_offsets;
             a.tile_prefix = g.d_tile_prefix + (size_t)l * (g.T + 1);
             a.perm = (l == 0) ? g.d_perm : nullptr;
-            a.out = (uint16_t*)g.act[l + 1];
-            const bool feeds_pool = (l + 1 < L) && g.family[l + 1].kind == MT_GLOBAL_AVG_POOL;
-            a.pool_partial = feeds_pool ? g.d_pool_partial : nullptr;
-            a.late_trigger = (conv_pair && l + 1 < L && g.family[l + 1].kind == MT_CONV3X3) ? 1 : 0;
-            a.early_lookup = (conv_pair && l > 0 && g.family[l - 1].kind == MT_CONV3X3) ? 1 : 0;
             a.H = f.h; a.W = f.w;
             a.Wp = g.conv.Wp; a.R = g.conv.R; a.tiles_per_strip = g.conv.tiles_per_strip;
             a.stage_bytes = g.conv.stage_bytes; a.n_stages = g.conv.n_stages;
             a.strips_per_image = g.conv.strips_per_image; a.box_bytes = g.conv.box_bytes;
             a.status = g.d_status;
-            // a layer that feeds the pool stores nothing: any valid map will do for it
-            if (conv_pair) CU_OK(launch_grouped_conv_pair(l == 0 ? in_rows2_map : g.act_rows2_map[l], l == 0 ? in_rows1_map : g.act_rows1_map[l],
-                                                          feeds_pool ? (l == 0 ? in_map : g.act_map[l]) : g.act_store_map[l + 1],
-                                                          a, g.sm_count, s));
-            else launch_grouped_conv(l == 0 ? in_map : g.act_map[l], a, g.conv.smem_bytes, g.sm_count, s);
+            const auto is_conv = [&](int k) { return k >= 0 && k < L && g.family[k].kind == MT_CONV3X3; };
+            const auto feeds_pool_at = [&](int k) { return k + 1 < L && g.family[k + 1].kind == MT_GLOBAL_AVG_POOL; };
+            if (conv_pair) {
+                // consecutive conv layers (at most kConvStackMax) as ONE launch with grid-wide barriers in between
+                int n_stack = 1;
+                while (n_stack < kConvStackMax && g.opt_conv_stack && is_conv(l + n_stack)) ++n_stack;
+                const int l_last = l + n_stack - 1;
+                ConvStackMaps maps;
+                for (int k = 0; k < n_stack; ++k) {
+                    const int lk = l + k;
+                    maps.x2[k] = lk == 0 ? in_rows2_map : g.act_rows2_map[lk];
+                    maps.x1[k] = lk == 0 ? in_rows1_map : g.act_rows1_map[lk];
+                    // a layer that feeds the pool stores nothing: any valid map will do for it
+                    maps.y[k] = feeds_pool_at(lk) ? (lk == 0 ? in_map : g.act_map[lk]) : g.act_store_map[lk + 1];
+                }
+                a.n_stack = n_stack;
+                a.grid_bar = g.d_grid_bar + (n_conv_launch++ & 7);
+                a.out = nullptr;
+                a.pool_partial = feeds_pool_at(l_last) ? g.d_pool_partial : nullptr;
+                a.late_trigger = is_conv(l_last + 1) ? 1 : 0;
+                a.early_lookup = is_conv(l - 1) ? 1 : 0;
+                CU_OK(launch_grouped_conv_pair(maps, a, g.sm_count, s));
+                l = l_last;
+            } else {
+                a.out = (uint16_t*)g.act[l + 1];
+                a.pool_partial = feeds_pool_at(l) ? g.d_pool_partial : nullptr;
+                launch_grouped_conv(l == 0 ? in_map : g.act_map[l], a, g.conv.smem_bytes, g.sm_count, s);
+            }
         } else if (pool_head && l == L - 2) {
             // pool + narrow last dense layer in one launch (the loop ends here: the head is done)
             Timer t(K_POOL, s);
@@ -879,6 +903,7 @@ mt_status mt_shutdown(void) {
     cudaFree(g.d_models); g.d_models = nullptr;
     cudaFree(g.d_brief); g.d_brief = nullptr;
     cudaFree(g.d_order); g.d_order = nullptr;
+    cudaFree(g.d_grid_bar); g.d_grid_bar = nullptr;
     cudaFree(g.d_wmaps); g.d_wmaps = nullptr;
     cudaFree(g.d_status); g.d_status = nullptr;
     cudaFree(g.d_ticket); g.d_ticket = nullptr;
@@ -1402,6 +1427,7 @@ mt_status mt_debug_set_option(const char* name, int32_t value) {
     else if (!strcmp(name, "pair")) g.opt_pair = on;
     else if (!strcmp(name, "conv_pair")) g.opt_conv_pair = on;
     else if (!strcmp(name, "pool_head")) g.opt_pool_head = on;
+    else if (!strcmp(name, "conv_stack")) g.opt_conv_stack = on;
     else if (!strcmp(name, "perm_gather")) g.opt_gather = value < 0 ? 0 : (value > 2 ? 2 : value);
     else return MT_ERR_INVALID_ARG;
     return MT_OK;

@@ -62,6 +62,7 @@ struct BucketArgs {
     int dst_ld_bytes;
     int item_grid;            // least number of CTAs of pass 2 (the work-item expansion wants the whole GPU)
     WorkItem* items[8];       // per dense layer: expanded work items (null for other layers)
+    unsigned* grid_bar;       // non-null: a word this call's conv launches use as their barrier counter; zeroed here
     int32_t* status;
 };
 
@@ -168,6 +169,8 @@ struct ConvArgs {
     // predecessor is complete when the next one starts.  early_lookup (only behind a launch with late_trigger, which is
     // not the bucketing itself): read the bucketing results and request the first weights BEFORE the dependency wait.
     int late_trigger = 0, early_lookup = 0;
+    int n_stack = 1;              // CTA-pair executor: conv layers run by this launch
+    unsigned* grid_bar = nullptr; // ... and the counter of their grid-wide barrier (zero when the launch starts)
     int32_t* status;
 };
 cudaError_t configure_grouped_conv();
@@ -181,11 +184,17 @@ constexpr int kConvPairImageOffset = 9 * 64 * 64;          // bf16 elements of t
 void launch_pretile_conv_pair(const uint16_t* w, uint16_t* out, cudaStream_t s);
 int conv_pair_smem_bytes();
 cudaError_t configure_grouped_conv_pair();
-// tmap_x2, tmap_x1: the layer's input (NHWC bf16) as boxes of 64 channels x 64 pixels x 2 rows and x 1 row (the executor
-// fetches the image in blocks of two rows, whatever ConvArgs says about strip stages); tmap_y: the layer's output as
-// boxes of 32 channels x 32 pixels x 1 row, 64-byte swizzle (unused by a layer that feeds the pool)
-cudaError_t launch_grouped_conv_pair(const CUtensorMap& tmap_x2, const CUtensorMap& tmap_x1, const CUtensorMap& tmap_y,
-                                     const ConvArgs& a, int sm_count, cudaStream_t s);
+// Up to kConvStackMax consecutive conv layers of one geometry run as ONE launch (ConvArgs::n_stack, from ConvArgs::layer
+// on; grid-wide barrier between layers on ConvArgs::grid_bar, a word the bucketing kernel of the call has zeroed).
+// Per layer of the stack: x2, x1 = its input (NHWC bf16) as boxes of 64 channels x 64 pixels x 2 rows and x 1 row (the
+// executor fetches the image in blocks of two rows, whatever ConvArgs says about strip stages); y = its output as boxes
+// of 32 channels x 32 pixels x 1 row, 64-byte swizzle (unused by a layer that feeds the pool).  ConvArgs::perm applies to
+// the stack's first layer, ConvArgs::pool_partial to its last.
+constexpr int kConvStackMax = 4;
+struct ConvStackMaps {
+    CUtensorMap x2[kConvStackMax], x1[kConvStackMax], y[kConvStackMax];
+};
+cudaError_t launch_grouped_conv_pair(const ConvStackMaps& maps, const ConvArgs& a, int sm_count, cudaStream_t s);
 
 // Second half of the fused pooling: sums the per-strip channel sums of each image and divides by H*W.
 void launch_pool_finalize(const float* partial, int n, int strips, int C, int HW, uint16_t* out, int ld_out,

@@ -28,10 +28,13 @@ def small_batch_path(request, monkeypatch):
     return request.param
 
 
-@pytest.fixture(params=["pair", "single"])
+@pytest.fixture(params=["pair", "pair_layerwise", "single"])
 def conv_path(request, monkeypatch):
-    """Conv layers whose padded row length is 64 pixels run on CTA pairs (two images of a tenant per cluster);
-    MT_CONV_PAIR=0 sends them to the one-CTA executor.  Tests that take this fixture run once on each."""
+    """Conv layers whose padded row length is 64 pixels run on CTA pairs (two images of a tenant per cluster), consecutive
+    conv layers as ONE launch with grid-wide barriers in between; MT_CONV_STACK=0 gives every conv layer a launch of its
+    own and MT_CONV_PAIR=0 sends them to the one-CTA executor.  Tests that take this fixture run once on each."""
     if request.param == "single":
         monkeypatch.setenv("MT_CONV_PAIR", "0")
+    elif request.param == "pair_layerwise":
+        monkeypatch.setenv("MT_CONV_STACK", "0")
     return request.param
