@@ -206,6 +206,8 @@ mt_status mt_debug_empty_launches(int32_t count, void* stream);
  *   "conv_pair"  (MT_CONV_PAIR)  CTA-pair conv executor for padded rows of 64 pixels; off: the one-CTA executor
  *   "conv_stack" (MT_CONV_STACK) consecutive conv layers of the CTA-pair executor as one launch with grid-wide barriers;
  *                off: one launch per conv layer
+ *   "conv_balance" (MT_CONV_BALANCE) the CTA-pair conv executor cuts its clusters' ranges by cost, a tenant border inside a
+ *                range counting as two units of work; off: ranges of equal length
  *   "pool_head"  (MT_POOL_HEAD)  pool + narrow head as one launch; off: pool_finalize + a grouped dense launch
  *   "perm_gather" (MT_PERM_GATHER) first dense layer reads the caller's rows through the permutation with TMA gathers
  *                instead of a row-move pass: 0 never, 1 (default) for batches of at most 256 requests, 2 always

@@ -140,10 +140,64 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ ConvStackMaps maps, const Co
     // contiguous range of pair-strips for this cluster: unit = (tenant, pair of images, strip of 2 tiles)
     const int total = p.tile_prefix[p.T];
     const int n_pairs = gridDim.x >> 1, pair_id = blockIdx.x >> 1;
-    const int s_begin = (int)(((long long)total * pair_id) / n_pairs);
-    const int s_end = (int)(((long long)total * (pair_id + 1)) / n_pairs);
+    int s_begin = (int)(((long long)total * pair_id) / n_pairs);
+    int s_end = (int)(((long long)total * (pair_id + 1)) / n_pairs);
     constexpr int Wp = 64;
     const int TS = p.tiles_per_strip;
+    // Ranges of equal COST rather than equal length: a tenant border inside a range stops the tensor pipe while the
+    // new weights come in, which is worth about p.border_units units of work (measured: the pairs that cross a border
+    // issue for 3 us longer than the others, and everybody waits for them at the end of each layer).  Every tenant
+    // border is charged that many units and the ranges split the total evenly; a range edge that falls into a border's
+    // charge snaps to the border itself, so neither neighbour pays for it.  The cost prefix over the tenants is built in
+    // shared memory (the output staging area is free before the first tile); more tenants than fit there keep the
+    // equal-length split.
+    constexpr int kMaxBalancedTenants = kCpOutStageBytes / 4 - 8;
+    if (p.border_units > 0 && p.T <= kMaxBalancedTenants && total > 0) {
+        int* s_cost = reinterpret_cast<int*>(out_stage_ptr);          // s_cost[t] = cost position of tenant t's first unit
+        if (warp == 2) {
+            // lane l scans its share of the tenants in order; the shares' border counts are then scanned across the warp
+            const int per = (p.T + 31) >> 5;
+            const int lo = min(lane * per, p.T), hi = min(lo + per, p.T);
+            int mine = 0;
+            for (int t = lo; t < hi; ++t) mine += (p.tile_prefix[t + 1] > p.tile_prefix[t]) ? 1 : 0;
+            int incl = mine;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int u = __shfl_up_sync(0xffffffffu, incl, d);
+                if (lane >= d) incl += u;
+            }
+            int before = incl - mine;                                 // tenants with units in front of this lane's share
+            for (int t = lo; t < hi; ++t) {
+                const int first = p.tile_prefix[t];
+                s_cost[t] = first + p.border_units * before;
+                before += (p.tile_prefix[t + 1] > first) ? 1 : 0;
+            }
+            if (lane == 31) s_cost[p.T] = total + p.border_units * max(before - 1, 0);   // total cost (the first tenant has no border)
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const long long total_cost = s_cost[p.T];
+            // unit at which cost position c is reached: the last tenant whose border charge starts at or before c
+            auto unit_at = [&](long long c) {
+                if (c <= 0) return 0;
+                if (c >= total_cost) return total;
+                int lo = 0, hi = p.T;                                  // largest t with s_cost[t] - border_units <= c
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if ((long long)s_cost[mid] - p.border_units <= c) lo = mid; else hi = mid;
+                }
+                const int first = p.tile_prefix[lo], units = p.tile_prefix[lo + 1] - first;
+                const long long into = c - s_cost[lo];
+                return first + (int)min((long long)units, max(into, 0LL));
+            };
+            s_first[6] = unit_at(total_cost * pair_id / n_pairs);
+            s_first[7] = unit_at(total_cost * (pair_id + 1) / n_pairs);
+        }
+        __syncthreads();
+        s_begin = s_first[6];
+        s_end = s_first[7];
+        __syncthreads();                                              // the staging area goes back to the epilogue
+    }
 
     // The first unit's tenant, its range of units and requests and its weight image: every thread looks at a few
     // tenants, all loads independent of one another, instead of a binary search of dependent loads by each role -
@@ -201,10 +255,9 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ ConvStackMaps maps, const Co
     // grid-wide counter and waits, for a bounded time, until all CTAs of the launch have (p.grid_bar was zeroed by the
     // bucketing kernel of this call).  Afterwards the layer's outputs may be read by anyone, also through TMA.
     auto layer_sync = [&](int k) {
-        asm volatile("fence.proxy.async;" ::: "memory");
-        __threadfence();
         __syncthreads();
         if (threadIdx.x == 0) {
+            __threadfence();            // cumulative: covers what the CTA's other threads wrote before the barrier above
             atomicAdd(p.grid_bar, 1u);
             const unsigned want = (unsigned)(k + 1) * gridDim.x;
             const uint64_t t0 = global_timer_ns();
@@ -560,7 +613,10 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ ConvStackMaps maps, const Co
         }
         if (k + 1 < n_stack) {
             // this layer's outputs must have reached memory before anyone passes the barrier
-            if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+            if (lane == 0) {
+                asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+                asm volatile("fence.proxy.async;" ::: "memory");
+            }
             __syncwarp();
             layer_sync(k);
         }

@@ -141,7 +141,7 @@ struct Ctx {
 
     // switches for tests and A/B timing: read from the environment once, at mt_init (MT_FUSED, MT_PAIR, MT_CONV_PAIR,
     // MT_POOL_HEAD; "0" turns the path off), changed afterwards only through mt_debug_set_option
-    bool opt_fused = true, opt_pair = true, opt_conv_pair = true, opt_pool_head = true, opt_conv_stack = true;
+    bool opt_fused = true, opt_pair = true, opt_conv_pair = true, opt_pool_head = true, opt_conv_stack = true, opt_conv_balance = true;
     int opt_gather = 1;                  // 0 never, 1 small batches, 2 always
 
     // tensor maps over the caller's images (first conv layer), kept while pointer and batch size stay the same
@@ -247,6 +247,7 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     g.opt_conv_pair = env_on("MT_CONV_PAIR");
     g.opt_pool_head = env_on("MT_POOL_HEAD");
     g.opt_conv_stack = env_on("MT_CONV_STACK");
+    g.opt_conv_balance = env_on("MT_CONV_BALANCE");
     { const char* v = getenv("MT_PERM_GATHER"); g.opt_gather = (v && v[0] >= '0' && v[0] <= '2') ? v[0] - '0' : 1; }
     g.init = true;
     return MT_OK;
@@ -839,6 +840,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
                     maps.y[k] = feeds_pool_at(lk) ? (lk == 0 ? in_map : g.act_map[lk]) : g.act_store_map[lk + 1];
                 }
                 a.n_stack = n_stack;
+                a.border_units = g.opt_conv_balance ? 2 : 0;
                 a.grid_bar = g.d_grid_bar + (n_conv_launch++ & 7);
                 a.out = nullptr;
                 a.pool_partial = feeds_pool_at(l_last) ? g.d_pool_partial : nullptr;
@@ -1428,6 +1430,7 @@ mt_status mt_debug_set_option(const char* name, int32_t value) {
     else if (!strcmp(name, "conv_pair")) g.opt_conv_pair = on;
     else if (!strcmp(name, "pool_head")) g.opt_pool_head = on;
     else if (!strcmp(name, "conv_stack")) g.opt_conv_stack = on;
+    else if (!strcmp(name, "conv_balance")) g.opt_conv_balance = on;
     else if (!strcmp(name, "perm_gather")) g.opt_gather = value < 0 ? 0 : (value > 2 ? 2 : value);
     else return MT_ERR_INVALID_ARG;
     return MT_OK;

@@ -169,6 +169,8 @@ struct ConvArgs {
     // predecessor is complete when the next one starts.  early_lookup (only behind a launch with late_trigger, which is
     // not the bucketing itself): read the bucketing results and request the first weights BEFORE the dependency wait.
     int late_trigger = 0, early_lookup = 0;
+    int border_units = 0;         // CTA-pair executor: work units a tenant border inside a cluster's range is charged when
+                                  // the ranges are cut (0: ranges of equal length)
     int n_stack = 1;              // CTA-pair executor: conv layers run by this launch
     unsigned* grid_bar = nullptr; // ... and the counter of their grid-wide barrier (zero when the launch starts)
     int32_t* status;
