@@ -267,15 +267,15 @@ bucket_hist_scan(const int32_t* __restrict__ ids, int n, int T, Brief br, int n_
 struct ItemPtrs { WorkItem* v[8]; };
 
 // Work item `item` of dense layer l: (tenant, row tile, column tile) and what the executor needs to know about it.
-__device__ __forceinline__ WorkItem make_work_item(int item, int l, int T, const ModelDev* __restrict__ models, Brief br,
-                                                   const int32_t* __restrict__ offsets,
+__device__ __forceinline__ WorkItem make_work_item(int item, int l, int T, const ModelDev* __restrict__ models,
+                                                   const int32_t* order_row, const int32_t* __restrict__ offsets,
                                                    const int32_t* __restrict__ prefix, int tile_m) {
     int lo = 0, hi = T;   // largest rank r with prefix[r] <= item
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
         if (prefix[mid] <= item) lo = mid; else hi = mid;
     }
-    const int t = tenant_at(br, l, lo);        // lo is a rank in the layer's cost order
+    const int t = order_row[lo];               // lo is a rank in the layer's cost order
     const LayerDev& L = models[t].layer[l];
     const int seg0 = offsets[t], n_t = offsets[t + 1] - seg0;
     const int m_tiles = (n_t + tile_m - 1) / tile_m;
@@ -422,7 +422,7 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
         for (int t = threadIdx.x; t < T1; t += nthr) s_cnt[t] = prefix[t];
         __syncthreads();
         const int n_items = s_cnt[T];
-        for (int item = threadIdx.x; item < n_items; item += nthr) out[item] = make_work_item(item, l, T, models, br, offsets, s_cnt, tn.m[l]);
+        for (int item = threadIdx.x; item < n_items; item += nthr) out[item] = make_work_item(item, l, T, models, br.order + (size_t)l * br.ld, offsets, s_cnt, tn.m[l]);
         __syncthreads();
     }
 }
@@ -438,7 +438,7 @@ bucket_scatter_expand(const int32_t* __restrict__ ids, int n, int T, const Model
                       const int32_t* __restrict__ block_hist, const int32_t* __restrict__ offsets,
                       int32_t* __restrict__ perm, int32_t* __restrict__ inv, const uint4* __restrict__ rows_src,
                       uint4* __restrict__ rows_dst, int row_vec, int dst_ld_vec, int n_layers, LayerTileN tn,
-                      const int32_t* __restrict__ tile_prefix, ItemPtrs items) {
+                      const int32_t* __restrict__ tile_prefix, ItemPtrs items, int all_layers_at_once) {
     pdl_launch_dependents();
     pdl_wait();
     extern __shared__ int32_t s_next[];   // T + 1: next free position of every bucket for this block; then s_pos[chunk]
@@ -516,7 +516,38 @@ bucket_scatter_expand(const int32_t* __restrict__ ids, int n, int T, const Model
         }
         __syncthreads();      // s_next is reused below
     }
-    // work items: the layer's unit prefix sums go to shared memory first, so the search per item stays on the SM
+    // work items: the layers' unit prefix sums (and their tenant orders) go to shared memory first, so the search per
+    // item stays on the SM
+    if (all_layers_at_once) {
+        // every dense layer's rows at once and ONE loop over the items of all layers: the chain of dependent loads
+        // (prefixes -> tenant -> its table entry and offsets) is paid once, not once per layer
+        int32_t* s_all = s_next;                     // per item layer q: prefix row [T1], then order row [T1]
+        int n_q = 0;
+        for (int l = 0; l < n_layers; ++l) {
+            if (!items.v[l]) continue;
+            const int32_t* prefix = tile_prefix + (size_t)l * (T + 1);
+            const int32_t* ord = br.order + (size_t)l * br.ld;
+            int32_t* row = s_all + (size_t)n_q * 2 * T1;
+            for (int t = threadIdx.x; t < T1; t += blockDim.x) { row[t] = prefix[t]; row[T1 + t] = (t < T) ? __ldg(ord + t) : 0; }
+            ++n_q;
+        }
+        __syncthreads();
+        int done = 0, q = 0;                         // items of the layers before the current one
+        for (int l = 0; l < n_layers; ++l) {
+            WorkItem* out = items.v[l];
+            if (!out) continue;
+            const int32_t* row = s_all + (size_t)q * 2 * T1;
+            const int total = row[T];
+            // global item numbers [done, done + total) belong to this layer; a thread's items keep the grid stride
+            const int first = blockIdx.x * blockDim.x + threadIdx.x, stride = gridDim.x * blockDim.x;
+            int g = first + ((done > first) ? ((done - first + stride - 1) / stride) * stride : 0);
+            for (; g < done + total; g += stride)
+                out[g - done] = make_work_item(g - done, l, T, models, row + T1, offsets, row, tn.m[l]);
+            done += total;
+            ++q;
+        }
+        return;
+    }
     for (int l = 0; l < n_layers; ++l) {
         WorkItem* out = items.v[l];
         if (!out) continue;
@@ -525,7 +556,7 @@ bucket_scatter_expand(const int32_t* __restrict__ ids, int n, int T, const Model
         __syncthreads();
         const int total = s_next[T];
         for (int item = blockIdx.x * blockDim.x + threadIdx.x; item < total; item += gridDim.x * blockDim.x)
-            out[item] = make_work_item(item, l, T, models, br, offsets, s_next, tn.m[l]);
+            out[item] = make_work_item(item, l, T, models, br.order + (size_t)l * br.ld, offsets, s_next, tn.m[l]);
         __syncthreads();
     }
 }
@@ -582,6 +613,12 @@ static int grid_for(long long total, int threads, int sm_count) {
     return (int)blocks;
 }
 
+constexpr size_t kScatterSmemMax = 96 * 1024;      // two CTAs of the scatter pass still fit an SM
+
+cudaError_t configure_bucketing() {
+    return cudaFuncSetAttribute(bucket_scatter_expand, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScatterSmemMax);
+}
+
 void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
     const int n_blocks = (a.n + kBucketChunk - 1) / kBucketChunk;
     const int n_hist_blocks = (a.n + kHistChunk - 1) / kHistChunk;
@@ -602,9 +639,16 @@ void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
     launch_pdl(bucket_hist_scan, dim3(n_hist_blocks), dim3(kHistChunk), smem, s, a.ids, a.n, a.T, br, a.n_layers, a.rows_per_unit, tn,
                a.block_hist, a.counts, a.offsets, a.tile_prefix, a.ticket, a.status, a.grid_bar);
     const int grid2 = n_blocks > a.item_grid ? n_blocks : a.item_grid;
-    launch_pdl(bucket_scatter_expand, dim3(grid2), dim3(kScatterThreads), smem + sizeof(int32_t) * kBucketChunk, s, a.ids, a.n, a.T, a.models, br,
+    // shared memory: the scatter's positions, or (larger) prefix and order rows of every layer that has work items
+    int item_layers = 0;
+    for (int l = 0; l < a.n_layers && l < 8; ++l) item_layers += a.items[l] ? 1 : 0;
+    const size_t smem_scatter = smem + sizeof(int32_t) * kBucketChunk;
+    const size_t smem_items = sizeof(int32_t) * 2 * (size_t)(a.T + 1) * item_layers;
+    const int at_once = (item_layers > 1 && smem_items <= kScatterSmemMax) ? 1 : 0;
+    launch_pdl(bucket_scatter_expand, dim3(grid2), dim3(kScatterThreads), (at_once && smem_items > smem_scatter) ? smem_items : smem_scatter, s,
+               a.ids, a.n, a.T, a.models, br,
                a.block_hist, a.offsets, a.perm, a.inv, (const uint4*)a.rows_src, (uint4*)a.rows_dst, a.row_bytes / 16,
-               a.dst_ld_bytes / 16, a.n_layers, tn, a.tile_prefix, ip);
+               a.dst_ld_bytes / 16, a.n_layers, tn, a.tile_prefix, ip, at_once);
 }
 
 void launch_gather_rows(const void* src, const int32_t* perm, int n, int row_bytes, void* dst, int dst_ld_bytes,

@@ -230,6 +230,7 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     CU_OK(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
     if (!fn || qres != cudaDriverEntryPointSuccess) return MT_ERR_CUDA;
     g.encode = reinterpret_cast<EncodeTiledFn>(fn);
+    CU_OK(configure_bucketing());
     CU_OK(configure_grouped_gemm());
     CU_OK(configure_grouped_conv());
     CU_OK(configure_grouped_gemm_pair());

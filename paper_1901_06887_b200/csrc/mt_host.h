@@ -66,6 +66,7 @@ struct BucketArgs {
     int32_t* status;
 };
 
+cudaError_t configure_bucketing();
 void launch_bucketing(const BucketArgs& a, cudaStream_t s);
 // One thread waits (bounded by limit_ns) on a barrier nobody completes; *gave_up = 1 and the status word is set.
 void launch_wait_timeout_probe(int32_t* status, unsigned long long limit_ns, int32_t* gave_up, cudaStream_t s);
