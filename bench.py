@@ -54,6 +54,10 @@ REFERENCE_SAMPLE = {1: 64, 2: 512, 3: 4096, 4: 6, 5: 24}
 # weights of the tenants that have requests, as the algorithmic bytes do); "bytes": measured at full size, per step.
 # An entry is deleted when its kernel changes and comes back with the next capture.
 TRAFFIC = {
+    2: {"ratio": 0.997, "source": "profiles/grouped_gemm_c2_reduced_ncu_full.md (16 tenants, 1024 requests: 843.0 MB "
+                                  "measured / 845.8 MB algorithmic), scaled by algorithmic bytes"},
+    3: {"ratio": 1.007, "source": "profiles/grouped_gemm128_c3_reduced_ncu_full.md (250 tenants, 4096 requests: 272.1 MB "
+                                  "measured / 270.0 MB algorithmic), scaled by algorithmic bytes"},
     4: {"bytes": 608.5e6, "source": "profiles/grouped_conv3x3_pair_c4_full_ncu_full.md (full size, four conv launches)"},
 }
 

@@ -80,7 +80,13 @@ mt_status mt_shutdown(void);
  * output element counts, same conv geometry.  Hidden dense widths may differ per model.
  * Kernel limits (else MT_ERR_UNSUPPORTED): 1..MT_MAX_LAYERS layers; dense in_ch a multiple of 64;
  * conv in_ch == out_ch == 64, w <= 126; a pool must follow a conv; a dense layer may not precede a conv.
- * Synchronous: returns after the copies have completed. */
+ * The call does not wait for the device: weights and biases in HOST memory are copied into the library's pinned
+ * staging before it returns (the caller may free them at once), and the copy to the device and the re-layout run on
+ * an internal stream, under whatever batches are in flight; the first mt_infer* / mt_prefetch that follows waits, on
+ * its own stream, for exactly the models it is the first to see.  Weights given as DEVICE pointers are read by that
+ * internal stream, for which the call then waits (not for the device).  A model wider than any before makes the next
+ * mt_infer* reallocate its workspace, which does synchronise the device.  MT_ASYNC_REGISTER=0 (option
+ * "async_register") selects the older path that synchronises the device once per layer. */
 mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32_t* model_id_out);
 
 /* predict(model, input) for a whole mixed batch (Sec. 3: a worker multiplexes requests across models).
@@ -122,7 +128,8 @@ mt_status mt_release(int32_t model_id);
  * so the time to bring it in is predictable, and GPU memory need only hold the models in demand).  By default every
  * registered model stays on the device.  mt_set_cache_bytes(B), called after mt_init while no model is registered,
  * switches to a cache of B device bytes (one arena, allocated once; 0 switches back): registration then also keeps the
- * model's block - weights in the executor's layout and biases - in pinned host memory, and the device holds the least
+ * model's block - weights in the executor's layout and biases - in pinned host memory (copied back from the device on
+ * the internal stream once the re-layout has run), and the device holds the least
  * recently used subset that fits.  MT_ERR_OOM: the arena cannot be allocated; a model larger than B is refused at
  * registration with MT_ERR_OOM.
  *
@@ -208,6 +215,7 @@ mt_status mt_debug_empty_launches(int32_t count, void* stream);
  *                off: one launch per conv layer
  *   "conv_balance" (MT_CONV_BALANCE) the CTA-pair conv executor cuts its clusters' ranges by cost, a tenant border inside a
  *                range counting as two units of work; off: ranges of equal length
+ *   "async_register" (MT_ASYNC_REGISTER) registration without device synchronisation; off: synchronous registration
  *   "pool_head"  (MT_POOL_HEAD)  pool + narrow head as one launch; off: pool_finalize + a grouped dense launch
  *   "perm_gather" (MT_PERM_GATHER) first dense layer reads the caller's rows through the permutation with TMA gathers
  *                instead of a row-move pass: 0 never, 1 (default) for batches of at most 256 requests, 2 always

@@ -41,6 +41,13 @@ struct HostModel {
     void* host_image = nullptr;
     std::vector<size_t> w_off, b_off;      // per layer: offsets of weights and bias inside the block
     uint64_t last_batch = 0;               // number of the last batch that may have read the block
+    cudaEvent_t ready = nullptr;           // asynchronous registration: the block's copies and re-layout have finished
+};
+
+// A change of the device tables that waits for the next call that names a stream (registration has none).
+struct PendingOp {
+    int id;
+    int kind;                              // 1: the model's block is (being made) ready - publish its entry; 2: evicted
 };
 
 // What a tenant's entry in the device tables becomes when its block is (re)loaded or evicted: passed BY VALUE to a
@@ -53,7 +60,8 @@ struct TableUpdate {
     int32_t id, n_wmaps;
 };
 
-__global__ void table_update_kernel(const __grid_constant__ TableUpdate u, ModelDev* models, int32_t* brief, CUtensorMap* wmaps) {
+__global__ void table_update_kernel(const __grid_constant__ TableUpdate u, ModelDev* models, int32_t* brief, int brief_ld,
+                                    CUtensorMap* wmaps) {
     const int t = threadIdx.x;
     if (u.alive == 1) {
         const int n_words = sizeof(ModelDev) / 4;
@@ -70,6 +78,8 @@ __global__ void table_update_kernel(const __grid_constant__ TableUpdate u, Model
         models[u.id].alive = u.alive;
     }
     if (t == 0) brief[u.id] = u.alive;
+    if (u.alive == 1 && t >= 1 && t <= MT_MAX_LAYERS)      // rows 1..: out features per layer (0: the model has no such layer)
+        brief[(size_t)t * brief_ld + u.id] = (t - 1 < u.md.n_layers) ? u.md.layer[t - 1].N : 0;
 }
 
 enum KernelId { K_BUCKET = 0, K_GATHER, K_GEMM, K_CONV, K_POOL, K_FUSED, K_COUNT };
@@ -162,6 +172,19 @@ struct Ctx {
     cudaEvent_t loads_done = nullptr;
     uint64_t request_hits = 0, request_misses = 0;
 
+    // asynchronous registration: staging for the caller's weights (pinned host + device mirror), table changes that
+    // wait for a stream, and the host mirror of the per-layer tenant order
+    void* reg_host = nullptr;
+    void* reg_dev = nullptr;
+    size_t reg_host_cap = 0, reg_dev_cap = 0;
+    cudaEvent_t reg_h2d_done = nullptr;                 // the staging copy of the last registration has left pinned memory
+    bool reg_h2d_pending = false;
+    std::vector<PendingOp> pending_ops;
+    int32_t* h_order = nullptr;                         // pinned, [MT_MAX_LAYERS][max_models]
+    bool order_dirty = false, order_copy_pending = false;
+    cudaEvent_t order_copied = nullptr;
+    bool opt_async_register = true;
+
     // timing
     int timing = 0;                      // 0 off, 1 every kernel, 2 only the layer executors, 3 the same on every 4th call
     int timing_now = 0;                  // the mode in force for the current call (0, 1 or 2)
@@ -210,11 +233,14 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     CU_OK(cudaMalloc(&g.d_grid_bar, sizeof(unsigned) * 8));
     CU_OK(cudaMemset(g.d_grid_bar, 0, sizeof(unsigned) * 8));
     CU_OK(cudaMalloc(&g.d_order, sizeof(int32_t) * (size_t)MT_MAX_LAYERS * max_models));
-    {
-        std::vector<int32_t> ident((size_t)MT_MAX_LAYERS * max_models);
-        for (size_t i = 0; i < ident.size(); ++i) ident[i] = (int32_t)(i % (size_t)max_models);
-        CU_OK(cudaMemcpy(g.d_order, ident.data(), sizeof(int32_t) * ident.size(), cudaMemcpyHostToDevice));
-    }
+    CU_OK(cudaMallocHost(&g.h_order, sizeof(int32_t) * (size_t)MT_MAX_LAYERS * max_models));
+    for (size_t i = 0; i < (size_t)MT_MAX_LAYERS * max_models; ++i) g.h_order[i] = (int32_t)(i % (size_t)max_models);
+    CU_OK(cudaMemcpy(g.d_order, g.h_order, sizeof(int32_t) * (size_t)MT_MAX_LAYERS * max_models, cudaMemcpyHostToDevice));
+    if (!g.load_stream) CU_OK(cudaStreamCreateWithFlags(&g.load_stream, cudaStreamNonBlocking));
+    if (!g.reg_h2d_done) CU_OK(cudaEventCreateWithFlags(&g.reg_h2d_done, cudaEventDisableTiming));
+    if (!g.order_copied) CU_OK(cudaEventCreateWithFlags(&g.order_copied, cudaEventDisableTiming));
+    g.order_dirty = false; g.order_copy_pending = false; g.reg_h2d_pending = false;
+    g.pending_ops.clear();
     CU_OK(cudaMalloc(&g.d_wmaps, sizeof(CUtensorMap) * (size_t)max_models * MT_MAX_LAYERS));
     CU_OK(cudaMalloc(&g.d_status, sizeof(int32_t) * ST_WORDS));
     CU_OK(cudaMalloc(&g.d_ticket, sizeof(int32_t)));
@@ -248,6 +274,7 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     g.opt_conv_pair = env_on("MT_CONV_PAIR");
     g.opt_pool_head = env_on("MT_POOL_HEAD");
     g.opt_conv_stack = env_on("MT_CONV_STACK");
+    g.opt_async_register = env_on("MT_ASYNC_REGISTER");
     g.opt_conv_balance = env_on("MT_CONV_BALANCE");
     { const char* v = getenv("MT_PERM_GATHER"); g.opt_gather = (v && v[0] >= '0' && v[0] <= '2') ? v[0] - '0' : 1; }
     g.init = true;
@@ -434,7 +461,43 @@ mt_status fill_table_update(int id, uint8_t* base, TableUpdate* u) {
 }
 
 void launch_table_update(const TableUpdate& u, cudaStream_t s) {
-    table_update_kernel<<<1, 128, 0, s>>>(u, g.d_models, g.d_brief, g.d_wmaps);
+    table_update_kernel<<<1, 128, 0, s>>>(u, g.d_models, g.d_brief, g.max_models, g.d_wmaps);
+}
+
+// Registration and release change the device tables without naming a stream; the changes are applied here, in stream
+// order, by the next call that does: a model whose block is ready (or becomes ready on the load stream: `s` waits for
+// its event) gets its table entry, an evicted one is marked, and the per-layer tenant order is uploaded from its
+// pinned mirror.
+mt_status flush_tables(cudaStream_t s) {
+    if (!g.pending_ops.empty()) {
+        for (const PendingOp& op : g.pending_ops) {
+            HostModel& hm = g.models[op.id];
+            TableUpdate u;
+            if (op.kind == 1) {
+                if (!hm.alive) continue;                                         // released in the meantime
+                if (g.cache_bytes && !g.cache.resident(op.id)) continue;         // evicted again before it was ever used
+                if (hm.ready) CU_OK(cudaStreamWaitEvent(s, hm.ready, 0));
+                uint8_t* base = g.cache_bytes ? g.arena + g.cache.find(op.id)->off : static_cast<uint8_t*>(hm.dev_block);
+                mt_status st = fill_table_update(op.id, base, &u);
+                if (st != MT_OK) return st;
+            } else {
+                if (!hm.alive || !g.cache_bytes || g.cache.resident(op.id)) continue;   // gone, or back already
+                memset(&u, 0, sizeof u);
+                u.id = op.id; u.alive = 2;
+            }
+            launch_table_update(u, s);
+        }
+        g.pending_ops.clear();
+        CU_OK(cudaGetLastError());
+    }
+    if (g.order_dirty) {
+        CU_OK(cudaMemcpyAsync(g.d_order, g.h_order, sizeof(int32_t) * (size_t)MT_MAX_LAYERS * g.max_models,
+                              cudaMemcpyHostToDevice, s));
+        CU_OK(cudaEventRecord(g.order_copied, s));
+        g.order_copy_pending = true;
+        g.order_dirty = false;
+    }
+    return MT_OK;
 }
 
 // Make the given tenants resident for the batch that is about to be enqueued on `s` (ids unique and live; reqs[i] =
@@ -445,6 +508,10 @@ void launch_table_update(const TableUpdate& u, cudaStream_t s) {
 // not fit the cache (nothing of this batch has been enqueued; tenants evicted on the way stay evicted).
 mt_status ensure_resident(const std::vector<int>& ids, const std::vector<int>& reqs, cudaStream_t s) {
     if (!g.cache_bytes || ids.empty()) return MT_OK;
+    {
+        mt_status fs = flush_tables(s);
+        if (fs != MT_OK) return fs;
+    }
     const uint64_t tick = ++g.cache_tick;
     struct Load { int id; size_t off; };
     std::vector<Load> loads;
@@ -540,6 +607,10 @@ double item_cost_cycles(int k_blocks, int n_cols, int rows) {
 // back and forth over their CTAs (longest-processing-time-first list scheduling with costs known a priori).
 mt_status recompute_order() {
     if (!g.has_family || g.T == 0) return MT_OK;
+    if (g.order_copy_pending) {             // the pinned mirror may still be the source of a copy in flight
+        CU_OK(cudaEventSynchronize(g.order_copied));
+        g.order_copy_pending = false;
+    }
     std::vector<int32_t> row(g.T);
     std::vector<double> cost(g.T);
     for (size_t l = 0; l < g.family.size(); ++l) {
@@ -554,8 +625,9 @@ mt_status recompute_order() {
         }
         if (g.family[l].kind == MT_DENSE)
             std::stable_sort(row.begin(), row.end(), [&](int32_t a, int32_t b) { return cost[a] > cost[b]; });
-        CU_OK(cudaMemcpy(g.d_order + l * (size_t)g.max_models, row.data(), sizeof(int32_t) * g.T, cudaMemcpyHostToDevice));
+        memcpy(g.h_order + l * (size_t)g.max_models, row.data(), sizeof(int32_t) * g.T);
     }
+    g.order_dirty = true;      // uploaded, in stream order, by the next call that names a stream (flush_tables)
     return MT_OK;
 }
 
@@ -680,6 +752,8 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
     if (!g.has_family || g.live == 0) return MT_ERR_BAD_MODEL_ID;
     CU_OK(cudaSetDevice(g.device));
     mt_status st = ensure_workspace(n);
+    if (st != MT_OK) return st;
+    st = flush_tables(s);
     if (st != MT_OK) return st;
     const int L = (int)g.family.size();
     const HostLayer& f0 = g.family[0];
@@ -874,6 +948,170 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
     return MT_OK;
 }
 
+// Host-side bookkeeping of a freshly registered model (both registration paths).
+mt_status adopt_model(int id, const std::vector<HostLayer>& hl, uint8_t* block, size_t total, void* host_image,
+                      const std::vector<size_t>& w_off, const std::vector<size_t>& b_off, cudaEvent_t ready) {
+    const int n_layers = (int)hl.size();
+    if (!g.has_family || g.live == 0) {
+        g.family = hl;
+        g.has_family = true;
+        g.in_elems = layer_in_elems(hl[0]);
+        g.out_elems = hl.back().out_ch;
+        for (const HostLayer& f : hl)
+            if (f.kind == MT_CONV3X3) plan_conv(f.h, f.w, &g.conv);   // cannot fail: validate_layers bounds w
+        for (int b = 0; b <= MT_MAX_LAYERS; ++b) g.width[b] = 0;
+        g.ws_dirty = true;
+        g.in_map_ptr = nullptr;
+        free_staging();   // sized for the previous family's rows (no model is live: nothing is in flight)
+    }
+    if ((size_t)n_layers > g.family.size()) {      // a deeper MLP joins: the family gains launches
+        for (size_t l = g.family.size(); l < (size_t)n_layers; ++l) g.family.push_back(hl[l]);
+        g.ws_dirty = true;
+    }
+    for (int l = 0; l < n_layers; ++l) {
+        const int wd = layer_in_elems(hl[l]);
+        if (wd > g.width[l]) { g.width[l] = wd; g.ws_dirty = true; }
+    }
+    HostModel& hm = g.models[id];
+    hm.alive = true;
+    hm.layers = hl;
+    hm.dev_block = g.cache_bytes ? nullptr : block;
+    hm.block_bytes = total;
+    hm.host_image = host_image;
+    hm.w_off = w_off;
+    hm.b_off = b_off;
+    hm.last_batch = 0;
+    if (hm.ready && hm.ready != ready) cudaEventDestroy(hm.ready);
+    hm.ready = ready;
+    g.live += 1;
+    if (id + 1 > g.T) g.T = id + 1;
+    recompute_tile_n();
+    return recompute_order();
+}
+
+// Registration without stalling the device.  The caller's weights and biases are copied into pinned staging on the
+// host (so the caller may free them on return, as before), everything else - the copy to the device, the re-layout
+// into the executor's tiled images, with the cache on also the copy of the finished block back to its pinned host
+// image - is enqueued on the library's load stream and overlaps whatever batches are running.  The model's entry in
+// the device tables is written by the next call that names a stream, which first waits for the model's event.
+// Weights given as DEVICE pointers are read by the load stream directly; the call then waits for that stream alone.
+mt_status register_async(const mt_layer_desc* layers, const std::vector<HostLayer>& hl, int id, size_t total,
+                         const std::vector<size_t>& w_off, const std::vector<size_t>& b_off, int32_t* model_id_out) {
+    const int n_layers = (int)hl.size();
+    // staging layout: per layer the raw weights, then the bias, 256-byte aligned pieces
+    std::vector<size_t> sw(n_layers, 0), sb(n_layers, 0);
+    size_t need = 0;
+    bool device_source = false;
+    for (int l = 0; l < n_layers; ++l) {
+        const HostLayer& h = hl[l];
+        if (h.kind == MT_GLOBAL_AVG_POOL) continue;
+        const size_t raw = (size_t)h.out_ch * h.in_ch * 2 * (h.kind == MT_CONV3X3 ? 9 : 1);
+        sw[l] = need; need += align_up(raw, 256);
+        sb[l] = need; need += align_up(sizeof(float) * h.out_ch, 256);
+        if (is_device_pointer(layers[l].weight) || (layers[l].bias && is_device_pointer(layers[l].bias))) device_source = true;
+    }
+    if (need > g.reg_host_cap || need > g.reg_dev_cap) {
+        // grow the staging (rare: sized for the largest model seen, with headroom); the load stream must be done with it
+        CU_OK(cudaStreamSynchronize(g.load_stream));
+        g.reg_h2d_pending = false;
+        const size_t cap = align_up(need + need / 2, (size_t)1 << 20);
+        if (g.reg_host) cudaFreeHost(g.reg_host);
+        cudaFree(g.reg_dev);
+        g.reg_host = nullptr; g.reg_dev = nullptr; g.reg_host_cap = g.reg_dev_cap = 0;
+        CU_OK(cudaMallocHost(&g.reg_host, cap));
+        CU_OK(cudaMalloc(&g.reg_dev, cap));
+        g.reg_host_cap = g.reg_dev_cap = cap;
+    }
+    uint8_t* block = nullptr;
+    std::vector<int> evicted;
+    if (g.cache_bytes) {
+        size_t off = 0;
+        if (g.cache.acquire(id, total, ++g.cache_tick, &off, &evicted) == WeightCache::kNoRoom) return MT_ERR_OOM;
+        block = g.arena + off;
+        // the victims' bytes may still be read by batches in flight; their table entries flip at the next flush
+        uint64_t youngest = 0;
+        for (int v : evicted) {
+            g.pending_ops.push_back({v, 2});
+            if (g.models[v].last_batch > youngest) youngest = g.models[v].last_batch;
+        }
+        if (youngest > g.synced_batch && youngest <= g.batch_no)
+            CU_OK(cudaStreamWaitEvent(g.load_stream, g.batch_done[youngest % Ctx::kBatchEvents], 0));
+    } else {
+        CU_OK(cudaMalloc(&block, total));
+    }
+    auto fail = [&](cudaError_t e) {
+        if (g.cache_bytes) g.cache.release(id); else cudaFree(block);
+        cudaGetLastError();
+        return e == cudaErrorMemoryAllocation ? MT_ERR_OOM : MT_ERR_CUDA;
+    };
+    // the previous registration's staging copy must have left pinned memory before it is overwritten
+    if (g.reg_h2d_pending) {
+        cudaError_t e = cudaEventSynchronize(g.reg_h2d_done);
+        if (e != cudaSuccess) return fail(e);
+        g.reg_h2d_pending = false;
+    }
+    uint8_t* hs = static_cast<uint8_t*>(g.reg_host);
+    uint8_t* ds = static_cast<uint8_t*>(g.reg_dev);
+    cudaStream_t ls = g.load_stream;
+    cudaError_t e = cudaMemsetAsync(block, 0, total, ls);
+    for (int l = 0; l < n_layers && e == cudaSuccess; ++l) {
+        const HostLayer& h = hl[l];
+        if (h.kind == MT_GLOBAL_AVG_POOL) continue;
+        const size_t raw = (size_t)h.out_ch * h.in_ch * 2 * (h.kind == MT_CONV3X3 ? 9 : 1);
+        if (is_device_pointer(layers[l].weight)) e = cudaMemcpyAsync(ds + sw[l], layers[l].weight, raw, cudaMemcpyDeviceToDevice, ls);
+        else memcpy(hs + sw[l], layers[l].weight, raw);
+        if (e != cudaSuccess) break;
+        if (layers[l].bias) {
+            if (is_device_pointer(layers[l].bias)) e = cudaMemcpyAsync(ds + sb[l], layers[l].bias, sizeof(float) * h.out_ch, cudaMemcpyDeviceToDevice, ls);
+            else memcpy(hs + sb[l], layers[l].bias, sizeof(float) * h.out_ch);
+        }
+    }
+    // host-resident pieces: one copy of the staging per piece (device-resident pieces were copied above)
+    for (int l = 0; l < n_layers && e == cudaSuccess; ++l) {
+        const HostLayer& h = hl[l];
+        if (h.kind == MT_GLOBAL_AVG_POOL) continue;
+        const size_t raw = (size_t)h.out_ch * h.in_ch * 2 * (h.kind == MT_CONV3X3 ? 9 : 1);
+        if (!is_device_pointer(layers[l].weight)) e = cudaMemcpyAsync(ds + sw[l], hs + sw[l], raw, cudaMemcpyHostToDevice, ls);
+        if (e == cudaSuccess && layers[l].bias && !is_device_pointer(layers[l].bias))
+            e = cudaMemcpyAsync(ds + sb[l], hs + sb[l], sizeof(float) * h.out_ch, cudaMemcpyHostToDevice, ls);
+    }
+    if (e == cudaSuccess) e = cudaEventRecord(g.reg_h2d_done, ls);
+    if (e != cudaSuccess) return fail(e);
+    g.reg_h2d_pending = true;
+    for (int l = 0; l < n_layers && e == cudaSuccess; ++l) {
+        const HostLayer& h = hl[l];
+        if (h.kind == MT_GLOBAL_AVG_POOL) continue;
+        const uint16_t* src = reinterpret_cast<const uint16_t*>(ds + sw[l]);
+        if (h.kind == MT_DENSE) launch_pretile_dense(src, h.out_ch, h.in_ch, (uint16_t*)(block + w_off[l]), ls);
+        else {
+            launch_pretile_conv(src, h.out_ch, h.in_ch, (uint16_t*)(block + w_off[l]), ls);
+            launch_pretile_conv_pair(src, (uint16_t*)(block + w_off[l]) + kConvPairImageOffset, ls);
+        }
+        e = cudaGetLastError();
+        if (e == cudaSuccess && layers[l].bias)
+            e = cudaMemcpyAsync(block + b_off[l], ds + sb[l], sizeof(float) * h.out_ch, cudaMemcpyDeviceToDevice, ls);
+    }
+    void* host_image = nullptr;
+    if (e == cudaSuccess && g.cache_bytes) {        // the host tier: the block's image in pinned memory
+        e = cudaMallocHost(&host_image, total);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(host_image, block, total, cudaMemcpyDeviceToHost, ls);
+    }
+    cudaEvent_t ready = nullptr;
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ready, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventRecord(ready, ls);
+    if (e == cudaSuccess && device_source) e = cudaStreamSynchronize(ls);   // the caller's device buffers may go away on return
+    if (e != cudaSuccess) {
+        if (host_image) cudaFreeHost(host_image);
+        if (ready) cudaEventDestroy(ready);
+        return fail(e);
+    }
+    g.pending_ops.push_back({id, 1});
+    mt_status st = adopt_model(id, hl, block, total, host_image, w_off, b_off, ready);
+    if (st != MT_OK) return st;
+    *model_id_out = id;
+    return MT_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -891,7 +1129,16 @@ mt_status mt_shutdown(void) {
     for (HostModel& m : g.models) {
         if (m.dev_block) { cudaFree(m.dev_block); m.dev_block = nullptr; }
         if (m.host_image) { cudaFreeHost(m.host_image); m.host_image = nullptr; }
+        if (m.ready) { cudaEventDestroy(m.ready); m.ready = nullptr; }
     }
+    if (g.h_order) { cudaFreeHost(g.h_order); g.h_order = nullptr; }
+    if (g.reg_host) { cudaFreeHost(g.reg_host); g.reg_host = nullptr; }
+    cudaFree(g.reg_dev); g.reg_dev = nullptr;
+    g.reg_host_cap = g.reg_dev_cap = 0;
+    if (g.reg_h2d_done) { cudaEventDestroy(g.reg_h2d_done); g.reg_h2d_done = nullptr; }
+    if (g.order_copied) { cudaEventDestroy(g.order_copied); g.order_copied = nullptr; }
+    g.pending_ops.clear();
+    g.order_dirty = g.order_copy_pending = g.reg_h2d_pending = false;
     g.models.clear();
     cudaFree(g.arena); g.arena = nullptr;
     g.cache.reset(0);
@@ -968,6 +1215,8 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
         b_off[l] = total; total += align_up(n_tiles * BN * sizeof(float), 1024);
         if (raw > raw_max) raw_max = raw;
     }
+    if (g.opt_async_register) return register_async(layers, hl, id, total, w_off, b_off, model_id_out);
+
     uint8_t* block = nullptr;
     if (g.cache_bytes) {
         // a place in the arena, over least-recently-used tenants if need be (registration is synchronous: nothing is
@@ -1046,39 +1295,7 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
         return e == cudaErrorMemoryAllocation ? MT_ERR_OOM : MT_ERR_CUDA;
     }
 
-    if (!g.has_family || g.live == 0) {
-        g.family = hl;
-        g.has_family = true;
-        g.in_elems = layer_in_elems(hl[0]);
-        g.out_elems = hl.back().out_ch;
-        for (const HostLayer& f : hl)
-            if (f.kind == MT_CONV3X3) plan_conv(f.h, f.w, &g.conv);   // cannot fail: validate_layers bounds w
-        for (int b = 0; b <= MT_MAX_LAYERS; ++b) g.width[b] = 0;
-        g.ws_dirty = true;
-        g.in_map_ptr = nullptr;
-        free_staging();   // sized for the previous family's rows (no model is live: nothing is in flight)
-    }
-    if ((size_t)n_layers > g.family.size()) {      // a deeper MLP joins: the family gains launches
-        for (size_t l = g.family.size(); l < (size_t)n_layers; ++l) g.family.push_back(hl[l]);
-        g.ws_dirty = true;
-    }
-    for (int l = 0; l < n_layers; ++l) {
-        const int wd = layer_in_elems(hl[l]);
-        if (wd > g.width[l]) { g.width[l] = wd; g.ws_dirty = true; }
-    }
-    HostModel& hm = g.models[id];
-    hm.alive = true;
-    hm.layers = hl;
-    hm.dev_block = g.cache_bytes ? nullptr : block;
-    hm.block_bytes = total;
-    hm.host_image = host_image;
-    hm.w_off = w_off;
-    hm.b_off = b_off;
-    hm.last_batch = 0;
-    g.live += 1;
-    if (id + 1 > g.T) g.T = id + 1;
-    recompute_tile_n();
-    st = recompute_order();
+    st = adopt_model(id, hl, block, total, host_image, w_off, b_off, nullptr);
     if (st != MT_OK) return st;
     *model_id_out = id;
     return MT_OK;
@@ -1431,6 +1648,7 @@ mt_status mt_debug_set_option(const char* name, int32_t value) {
     else if (!strcmp(name, "conv_pair")) g.opt_conv_pair = on;
     else if (!strcmp(name, "pool_head")) g.opt_pool_head = on;
     else if (!strcmp(name, "conv_stack")) g.opt_conv_stack = on;
+    else if (!strcmp(name, "async_register")) g.opt_async_register = on;
     else if (!strcmp(name, "conv_balance")) g.opt_conv_balance = on;
     else if (!strcmp(name, "perm_gather")) g.opt_gather = value < 0 ? 0 : (value > 2 ? 2 : value);
     else return MT_ERR_INVALID_ARG;

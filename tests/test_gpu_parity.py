@@ -338,3 +338,60 @@ def test_host_entries_after_a_wider_family_replaces_a_narrow_one(entry):
     wide = [synth.make_mlp(2, 10 + t, (512, 256, 200)) for t in range(2)]
     assert harness.register_models(wide) == [0, 1]
     host_call(wide, rng.integers(0, 2, n).astype(np.int32), bits(rng.standard_normal((n, 512))), 200)
+
+
+@pytest.mark.parametrize("mode", ["async", "sync"])
+def test_models_registered_while_batches_are_in_flight(mode, monkeypatch):
+    # registration does not wait for the device (MT_ASYNC_REGISTER=0: the older path that does): models are added
+    # between batches that are still running, the next batch uses them at once, nothing is synchronised in between
+    if mode == "sync":
+        monkeypatch.setenv("MT_ASYNC_REGISTER", "0")
+    models = [synth.make_mlp(13, t, (256, 512, 384, 64)) for t in range(6)]
+    rng = np.random.default_rng(31)
+    fresh()
+    harness.register_models(models[:3])
+    n = 900
+    batches, outs, keep = [], [], []
+
+    def enqueue(n_live):
+        ids = rng.integers(0, n_live, n).astype(np.int32)
+        x = bits(rng.standard_normal((n, 256)))
+        d_x, d_ids = harness.bf16_bits_to_device(x), torch.from_numpy(ids).cuda()
+        out = torch.full((n, 64), float("nan"), dtype=torch.float32, device="cuda")
+        mt.mt_infer(d_x, d_ids, n, out)
+        batches.append((ids, x)); outs.append(out); keep.append((d_x, d_ids))
+
+    for _ in range(3):
+        enqueue(3)
+    assert mt.mt_register_model(models[3]) == 3            # while the three batches above are running
+    enqueue(4)
+    assert harness.register_models(models[4:]) == [4, 5]
+    for _ in range(2):
+        enqueue(6)
+    torch.cuda.synchronize()
+    assert mt.mt_get_async_status() == (0, -1)
+    for (ids, x), out in zip(batches, outs):
+        got = out.cpu().numpy()
+        assert np.isfinite(got).all()
+        assert harness.scaled_error(got, oracle.forward(models, ids, x)).max() <= TOL
+
+
+def test_weights_given_as_device_tensors():
+    # weights and biases may be device pointers (also unaligned ones): the library reads them on its own stream and the
+    # caller may drop them when the call returns
+    models = [synth.make_mlp(13, 20 + t, (128, 192, 40)) for t in range(3)]
+    fresh()
+    for m in models:
+        dev_layers = []
+        for l in m:
+            w = torch.from_numpy(l.weight.view(np.int16).reshape(-1)).cuda()
+            pad = torch.empty(w.numel() + 1, dtype=torch.int16, device="cuda")
+            pad[1:] = w                                     # 2-byte aligned only
+            b = torch.from_numpy(l.bias).cuda()
+            dev_layers.append(Layer(l.kind, l.in_ch, l.out_ch, relu=l.relu, weight=pad[1:], bias=b))
+        mt.mt_register_model(dev_layers)
+        del dev_layers, pad, w, b
+        torch.cuda.empty_cache()
+    rng = np.random.default_rng(32)
+    ids = rng.integers(0, 3, 700).astype(np.int32)
+    run_and_check(models, ids, bits(rng.standard_normal((700, 128))), register=False)
