@@ -58,7 +58,7 @@ TRAFFIC = {
                                   "measured / 845.8 MB algorithmic), scaled by algorithmic bytes"},
     3: {"ratio": 1.007, "source": "profiles/grouped_gemm128_c3_reduced_ncu_full.md (250 tenants, 4096 requests: 272.1 MB "
                                   "measured / 270.0 MB algorithmic), scaled by algorithmic bytes"},
-    4: {"bytes": 608.5e6, "source": "profiles/grouped_conv3x3_pair_c4_full_ncu_full.md (full size, four conv launches)"},
+    4: {"bytes": 722.9e6, "source": "profiles/grouped_conv3x3_pair_c4_full_ncu_full.md (full size, the four conv layers of a step in one launch)"},
 }
 
 
@@ -281,13 +281,13 @@ def run_cache_sweep(args, ctx):
     h_outs = [torch.empty((nb, out_elems), dtype=torch.float32).pin_memory() for _ in range(2)]
     two = [torch.cuda.Stream(), torch.cuda.Stream()]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    # PCIe rate of this machine: one 256 MB pinned host -> device copy, best of 5
-    probe_h = torch.empty(256 << 20, dtype=torch.uint8).pin_memory()
-    probe_d = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    # PCIe rate of this machine: a 512 MB pinned host -> device copy, best of 8
+    probe_h = torch.empty(512 << 20, dtype=torch.uint8).pin_memory()
+    probe_d = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
     pcie = 0.0
-    for _ in range(5):
+    for _ in range(8):
         e0.record(); probe_d.copy_(probe_h, non_blocking=True); e1.record(); torch.cuda.synchronize()
-        pcie = max(pcie, (256 << 20) / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+        pcie = max(pcie, (512 << 20) / (e0.elapsed_time(e1) * 1e-3) / 1e9)
     del probe_h, probe_d
     rows = []
     block = None
