@@ -99,7 +99,9 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
  * of at most 512 requests against dense layers at most 256 wide runs as ONE launch that does all of it.  No host<->device synchronisation happens unless the
  * workspace must grow (n larger than any earlier call, or a wider model registered since): then the
  * call synchronises the device and reallocates first - make one call at the largest n before timing.
- * inputs must be 16-byte aligned.  n == 0 is a no-op.
+ * inputs must be 16-byte aligned.  n == 0 is a no-op.  Once the workspace exists and the models in use have been seen by
+ * one earlier call, the call only launches kernels on `stream`, so it may be captured into a CUDA graph and replayed on
+ * new contents of the same buffers (tests/test_gpu_parity.py does).
  * A request whose id is not a live model never faults: its output row is NaN, a sticky status is set
  * (see mt_get_async_status) and all other requests complete normally. */
 mt_status mt_infer(const void* inputs, const int32_t* model_ids, int32_t n, void* outputs, void* stream);

@@ -395,3 +395,46 @@ def test_weights_given_as_device_tensors():
     rng = np.random.default_rng(32)
     ids = rng.integers(0, 3, 700).astype(np.int32)
     run_and_check(models, ids, bits(rng.standard_normal((700, 128))), register=False)
+
+
+@pytest.mark.parametrize("family", ["mlp", "small_mlp", "conv"])
+def test_mt_infer_replays_from_a_cuda_graph(family):
+    # mt_infer only enqueues work (no allocation, no synchronisation once the workspace exists), so a call can be
+    # captured into a CUDA graph - programmatic dependent launches included - and replayed on new inputs in the same
+    # buffers: every replay must match the oracle
+    if family == "mlp":
+        wl = synth.make_workload(3, n=900, n_tenants=40)
+        mk = lambda k: synth.make_requests(3, wl.models, n=900, salt=90 + k)
+    elif family == "small_mlp":
+        wl = synth.make_workload(1, n=64)
+        mk = lambda k: synth.make_requests(1, wl.models, n=64, salt=90 + k)
+    else:
+        wl = synth.make_workload(4, n=12, n_tenants=3, h=56, w=56, n_conv=3)
+        mk = lambda k: synth.make_requests(4, wl.models, n=12, salt=90 + k)
+    n = wl.n
+    fresh(max(64, len(wl.models)))
+    harness.register_models(wl.models)
+    x = harness.bf16_bits_to_device(wl.inputs.reshape(n, -1)).clone()
+    ids = torch.from_numpy(wl.model_ids).cuda()
+    out = torch.full((n, wl.out_elems), float("nan"), dtype=torch.float32, device="cuda")
+    mt.mt_infer(x, ids, n, out)                       # sizes the workspace, publishes the models' table entries
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        graph.capture_begin()
+        mt.mt_infer(x, ids, n, out, side)
+        graph.capture_end()
+    torch.cuda.current_stream().wait_stream(side)
+    for k in range(3):
+        new_ids, new_x = mk(k)
+        x.copy_(harness.bf16_bits_to_device(new_x.reshape(n, -1)))
+        ids.copy_(torch.from_numpy(new_ids).cuda())
+        out.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert mt.mt_get_async_status() == (0, -1)
+        got = out.cpu().numpy()
+        ref = oracle.forward(wl.models, new_ids, new_x)
+        assert np.isfinite(got).all() and harness.scaled_error(got, ref).max() <= TOL, k
