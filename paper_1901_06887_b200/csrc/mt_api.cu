@@ -670,13 +670,15 @@ bool all_dense(const std::vector<HostLayer>& m) {
     return true;
 }
 
-// What the models of one context share: input and output element counts, and the layer kinds index by index.  MLPs
-// (dense layers only) may differ in depth and in hidden widths; a tenant's layer j runs in the family's j-th launch
-// and its last layer, whichever launch that is, writes the output.  Conv families keep one depth and geometry.
+// What the models of one context share: the input element count and the layer kinds index by index.  MLPs (dense
+// layers only) may differ in depth, hidden widths and output width; a tenant's layer j runs in the family's j-th
+// launch and its last layer, whichever launch that is, writes the output - its own out_ch columns of a row whose
+// stride is the widest model's output.  Conv families keep one depth, geometry and output width.
 mt_status check_family(const std::vector<HostLayer>& m) {
     if (!g.has_family || g.live == 0) return MT_OK;
-    if (layer_in_elems(m[0]) != g.in_elems || m.back().out_ch != g.out_elems) return MT_ERR_SHAPE;
-    if (all_dense(m) && all_dense(g.family)) return MT_OK;
+    if (layer_in_elems(m[0]) != g.in_elems) return MT_ERR_SHAPE;
+    if (all_dense(m) && all_dense(g.family)) return MT_OK;      // MLPs: any depth, any hidden and output widths
+    if (m.back().out_ch != g.out_elems) return MT_ERR_SHAPE;
     if (m.size() != g.family.size()) return MT_ERR_SHAPE;
     for (size_t l = 0; l < m.size(); ++l) {
         const HostLayer &a = m[l], &f = g.family[l];
@@ -971,6 +973,10 @@ mt_status adopt_model(int id, const std::vector<HostLayer>& hl, uint8_t* block, 
     for (int l = 0; l < n_layers; ++l) {
         const int wd = layer_in_elems(hl[l]);
         if (wd > g.width[l]) { g.width[l] = wd; g.ws_dirty = true; }
+    }
+    if (hl.back().out_ch > g.out_elems) {          // a wider output: the rows of the output buffer get longer
+        g.out_elems = hl.back().out_ch;
+        g.ws_dirty = true;
     }
     HostModel& hm = g.models[id];
     hm.alive = true;
@@ -1428,6 +1434,14 @@ mt_status mt_infer_host_async(const void* inputs_host, const int32_t* model_ids_
     CU_OK(cudaMemcpyAsync(outputs_host, g.as_out[k], out_bytes, cudaMemcpyDeviceToHost, s));
     CU_OK(cudaEventRecord(g.as_slot_done[k], s));
     g.as_slot_used[k] = true;
+    return MT_OK;
+}
+
+mt_status mt_output_elems(int32_t* out_elems_out) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g.init) return MT_ERR_NOT_INIT;
+    if (!out_elems_out) return MT_ERR_INVALID_ARG;
+    *out_elems_out = (g.has_family && g.live > 0) ? g.out_elems : 0;
     return MT_OK;
 }
 

@@ -297,10 +297,9 @@ def test_growing_batches_and_wider_models_reallocate_correctly(small_batch_path)
 def test_family_mismatch_is_rejected():
     fresh()
     assert mt.mt_register_model(synth.make_mlp(1, 0, (64, 128, 10))) == 0
-    for widths in ((128, 128, 10), (64, 128, 12)):           # other input or output width (depth may differ)
-        with pytest.raises(mt.MtError) as e:
-            mt.mt_register_model(synth.make_mlp(1, 1, widths))
-        assert e.value.code == 3
+    with pytest.raises(mt.MtError) as e:                     # another input width (depth and output width may differ)
+        mt.mt_register_model(synth.make_mlp(1, 1, (128, 128, 10)))
+    assert e.value.code == 3
     assert mt.mt_register_model(synth.make_mlp(1, 1, (64, 512, 10))) == 1      # hidden width may differ
     with pytest.raises(mt.MtError) as e:
         mt.mt_release(5)

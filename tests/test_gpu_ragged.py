@@ -73,15 +73,17 @@ def test_mixed_depths_cta_pair_executor_and_rejected_ids():
     assert np.isfinite(got[good]).all() and harness.scaled_error(got[good], ref).max() <= TOL
 
 
-def test_a_family_still_needs_one_input_and_output_shape():
+def test_a_family_still_needs_one_input_shape_and_conv_families_one_output():
     fresh()
     assert mt.mt_register_model(synth.make_mlp(11, 0, (64, 128, 10))) == 0
     assert mt.mt_register_model(synth.make_mlp(11, 1, (64, 10))) == 1                  # shallower: accepted
     assert mt.mt_register_model(synth.make_mlp(11, 2, (64, 64, 64, 64, 10))) == 2      # deeper: accepted
-    for widths in ((128, 128, 10), (64, 128, 12)):
-        with pytest.raises(mt.MtError) as e:
-            mt.mt_register_model(synth.make_mlp(11, 3, widths))
-        assert e.value.code == 3
+    with pytest.raises(mt.MtError) as e:
+        mt.mt_register_model(synth.make_mlp(11, 3, (128, 128, 10)))                  # another input width
+    assert e.value.code == 3
+    assert mt.mt_output_elems() == 10
+    assert mt.mt_register_model(synth.make_mlp(11, 3, (64, 128, 12))) == 3           # a wider output: accepted
+    assert mt.mt_output_elems() == 12
     # conv families keep one depth
     fresh()
     wl = synth.make_workload(4, n=4, n_tenants=1, h=8, w=8, n_conv=2)
@@ -90,3 +92,27 @@ def test_a_family_still_needs_one_input_and_output_shape():
     with pytest.raises(mt.MtError) as e:
         mt.mt_register_model(deeper)
     assert e.value.code == 3
+
+
+@pytest.mark.parametrize("n", [300, 2500])
+def test_tenants_with_different_output_widths(n, small_batch_path):
+    # outputs of 10, 64, 200 and 33 columns in one batch: the buffer's rows are as long as the widest output
+    # (mt_output_elems), every request gets its own model's columns and the rest of its row is left alone
+    outs = [10, 64, 200, 33]
+    models = [synth.make_mlp(14, t, (128, 256 if t % 2 else 128, outs[t])) for t in range(4)]
+    rng = np.random.default_rng(n)
+    ids = rng.integers(0, 4, n).astype(np.int32)
+    x = bits(rng.standard_normal((n, 128)))
+    fresh()
+    harness.register_models(models)
+    stride = mt.mt_output_elems()
+    assert stride == 200
+    out = torch.full((n, stride), -7.0, dtype=torch.float32, device="cuda")
+    mt.mt_infer(harness.bf16_bits_to_device(x), torch.from_numpy(ids).cuda(), n, out)
+    assert mt.mt_get_async_status() == (0, -1)
+    got = out.cpu().numpy()
+    for t in range(4):
+        rows = np.flatnonzero(ids == t)
+        ref = oracle.forward([models[t]], np.zeros(len(rows), np.int32), x[rows])
+        assert harness.scaled_error(got[rows, :outs[t]], ref).max() <= TOL
+        assert (got[rows, outs[t]:] == -7.0).all()
