@@ -76,11 +76,12 @@ mt_status mt_shutdown(void);
 
 /* "Upload your model" (Sec. 1.2 / Sec. 3): validate the layer list, copy the weights to the device in
  * the executor's tiled layout and return a small dense id (lowest free slot first) in *model_id_out.
- * All models hosted by one context form one family: the same input element count and the same layer kinds index by
- * index.  MLPs (dense layers only) may differ in depth, hidden widths and output width; conv families keep one depth,
- * geometry and output width.  The row stride of mt_infer's output buffer is the WIDEST registered model's output
+ * All models hosted by one context form one family: the same layer kinds index by index.  MLPs (dense layers only)
+ * may differ in depth and in every width - input, hidden and output; conv families keep one depth, geometry, input and
+ * output width.  The row stride of mt_infer's output buffer is the WIDEST registered model's output
  * (mt_output_elems); a model with fewer outputs writes the first out_ch columns of its requests' rows and leaves the rest
- * untouched.
+ * untouched.  The row stride of the input buffer is the WIDEST registered model's input (mt_input_elems); a request of a
+ * model with fewer inputs carries them at the start of its row and the rest of the row is never read.
  * Kernel limits (else MT_ERR_UNSUPPORTED): 1..MT_MAX_LAYERS layers; dense in_ch a multiple of 64;
  * conv in_ch == out_ch == 64, w <= 126; a pool must follow a conv; a dense layer may not precede a conv.
  * The call does not wait for the device: weights and biases in HOST memory are copied into the library's pinned
@@ -92,11 +93,17 @@ mt_status mt_shutdown(void);
  * "async_register") selects the older path that synchronises the device once per layer. */
 mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32_t* model_id_out);
 
-/* Elements per row of the output buffer as of now: the widest live model's output width (0 if none is registered). */
+/* Elements per row of the output buffer as of now: the widest output among the models registered since the context
+ * last held none (0 if none is registered); releasing a model never shortens the rows. */
 mt_status mt_output_elems(int32_t* out_elems_out);
 
+/* Elements per row of the input buffer as of now: the widest input among the models registered since the context
+ * last held none (0 if none is registered). */
+mt_status mt_input_elems(int32_t* in_elems_out);
+
 /* predict(model, input) for a whole mixed batch (Sec. 3: a worker multiplexes requests across models).
- *   inputs    device, bf16, [n][in_elems] row-major (NHWC per request for conv), arrival order
+ *   inputs    device, bf16, [n][in_elems] row-major (NHWC per request for conv), arrival order (in_elems: see
+ *             mt_input_elems)
  *   model_ids device, int32 [n]; request i is evaluated by model model_ids[i]
  *   outputs   device, fp32, [n][out_elems], arrival order (out_elems: see mt_output_elems)
  *   stream    cudaStream_t (NULL = default stream)

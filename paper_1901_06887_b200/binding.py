@@ -24,7 +24,7 @@ EXPORTS = ["mt_init", "mt_shutdown", "mt_register_model", "mt_infer", "mt_infer_
            "mt_get_async_status", "mt_status_string", "mt_debug_last_bucketing", "mt_set_kernel_timing",
            "mt_get_kernel_times", "mt_bucket_noalloc", "mt_debug_wait_timeout", "mt_debug_launch_count", "mt_debug_set_option", "mt_debug_empty_launches", "mt_debug_item_cost",
            "mt_debug_schedule_balance", "mt_set_cache_bytes", "mt_prefetch", "mt_get_cache_stats", "mt_cache_sim_create",
-           "mt_cache_sim_access", "mt_cache_sim_release", "mt_cache_sim_stats", "mt_cache_sim_destroy", "mt_output_elems"]
+           "mt_cache_sim_access", "mt_cache_sim_release", "mt_cache_sim_stats", "mt_cache_sim_destroy", "mt_output_elems", "mt_input_elems"]
 
 
 class MtError(RuntimeError):
@@ -78,6 +78,7 @@ def lib() -> ctypes.CDLL:
         l.mt_debug_set_option.argtypes = [ctypes.c_char_p, i32]
         l.mt_debug_empty_launches.argtypes = [i32, vp]
         l.mt_output_elems.argtypes = [ctypes.POINTER(i32)]
+        l.mt_input_elems.argtypes = [ctypes.POINTER(i32)]
         l.mt_set_cache_bytes.argtypes = [ctypes.c_size_t]
         l.mt_prefetch.argtypes = [vp, i32, vp]
         l.mt_get_cache_stats.argtypes = [ctypes.POINTER(CacheStats), i32]
@@ -203,6 +204,13 @@ def mt_output_elems() -> int:
     """Row stride (elements) of mt_infer's output buffer: the widest registered model's output width."""
     v = ctypes.c_int32(0)
     _check(lib().mt_output_elems(ctypes.byref(v)), "mt_output_elems")
+    return int(v.value)
+
+
+def mt_input_elems() -> int:
+    """Row stride (elements) of mt_infer's input buffer: the widest registered model's input width."""
+    v = ctypes.c_int32(0)
+    _check(lib().mt_input_elems(ctypes.byref(v)), "mt_input_elems")
     return int(v.value)
 
 

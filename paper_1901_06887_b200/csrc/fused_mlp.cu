@@ -248,10 +248,11 @@ fused_mlp_kernel(const FusedArgs p) {
                 for (int e = et; e < p.out_elems; e += kFusedEpiThreads) dst[e] = __int_as_float(0x7fc00000);
             }
         }
-        const int cpr = p.K0 >> 3;                  // 16-byte chunks per input row
+        const int ld_ch = p.K0 >> 3;                // 16-byte chunks per row of the caller's buffer (the widest input)
         for (int u = blockIdx.x; ok && u < total_units; u += gridDim.x) {
             const UnitCoord c = locate(u);
             const int L = p.models[c.t].n_layers;
+            const int cpr = p.models[c.t].layer[0].k_blocks << 3;    // chunks of a row that this tenant's first layer reads
             // gather the unit's rows (arrival order -> bucketed rows) into the operand buffer: row rr, chunk ch of the
             // row goes to K block ch / 8, 16-byte position (ch % 8) ^ (rr % 8) of the 128-byte swizzle row
             const uint4* src = reinterpret_cast<const uint4*>(p.inputs);
@@ -265,7 +266,7 @@ fused_mlp_kernel(const FusedArgs p) {
                     for (int k = 0; k < 4; ++k) {
                         const int e = idx + k * kFusedEpiThreads;
                         rr[k] = e / cpr; ch[k] = e - rr[k] * cpr;
-                        v[k] = __ldg(src + (size_t)s_perm[c.j0 + rr[k]] * cpr + ch[k]);
+                        v[k] = __ldg(src + (size_t)s_perm[c.j0 + rr[k]] * ld_ch + ch[k]);
                     }
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
@@ -273,7 +274,7 @@ fused_mlp_kernel(const FusedArgs p) {
                 }
                 for (; idx < total_ch; idx += kFusedEpiThreads) {
                     const int rr = idx / cpr, ch = idx - rr * cpr;
-                    const uint4 v = __ldg(src + (size_t)s_perm[c.j0 + rr] * cpr + ch);
+                    const uint4 v = __ldg(src + (size_t)s_perm[c.j0 + rr] * ld_ch + ch);
                     *reinterpret_cast<uint4*>(smem + (ch >> 3) * TILE_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4)) = v;
                 }
             }

@@ -670,14 +670,15 @@ bool all_dense(const std::vector<HostLayer>& m) {
     return true;
 }
 
-// What the models of one context share: the input element count and the layer kinds index by index.  MLPs (dense
-// layers only) may differ in depth, hidden widths and output width; a tenant's layer j runs in the family's j-th
-// launch and its last layer, whichever launch that is, writes the output - its own out_ch columns of a row whose
-// stride is the widest model's output.  Conv families keep one depth, geometry and output width.
+// What the models of one context share: the layer kinds index by index.  MLPs (dense layers only) may differ in
+// depth and in every width, the input's included; a tenant's layer j runs in the family's j-th launch and its last
+// layer, whichever launch that is, writes the output - its own out_ch columns of a row whose stride is the widest
+// model's output.  Likewise the rows of the input buffer are as long as the widest model's input and a request's row
+// holds its own model's features first.  Conv families keep one depth, geometry, input and output width.
 mt_status check_family(const std::vector<HostLayer>& m) {
     if (!g.has_family || g.live == 0) return MT_OK;
+    if (all_dense(m) && all_dense(g.family)) return MT_OK;      // MLPs: any depth, any input, hidden and output widths
     if (layer_in_elems(m[0]) != g.in_elems) return MT_ERR_SHAPE;
-    if (all_dense(m) && all_dense(g.family)) return MT_OK;      // MLPs: any depth, any hidden and output widths
     if (m.back().out_ch != g.out_elems) return MT_ERR_SHAPE;
     if (m.size() != g.family.size()) return MT_ERR_SHAPE;
     for (size_t l = 0; l < m.size(); ++l) {
@@ -977,6 +978,11 @@ mt_status adopt_model(int id, const std::vector<HostLayer>& hl, uint8_t* block, 
     if (hl.back().out_ch > g.out_elems) {          // a wider output: the rows of the output buffer get longer
         g.out_elems = hl.back().out_ch;
         g.ws_dirty = true;
+    }
+    if (layer_in_elems(hl[0]) > g.in_elems) {      // a wider input (MLP families only): so do the input buffer's
+        g.in_elems = layer_in_elems(hl[0]);
+        g.ws_dirty = true;
+        g.in_map_ptr = nullptr;
     }
     HostModel& hm = g.models[id];
     hm.alive = true;
@@ -1442,6 +1448,14 @@ mt_status mt_output_elems(int32_t* out_elems_out) {
     if (!g.init) return MT_ERR_NOT_INIT;
     if (!out_elems_out) return MT_ERR_INVALID_ARG;
     *out_elems_out = (g.has_family && g.live > 0) ? g.out_elems : 0;
+    return MT_OK;
+}
+
+mt_status mt_input_elems(int32_t* in_elems_out) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g.init) return MT_ERR_NOT_INIT;
+    if (!in_elems_out) return MT_ERR_INVALID_ARG;
+    *in_elems_out = (g.has_family && g.live > 0) ? g.in_elems : 0;
     return MT_OK;
 }
 

@@ -123,7 +123,7 @@ struct FusedArgs {
     int T;
     const ModelDev* models;
     int n_layers;
-    int K0;                   // input features (multiple of 64, at most 256)
+    int K0;                   // features per row of `inputs`: the widest model's input (multiple of 64, at most 256)
     int out_elems;            // output features (at most 256)
     float* out;               // fp32 [n][out_elems], arrival order (the caller's buffer)
     int32_t* counts;          // [T + 1]   bucketing results, written by CTA 0

@@ -297,8 +297,8 @@ def test_growing_batches_and_wider_models_reallocate_correctly(small_batch_path)
 def test_family_mismatch_is_rejected():
     fresh()
     assert mt.mt_register_model(synth.make_mlp(1, 0, (64, 128, 10))) == 0
-    with pytest.raises(mt.MtError) as e:                     # another input width (depth and output width may differ)
-        mt.mt_register_model(synth.make_mlp(1, 1, (128, 128, 10)))
+    with pytest.raises(mt.MtError) as e:                     # a conv model cannot join an MLP family (widths may differ)
+        mt.mt_register_model(synth.make_workload(4, n=4, n_tenants=1, h=8, w=8, n_conv=2).models[0])
     assert e.value.code == 3
     assert mt.mt_register_model(synth.make_mlp(1, 1, (64, 512, 10))) == 1      # hidden width may differ
     with pytest.raises(mt.MtError) as e:

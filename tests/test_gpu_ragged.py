@@ -73,24 +73,36 @@ def test_mixed_depths_cta_pair_executor_and_rejected_ids():
     assert np.isfinite(got[good]).all() and harness.scaled_error(got[good], ref).max() <= TOL
 
 
-def test_a_family_still_needs_one_input_shape_and_conv_families_one_output():
+def test_what_a_family_may_mix_and_what_conv_families_keep():
     fresh()
+    assert mt.mt_input_elems() == 0 and mt.mt_output_elems() == 0
     assert mt.mt_register_model(synth.make_mlp(11, 0, (64, 128, 10))) == 0
     assert mt.mt_register_model(synth.make_mlp(11, 1, (64, 10))) == 1                  # shallower: accepted
     assert mt.mt_register_model(synth.make_mlp(11, 2, (64, 64, 64, 64, 10))) == 2      # deeper: accepted
-    with pytest.raises(mt.MtError) as e:
-        mt.mt_register_model(synth.make_mlp(11, 3, (128, 128, 10)))                  # another input width
-    assert e.value.code == 3
-    assert mt.mt_output_elems() == 10
+    assert (mt.mt_input_elems(), mt.mt_output_elems()) == (64, 10)
     assert mt.mt_register_model(synth.make_mlp(11, 3, (64, 128, 12))) == 3           # a wider output: accepted
-    assert mt.mt_output_elems() == 12
-    # conv families keep one depth
+    assert (mt.mt_input_elems(), mt.mt_output_elems()) == (64, 12)
+    assert mt.mt_register_model(synth.make_mlp(11, 4, (192, 128, 10))) == 4          # a wider input: accepted
+    assert (mt.mt_input_elems(), mt.mt_output_elems()) == (192, 12)
+    mt.mt_release(4)                                                                 # rows never get shorter
+    assert (mt.mt_input_elems(), mt.mt_output_elems()) == (192, 12)
+    with pytest.raises(mt.MtError) as e:
+        mt.mt_register_model(synth.make_mlp(11, 5, (100, 128, 10)))                  # not a multiple of 64
+    assert e.value.code == 4
+    # conv families keep one depth and one input shape
     fresh()
     wl = synth.make_workload(4, n=4, n_tenants=1, h=8, w=8, n_conv=2)
     assert mt.mt_register_model(wl.models[0]) == 0
     deeper = synth.make_workload(4, n=4, n_tenants=1, h=8, w=8, n_conv=3).models[0]
     with pytest.raises(mt.MtError) as e:
         mt.mt_register_model(deeper)
+    assert e.value.code == 3
+    larger = synth.make_workload(4, n=4, n_tenants=1, h=16, w=8, n_conv=2).models[0]
+    with pytest.raises(mt.MtError) as e:
+        mt.mt_register_model(larger)
+    assert e.value.code == 3
+    with pytest.raises(mt.MtError) as e:
+        mt.mt_register_model(synth.make_mlp(11, 0, (64 * 8 * 8, 10)))                # an MLP cannot join a conv family
     assert e.value.code == 3
 
 
@@ -116,3 +128,60 @@ def test_tenants_with_different_output_widths(n, small_batch_path):
         ref = oracle.forward([models[t]], np.zeros(len(rows), np.int32), x[rows])
         assert harness.scaled_error(got[rows, :outs[t]], ref).max() <= TOL
         assert (got[rows, outs[t]:] == -7.0).all()
+
+
+@pytest.mark.parametrize("n,ins", [(350, [64, 256, 128, 192]), (2500, [128, 512, 64, 320]), (6000, [256, 1024, 64, 576])])
+def test_tenants_with_different_input_widths(n, ins, small_batch_path):
+    # inputs of four widths in one batch: the buffer's rows are as long as the widest input (mt_input_elems); a request
+    # carries its own model's features first, and what follows in its row is never read - the test puts NaN there
+    T = len(ins)
+    models = [synth.make_mlp(15, t, (ins[t], 256 if t % 2 else 128, 40)) for t in range(T)]
+    rng = np.random.default_rng(n)
+    ids = synth.zipf_ids(4, n, T, 0.8, salt=n)
+    fresh()
+    harness.register_models(models)
+    stride = mt.mt_input_elems()
+    assert stride == max(ins)
+    x = rng.standard_normal((n, stride)).astype(np.float32)
+    for t in range(T):
+        x[ids == t, ins[t]:] = np.nan
+    xb = bits(x)
+    got = harness.run_batch(ids, xb, 40)
+    assert mt.mt_get_async_status() == (0, -1)
+    assert np.isfinite(got).all()
+    for t in range(T):
+        rows = np.flatnonzero(ids == t)
+        ref = oracle.forward([models[t]], np.zeros(len(rows), np.int32), np.ascontiguousarray(xb[rows, :ins[t]]))
+        assert harness.scaled_error(got[rows], ref).max() <= TOL
+    # the same batch through the first layer's TMA gather (rows read through perm) gives the same bits
+    mt.mt_debug_set_option("perm_gather", 2)
+    try:
+        got2 = harness.run_batch(ids, xb, 40)
+    finally:
+        mt.mt_debug_set_option("perm_gather", 1)
+    assert np.array_equal(got, got2)
+
+
+def test_a_wider_input_registered_between_batches_lengthens_the_rows():
+    m0 = synth.make_mlp(16, 0, (128, 256, 16))
+    m1 = synth.make_mlp(16, 1, (384, 128, 16))
+    rng = np.random.default_rng(3)
+    n = 900
+    fresh()
+    harness.register_models([m0])
+    x0 = bits(rng.standard_normal((n, 128)))
+    ids0 = np.zeros(n, np.int32)
+    first = harness.run_batch(ids0, x0, 16)
+    harness.register_models([m1])
+    assert mt.mt_input_elems() == 384
+    ids = rng.integers(0, 2, n).astype(np.int32)
+    x = rng.standard_normal((n, 384)).astype(np.float32)
+    x[:, :128] = synth.bf16_bits_to_f32(x0)
+    xb = bits(x)
+    got = harness.run_batch(ids, xb, 16)
+    for t, m, k in ((0, m0, 128), (1, m1, 384)):
+        rows = np.flatnonzero(ids == t)
+        ref = oracle.forward([m], np.zeros(len(rows), np.int32), np.ascontiguousarray(xb[rows, :k]))
+        assert harness.scaled_error(got[rows], ref).max() <= TOL
+    rows = np.flatnonzero(ids == 0)
+    assert np.array_equal(got[rows], first[rows])      # model 0's requests: same inputs, same bits as before
