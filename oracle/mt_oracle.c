@@ -27,6 +27,11 @@
  *            weights [out][ky][kx][in]; tap (ky,kx) reads pixel (y+ky-1, x+kx-1)
  *   global average pool: mean over all H*W positions, per channel
  *   ReLU: max(z, 0)
+ *   identity shortcut (the residual block of the network the paper uses as
+ *            its running example, Sec. 1.1: resnet18): a conv layer marked
+ *            `residual` adds the INPUT of the layer before it to its own
+ *            pre-activation, a_{l+1} = act(conv(a_l) + b + a_{l-1}), which
+ *            closes a block of two conv layers
  *
  * Precision: every value is held in double from the bf16 input to the output;
  * nothing is rounded between layers.  bf16 and fp32 inputs are exact in double.
@@ -35,7 +40,9 @@
  * identity and zero weights (closed forms), a separately written triple-loop
  * matmul, numpy float64 matmul, brute-force padded-copy conv, scipy
  * correlate2d, shifted-tap and all-ones closed forms, numpy stable argsort and
- * an O(n*T) brute-force bucketing.  No function here is left unpinned.
+ * an O(n*T) brute-force bucketing; the shortcut by a zero-weight block
+ * (a closed form of the block's input alone) and a scipy restatement.
+ * No function here is left unpinned.
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -51,6 +58,7 @@ typedef struct {
     int32_t in_ch, out_ch;
     int32_t h, w;          /* spatial size for conv / pool; 0 for dense */
     int32_t relu;          /* 1: apply max(z,0) after the layer */
+    int32_t residual;      /* conv only, 1: add the previous layer's input before the activation */
     const uint16_t* weight; /* bf16 bit patterns; NULL for pool */
     const float* bias;      /* fp32 [out_ch]; NULL means zeros */
 } orc_layer;
@@ -102,8 +110,9 @@ int orc_bucket(const int32_t* ids, int32_t n, int32_t T,
     return 0;
 }
 
-/* One layer: a (in) -> z (out), both double. */
-static void layer_apply(const orc_layer* l, const double* a, double* z)
+/* One layer: a (in) -> z (out), both double.  skip: the tensor a residual
+ * layer adds before its activation (same shape as z), else NULL. */
+static void layer_apply(const orc_layer* l, const double* a, const double* skip, double* z)
 {
     if (l->kind == ORC_DENSE) {
         for (int32_t o = 0; o < l->out_ch; ++o) {
@@ -141,6 +150,10 @@ static void layer_apply(const orc_layer* l, const double* a, double* z)
             z[c] = s / (double)P;
         }
     }
+    if (skip) {
+        const int64_t n_out = layer_out_elems(l);
+        for (int64_t j = 0; j < n_out; ++j) z[j] += skip[j];
+    }
     if (l->relu) {
         const int64_t n_out = layer_out_elems(l);
         for (int64_t j = 0; j < n_out; ++j)
@@ -158,19 +171,27 @@ int orc_forward_one(const orc_layer* layers, int32_t n_layers, const uint16_t* i
     for (int32_t li = 0; li < n_layers; ++li) {
         if (li > 0 && layer_in_elems(&layers[li]) != layer_out_elems(&layers[li - 1])) return -1;
         if (layer_out_elems(&layers[li]) > max_elems) max_elems = layer_out_elems(&layers[li]);
+        if (layers[li].residual) {
+            /* the shortcut joins the output of this layer with the input of the one before: both are conv
+             * layers and the three tensors have one shape */
+            if (li == 0 || layers[li].kind != ORC_CONV3X3 || layers[li - 1].kind != ORC_CONV3X3) return -1;
+            if (layer_in_elems(&layers[li - 1]) != layer_out_elems(&layers[li])) return -1;
+        }
     }
+    /* three tensors are alive at a time: the previous layer's input, this layer's input, its output */
+    double* before = (double*)malloc(sizeof(double) * (size_t)max_elems);
     double* a = (double*)malloc(sizeof(double) * (size_t)max_elems);
     double* z = (double*)malloc(sizeof(double) * (size_t)max_elems);
-    if (!a || !z) { free(a); free(z); return -2; }
+    if (!before || !a || !z) { free(before); free(a); free(z); return -2; }
     const int64_t n_in = layer_in_elems(&layers[0]);
     for (int64_t j = 0; j < n_in; ++j) a[j] = bf16_to_double(input[j]);
     for (int32_t li = 0; li < n_layers; ++li) {
-        layer_apply(&layers[li], a, z);
-        double* t = a; a = z; z = t;
+        layer_apply(&layers[li], a, layers[li].residual ? before : NULL, z);
+        double* t = before; before = a; a = z; z = t;
     }
     const int64_t n_out = layer_out_elems(&layers[n_layers - 1]);
     for (int64_t j = 0; j < n_out; ++j) out[j] = a[j];
-    free(a); free(z);
+    free(before); free(a); free(z);
     return 0;
 }
 

@@ -1,7 +1,8 @@
 """ctypes front end of the plain-C fp64 oracle in ``mt_oracle.c`` (test infrastructure only).
 
 Models are passed as lists of layer objects with the attributes ``kind, in_ch, out_ch, h, w, relu,
-weight, bias`` (weight: uint16 array of bf16 bit patterns or None; bias: float32 array or None).
+weight, bias`` and optionally ``residual`` (weight: uint16 array of bf16 bit patterns or None; bias: float32
+array or None).
 Nothing here computes: it only marshals arrays into the C routines.
 """
 from __future__ import annotations
@@ -41,7 +42,7 @@ def build(force: bool = False) -> str:
 class _CLayer(ctypes.Structure):
     _fields_ = [("kind", ctypes.c_int32), ("in_ch", ctypes.c_int32), ("out_ch", ctypes.c_int32),
                 ("h", ctypes.c_int32), ("w", ctypes.c_int32), ("relu", ctypes.c_int32),
-                ("weight", ctypes.c_void_p), ("bias", ctypes.c_void_p)]
+                ("residual", ctypes.c_int32), ("weight", ctypes.c_void_p), ("bias", ctypes.c_void_p)]
 
 
 def _load():
@@ -77,7 +78,7 @@ def _pack_model(layers: Sequence, keep: list):
             b = np.ascontiguousarray(l.bias, dtype=np.float32)
             keep.append(b)
         arr[i] = _CLayer(int(l.kind), int(l.in_ch), int(l.out_ch), int(l.h), int(l.w), int(l.relu),
-                         w.ctypes.data if w is not None else None,
+                         int(getattr(l, "residual", 0)), w.ctypes.data if w is not None else None,
                          b.ctypes.data if b is not None else None)
     keep.append(arr)
     return arr

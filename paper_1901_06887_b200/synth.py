@@ -67,6 +67,7 @@ class Layer:
     relu: int = 0
     weight: Optional[np.ndarray] = None  # uint16 bf16 bits; None for pooling
     bias: Optional[np.ndarray] = None    # float32 [out_ch]; None for pooling
+    residual: int = 0                    # conv only, 1: the previous layer's input is added before the activation
 
     @property
     def in_elems(self) -> int:
@@ -124,12 +125,14 @@ def make_mlp(config: int, tenant: int, widths: Sequence[int]) -> List[Layer]:
     return layers
 
 
-def make_conv_stack(config: int, tenant: int, n_conv: int, ch: int, h: int, w: int, n_out: int) -> List[Layer]:
-    """n_conv x (3x3 conv ch->ch, stride 1, pad 1, ReLU) -> global avg pool -> dense ch->n_out."""
+def make_conv_stack(config: int, tenant: int, n_conv: int, ch: int, h: int, w: int, n_out: int,
+                    shortcuts: Sequence[int] = ()) -> List[Layer]:
+    """n_conv x (3x3 conv ch->ch, stride 1, pad 1, ReLU) -> global avg pool -> dense ch->n_out.
+    shortcuts: indices (>= 1) of conv layers that close a two-layer residual block (identity shortcut)."""
     layers = []
     for li in range(n_conv):
         layers.append(Layer(
-            kind=CONV3X3, in_ch=ch, out_ch=ch, h=h, w=w, relu=1,
+            kind=CONV3X3, in_ch=ch, out_ch=ch, h=h, w=w, relu=1, residual=int(li in shortcuts),
             weight=_he_uniform_bf16(stream(config, "weights", tenant, li), (ch, 3, 3, ch), 9 * ch),
             bias=_bias(stream(config, "biases", tenant, li), ch)))
     layers.append(Layer(kind=GLOBAL_AVG_POOL, in_ch=ch, out_ch=ch, h=h, w=w))

@@ -225,6 +225,70 @@ def test_conv_via_im2col_and_triple_loop(oracle_mod):
     assert np.allclose(out.reshape(H * W, O), ref, rtol=1e-12, atol=1e-12)
 
 
+# ----------------------------------------------------------------- identity shortcut (two-layer residual block)
+def test_shortcut_with_zero_weights_is_a_closed_form_of_the_block_input(oracle_mod):
+    # block: a1 = relu(conv0(a0)); a2 = relu(conv1(a1) + b1 + a0).  With conv1's weights zero, a2 = relu(b1 + a0): it
+    # depends on the BLOCK'S input alone.  A shortcut that is dropped gives relu(b1); one taken from a1 gives
+    # relu(b1 + a1); one added after the activation gives relu(b1) + a0 (a0 has negative values, so that differs too).
+    rng = np.random.default_rng(21)
+    H, W, C = 4, 5, 3
+    b1 = np.array([0.25, -0.5, 1.0], np.float32)
+    l0 = Layer(CONV3X3, C, C, h=H, w=W, relu=1, weight=rand_bits(rng, (C, 3, 3, C)), bias=rng.standard_normal(C).astype(np.float32))
+    l1 = Layer(CONV3X3, C, C, h=H, w=W, relu=1, weight=bits(np.zeros((C, 3, 3, C))), bias=b1, residual=1)
+    xb = rand_bits(rng, (H * W * C,))
+    a0 = f64(xb).reshape(H, W, C)
+    out = oracle_mod.forward_one([l0, l1], xb).reshape(H, W, C)
+    want = np.maximum(a0 + b1.astype(np.float64), 0.0)
+    assert np.array_equal(out, want)
+    assert (a0 < 0).any() and not np.array_equal(want, np.maximum(b1.astype(np.float64), 0.0) + 0 * a0)
+    # without the activation the sum itself comes out
+    l1n = Layer(CONV3X3, C, C, h=H, w=W, relu=0, weight=l1.weight, bias=b1, residual=1)
+    assert np.array_equal(oracle_mod.forward_one([l0, l1n], xb).reshape(H, W, C), a0 + b1.astype(np.float64))
+    # and a layer without the flag ignores the block's input
+    l1p = Layer(CONV3X3, C, C, h=H, w=W, relu=1, weight=l1.weight, bias=b1, residual=0)
+    assert np.array_equal(oracle_mod.forward_one([l0, l1p], xb).reshape(H, W, C),
+                          np.broadcast_to(np.maximum(b1.astype(np.float64), 0.0), (H, W, C)))
+
+
+def test_shortcut_blocks_vs_scipy(oracle_mod):
+    # two blocks in a row, then pool and head; the second block's input is the first block's output
+    rng = np.random.default_rng(22)
+    H, W, C = 5, 4, 2
+    convs = [Layer(CONV3X3, C, C, h=H, w=W, relu=1, weight=rand_bits(rng, (C, 3, 3, C), 0.5),
+                   bias=rng.standard_normal(C).astype(np.float32), residual=int(i in (1, 3))) for i in range(4)]
+    head = Layer(DENSE, C, 3, relu=0, weight=rand_bits(rng, (3, C)), bias=rng.standard_normal(3).astype(np.float32))
+    xb = rand_bits(rng, (H * W * C,))
+
+    def lib_conv(x, l):
+        w = f64(l.weight)
+        y = np.zeros((H, W, C))
+        for o in range(C):
+            y[:, :, o] = l.bias[o] + sum(correlate2d(x[:, :, c], w[o, :, :, c], mode="same", boundary="fill", fillvalue=0.0)
+                                         for c in range(C))
+        return y
+
+    a0 = f64(xb).reshape(H, W, C)
+    a1 = np.maximum(lib_conv(a0, convs[0]), 0.0)
+    a2 = np.maximum(lib_conv(a1, convs[1]) + a0, 0.0)
+    a3 = np.maximum(lib_conv(a2, convs[2]), 0.0)
+    a4 = np.maximum(lib_conv(a3, convs[3]) + a2, 0.0)
+    out = oracle_mod.forward_one(convs, xb).reshape(H, W, C)
+    assert np.allclose(out, a4, rtol=1e-10, atol=1e-10)
+    assert not np.allclose(out, np.maximum(lib_conv(a3, convs[3]) + a3, 0.0), atol=1e-3)    # the wrong tensor is far off
+    full = oracle_mod.forward_one(convs + [Layer(GLOBAL_AVG_POOL, C, C, h=H, w=W), head], xb)
+    assert np.allclose(full, f64(head.weight) @ a4.reshape(H * W, C).mean(axis=0) + head.bias, rtol=1e-10, atol=1e-10)
+
+
+def test_shortcut_needs_two_conv_layers_of_one_shape(oracle_mod):
+    rng = np.random.default_rng(23)
+    conv = lambda c, o, res: Layer(CONV3X3, c, o, h=3, w=3, relu=1, weight=rand_bits(rng, (o, 3, 3, c)), bias=None, residual=res)
+    xb = rand_bits(rng, (3 * 3 * 2,))
+    with pytest.raises(Exception):
+        oracle_mod.forward_one([conv(2, 2, 1)], xb)                      # nothing before it
+    with pytest.raises(Exception):
+        oracle_mod.forward_one([conv(2, 4, 0), conv(4, 4, 1)], xb)       # the block's input has another shape
+
+
 def test_conv_relu_and_stack_with_pool_and_head(oracle_mod):
     rng = np.random.default_rng(11)
     H, W, C = 4, 3, 2
