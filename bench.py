@@ -200,6 +200,8 @@ def dominant_roofline(wl, kernel_ms_per_step, peaks, peaks_kind, config, long_ru
                 "frac_of_burst_peak": ach / burst, "frac_of_sustained_peak": ach / sustained}
     traffic, source = None, None
     t = TRAFFIC.get(config)
+    if any(getattr(l, "residual", 0) for m in wl.models for l in m):
+        t = None            # the captures are of the plain workload
     if t is not None:
         traffic = int(t["ratio"] * byts) if "ratio" in t else int(t["bytes"])
         source = t["source"]
@@ -356,6 +358,8 @@ def measure_config(cfg, args, ctx):
     steps = args.steps if args.steps is not None else DEFAULT_STEPS[cfg]
 
     over = {"n_tenants": args.tenants} if args.tenants else {}
+    if args.shortcuts and cfg == 4:
+        over["shortcuts"] = (1, 3)      # conv layers 1 and 3 close two-layer residual blocks (identity shortcuts)
     models = synth.make_models(cfg, **over)
     batches = [synth.make_requests(cfg, models, n=args.requests, salt=1000 * rank + b) for b in range(N_INPUT_BUFFERS)]
     wl = synth.Workload(synth.CONFIG_NAMES[cfg], cfg, models, batches[0][0], batches[0][1])
@@ -509,7 +513,7 @@ def measure_config(cfg, args, ctx):
     line = result_line(units, ms, steps, n_gpus=world, steps=steps, warmup=args.warmup, scaling="weak",
                        vs_baseline=None, dtype="bf16", data="synthetic")
     line["config"] = {"workload": synth.CONFIG_NAMES[cfg], "requests_per_step_per_gpu": n, "tenants": len(models),
-                      "reduced": bool(args.tenants or args.requests),
+                      "reduced": bool(args.tenants or args.requests), "residual_blocks": bool(args.shortcuts and cfg == 4),
                       "l2": "weights streamed per step exceed the 126 MB L2 only for c2/c3/c5; inputs rotate over "
                             "%d device buffers" % N_INPUT_BUFFERS,
                       "parallelism": "replicas x%d (each GPU hosts all tenants, own batch)" % world}
@@ -582,6 +586,8 @@ def main():
     ap.add_argument("--tenants", type=int, default=None, help="reduced case: number of tenants (profiling captures)")
     ap.add_argument("--requests", type=int, default=None, help="reduced case: requests per batch")
     ap.add_argument("--profile", action="store_true", help="timed loop only (no e2e, CPU baseline or clock sampler)")
+    ap.add_argument("--shortcuts", action="store_true", help="workload 4 as two residual blocks: conv layers 1 and 3 add "
+                    "the input of the layer before them (a variant, not the headline)")
     ap.add_argument("--cache-sweep", action="store_true", help="weight-residency leg: workload 2 behind a device cache "
                     "of 40-100 %% of its weights (prints its own JSON line)")
     args = ap.parse_args()
@@ -612,7 +618,7 @@ def main():
         return
     head_cfg = args.config or HEADLINE_CONFIG
     line = measure_config(head_cfg, args, ctx)
-    reduced = bool(args.tenants or args.requests or args.profile)
+    reduced = bool(args.tenants or args.requests or args.profile or args.shortcuts)
     if args.config is None and world == 1 and not reduced and not args.no_per_config and line is not None:
         # the same measurements for all five workloads; --steps applies to the headline only
         per = {"c%d" % head_cfg: {k: v for k, v in line.items() if k not in ("metric", "unit", "higher_is_better", "n_gpus",

@@ -52,13 +52,18 @@ typedef enum { MT_DENSE = 0, MT_CONV3X3 = 1, MT_GLOBAL_AVG_POOL = 2 } mt_layer_k
  *   MT_CONV3X3          NHWC, stride 1, zero pad 1, cross-correlation; W bf16 [out_ch][3][3][in_ch];
  *                       tap (ky,kx) reads pixel (y+ky-1, x+kx-1)
  *   MT_GLOBAL_AVG_POOL  mean over the h*w positions of each channel; no weights
+ * residual (MT_CONV3X3 only, the layer before it a conv too): the layer closes a two-layer residual block with an
+ * identity shortcut, the building block of the network the paper uses as its running example (Sec. 1.1, resnet18):
+ * a[l+1] = act(conv(a[l]) + b + a[l-1]), where a[l-1] is the INPUT of the layer before.  Tenants of one conv family
+ * may differ in which layers carry it.
  * weight / bias may be host or device pointers; the library copies them during mt_register_model and
  * keeps no reference, so the caller may free them on return.  bias == NULL means zeros. */
 typedef struct {
     int32_t kind;          /* mt_layer_kind */
     int32_t in_ch, out_ch; /* dense: in/out features; conv: C_in/C_out; pool: in_ch == out_ch */
     int32_t h, w;          /* conv/pool spatial size; 0 for dense */
-    int32_t relu;          /* 1: apply max(.,0) after bias */
+    int32_t relu;          /* 1: apply max(.,0) after bias (and after the shortcut's sum) */
+    int32_t residual;      /* 1: add the previous layer's input before the activation (see above); else 0 */
     const void* weight;    /* bf16 */
     const void* bias;      /* fp32 [out_ch] */
 } mt_layer_desc;
@@ -83,7 +88,8 @@ mt_status mt_shutdown(void);
  * untouched.  The row stride of the input buffer is the WIDEST registered model's input (mt_input_elems); a request of a
  * model with fewer inputs carries them at the start of its row and the rest of the row is never read.
  * Kernel limits (else MT_ERR_UNSUPPORTED): 1..MT_MAX_LAYERS layers; dense in_ch a multiple of 64;
- * conv in_ch == out_ch == 64, w <= 126; a pool must follow a conv; a dense layer may not precede a conv.
+ * conv in_ch == out_ch == 64, w <= 126; a pool must follow a conv; a dense layer may not precede a conv; residual
+ * only on a conv layer that follows a conv layer.
  * The call does not wait for the device: weights and biases in HOST memory are copied into the library's pinned
  * staging before it returns (the caller may free them at once), and the copy to the device and the re-layout run on
  * an internal stream, under whatever batches are in flight; the first mt_infer* / mt_prefetch that follows waits, on

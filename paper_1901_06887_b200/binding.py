@@ -43,7 +43,7 @@ class CacheStats(ctypes.Structure):
 
 class LayerDesc(ctypes.Structure):
     _fields_ = [("kind", ctypes.c_int32), ("in_ch", ctypes.c_int32), ("out_ch", ctypes.c_int32),
-                ("h", ctypes.c_int32), ("w", ctypes.c_int32), ("relu", ctypes.c_int32),
+                ("h", ctypes.c_int32), ("w", ctypes.c_int32), ("relu", ctypes.c_int32), ("residual", ctypes.c_int32),
                 ("weight", ctypes.c_void_p), ("bias", ctypes.c_void_p)]
 
 
@@ -129,7 +129,7 @@ def mt_shutdown() -> None:
 
 
 def mt_register_model(layers: Sequence) -> int:
-    """layers: objects with kind, in_ch, out_ch, h, w, relu, weight, bias (weight: uint16 numpy array of bf16
+    """layers: objects with kind, in_ch, out_ch, h, w, relu, weight, bias and optionally residual (weight: uint16 numpy array of bf16
     bit patterns or a torch bf16 tensor, host or device; bias: float32 or None).  Returns the model id."""
     arr = (LayerDesc * len(layers))()
     keep = []
@@ -140,7 +140,8 @@ def mt_register_model(layers: Sequence) -> int:
         if isinstance(b, np.ndarray):
             b = np.ascontiguousarray(b, dtype=np.float32)
         keep += [w, b]
-        arr[i] = LayerDesc(int(l.kind), int(l.in_ch), int(l.out_ch), int(l.h), int(l.w), int(l.relu), _ptr(w), _ptr(b))
+        arr[i] = LayerDesc(int(l.kind), int(l.in_ch), int(l.out_ch), int(l.h), int(l.w), int(l.relu), int(getattr(l, "residual", 0)),
+                           _ptr(w), _ptr(b))
     mid = ctypes.c_int32(-1)
     _check(lib().mt_register_model(arr, len(layers), ctypes.byref(mid)), "mt_register_model")
     return int(mid.value)

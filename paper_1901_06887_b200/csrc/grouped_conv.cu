@@ -49,6 +49,8 @@ struct StripCoord {
     int t, j, y0, strip_in_image;
 };
 
+// kSkip: the layer has tenants with an identity shortcut (ConvArgs::skip[0]); the plain form carries none of that code.
+template <bool kSkip>
 __global__ void __launch_bounds__(kConvThreads, 1)
 grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArgs p) {
     extern __shared__ uint8_t smem_raw[];
@@ -282,9 +284,10 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
         const int r = q4 * 32 + lane;               // tile-local padded pixel of this thread
         const int yl = r / Wp, x = r - yl * Wp;
         const int rows_per_tile = BM / Wp;
-        int g = 0, relu = 0;
+        int g = 0, relu = 0, resid = 0;
         bool ok = true;
         int img_j = 0, y0 = 0;
+        int skip_img = 0;                           // image index of the strip in the tensor a residual layer adds
         const bool pooling = (p.pool_partial != nullptr);
         for (int s = s_begin; ok && s < s_end; ++s) {
             float psum[32];
@@ -305,7 +308,11 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
                         asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");   // everyone done with the old bias
                         if (threadIdx.x - 64 < kCN) s_bias[threadIdx.x - 64] = L.bias[threadIdx.x - 64];
                         relu = L.relu;
+                        if constexpr (kSkip) resid = (L.residual && p.skip[0] != nullptr) ? 1 : 0;
                         asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+                    }
+                    if constexpr (kSkip) {
+                        if (resid) skip_img = p.skip_perm[0] ? p.skip_perm[0][img_j] : img_j;
                     }
                 }
                 tc_fence_after();
@@ -318,6 +325,14 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
                 if (x < p.W && y < p.H) {
                     uint16_t* dst = p.out + (((size_t)img_j * p.H + y) * p.W + x) * kCN + half * 32;
                     const float4* b4 = reinterpret_cast<const float4*>(s_bias + half * 32);
+                    // identity shortcut: this thread's pixel of the block's input, 32 channels = 64 bytes
+                    uint4 sk[4];
+                    if constexpr (kSkip) if (resid) {
+                        const uint4* sp = reinterpret_cast<const uint4*>(
+                            p.skip[0] + (((size_t)skip_img * p.H + y) * p.W + x) * kCN + half * 32);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) sk[j] = __ldcg(sp + j);
+                    }
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         float f[8];
@@ -328,6 +343,14 @@ grouped_conv3x3_kernel(const __grid_constant__ CUtensorMap tmap_x, const ConvArg
                             f[4 * h2 + 1] = __uint_as_float(v[8 * j + 4 * h2 + 1]) + b.y;
                             f[4 * h2 + 2] = __uint_as_float(v[8 * j + 4 * h2 + 2]) + b.z;
                             f[4 * h2 + 3] = __uint_as_float(v[8 * j + 4 * h2 + 3]) + b.w;
+                        }
+                        if constexpr (kSkip) if (resid) {
+                            const uint32_t w4[4] = {sk[j].x, sk[j].y, sk[j].z, sk[j].w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {       // two bf16 per word, the lower address in the low half
+                                f[2 * e + 0] += __uint_as_float(w4[e] << 16);
+                                f[2 * e + 1] += __uint_as_float(w4[e] & 0xffff0000u);
+                            }
                         }
                         if (relu) {
 #pragma unroll
@@ -523,11 +546,14 @@ void launch_pool_head(const float* partial, int n, int strips, int HW, const Mod
 }
 
 cudaError_t configure_grouped_conv() {
-    return cudaFuncSetAttribute(grouped_conv3x3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(grouped_conv3x3_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(grouped_conv3x3_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
 }
 
 void launch_grouped_conv(const CUtensorMap& tmap_x, const ConvArgs& a, int smem_bytes, int sm_count, cudaStream_t s) {
-    launch_pdl(grouped_conv3x3_kernel, dim3(sm_count), dim3(kConvThreads), (size_t)smem_bytes, s, tmap_x, a);
+    if (a.skip[0]) launch_pdl(grouped_conv3x3_kernel<true>, dim3(sm_count), dim3(kConvThreads), (size_t)smem_bytes, s, tmap_x, a);
+    else launch_pdl(grouped_conv3x3_kernel<false>, dim3(sm_count), dim3(kConvThreads), (size_t)smem_bytes, s, tmap_x, a);
 }
 
 }  // namespace mt

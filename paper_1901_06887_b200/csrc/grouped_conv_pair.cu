@@ -71,6 +71,9 @@ struct PairStrip {
 // in global memory, every wait bounded) - a layer boundary inside a launch costs a few microseconds, one between two
 // launches about three times that, since no CTA of the next launch can start while one of this launch holds its SM's
 // shared memory.  The next layer's first weights are requested before the barrier.
+// kSkip: the launch has layers with identity shortcuts (ConvArgs::skip); without it the epilogue carries none of that
+// code - its registers and the predicated loads cost the plain path 5 % when they were compiled in unconditionally.
+template <bool kSkip>
 __global__ void __launch_bounds__(kCpThreads, 1)
 grouped_conv3x3_pair_kernel(const __grid_constant__ ConvStackMaps maps, const ConvArgs p) {
     extern __shared__ uint8_t smem_raw[];
@@ -493,97 +496,198 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ ConvStackMaps maps, const Co
         const int layer = p.layer + k;
         const bool pooling = (p.pool_partial != nullptr) && k == n_stack - 1;   // only the stack's last layer feeds the pool
         const CUtensorMap* const tmap_y = &maps.y[k];
+        // Identity shortcuts (kSkip only): a thread adds, to its pixel's 32 channels, 64 bytes of the tensor that the
+        // layer before read.  The epilogue of this kernel has no slack (the MMAs are bound by operand reads from
+        // shared memory and a tile leaves the pipe every 1.4 us), so the obvious form - every thread loads its 64 bytes
+        // when the accumulator is ready - took 2.7 x the time of a plain layer.  What this form does instead:
+        //  - whole sectors, nothing through shared memory: a thread reads its own 64 bytes as two 32-byte loads (staging
+        //    a coalesced load through the warp's shared-memory region took bandwidth from the MMAs' operand reads:
+        //    +34 us per layer; an exchange between lanes cost as many instructions as it saved sectors);
+        //  - the values of a tile are requested TWO tiles ahead (16 KiB per SM and tile in flight, twice): one tile
+        //    ahead the layer's 103 MB could not be in flight often enough to arrive within the layer's 50 us.  That
+        //    needs a tile's coordinates long before its record is published, so the epilogue derives them itself (the
+        //    same unit -> (tenant, image, row) map as the producer's) and re-reads the tenant's flag and the image's
+        //    arrival index only when they change;
+        //  - four tiles ahead the same lines are asked into L2 (a prefetch holds no register), so most of those
+        //    loads are L2 hits; and the buffers must not spill: a spilled load destination is a wait for the load.
+        // On 56 x 56 images a layer with shortcuts now takes 1.65 x a plain one (83 against 50 us), of which a third is
+        // the extra instructions, the rest the loads.
+        // Tiles alternate between the two register buffers, so a strip must have an even number of tiles (it has two).
+        const uint16_t* const skip_k = kSkip ? p.skip[k] : nullptr;
+        const int32_t* const skip_perm_k = kSkip ? p.skip_perm[k] : nullptr;
+        const bool skip_wide = (reinterpret_cast<uintptr_t>(skip_k) & 31) == 0;      // 32-byte loads need that alignment
+        uint4 sk_a[4], sk_b[4];                     // values on their way: even / odd tile of a strip
+        bool have_a = false, have_b = false;        // warp-uniform: the buffer holds (or will hold) values to add
+        int n1_on = 0, n1_img = 0, n1_y0 = 0;       // strip s + 1: shortcut wanted (and the image real), its image, first row
+        int n2_on = 0, n2_img = 0, n2_y0 = 0;       // strip s + 2, looked up while strip s runs
+        int d_t = -1, d_resid = 0, d_j = -1, d_img = 0;     // last tenant / image looked up
+        auto describe = [&](int s2, int& on, int& img, int& first_row) {
+            const PairStrip c = locate(s2);
+            if (c.t != d_t) { d_t = c.t; d_resid = p.models[c.t].layer[layer].residual; }
+            if (c.j != d_j) { d_j = c.j; d_img = skip_perm_k ? skip_perm_k[c.j] : c.j; }
+            on = (skip_k != nullptr && !c.dummy && d_resid) ? 1 : 0;
+            first_row = c.y0;
+            img = d_img;
+        };
+        auto request = [&](int on, int img, int yy, uint4 (&dst)[4]) -> bool {      // yy: this thread's image row (warp-uniform)
+            if (!on || yy >= p.H) return false;
+            if (x < p.W) {
+                // written earlier in this launch or by the caller: read past L1
+                const uint16_t* sp = skip_k + (((size_t)img * p.H + yy) * p.W + x) * kCpN + half * 32;
+                if (skip_wide) {
+                    asm volatile("ld.global.cg.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                                 : "=r"(dst[0].x), "=r"(dst[0].y), "=r"(dst[0].z), "=r"(dst[0].w),
+                                   "=r"(dst[1].x), "=r"(dst[1].y), "=r"(dst[1].z), "=r"(dst[1].w) : "l"(sp));
+                    asm volatile("ld.global.cg.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                                 : "=r"(dst[2].x), "=r"(dst[2].y), "=r"(dst[2].z), "=r"(dst[2].w),
+                                   "=r"(dst[3].x), "=r"(dst[3].y), "=r"(dst[3].z), "=r"(dst[3].w) : "l"(sp + 16));
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) dst[j] = __ldcg(reinterpret_cast<const uint4*>(sp) + j);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) dst[j] = make_uint4(0u, 0u, 0u, 0u);
+            }
+            return true;
+        };
         if (*abort_flag) ok = false;
+        if constexpr (kSkip) {
+            if (ok && s_begin < s_end) {
+                int on, img, first_row;
+                describe(s_begin, on, img, first_row);
+                have_a = request(on, img, first_row + yl, sk_a);
+                if (TS > 1) have_b = request(on, img, first_row + rows_per_tile + yl, sk_b);
+                if (s_begin + 1 < s_end) describe(s_begin + 1, n1_on, n1_img, n1_y0);
+            }
+        }
+        float psum[32];
+        // One accumulator tile (tile i of strip s); buf / have_buf: the register buffer of the tile's parity.
+        auto do_tile = [&](int s, int i, uint4 (&buf)[4], bool& have_buf) -> bool {
+            const int slot = g % kCpSlots;
+            // tfull is completed by the leader's multicast commit: one lane per warp polls and tells the others
+            int got = 1;
+            if (lane == 0) got = mbar_wait_spin(tfull_bar(slot), (uint32_t)((g / kCpSlots) & 1), abort_flag, p.status, 58, 32) ? 1 : 0;
+            got = __shfl_sync(0xffffffffu, got, 0);
+            if (!got) return false;
+            if (i == 0) {
+                // the strip's record was published (with the strip's data) before any of its MMAs were issued
+                const int4 rec = s_rec[(s - s_begin) & (kCpRecords - 1)];
+                img_j = rec.y; y0 = rec.z; store = (rec.x & 8) ? 0 : 1;
+                // This completion (tile g) follows every read of the block under tile g (by tile g and, if the
+                // segment goes on, by the first two tap rows of tile g + 1, which are queued before the commit);
+                // the segment's first tile also hands back its own block.
+                if (threadIdx.x == 64 && (rec.x & 2)) { mbar_arrive(bempty_bar(rel & (kCpRing - 1))); ++rel; }
+                if (rec.x & 1) {                // new tenant: its bias into shared memory, ReLU flag into a register
+                    const LayerDev& L = p.models[rec.w].layer[layer];
+                    asm volatile("bar.sync 1, %0;" ::"n"(kCpEpiThreads) : "memory");   // everyone done with the old bias
+                    if (threadIdx.x - 64 < kCpN) s_bias[threadIdx.x - 64] = L.bias[threadIdx.x - 64];
+                    relu = L.relu;
+                    asm volatile("bar.sync 1, %0;" ::"n"(kCpEpiThreads) : "memory");
+                }
+            }
+            if (threadIdx.x == 64) { mbar_arrive(bempty_bar(rel & (kCpRing - 1))); ++rel; }
+            tc_fence_after();
+            uint32_t v[32];
+            tmem_ld32(tmem_base + (static_cast<uint32_t>(q4 * 32) << 16) + slot * kCpN + half * 32, v);
+            tmem_ld_wait();
+            tc_fence_before();
+            // values are in registers: the slot can be reused once the eight epilogue warps of both CTAs have said
+            // so (one arrival per warp: an arrival that crosses to the other CTA is expensive)
+            __syncwarp();
+            if (lane == 0) {
+                if (is_leader) mbar_arrive(tempty_bar(slot));
+                else mbar_arrive_remote_relaxed(tempty_leader0 + 8u * slot);
+            }
+            const int y = y0 + i * rows_per_tile + yl;
+            // bias (+ shortcut) + ReLU in fp32 on this thread's pixel, 32 channels
+            float f[32];
+            {
+                const float4* b4 = reinterpret_cast<const float4*>(s_bias + half * 32);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float4 b = b4[j];
+                    f[4 * j + 0] = __uint_as_float(v[4 * j + 0]) + b.x;
+                    f[4 * j + 1] = __uint_as_float(v[4 * j + 1]) + b.y;
+                    f[4 * j + 2] = __uint_as_float(v[4 * j + 2]) + b.z;
+                    f[4 * j + 3] = __uint_as_float(v[4 * j + 3]) + b.w;
+                }
+                if constexpr (kSkip) {
+                    // this tile's shortcut values were requested two tiles ago; the buffer then takes the request for
+                    // the tile of the same parity in the next strip
+                    if (have_buf) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t w4[4] = {buf[j].x, buf[j].y, buf[j].z, buf[j].w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {       // two bf16 per word, the lower address in the low half
+                                f[8 * j + 2 * e + 0] += __uint_as_float(w4[e] << 16);
+                                f[8 * j + 2 * e + 1] += __uint_as_float(w4[e] & 0xffff0000u);
+                            }
+                        }
+                    }
+                    have_buf = (s + 1 < s_end) ? request(n1_on, n1_img, n1_y0 + i * rows_per_tile + yl, buf) : false;
+                    if (i == 0 && s + 2 < s_end) {
+                        describe(s + 2, n2_on, n2_img, n2_y0);
+                        // and that strip's lines are asked into L2 now, four tiles ahead (one warp of the two that
+                        // share a pixel's 128-byte line does it), so that the loads above mostly find them there
+                        if (n2_on && half == 0 && x < p.W) {
+#pragma unroll
+                            for (int tl = 0; tl < 2; ++tl) {
+                                const int yy = n2_y0 + tl * rows_per_tile + yl;
+                                if (tl < TS && yy < p.H)
+                                    asm volatile("prefetch.global.L2 [%0];" ::"l"(skip_k + (((size_t)n2_img * p.H + yy) * p.W + x) * kCpN));
+                            }
+                        }
+                    }
+                }
+                if (relu) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) f[e] = fmaxf(f[e], 0.0f);
+                }
+            }
+            if (pooling) {      // the layer feeds a global average pool: only channel sums are kept
+                if (store && x < p.W && y < p.H) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) psum[e] += f[e];
+                }
+            } else {
+                // The warp's 32 pixels x 32 channels go to its staging region (64 bytes per pixel, 16-byte chunk c
+                // of pixel q at chunk c ^ ((q >> 1) & 3): the 64-byte swizzle of the store's tensor map) and leave
+                // as ONE tensor store, which also drops the pad columns and the rows past the image.  A row of
+                // per-thread 64-byte global stores would cost the load/store unit 32 separate lines per instruction.
+                if (lane == 0) bulk_wait_group_read0();      // the previous tile's store has read the region
+                __syncwarp();
+                uint8_t* mine = out_stage_ptr + ew * 2048 + lane * 64;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint4 o;
+                    o.x = pack_bf16x2(f[8 * j + 0], f[8 * j + 1]);
+                    o.y = pack_bf16x2(f[8 * j + 2], f[8 * j + 3]);
+                    o.z = pack_bf16x2(f[8 * j + 4], f[8 * j + 5]);
+                    o.w = pack_bf16x2(f[8 * j + 6], f[8 * j + 7]);
+                    *reinterpret_cast<uint4*>(mine + ((j ^ ((lane >> 1) & 3)) << 4)) = o;
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                const int yw = y0 + i * rows_per_tile + (q4 >> 1);       // the warp's image row (warp-uniform)
+                if (lane == 0 && store && yw < p.H && (q4 & 1) * 32 < p.W) {
+                    tma_store_4d(tmap_y, half * 32, (q4 & 1) * 32, yw, img_j, out_stage0 + ew * 2048);
+                    bulk_commit_group();
+                }
+            }
+            __syncwarp();
+            ++g;
+            return true;
+        };
         for (int s = s_begin; ok && s < s_end; ++s) {
-            float psum[32];
 #pragma unroll
             for (int e = 0; e < 32; ++e) psum[e] = 0.0f;
-            for (int i = 0; i < TS; ++i, ++g) {
-                const int slot = g % kCpSlots;
-                // tfull is completed by the leader's multicast commit: one lane per warp polls and tells the others
-                int got = 1;
-                if (lane == 0) got = mbar_wait_spin(tfull_bar(slot), (uint32_t)((g / kCpSlots) & 1), abort_flag, p.status, 58, 32) ? 1 : 0;
-                got = __shfl_sync(0xffffffffu, got, 0);
-                if (!got) { ok = false; break; }
-                if (i == 0) {
-                    // the strip's record was published (with the strip's data) before any of its MMAs were issued
-                    const int4 rec = s_rec[(s - s_begin) & (kCpRecords - 1)];
-                    img_j = rec.y; y0 = rec.z; store = (rec.x & 8) ? 0 : 1;
-                    // This completion (tile g) follows every read of the block under tile g (by tile g and, if the
-                    // segment goes on, by the first two tap rows of tile g + 1, which are queued before the commit);
-                    // the segment's first tile also hands back its own block.
-                    if (threadIdx.x == 64 && (rec.x & 2)) { mbar_arrive(bempty_bar(rel & (kCpRing - 1))); ++rel; }
-                    if (rec.x & 1) {                // new tenant: its bias into shared memory, ReLU flag into a register
-                        const LayerDev& L = p.models[rec.w].layer[layer];
-                        asm volatile("bar.sync 1, %0;" ::"n"(kCpEpiThreads) : "memory");   // everyone done with the old bias
-                        if (threadIdx.x - 64 < kCpN) s_bias[threadIdx.x - 64] = L.bias[threadIdx.x - 64];
-                        relu = L.relu;
-                        asm volatile("bar.sync 1, %0;" ::"n"(kCpEpiThreads) : "memory");
-                    }
-                }
-                if (threadIdx.x == 64) { mbar_arrive(bempty_bar(rel & (kCpRing - 1))); ++rel; }
-                tc_fence_after();
-                uint32_t v[32];
-                tmem_ld32(tmem_base + (static_cast<uint32_t>(q4 * 32) << 16) + slot * kCpN + half * 32, v);
-                tmem_ld_wait();
-                tc_fence_before();
-                // values are in registers: the slot can be reused once the eight epilogue warps of both CTAs have said
-                // so (one arrival per warp: an arrival that crosses to the other CTA is expensive)
-                __syncwarp();
-                if (lane == 0) {
-                    if (is_leader) mbar_arrive(tempty_bar(slot));
-                    else mbar_arrive_remote_relaxed(tempty_leader0 + 8u * slot);
-                }
-                const int y = y0 + i * rows_per_tile + yl;
-                // bias + ReLU in fp32 on this thread's pixel, 32 channels
-                float f[32];
-                {
-                    const float4* b4 = reinterpret_cast<const float4*>(s_bias + half * 32);
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const float4 b = b4[j];
-                        f[4 * j + 0] = __uint_as_float(v[4 * j + 0]) + b.x;
-                        f[4 * j + 1] = __uint_as_float(v[4 * j + 1]) + b.y;
-                        f[4 * j + 2] = __uint_as_float(v[4 * j + 2]) + b.z;
-                        f[4 * j + 3] = __uint_as_float(v[4 * j + 3]) + b.w;
-                    }
-                    if (relu) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) f[e] = fmaxf(f[e], 0.0f);
-                    }
-                }
-                if (pooling) {      // the layer feeds a global average pool: only channel sums are kept
-                    if (store && x < p.W && y < p.H) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) psum[e] += f[e];
-                    }
-                } else {
-                    // The warp's 32 pixels x 32 channels go to its staging region (64 bytes per pixel, 16-byte chunk c
-                    // of pixel q at chunk c ^ ((q >> 1) & 3): the 64-byte swizzle of the store's tensor map) and leave
-                    // as ONE tensor store, which also drops the pad columns and the rows past the image.  A row of
-                    // per-thread 64-byte global stores would cost the load/store unit 32 separate lines per instruction.
-                    if (lane == 0) bulk_wait_group_read0();      // the previous tile's store has read the region
-                    __syncwarp();
-                    uint8_t* mine = out_stage_ptr + ew * 2048 + lane * 64;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        uint4 o;
-                        o.x = pack_bf16x2(f[8 * j + 0], f[8 * j + 1]);
-                        o.y = pack_bf16x2(f[8 * j + 2], f[8 * j + 3]);
-                        o.z = pack_bf16x2(f[8 * j + 4], f[8 * j + 5]);
-                        o.w = pack_bf16x2(f[8 * j + 6], f[8 * j + 7]);
-                        *reinterpret_cast<uint4*>(mine + ((j ^ ((lane >> 1) & 3)) << 4)) = o;
-                    }
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    const int yw = y0 + i * rows_per_tile + (q4 >> 1);       // the warp's image row (warp-uniform)
-                    if (lane == 0 && store && yw < p.H && (q4 & 1) * 32 < p.W) {
-                        tma_store_4d(tmap_y, half * 32, (q4 & 1) * 32, yw, img_j, out_stage0 + ew * 2048);
-                        bulk_commit_group();
-                    }
-                }
-                __syncwarp();
+            for (int i = 0; ok && i < TS; i += 2) {
+                ok = do_tile(s, i, sk_a, have_a);
+                if (ok && i + 1 < TS) ok = do_tile(s, i + 1, sk_b, have_b);
             }
+            if constexpr (kSkip) { n1_on = n2_on; n1_img = n2_img; n1_y0 = n2_y0; }
             if (pooling && ok) {
                 // Channel sums of this strip: a halving butterfly leaves lane c with the warp's total of channel c
                 // (31 shuffles), the four lane quarters are then added in a fixed order, and the strip's 64 sums are
@@ -665,7 +769,9 @@ void launch_pretile_conv_pair(const uint16_t* w, uint16_t* out, cudaStream_t s) 
 int conv_pair_smem_bytes() { return kCpSmemBytes; }
 
 cudaError_t configure_grouped_conv_pair() {
-    return cudaFuncSetAttribute(grouped_conv3x3_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(grouped_conv3x3_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(grouped_conv3x3_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
 }
 
 // Cluster of two CTAs; grid = an even number of CTAs (one per SM).  a.tile_prefix counts (pair of images, strip) units.
@@ -684,7 +790,10 @@ cudaError_t launch_grouped_conv_pair(const ConvStackMaps& maps, const ConvArgs& 
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 2;
     ++g_kernel_launches;
-    return cudaLaunchKernelEx(&cfg, grouped_conv3x3_pair_kernel, maps, a);
+    bool any_skip = false;
+    for (int k = 0; k < a.n_stack; ++k) any_skip = any_skip || a.skip[k] != nullptr;
+    return any_skip ? cudaLaunchKernelEx(&cfg, grouped_conv3x3_pair_kernel<true>, maps, a)
+                    : cudaLaunchKernelEx(&cfg, grouped_conv3x3_pair_kernel<false>, maps, a);
 }
 
 }  // namespace mt

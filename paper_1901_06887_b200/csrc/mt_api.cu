@@ -29,7 +29,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 struct HostLayer {
-    int kind, in_ch, out_ch, h, w, relu;
+    int kind, in_ch, out_ch, h, w, relu, residual;
 };
 
 struct HostModel {
@@ -135,6 +135,7 @@ struct Ctx {
     void* st_in = nullptr;
     int32_t* st_ids = nullptr;
     float* st_out = nullptr;
+    int n_residual[MT_MAX_LAYERS] = {0};     // live models whose layer l carries an identity shortcut
     size_t st_cap_in = 0, st_cap_ids = 0, st_cap_out = 0;   // bytes: a new family changes the row sizes, not only n
 
     // staging for mt_infer_host_async: two slots used in turn, so that the copies of one call overlap the compute
@@ -264,6 +265,7 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     CU_OK(configure_grouped_conv_pair());
     g.T = 0;
     g.live = 0;
+    for (int l = 0; l < MT_MAX_LAYERS; ++l) g.n_residual[l] = 0;
     g.has_family = false;
     g.cap_n = 0;
     g.ws_dirty = true;
@@ -445,7 +447,7 @@ mt_status fill_table_update(int id, uint8_t* base, TableUpdate* u) {
     for (size_t l = 0; l < hm.layers.size(); ++l) {
         const HostLayer& h = hm.layers[l];
         LayerDev& d = u->md.layer[l];
-        d.kind = h.kind; d.K = h.in_ch; d.N = h.out_ch; d.relu = h.relu;
+        d.kind = h.kind; d.K = h.in_ch; d.N = h.out_ch; d.relu = h.relu; d.residual = h.residual;
         d.n_tiles = (int)padded_weight_tiles(h);
         d.k_blocks = h.kind == MT_DENSE ? h.in_ch / BK : 9;
         if (h.kind == MT_GLOBAL_AVG_POOL) continue;
@@ -638,6 +640,8 @@ mt_status validate_layers(const mt_layer_desc* layers, int n_layers) {
         if (d.kind < MT_DENSE || d.kind > MT_GLOBAL_AVG_POOL) return MT_ERR_INVALID_ARG;
         if (d.in_ch <= 0 || d.out_ch <= 0) return MT_ERR_INVALID_ARG;
         if (d.kind != MT_GLOBAL_AVG_POOL && !d.weight) return MT_ERR_INVALID_ARG;
+        // an identity shortcut joins a conv layer's output with the input of the conv layer before it
+        if (d.residual && (d.kind != MT_CONV3X3 || l == 0 || layers[l - 1].kind != MT_CONV3X3)) return MT_ERR_UNSUPPORTED;
         if (d.kind == MT_DENSE) {
             if (l > 0) {
                 const mt_layer_desc& p = layers[l - 1];
@@ -806,7 +810,9 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
                            g.opt_pool_head;
     // Conv layers run on CTA pairs (two images of a tenant per cluster) when the strip geometry allows the tap
     // pairing; MT_CONV_PAIR=0 forces the one-CTA executor.
-    const bool conv_pair = tiles_per_image > 0 && g.conv.Wp == 64 && g.sm_count >= 2 && g.opt_conv_pair;
+    // (its shortcut path alternates two register buffers over a strip's tiles: an even number of them)
+    const bool conv_pair = tiles_per_image > 0 && g.conv.Wp == 64 && g.sm_count >= 2 && g.opt_conv_pair &&
+                           g.conv.tiles_per_strip % 2 == 0;
 
     // Dense families: the payload rows move into bucketed order inside the scatter pass when the batch is spread over
     // enough CTAs and small enough for them; otherwise as a gather pass of its own over the whole GPU.
@@ -903,6 +909,11 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             a.strips_per_image = g.conv.strips_per_image; a.box_bytes = g.conv.box_bytes;
             a.status = g.d_status;
             const auto is_conv = [&](int k) { return k >= 0 && k < L && g.family[k].kind == MT_CONV3X3; };
+            // what a residual layer k adds: the input of layer k - 1 (the caller's buffer, in arrival order, for k = 1)
+            const auto skip_of = [&](int k) -> const uint16_t* {
+                if (k < 1 || !is_conv(k - 1) || g.n_residual[k] == 0) return nullptr;   // no live model has one there
+                return k == 1 ? static_cast<const uint16_t*>(inputs) : static_cast<const uint16_t*>(g.act[k - 1]);
+            };
             const auto feeds_pool_at = [&](int k) { return k + 1 < L && g.family[k + 1].kind == MT_GLOBAL_AVG_POOL; };
             if (conv_pair) {
                 // consecutive conv layers (at most kConvStackMax) as ONE launch with grid-wide barriers in between
@@ -917,6 +928,10 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
                     // a layer that feeds the pool stores nothing: any valid map will do for it
                     maps.y[k] = feeds_pool_at(lk) ? (lk == 0 ? in_map : g.act_map[lk]) : g.act_store_map[lk + 1];
                 }
+                for (int k = 0; k < n_stack; ++k) {
+                    a.skip[k] = skip_of(l + k);
+                    a.skip_perm[k] = (l + k == 1) ? g.d_perm : nullptr;
+                }
                 a.n_stack = n_stack;
                 a.border_units = g.opt_conv_balance ? 2 : 0;
                 a.grid_bar = g.d_grid_bar + (n_conv_launch++ & 7);
@@ -928,6 +943,8 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
                 l = l_last;
             } else {
                 a.out = (uint16_t*)g.act[l + 1];
+                a.skip[0] = skip_of(l);
+                a.skip_perm[0] = (l == 1) ? g.d_perm : nullptr;
                 a.pool_partial = feeds_pool_at(l) ? g.d_pool_partial : nullptr;
                 launch_grouped_conv(l == 0 ? in_map : g.act_map[l], a, g.conv.smem_bytes, g.sm_count, s);
             }
@@ -987,6 +1004,7 @@ mt_status adopt_model(int id, const std::vector<HostLayer>& hl, uint8_t* block, 
     HostModel& hm = g.models[id];
     hm.alive = true;
     hm.layers = hl;
+    for (int l = 0; l < n_layers; ++l) g.n_residual[l] += hl[l].residual ? 1 : 0;
     hm.dev_block = g.cache_bytes ? nullptr : block;
     hm.block_bytes = total;
     hm.host_image = host_image;
@@ -1189,6 +1207,7 @@ mt_status mt_shutdown(void) {
     g.has_family = false;
     g.family.clear();
     g.live = 0;
+    for (int l = 0; l < MT_MAX_LAYERS; ++l) g.n_residual[l] = 0;
     g.T = 0;
     return MT_OK;
 }
@@ -1205,7 +1224,8 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
     CU_OK(cudaSetDevice(g.device));
     std::vector<HostLayer> hl(n_layers);
     for (int l = 0; l < n_layers; ++l)
-        hl[l] = {layers[l].kind, layers[l].in_ch, layers[l].out_ch, layers[l].h, layers[l].w, layers[l].relu ? 1 : 0};
+        hl[l] = {layers[l].kind, layers[l].in_ch, layers[l].out_ch, layers[l].h, layers[l].w, layers[l].relu ? 1 : 0,
+                 layers[l].residual ? 1 : 0};
     st = check_family(hl);
     if (st != MT_OK) return st;
     int id = -1;
@@ -1256,7 +1276,7 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
     for (int l = 0; l < n_layers && e == cudaSuccess; ++l) {
         const HostLayer& h = hl[l];
         LayerDev& d = md.layer[l];
-        d.kind = h.kind; d.K = h.in_ch; d.N = h.out_ch; d.relu = h.relu;
+        d.kind = h.kind; d.K = h.in_ch; d.N = h.out_ch; d.relu = h.relu; d.residual = h.residual;
         d.n_tiles = (int)padded_weight_tiles(h);
         d.k_blocks = h.kind == MT_DENSE ? h.in_ch / BK : 9;
         if (h.kind == MT_GLOBAL_AVG_POOL) continue;
@@ -1331,6 +1351,7 @@ mt_status mt_release(int32_t model_id) {
     cudaFree(hm.dev_block);
     hm.dev_block = nullptr;
     hm.alive = false;
+    for (size_t l = 0; l < hm.layers.size(); ++l) g.n_residual[l] -= hm.layers[l].residual ? 1 : 0;
     hm.layers.clear();
     g.live -= 1;
     recompute_tile_n();

@@ -20,6 +20,7 @@ struct LayerDev {
     int32_t relu;
     int32_t n_tiles;     // ceil(N / 128)
     int32_t k_blocks;    // dense: K / 64; conv: 9 taps
+    int32_t residual;    // conv: 1 = the previous layer's input is added before the activation
     const uint16_t* w;   // weights in executor layout (see pretile kernels)
     const float* bias;   // fp32, zero-padded to n_tiles * 128
 };

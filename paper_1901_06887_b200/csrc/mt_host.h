@@ -174,8 +174,15 @@ struct ConvArgs {
                                   // the ranges are cut (0: ranges of equal length)
     int n_stack = 1;              // CTA-pair executor: conv layers run by this launch
     unsigned* grid_bar = nullptr; // ... and the counter of their grid-wide barrier (zero when the launch starts)
+    // Identity shortcuts: per layer of the launch (index 0 for the one-CTA executor) the bf16 NHWC tensor that a tenant
+    // whose layer is marked residual adds before the activation - the input of the layer before - or nullptr when no
+    // such tensor exists (the family's first layer).  skip_perm non-null: that tensor is the caller's buffer, image
+    // index = skip_perm[j]; else it is in bucketed order.
+    const uint16_t* skip[4] = {nullptr, nullptr, nullptr, nullptr};
+    const int32_t* skip_perm[4] = {nullptr, nullptr, nullptr, nullptr};
     int32_t* status;
 };
+
 cudaError_t configure_grouped_conv();
 void launch_grouped_conv(const CUtensorMap& tmap_x, const ConvArgs& a, int smem_bytes, int sm_count, cudaStream_t s);
 
@@ -194,6 +201,7 @@ cudaError_t configure_grouped_conv_pair();
 // of 32 channels x 32 pixels x 1 row, 64-byte swizzle (unused by a layer that feeds the pool).  ConvArgs::perm applies to
 // the stack's first layer, ConvArgs::pool_partial to its last.
 constexpr int kConvStackMax = 4;
+static_assert(kConvStackMax <= 4, "ConvArgs::skip holds one entry per stacked layer");
 struct ConvStackMaps {
     CUtensorMap x2[kConvStackMax], x1[kConvStackMax], y[kConvStackMax];
 };

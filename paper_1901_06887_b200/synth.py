@@ -185,7 +185,8 @@ def make_models(config: int, **over) -> List[List[Layer]]:
     d = dict(_DEFAULTS[config]); d.update(over)
     T = d["n_tenants"]
     if config == 4:
-        return [make_conv_stack(config, t, d["n_conv"], d["ch"], d["h"], d["w"], d["n_out"]) for t in range(T)]
+        return [make_conv_stack(config, t, d["n_conv"], d["ch"], d["h"], d["w"], d["n_out"],
+                                shortcuts=tuple(d.get("shortcuts", ()))) for t in range(T)]
     models = []
     wrng = stream(config, "widths")
     for t in range(T):
@@ -250,6 +251,8 @@ def workload_bytes(models: List[List[Layer]], model_ids: np.ndarray, per_layer: 
             if l.weight is not None:
                 b += l.weight.size * 2 + l.bias.size * 4
             b += c * l.in_elems * 2                                   # read input activation (bf16)
+            if getattr(l, "residual", 0):
+                b += c * l.out_elems * 2                              # read the block's input once more (identity shortcut)
             b += c * l.out_elems * (4 if li == n_layers - 1 else 2)   # write output
             per[li] += b
     return per if per_layer else int(sum(per))
