@@ -126,7 +126,9 @@ mt_status mt_input_elems(int32_t* in_elems_out);
 mt_status mt_infer(const void* inputs, const int32_t* model_ids, int32_t n, void* outputs, void* stream);
 
 /* Same as mt_infer with HOST buffers (pinned memory recommended): copies inputs and ids to device
- * staging buffers on `stream`, runs the pass, copies the outputs back and synchronises `stream`. */
+ * staging buffers on `stream`, runs the pass, copies the outputs back and synchronises `stream`.
+ * The whole [n][out_elems] buffer is written: where models differ in output width, the columns of a row beyond its
+ * model's own come back as NaN (mt_infer, which writes the caller's device buffer directly, leaves them untouched). */
 mt_status mt_infer_host(const void* inputs_host, const int32_t* model_ids_host, int32_t n,
                         void* outputs_host, void* stream);
 

@@ -136,6 +136,7 @@ struct Ctx {
     int32_t* st_ids = nullptr;
     float* st_out = nullptr;
     int n_residual[MT_MAX_LAYERS] = {0};     // live models whose layer l carries an identity shortcut
+    bool out_mixed = false;                  // models of different output widths have been registered in this family
     size_t st_cap_in = 0, st_cap_ids = 0, st_cap_out = 0;   // bytes: a new family changes the row sizes, not only n
 
     // staging for mt_infer_host_async: two slots used in turn, so that the copies of one call overlap the compute
@@ -977,6 +978,7 @@ mt_status adopt_model(int id, const std::vector<HostLayer>& hl, uint8_t* block, 
         g.has_family = true;
         g.in_elems = layer_in_elems(hl[0]);
         g.out_elems = hl.back().out_ch;
+        g.out_mixed = false;
         for (const HostLayer& f : hl)
             if (f.kind == MT_CONV3X3) plan_conv(f.h, f.w, &g.conv);   // cannot fail: validate_layers bounds w
         for (int b = 0; b <= MT_MAX_LAYERS; ++b) g.width[b] = 0;
@@ -992,6 +994,7 @@ mt_status adopt_model(int id, const std::vector<HostLayer>& hl, uint8_t* block, 
         const int wd = layer_in_elems(hl[l]);
         if (wd > g.width[l]) { g.width[l] = wd; g.ws_dirty = true; }
     }
+    if (hl.back().out_ch != g.out_elems) g.out_mixed = true;
     if (hl.back().out_ch > g.out_elems) {          // a wider output: the rows of the output buffer get longer
         g.out_elems = hl.back().out_ch;
         g.ws_dirty = true;
@@ -1396,6 +1399,8 @@ mt_status mt_infer_host(const void* inputs_host, const int32_t* model_ids_host, 
     }
     CU_OK(cudaMemcpyAsync(g.st_in, inputs_host, in_bytes, cudaMemcpyHostToDevice, s));
     CU_OK(cudaMemcpyAsync(g.st_ids, model_ids_host, id_bytes, cudaMemcpyHostToDevice, s));
+    // columns beyond a model's own are never written: what the caller gets there must not be an earlier batch's values
+    if (g.out_mixed) CU_OK(cudaMemsetAsync(g.st_out, 0xFF, out_bytes, s));      // all ones: a NaN
     mt_status st = infer_device(g.st_in, g.st_ids, n, g.st_out, s);
     if (st != MT_OK) return st;
     st = cache_end_batch(s);
@@ -1452,6 +1457,7 @@ mt_status mt_infer_host_async(const void* inputs_host, const int32_t* model_ids_
         mt_status rs = ensure_resident(set, reqs, s);
         if (rs != MT_OK) return rs;
     }
+    if (g.out_mixed) CU_OK(cudaMemsetAsync(g.as_out[k], 0xFF, out_bytes, s));   // see mt_infer_host
     st = infer_device(g.as_in[k], g.as_ids[k], n, g.as_out[k], s);
     if (st != MT_OK) return st;
     st = cache_end_batch(s);
