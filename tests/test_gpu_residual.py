@@ -85,3 +85,40 @@ def test_flag_is_per_tenant_and_where_it_is_refused():
     with pytest.raises(mt.MtError) as e:
         mt.mt_register_model(mlp)
     assert e.value.code == 4
+
+
+def test_models_with_shortcuts_come_and_go(conv_path):
+    # the executors pick their shortcut form only while a live model has one on that layer: register a plain family,
+    # add a model with shortcuts, release it again, bring another in on a different layer - every batch against the oracle
+    H, W = 10, 44
+    plain = [synth.make_conv_stack(21, t, 3, 64, H, W, 10) for t in range(2)]
+    late = synth.make_conv_stack(21, 7, 3, 64, H, W, 10, shortcuts=(2,))
+    early = synth.make_conv_stack(21, 8, 3, 64, H, W, 10, shortcuts=(1,))
+    rng = np.random.default_rng(9)
+
+    def batch(models_by_id, n=13):
+        ids = np.asarray(rng.choice(sorted(models_by_id), size=n), np.int32)
+        xb = bits(rng.standard_normal((n, H * W * 64)))
+        got = harness.run_batch(ids, xb, 10)
+        assert mt.mt_get_async_status() == (0, -1)
+        for t, m in models_by_id.items():
+            rows = np.flatnonzero(ids == t)
+            if len(rows):
+                ref = oracle.forward([m], np.zeros(len(rows), np.int32), xb[rows])
+                assert harness.scaled_error(got[rows], ref).max() <= TOL
+
+    fresh()
+    live = {mt.mt_register_model(m): m for m in plain}
+    batch(live)
+    t_late = mt.mt_register_model(late)
+    live[t_late] = late
+    batch(live)
+    mt.mt_release(t_late)
+    del live[t_late]
+    batch(live)
+    t_early = mt.mt_register_model(early)
+    assert t_early == t_late                      # the slot is reused, with other flags
+    live[t_early] = early
+    batch(live)
+    live[mt.mt_register_model(late)] = late
+    batch(live, n=31)
