@@ -4,6 +4,7 @@ before it to its pre-activation.  Tenants of one family may differ in which laye
 against the per-request oracle on every conv path, and against closed forms."""
 import numpy as np
 import pytest
+import torch
 
 import oracle
 from paper_1901_06887_b200 import binding as mt, harness, synth
@@ -122,3 +123,26 @@ def test_models_with_shortcuts_come_and_go(conv_path):
     batch(live)
     live[mt.mt_register_model(late)] = late
     batch(live, n=31)
+
+
+def test_shortcut_from_a_caller_buffer_that_is_only_16_byte_aligned(conv_path):
+    # layer 1's shortcut reads the caller's input buffer; mt_infer asks for 16-byte alignment only, and the 32-byte
+    # loads of the CTA-pair executor's shortcut path need more: it must fall back to 16-byte loads, same results
+    H, W, n = 8, 40, 9
+    models = [synth.make_conv_stack(21, t, 2, 64, H, W, 10, shortcuts=(1,)) for t in range(2)]
+    rng = np.random.default_rng(12)
+    ids = rng.integers(0, 2, n).astype(np.int32)
+    xb = bits(rng.standard_normal((n, H * W * 64)))
+    fresh()
+    harness.register_models(models)
+    want = harness.run_batch(ids, xb, 10)
+    flat = torch.zeros(xb.size + 8, dtype=torch.int16, device="cuda")
+    shifted = flat[8:]                                           # 16 bytes past a 256-byte boundary
+    assert shifted.data_ptr() % 32 == 16
+    shifted.copy_(torch.from_numpy(xb.view(np.int16).reshape(-1)).cuda())
+    out = torch.full((n, 10), float("nan"), dtype=torch.float32, device="cuda")
+    mt.mt_infer(shifted, torch.from_numpy(ids).cuda(), n, out)
+    assert mt.mt_get_async_status() == (0, -1)
+    assert np.array_equal(out.cpu().numpy(), want)
+    ref = oracle.forward(models, ids, xb)
+    assert harness.scaled_error(want, ref).max() <= TOL
