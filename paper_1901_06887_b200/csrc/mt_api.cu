@@ -1059,14 +1059,16 @@ mt_status register_async(const mt_layer_desc* layers, const std::vector<HostLaye
     std::vector<int> evicted;
     if (g.cache_bytes) {
         size_t off = 0;
-        if (g.cache.acquire(id, total, ++g.cache_tick, &off, &evicted) == WeightCache::kNoRoom) return MT_ERR_OOM;
+        const WeightCache::Result got = g.cache.acquire(id, total, ++g.cache_tick, &off, &evicted);
         block = g.arena + off;
         // the victims' bytes may still be read by batches in flight; their table entries flip at the next flush
+        // (also when no room could be made in the end: what was evicted on the way stays evicted)
         uint64_t youngest = 0;
         for (int v : evicted) {
             g.pending_ops.push_back({v, 2});
             if (g.models[v].last_batch > youngest) youngest = g.models[v].last_batch;
         }
+        if (got == WeightCache::kNoRoom) return MT_ERR_OOM;
         if (youngest > g.synced_batch && youngest <= g.batch_no)
             CU_OK(cudaStreamWaitEvent(g.load_stream, g.batch_done[youngest % Ctx::kBatchEvents], 0));
     } else {
@@ -1258,14 +1260,15 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
         // in flight once the device has been synchronised, so the victims' table entries are switched directly)
         std::vector<int> evicted;
         size_t off = 0;
-        if (g.cache.acquire(id, total, ++g.cache_tick, &off, &evicted) == WeightCache::kNoRoom) return MT_ERR_OOM;
+        const WeightCache::Result got = g.cache.acquire(id, total, ++g.cache_tick, &off, &evicted);
         CU_OK(cudaDeviceSynchronize());
         g.synced_batch = g.batch_no;
-        for (int v : evicted) {
+        for (int v : evicted) {     // also when no room could be made in the end: what was evicted on the way stays evicted
             const int32_t two = 2;
             CU_OK(cudaMemcpy(g.d_brief + v, &two, sizeof two, cudaMemcpyHostToDevice));
             CU_OK(cudaMemcpy(&g.d_models[v].alive, &two, sizeof two, cudaMemcpyHostToDevice));
         }
+        if (got == WeightCache::kNoRoom) return MT_ERR_OOM;
         block = g.arena + off;
     } else {
         CU_OK(cudaMalloc(&block, total));
