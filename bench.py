@@ -58,7 +58,7 @@ TRAFFIC = {
                                   "measured / 845.8 MB algorithmic), scaled by algorithmic bytes"},
     3: {"ratio": 1.007, "source": "profiles/grouped_gemm128_c3_reduced_ncu_full.md (250 tenants, 4096 requests: 272.1 MB "
                                   "measured / 270.0 MB algorithmic), scaled by algorithmic bytes"},
-    4: {"bytes": 722.9e6, "source": "profiles/grouped_conv3x3_pair_c4_full_ncu_full.md (full size, the four conv layers of a step in one launch)"},
+    4: {"bytes": 720.7e6, "source": "profiles/grouped_conv3x3_pair_c4_full_ncu_full.md (full size, the four conv layers of a step in one launch)"},
 }
 
 

@@ -115,7 +115,8 @@ mt_status mt_input_elems(int32_t* in_elems_out);
  *   stream    cudaStream_t (NULL = default stream)
  * Only enqueues work on `stream`: bucketing (histogram, exclusive scan, stable scatter, row gather), one
  * persistent grouped launch per layer (the last one writes its rows straight back in arrival order).  A batch
- * of at most 512 requests against dense layers at most 256 wide runs as ONE launch that does all of it.  No host<->device synchronisation happens unless the
+ * of at most 512 requests against dense layers at most 256 wide runs as ONE launch that does all of it; a conv
+ * batch of at most 512 requests is bucketed inside its first conv launch.  No host<->device synchronisation happens unless the
  * workspace must grow (n larger than any earlier call, or a wider model registered since): then the
  * call synchronises the device and reallocates first - make one call at the largest n before timing.
  * inputs must be 16-byte aligned.  n == 0 is a no-op.  Once the workspace exists and the models in use have been seen by

@@ -454,9 +454,10 @@ void launch_pretile_conv(const uint16_t* w, int C_out, int C_in, uint16_t* out, 
 
 // g[j][c] = (1 / HW) * sum over the image's strips of pool_partial[j][strip][c] (fixed order), rounded to bf16.
 __global__ void pool_finalize_kernel(const float* __restrict__ partial, int n, int strips, int C, float inv_hw,
-                                     uint16_t* __restrict__ out, int ld_out) {
+                                     uint16_t* __restrict__ out, int ld_out, unsigned* grid_bar) {
     pdl_launch_dependents();
     pdl_wait();
+    if (grid_bar && blockIdx.x == 0 && threadIdx.x < 8) grid_bar[threadIdx.x] = 0u;   // the conv launches are done with them
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= n * C) return;
     const int j = idx / C, c = idx - j * C;
@@ -466,8 +467,9 @@ __global__ void pool_finalize_kernel(const float* __restrict__ partial, int n, i
 }
 
 void launch_pool_finalize(const float* partial, int n, int strips, int C, int HW, uint16_t* out, int ld_out,
-                          cudaStream_t s) {
-    launch_pdl(pool_finalize_kernel, dim3((n * C + 255) / 256), dim3(256), 0, s, partial, n, strips, C, 1.0f / (float)HW, out, ld_out);
+                          unsigned* grid_bar, cudaStream_t s) {
+    launch_pdl(pool_finalize_kernel, dim3((n * C + 255) / 256), dim3(256), 0, s, partial, n, strips, C, 1.0f / (float)HW, out, ld_out,
+               grid_bar);
 }
 
 // Pool + narrow head in one launch: for every image, finish the global average pool (sum the strips' channel sums in
@@ -479,9 +481,10 @@ void launch_pool_finalize(const float* partial, int n, int strips, int C, int HW
 __global__ void __launch_bounds__(256)
 pool_head_kernel(const float* __restrict__ partial, int n, int strips, float inv_hw, const ModelDev* __restrict__ models,
                  int layer, const int32_t* __restrict__ offsets, int T, const int32_t* __restrict__ perm,
-                 float* __restrict__ out, int out_elems) {
+                 float* __restrict__ out, int out_elems, unsigned* grid_bar) {
     pdl_launch_dependents();
     pdl_wait();
+    if (grid_bar && blockIdx.x == 0 && threadIdx.x < 8) grid_bar[threadIdx.x] = 0u;   // the conv launches are done with them
     const int lane = threadIdx.x & 31;
     const int j = blockIdx.x * 8 + (threadIdx.x >> 5);          // bucketed row = image
     if (j >= n) return;
@@ -540,9 +543,10 @@ pool_head_kernel(const float* __restrict__ partial, int n, int strips, float inv
 }
 
 void launch_pool_head(const float* partial, int n, int strips, int HW, const ModelDev* models, int layer,
-                      const int32_t* offsets, int T, const int32_t* perm, float* out, int out_elems, cudaStream_t s) {
+                      const int32_t* offsets, int T, const int32_t* perm, float* out, int out_elems, unsigned* grid_bar,
+                      cudaStream_t s) {
     launch_pdl(pool_head_kernel, dim3((n + 7) / 8), dim3(256), 0, s, partial, n, strips, 1.0f / (float)HW, models, layer,
-               offsets, T, perm, out, out_elems);
+               offsets, T, perm, out, out_elems, grid_bar);
 }
 
 cudaError_t configure_grouped_conv() {

@@ -52,7 +52,12 @@ constexpr int kCpSlots = 8;                               // TMEM ring: 8 accumu
 constexpr int kCpBarBytes = 2048;
 constexpr int kCpRecords = 16;
 constexpr int kCpOutStageBytes = 8 * 2048;                // per epilogue warp: 32 pixels x 64 bytes
-constexpr int kCpSmemBytes = kConvPairWeightBytes + kCpRing * kCpBlockBytes + kCpGhostBytes + kCpOutStageBytes + kCpBarBytes + 1024;
+// the launch's own bucketing results (small batches): offsets (T + 2), unit prefixes (T + 1), perm (n)
+constexpr int kCpSortBytes = 4 * ((kConvSelfBucketMaxT + 2) + (kConvSelfBucketMaxT + 1) + kConvSelfBucketMaxN + 13);
+constexpr int kCpSmemBytes = kConvPairWeightBytes + kCpRing * kCpBlockBytes + kCpGhostBytes + kCpOutStageBytes + kCpBarBytes +
+                             kCpSortBytes + 1024;
+static_assert(kCpSmemBytes <= 227 * 1024, "shared memory of the pair conv executor");
+static_assert(16 * (kConvSelfBucketMaxT + 1) * 4 <= kCpRing * kCpBlockBytes, "chunk histograms borrow the block ring");
 
 __device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
                                                  uint32_t leader_bar) {
@@ -105,6 +110,9 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ ConvStackMaps maps, const Co
     float* s_pool = reinterpret_cast<float*>(bar_ptr + 1024);         // 8 warps x 32 channel sums (fused pooling)
     int* s_first = reinterpret_cast<int*>(bar_ptr + 320);             // the first unit's tenant: id, units, requests
     const uint16_t** s_first_w = reinterpret_cast<const uint16_t**>(bar_ptr + 352);   // ... and its weight block
+    int32_t* const s_off = reinterpret_cast<int32_t*>(bar_ptr + kCpBarBytes);        // own bucketing: offsets, T + 2
+    int32_t* const s_prefix = s_off + kConvSelfBucketMaxT + 2;                        // ... unit prefixes, T + 1
+    int32_t* const s_perm = s_prefix + kConvSelfBucketMaxT + 1;                       // ... perm, n
 
     if (!p.late_trigger) pdl_launch_dependents();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -140,8 +148,99 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ ConvStackMaps maps, const Co
     // layer of the same call (early_lookup) the wait comes a little later: the bucketing results read next are older
     // than that layer's own dependency, which it let pass before it allowed this launch to start.
     if (!p.early_lookup) pdl_wait();
+    // Where the bucketing results come from: the arrays a bucketing launch filled, or - small batches - this CTA's own
+    // stable counting sort of the ids (every CTA of the launch repeats it; it costs a few microseconds where a launch of
+    // its own costs about twenty, a twelfth of a step on 56 x 56 images).
+    const int32_t* tile_prefix = p.tile_prefix;
+    const int32_t* offsets = p.offsets;
+    const int32_t* perm_first = p.perm;              // the launch's first layer reads the caller's images through it
+    const bool self_bucket = p.ids != nullptr;
+    if (self_bucket) {
+        const int T = p.T, T1 = p.T + 1, n = p.n;
+        const int n_chunks = (n + 31) >> 5;           // chunk c = requests [32c, 32c + 32)
+        int32_t* s_chist = reinterpret_cast<int32_t*>(smem + kConvPairWeightBytes);   // [chunks][T1], in the idle block ring
+        for (int k = threadIdx.x; k < n_chunks * T1; k += kCpThreads) s_chist[k] = 0;
+        __syncthreads();
+        constexpr int kWarps = kCpThreads / 32;
+        constexpr int kMaxOwn = (kConvSelfBucketMaxN / 32 + kWarps - 1) / kWarps;     // chunks a warp may own
+        int own_b[kMaxOwn], own_rank[kMaxOwn];
+#pragma unroll
+        for (int q = 0; q < kMaxOwn; ++q) {
+            own_b[q] = -1; own_rank[q] = 0;
+            const int c = warp + kWarps * q;
+            const int i = c * 32 + lane;
+            if (c < n_chunks && i < n) {
+                const int id = p.ids[i];
+                const int alive = (id < 0 || id >= T) ? 0 : p.models[id].alive;     // 1 resident, 2 registered but evicted
+                const int b = alive == 1 ? id : T;
+                if (b == T && blockIdx.x == 0) {
+                    atomicCAS(&p.status[ST_CODE], MT_OK, alive == 2 ? MT_ERR_NOT_RESIDENT : MT_ERR_BAD_MODEL_ID);
+                    atomicMin(&p.status[ST_BAD_INDEX], i);
+                }
+                // rank among the chunk's requests of the same bucket, from the warp's match mask (the lanes with a
+                // request are lanes 0 .. n - 32c - 1)
+                const unsigned live = (n - c * 32 >= 32) ? 0xffffffffu : ((1u << (n - c * 32)) - 1u);
+                const unsigned peers = __match_any_sync(live, b);
+                const int rank_in_chunk = __popc(peers & ((1u << lane) - 1u));
+                if (rank_in_chunk == 0) s_chist[c * T1 + b] = __popc(peers);
+                own_b[q] = b; own_rank[q] = rank_in_chunk;
+            }
+        }
+        __syncthreads();
+        for (int t = threadIdx.x; t < T1; t += kCpThreads) {      // per bucket: exclusive prefix over the chunks; the count
+            int run = 0;
+            for (int c = 0; c < n_chunks; ++c) {
+                const int v = s_chist[c * T1 + t];
+                s_chist[c * T1 + t] = run;
+                run += v;
+            }
+            s_prefix[t] = run;                                    // (counts for now)
+        }
+        __syncthreads();
+        if (warp == 0) {                                          // offsets and unit prefixes over the buckets
+            const int per = (T1 + 31) >> 5;
+            const int lo = min(lane * per, T1), hi = min(lo + per, T1);
+            int sum = 0, usum = 0;
+            for (int t = lo; t < hi; ++t) { sum += s_prefix[t]; if (t < T) usum += ((s_prefix[t] + 1) >> 1) * p.strips_per_image; }
+            int incl = sum, uincl = usum;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int u = __shfl_up_sync(0xffffffffu, incl, d);
+                const int uu = __shfl_up_sync(0xffffffffu, uincl, d);
+                if (lane >= d) { incl += u; uincl += uu; }
+            }
+            int run = incl - sum, urun = uincl - usum;
+            for (int t = lo; t < hi; ++t) {
+                const int cnt = s_prefix[t];
+                if (blockIdx.x == 0) p.counts_out[t] = cnt;
+                s_off[t] = run; run += cnt;
+                if (t < T) { s_prefix[t] = urun; urun += ((cnt + 1) >> 1) * p.strips_per_image; }
+            }
+            __syncwarp();
+            if (lane == 31) { s_off[T1] = incl; s_prefix[T] = uincl; }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < kMaxOwn; ++q) {
+            const int c = warp + kWarps * q;
+            const int i = c * 32 + lane;
+            if (own_b[q] >= 0) {
+                const int pos = s_off[own_b[q]] + s_chist[c * T1 + own_b[q]] + own_rank[q];
+                s_perm[pos] = i;
+                if (blockIdx.x == 0) { p.perm_out[pos] = i; p.inv_out[i] = pos; }
+            }
+        }
+        if (blockIdx.x == 0) {        // for the launches that follow (more conv layers, the pool and the head)
+            for (int t = threadIdx.x; t <= T1; t += kCpThreads) p.offsets_out[t] = s_off[t];
+            for (int k = threadIdx.x; k < p.prefix_rows * T1; k += kCpThreads) p.prefix_out[k] = s_prefix[k % T1];
+        }
+        __syncthreads();              // the block ring is free again; s_off, s_prefix and s_perm are complete
+        tile_prefix = s_prefix;
+        offsets = s_off;
+        perm_first = s_perm;
+    }
     // contiguous range of pair-strips for this cluster: unit = (tenant, pair of images, strip of 2 tiles)
-    const int total = p.tile_prefix[p.T];
+    const int total = tile_prefix[p.T];
     const int n_pairs = gridDim.x >> 1, pair_id = blockIdx.x >> 1;
     int s_begin = (int)(((long long)total * pair_id) / n_pairs);
     int s_end = (int)(((long long)total * (pair_id + 1)) / n_pairs);
@@ -162,7 +261,7 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ ConvStackMaps maps, const Co
             const int per = (p.T + 31) >> 5;
             const int lo = min(lane * per, p.T), hi = min(lo + per, p.T);
             int mine = 0;
-            for (int t = lo; t < hi; ++t) mine += (p.tile_prefix[t + 1] > p.tile_prefix[t]) ? 1 : 0;
+            for (int t = lo; t < hi; ++t) mine += (tile_prefix[t + 1] > tile_prefix[t]) ? 1 : 0;
             int incl = mine;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
@@ -171,9 +270,9 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ ConvStackMaps maps, const Co
             }
             int before = incl - mine;                                 // tenants with units in front of this lane's share
             for (int t = lo; t < hi; ++t) {
-                const int first = p.tile_prefix[t];
+                const int first = tile_prefix[t];
                 s_cost[t] = first + p.border_units * before;
-                before += (p.tile_prefix[t + 1] > first) ? 1 : 0;
+                before += (tile_prefix[t + 1] > first) ? 1 : 0;
             }
             if (lane == 31) s_cost[p.T] = total + p.border_units * max(before - 1, 0);   // total cost (the first tenant has no border)
         }
@@ -189,7 +288,7 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ ConvStackMaps maps, const Co
                     const int mid = (lo + hi) >> 1;
                     if ((long long)s_cost[mid] - p.border_units <= c) lo = mid; else hi = mid;
                 }
-                const int first = p.tile_prefix[lo], units = p.tile_prefix[lo + 1] - first;
+                const int first = tile_prefix[lo], units = tile_prefix[lo + 1] - first;
                 const long long into = c - s_cost[lo];
                 return first + (int)min((long long)units, max(into, 0LL));
             };
@@ -207,8 +306,8 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ ConvStackMaps maps, const Co
     // this sits between the previous layer's end and the first MMA.
     if (s_begin < s_end) {
         for (int i = threadIdx.x; i < p.T; i += blockDim.x) {
-            const int lo = p.tile_prefix[i], hi = p.tile_prefix[i + 1];
-            const int seg = p.offsets[i], seg_hi = p.offsets[i + 1];
+            const int lo = tile_prefix[i], hi = tile_prefix[i + 1];
+            const int seg = offsets[i], seg_hi = offsets[i + 1];
             const uint16_t* w = p.models[i].layer[p.layer].w;
             if (lo <= s_begin && s_begin < hi) {
                 s_first[0] = i; s_first[1] = lo; s_first[2] = hi; s_first[3] = seg; s_first[4] = seg_hi - seg;
@@ -236,10 +335,10 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ ConvStackMaps maps, const Co
             int lo = 0, hi = p.T;
             while (hi - lo > 1) {
                 const int mid = (lo + hi) >> 1;
-                if (p.tile_prefix[mid] <= s) lo = mid; else hi = mid;
+                if (tile_prefix[mid] <= s) lo = mid; else hi = mid;
             }
-            cur_t = lo; cur_lo = p.tile_prefix[lo]; cur_hi = p.tile_prefix[lo + 1];
-            cur_seg = p.offsets[lo]; cur_n = p.offsets[lo + 1] - cur_seg;
+            cur_t = lo; cur_lo = tile_prefix[lo]; cur_hi = tile_prefix[lo + 1];
+            cur_seg = offsets[lo]; cur_n = offsets[lo + 1] - cur_seg;
         }
         PairStrip c;
         const int local = s - cur_lo;
@@ -296,7 +395,7 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ ConvStackMaps maps, const Co
             const int layer = p.layer + k;
             const CUtensorMap* const tmap_x = &maps.x2[k];
             const CUtensorMap* const tmap_x1 = &maps.x1[k];
-            const int32_t* const perm = (k == 0) ? p.perm : nullptr;
+            const int32_t* const perm = (k == 0) ? perm_first : nullptr;
             if (k > 0) w_tenant = -1;   // same tenants, other weights
             {
             // (indentation kept from the single-layer form)
@@ -514,7 +613,7 @@ grouped_conv3x3_pair_kernel(const __grid_constant__ ConvStackMaps maps, const Co
         // the extra instructions, the rest the loads.
         // Tiles alternate between the two register buffers, so a strip must have an even number of tiles (it has two).
         const uint16_t* const skip_k = kSkip ? p.skip[k] : nullptr;
-        const int32_t* const skip_perm_k = kSkip ? p.skip_perm[k] : nullptr;
+        const int32_t* const skip_perm_k = (kSkip && p.skip_perm[k]) ? (self_bucket ? s_perm : p.skip_perm[k]) : nullptr;
         const bool skip_wide = (reinterpret_cast<uintptr_t>(skip_k) & 31) == 0;      // 32-byte loads need that alignment
         uint4 sk_a[4], sk_b[4];                     // values on their way: even / odd tile of a strip
         bool have_a = false, have_b = false;        // warp-uniform: the buffer holds (or will hold) values to add

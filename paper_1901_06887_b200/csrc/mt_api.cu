@@ -153,7 +153,8 @@ struct Ctx {
 
     // switches for tests and A/B timing: read from the environment once, at mt_init (MT_FUSED, MT_PAIR, MT_CONV_PAIR,
     // MT_POOL_HEAD; "0" turns the path off), changed afterwards only through mt_debug_set_option
-    bool opt_fused = true, opt_pair = true, opt_conv_pair = true, opt_pool_head = true, opt_conv_stack = true, opt_conv_balance = true;
+    bool opt_fused = true, opt_pair = true, opt_conv_pair = true, opt_pool_head = true, opt_conv_stack = true, opt_conv_balance = true,
+         opt_conv_self_bucket = true;
     int opt_gather = 1;                  // 0 never, 1 small batches, 2 always
 
     // tensor maps over the caller's images (first conv layer), kept while pointer and batch size stay the same
@@ -279,6 +280,7 @@ mt_status do_init(int device, int max_models, int /*max_batch*/) {
     g.opt_conv_stack = env_on("MT_CONV_STACK");
     g.opt_async_register = env_on("MT_ASYNC_REGISTER");
     g.opt_conv_balance = env_on("MT_CONV_BALANCE");
+    g.opt_conv_self_bucket = env_on("MT_CONV_SELF_BUCKET");
     { const char* v = getenv("MT_PERM_GATHER"); g.opt_gather = (v && v[0] >= '0' && v[0] <= '2') ? v[0] - '0' : 1; }
     g.init = true;
     return MT_OK;
@@ -823,9 +825,15 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
     // requests moving each row once is cheaper (config 3: +57 us, config 5: +10 ms with gathers; at 512 requests the
     // two are level).  "perm_gather" = 2
     // forces the gather for any batch size (tests).
+    // Small conv batches on the CTA-pair executor, when pool + head end the pass (so that no dense work items are
+    // needed): no bucketing launch; the first conv launch sorts the ids itself, in every CTA (MT_CONV_SELF_BUCKET=0:
+    // the bucketing launch as for larger batches).
+    bool convs_then_pool = conv_pair && pool_head;
+    for (int l = 0; l + 2 < L; ++l) convs_then_pool = convs_then_pool && g.family[l].kind == MT_CONV3X3;
+    const bool self_bucket = convs_then_pool && g.opt_conv_self_bucket && n <= kConvSelfBucketMaxN && g.T <= kConvSelfBucketMaxT;
     const bool perm_gather = f0.kind == MT_DENSE && (g.opt_gather == 2 || (g.opt_gather == 1 && n <= 256));
     const bool rows_in_scatter = f0.kind == MT_DENSE && !perm_gather && n > 512 && (size_t)n * g.in_elems * 2 <= ((size_t)64 << 20);
-    {
+    if (!self_bucket) {
         Timer t(K_BUCKET, s);
         BucketArgs a;
         a.ids = ids; a.n = n; a.T = g.T; a.models = g.d_models; a.n_layers = L; a.rows_per_unit = tiles_per_image;
@@ -933,6 +941,11 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
                     a.skip[k] = skip_of(l + k);
                     a.skip_perm[k] = (l + k == 1) ? g.d_perm : nullptr;
                 }
+                if (self_bucket && l == 0) {
+                    a.ids = ids; a.n = n;
+                    a.counts_out = g.d_counts; a.offsets_out = g.d_offsets; a.perm_out = g.d_perm; a.inv_out = g.d_inv;
+                    a.prefix_out = g.d_tile_prefix; a.prefix_rows = L - 2;      // one row per conv layer
+                }
                 a.n_stack = n_stack;
                 a.border_units = g.opt_conv_balance ? 2 : 0;
                 a.grid_bar = g.d_grid_bar + (n_conv_launch++ & 7);
@@ -953,14 +966,14 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             // pool + narrow last dense layer in one launch (the loop ends here: the head is done)
             Timer t(K_POOL, s);
             launch_pool_head(g.d_pool_partial, n, g.conv.strips_per_image, f.h * f.w, g.d_models, L - 1, g.d_offsets, g.T,
-                             g.d_perm, (float*)outputs, g.out_elems, s);
+                             g.d_perm, (float*)outputs, g.out_elems, g.d_grid_bar, s);
             break;
         } else {
             Timer t(K_POOL, s);
             // a pool always follows a conv (checked at registration), whose epilogue already reduced every strip
             // to channel sums
             launch_pool_finalize(g.d_pool_partial, n, g.conv.strips_per_image, f.in_ch, f.h * f.w,
-                                 (uint16_t*)g.act[l + 1], g.act_ld[l + 1], s);
+                                 (uint16_t*)g.act[l + 1], g.act_ld[l + 1], g.d_grid_bar, s);
         }
     }
     Timer::close_group(s);
@@ -1708,6 +1721,7 @@ mt_status mt_debug_set_option(const char* name, int32_t value) {
     else if (!strcmp(name, "conv_stack")) g.opt_conv_stack = on;
     else if (!strcmp(name, "async_register")) g.opt_async_register = on;
     else if (!strcmp(name, "conv_balance")) g.opt_conv_balance = on;
+    else if (!strcmp(name, "conv_self_bucket")) g.opt_conv_self_bucket = on;
     else if (!strcmp(name, "perm_gather")) g.opt_gather = value < 0 ? 0 : (value > 2 ? 2 : value);
     else return MT_ERR_INVALID_ARG;
     return MT_OK;

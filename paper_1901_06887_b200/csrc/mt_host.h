@@ -180,8 +180,22 @@ struct ConvArgs {
     // index = skip_perm[j]; else it is in bucketed order.
     const uint16_t* skip[4] = {nullptr, nullptr, nullptr, nullptr};
     const int32_t* skip_perm[4] = {nullptr, nullptr, nullptr, nullptr};
+    // CTA-pair executor, small batches (kConvSelfBucketMaxN requests, kConvSelfBucketMaxT tenants at most): ids non-null
+    // = no bucketing launch ran for this call; every CTA repeats the stable counting sort of the n ids in shared memory
+    // (as the one-launch MLP path does) and takes offsets, unit prefixes and perm from there; CTA 0 also writes them,
+    // counts and inv to the arrays below for the launches that follow (prefix_rows rows of T + 1 unit prefixes).
+    const int32_t* ids = nullptr;
+    int n = 0;
+    int32_t* counts_out = nullptr;
+    int32_t* offsets_out = nullptr;
+    int32_t* perm_out = nullptr;
+    int32_t* inv_out = nullptr;
+    int32_t* prefix_out = nullptr;
+    int prefix_rows = 0;
     int32_t* status;
 };
+constexpr int kConvSelfBucketMaxN = 512;
+constexpr int kConvSelfBucketMaxT = 512;
 
 cudaError_t configure_grouped_conv();
 void launch_grouped_conv(const CUtensorMap& tmap_x, const ConvArgs& a, int smem_bytes, int sm_count, cudaStream_t s);
@@ -208,12 +222,15 @@ struct ConvStackMaps {
 cudaError_t launch_grouped_conv_pair(const ConvStackMaps& maps, const ConvArgs& a, int sm_count, cudaStream_t s);
 
 // Second half of the fused pooling: sums the per-strip channel sums of each image and divides by H*W.
+// grid_bar (may be null): the eight barrier counters of the call's stacked conv launches, set back to zero here - a
+// pool always follows the last conv layer, so the counters are zero whenever a call starts.
 void launch_pool_finalize(const float* partial, int n, int strips, int C, int HW, uint16_t* out, int ld_out,
-                          cudaStream_t s);
+                          unsigned* grid_bar, cudaStream_t s);
 
 // The same fused with the model's last layer when that is a dense layer from the pooled 64 channels to at most 64
 // outputs: pooled values (rounded to bf16) x head weights, bias, optional ReLU, fp32 rows written to arrival order.
 void launch_pool_head(const float* partial, int n, int strips, int HW, const ModelDev* models, int layer,
-                      const int32_t* offsets, int T, const int32_t* perm, float* out, int out_elems, cudaStream_t s);
+                      const int32_t* offsets, int T, const int32_t* perm, float* out, int out_elems, unsigned* grid_bar,
+                      cudaStream_t s);
 
 }  // namespace mt

@@ -28,13 +28,17 @@ def small_batch_path(request, monkeypatch):
     return request.param
 
 
-@pytest.fixture(params=["pair", "pair_layerwise", "single"])
+@pytest.fixture(params=["pair", "pair_layerwise", "pair_bucketing_launch", "single"])
 def conv_path(request, monkeypatch):
     """Conv layers whose padded row length is 64 pixels run on CTA pairs (two images of a tenant per cluster), consecutive
-    conv layers as ONE launch with grid-wide barriers in between; MT_CONV_STACK=0 gives every conv layer a launch of its
-    own and MT_CONV_PAIR=0 sends them to the one-CTA executor.  Tests that take this fixture run once on each."""
+    conv layers as ONE launch with grid-wide barriers in between, and batches of at most 512 requests are bucketed by
+    that launch itself; MT_CONV_STACK=0 gives every conv layer a launch of its own, MT_CONV_SELF_BUCKET=0 keeps the
+    bucketing launch and MT_CONV_PAIR=0 sends the layers to the one-CTA executor.  Tests that take this fixture run once
+    on each."""
     if request.param == "single":
         monkeypatch.setenv("MT_CONV_PAIR", "0")
     elif request.param == "pair_layerwise":
         monkeypatch.setenv("MT_CONV_STACK", "0")
+    elif request.param == "pair_bucketing_launch":
+        monkeypatch.setenv("MT_CONV_SELF_BUCKET", "0")
     return request.param

@@ -205,3 +205,41 @@ def test_work_item_order_follows_cost_after_release_and_reregistration():
     assert harness.scaled_error(got[live], oracle.forward(models, ids[live], x[live])).max() <= TOL
     assert mt.mt_register_model(models[3]) == 3
     run_and_check(models, ids, x, register=False)
+
+
+def test_small_conv_batches_are_bucketed_by_the_conv_launch_itself():
+    # at most 512 requests on the CTA-pair conv executor, pool + head at the end: no bucketing launch - every CTA of the
+    # first conv launch repeats the stable counting sort in shared memory and CTA 0 publishes it for the launches behind
+    # it (a second conv launch when there are more than four conv layers, the pool + head launch).  Same bits as with
+    # the bucketing launch; rejected ids come back as NaN rows with the status of the smallest offending index.
+    for n_conv, n, T, h, w in ((4, 37, 5, 9, 40), (6, 50, 3, 6, 44), (2, 512, 16, 3, 33)):
+        wl = synth.make_workload(4, n=n, n_tenants=T, h=h, w=w, n_conv=n_conv)
+        ids = wl.model_ids.copy()
+        ids[[3, n - 2]] = [T + 4, -1]                               # never issued / negative
+        fresh(max_models=max(64, T))
+        harness.register_models(wl.models)
+        want_launches = (2 if n_conv <= 4 else 3)                   # conv stack(s) + pool-and-head
+        got, k = launches_of(lambda: harness.run_batch(ids, wl.inputs, 10))
+        assert k == want_launches
+        assert mt.mt_get_async_status() == (2, 3)
+        good = (ids >= 0) & (ids < T)
+        assert np.isnan(got[~good]).all() and np.isfinite(got[good]).all()
+        counts, offsets, perm, inv = mt.mt_debug_last_bucketing(n)
+        oc, oo, op, oi = oracle.bucket(np.where(good, ids, T).astype(np.int32), T + 1)
+        assert np.array_equal(counts[:T], oc[:T]) and np.array_equal(offsets[:T + 1], oo[:T + 1]) and offsets[T + 1] == n
+        assert np.array_equal(perm, op) and np.array_equal(inv, oi)
+        ref = oracle.forward(wl.models, ids[good], wl.inputs[good])
+        assert harness.scaled_error(got[good], ref).max() <= TOL
+        mt.mt_debug_set_option("conv_self_bucket", 0)
+        try:
+            other, k2 = launches_of(lambda: harness.run_batch(ids, wl.inputs, 10))
+        finally:
+            mt.mt_debug_set_option("conv_self_bucket", 1)
+        assert k2 == want_launches + 1 and mt.mt_get_async_status() == (2, 3)
+        assert np.array_equal(np.nan_to_num(got, nan=-1.0), np.nan_to_num(other, nan=-1.0))
+        # a larger batch on the same context takes the bucketing launch again, then a small one the short way
+        big = synth.make_requests(4, wl.models, n=600, salt=7)
+        run_and_check(wl.models, big[0], big[1], register=False)
+        small = synth.make_requests(4, wl.models, n=11, salt=8)
+        _, k3 = launches_of(lambda: run_and_check(wl.models, small[0], small[1], register=False))
+        assert k3 == want_launches
