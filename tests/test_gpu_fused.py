@@ -212,7 +212,7 @@ def test_small_conv_batches_are_bucketed_by_the_conv_launch_itself():
     # first conv launch repeats the stable counting sort in shared memory and CTA 0 publishes it for the launches behind
     # it (a second conv launch when there are more than four conv layers, the pool + head launch).  Same bits as with
     # the bucketing launch; rejected ids come back as NaN rows with the status of the smallest offending index.
-    for n_conv, n, T, h, w in ((4, 37, 5, 9, 40), (6, 50, 3, 6, 44), (2, 512, 16, 3, 33)):
+    for n_conv, n, T, h, w in ((4, 37, 5, 9, 40), (6, 50, 3, 6, 44), (2, 512, 16, 3, 33), (2, 500, 300, 2, 33)):
         wl = synth.make_workload(4, n=n, n_tenants=T, h=h, w=w, n_conv=n_conv)
         ids = wl.model_ids.copy()
         ids[[3, n - 2]] = [T + 4, -1]                               # never issued / negative
@@ -243,3 +243,18 @@ def test_small_conv_batches_are_bucketed_by_the_conv_launch_itself():
         small = synth.make_requests(4, wl.models, n=11, salt=8)
         _, k3 = launches_of(lambda: run_and_check(wl.models, small[0], small[1], register=False))
         assert k3 == want_launches
+
+
+def test_conv_context_with_more_id_slots_than_the_conv_launch_sorts_keeps_the_bucketing_launch():
+    # the in-launch sort holds its tables for at most 512 id slots: with 513 registered models the batch is bucketed
+    # by a launch of its own again, same results against the oracle
+    T, h, w = 513, 2, 33
+    wl = synth.make_workload(4, n=40, n_tenants=T, h=h, w=w, n_conv=2)
+    fresh(max_models=T)
+    harness.register_models(wl.models)
+    (got, _), k = launches_of(lambda: run_and_check(wl.models, wl.model_ids, wl.inputs, register=False))
+    assert k == 3
+    mt.mt_release(T - 1)                                           # id slots stay 513: still the bucketing launch
+    keep = wl.model_ids != T - 1
+    _, k = launches_of(lambda: run_and_check(wl.models, wl.model_ids[keep], wl.inputs[keep], register=False))
+    assert k == 3
