@@ -79,7 +79,7 @@ mt_status mt_init(int32_t device, int32_t max_models, int32_t max_batch);
 /* Release every model, workspace and the context.  Synchronises the device. */
 mt_status mt_shutdown(void);
 
-/* "Upload your model" (Sec. 1.2 / Sec. 3): validate the layer list, copy the weights to the device in
+/* A tenant hands its model to the service (Sec. 1.2 / Sec. 3): validate the layer list, copy the weights to the device in
  * the executor's tiled layout and return a small dense id (lowest free slot first) in *model_id_out.
  * All models hosted by one context form one family: the same layer kinds index by index.  MLPs (dense layers only)
  * may differ in depth and in every width - input, hidden and output; conv families keep one depth, geometry, input and
@@ -107,7 +107,7 @@ mt_status mt_output_elems(int32_t* out_elems_out);
  * last held none (0 if none is registered). */
 mt_status mt_input_elems(int32_t* in_elems_out);
 
-/* predict(model, input) for a whole mixed batch (Sec. 3: a worker multiplexes requests across models).
+/* One inference per request for a whole mixed batch (Sec. 3: a worker multiplexes requests across models).
  *   inputs    device, bf16, [n][in_elems] row-major (NHWC per request for conv), arrival order (in_elems: see
  *             mt_input_elems)
  *   model_ids device, int32 [n]; request i is evaluated by model model_ids[i]
