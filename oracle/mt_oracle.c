@@ -8,8 +8,9 @@
  * What it computes, and where the paper says so:
  *   - A DNN is a stateless, deterministic function of (weights, input)
  *     (Sec. 1.1): orc_forward_one depends on nothing but its arguments.
- *   - A DNN is evaluated by "performing the operation of each layer in turn"
- *     (Sec. 1.1): the loop over layers below, no fusion, no reordering.
+ *   - A DNN is evaluated one layer after the other, each layer's operation
+ *     applied to the previous layer's output (Sec. 1.1): the loop over layers
+ *     below, no fusion, no reordering.
  *   - A fully-connected layer multiplies the previous layer's output by a
  *     tensor of learned constants (Sec. 1.1).  Reading used here (the paper
  *     gives no orientation or bias): z = W a + b, W stored [out][in].
