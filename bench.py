@@ -430,6 +430,25 @@ def measure_config(cfg, args, ctx):
     breakdown = mt.mt_get_kernel_times()
     units, ms = aggregate(n * steps, local_ms, world)
 
+    # Workload 4's batch is bucketed inside its conv launch, so the timed conv kernel contains that sort.  For the conv
+    # layers alone: the same steps once more with the bucketing as a launch of its own (right after the blocks above,
+    # i.e. in the power-capped regime).
+    alone = None
+    if cfg == 4 and world == 1 and not args.profile:
+        mt.mt_debug_set_option("conv_self_bucket", 0)
+        for i in range(10):
+            step(i)
+        torch.cuda.synchronize()
+        mt.mt_set_kernel_timing(3)
+        e0.record(stream)
+        for i in range(steps):
+            step(i)
+        mt.mt_set_kernel_timing(0)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        alone = (e0.elapsed_time(e1) / steps, mt.mt_get_kernel_times())
+        mt.mt_debug_set_option("conv_self_bucket", 1)
+
     if args.profile:
         mt.mt_shutdown()
         return {"profile_run": True, "ms_per_step": ms / steps, "kernels": {nm: t / max(c, 1) for nm, t, c in breakdown}}
@@ -530,6 +549,14 @@ def measure_config(cfg, args, ctx):
 
     line["whole_pass_roofline"] = whole_pass(line["ms_per_step"], long_first)
     line["roofline"] = roof
+    if alone is not None:
+        r2 = dominant_roofline(wl, dom_ms(alone[1]), peaks, peaks_kind, cfg, True)
+        line["conv_layers_alone"] = {
+            "note": "the same steps with the bucketing as a launch of its own (conv_self_bucket = 0), measured after the "
+                    "repeated blocks (power-capped regime): the conv launch then holds the conv layers only",
+            "ms_per_step": alone[0], "kernel_ms_per_step": r2["kernel_ms_per_step"], "achieved": r2["achieved"],
+            "unit": r2["unit"], "frac_of_burst_peak": r2.get("frac_of_burst_peak"),
+            "frac_of_sustained_peak": r2.get("frac_of_sustained_peak")}
     if len(blocks) > 1 or blocks[0][0] >= SUSTAIN_MS:
         # the later half of the blocks: the GPU has been busy for at least a second by then
         tail = list(range(len(blocks) // 2, len(blocks)))
