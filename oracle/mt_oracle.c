@@ -26,6 +26,8 @@
  * the textbook definitions:
  *   conv3x3: cross-correlation, stride 1, zero padding 1, NHWC activations,
  *            weights [out][ky][kx][in]; tap (ky,kx) reads pixel (y+ky-1, x+kx-1)
+ *   conv1x1: the fully-connected layer applied at every pixel, NHWC,
+ *            weights [out][in]: z[p][o] = b[o] + sum_c W[o][c] a[p][c]
  *   global average pool: mean over all H*W positions, per channel
  *   ReLU: max(z, 0)
  *   identity shortcut (the residual block of the network the paper uses as
@@ -41,7 +43,9 @@
  * identity and zero weights (closed forms), a separately written triple-loop
  * matmul, numpy float64 matmul, brute-force padded-copy conv, scipy
  * correlate2d, shifted-tap and all-ones closed forms, numpy stable argsort and
- * an O(n*T) brute-force bucketing; the shortcut by a zero-weight block
+ * an O(n*T) brute-force bucketing; conv1x1 by the dense layer applied pixel
+ * by pixel and by a conv3x3 whose only non-zero tap is the centre one; the
+ * shortcut by a zero-weight block
  * (a closed form of the block's input alone) and a scipy restatement.
  * No function here is left unpinned.
  */
@@ -52,7 +56,7 @@
 #include <omp.h>
 #endif
 
-enum { ORC_DENSE = 0, ORC_CONV3X3 = 1, ORC_GLOBAL_AVG_POOL = 2 };
+enum { ORC_DENSE = 0, ORC_CONV3X3 = 1, ORC_GLOBAL_AVG_POOL = 2, ORC_CONV1X1 = 3 };
 
 typedef struct {
     int32_t kind;
@@ -79,7 +83,7 @@ static int64_t layer_in_elems(const orc_layer* l)
 
 static int64_t layer_out_elems(const orc_layer* l)
 {
-    return l->kind == ORC_CONV3X3 ? (int64_t)l->out_ch * l->h * l->w : (int64_t)l->out_ch;
+    return (l->kind == ORC_CONV3X3 || l->kind == ORC_CONV1X1) ? (int64_t)l->out_ch * l->h * l->w : (int64_t)l->out_ch;
 }
 
 /* Stable counting sort of request indices by model id.
@@ -143,6 +147,17 @@ static void layer_apply(const orc_layer* l, const double* a, const double* skip,
                     }
                     z[((int64_t)y * W + x) * O + o] = acc;
                 }
+    } else if (l->kind == ORC_CONV1X1) {
+        const int64_t P = (int64_t)l->h * l->w;
+        for (int64_t p = 0; p < P; ++p)
+            for (int32_t o = 0; o < l->out_ch; ++o) {
+                double acc = l->bias ? (double)l->bias[o] : 0.0;
+                const uint16_t* wrow = l->weight + (int64_t)o * l->in_ch;
+                const double* av = a + p * l->in_ch;
+                for (int32_t c = 0; c < l->in_ch; ++c)
+                    acc += bf16_to_double(wrow[c]) * av[c];
+                z[p * l->out_ch + o] = acc;
+            }
     } else { /* global average pool */
         const int64_t P = (int64_t)l->h * l->w;
         for (int32_t c = 0; c < l->in_ch; ++c) {

@@ -85,7 +85,7 @@ def _pack_model(layers: Sequence, keep: list):
 
 
 def _out_elems(l) -> int:
-    return int(l.out_ch) * (int(l.h) * int(l.w) if int(l.kind) == 1 else 1)
+    return int(l.out_ch) * (int(l.h) * int(l.w) if int(l.kind) in (1, 3) else 1)      # conv3x3 and conv1x1 keep the image
 
 
 def bucket(model_ids: np.ndarray, n_tenants: int):

@@ -33,6 +33,7 @@ BASE_SEED = 190106887
 DENSE = 0
 CONV3X3 = 1
 GLOBAL_AVG_POOL = 2
+CONV1X1 = 3
 
 _PURPOSE = {"widths": 1, "weights": 2, "biases": 3, "ids": 4, "rankperm": 5, "inputs": 6}
 
@@ -75,7 +76,7 @@ class Layer:
 
     @property
     def out_elems(self) -> int:
-        return self.out_ch * (self.h * self.w if self.kind == CONV3X3 else 1)
+        return self.out_ch * (self.h * self.w if self.kind in (CONV3X3, CONV1X1) else 1)
 
 
 @dataclass
@@ -140,6 +141,23 @@ def make_conv_stack(config: int, tenant: int, n_conv: int, ch: int, h: int, w: i
         kind=DENSE, in_ch=ch, out_ch=n_out, relu=0,
         weight=_he_uniform_bf16(stream(config, "weights", tenant, n_conv + 1), (n_out, ch), ch),
         bias=_bias(stream(config, "biases", tenant, n_conv + 1), n_out)))
+    return layers
+
+
+def make_pointwise_stack(config: int, tenant: int, mid_ch: int, h: int, w: int, n_out: int) -> List[Layer]:
+    """conv3x3 64->64 -> conv1x1 64->mid_ch -> conv1x1 mid_ch->64 -> conv3x3 64->64 -> global avg pool -> dense 64->n_out,
+    ReLU after every conv: 3x3 layers around a pair of pointwise ones."""
+    def conv(li, kind, cin, cout):
+        taps = 9 if kind == CONV3X3 else 1
+        shape = (cout, 3, 3, cin) if kind == CONV3X3 else (cout, cin)
+        return Layer(kind=kind, in_ch=cin, out_ch=cout, h=h, w=w, relu=1,
+                     weight=_he_uniform_bf16(stream(config, "weights", tenant, li), shape, taps * cin),
+                     bias=_bias(stream(config, "biases", tenant, li), cout))
+    layers = [conv(0, CONV3X3, 64, 64), conv(1, CONV1X1, 64, mid_ch), conv(2, CONV1X1, mid_ch, 64), conv(3, CONV3X3, 64, 64)]
+    layers.append(Layer(kind=GLOBAL_AVG_POOL, in_ch=64, out_ch=64, h=h, w=w))
+    layers.append(Layer(kind=DENSE, in_ch=64, out_ch=n_out, relu=0,
+                        weight=_he_uniform_bf16(stream(config, "weights", tenant, 5), (n_out, 64), 64),
+                        bias=_bias(stream(config, "biases", tenant, 5), n_out)))
     return layers
 
 
@@ -227,6 +245,8 @@ def layer_flops(layer: Layer) -> int:
         return 2 * layer.in_ch * layer.out_ch
     if layer.kind == CONV3X3:
         return 2 * 9 * layer.in_ch * layer.out_ch * layer.h * layer.w
+    if layer.kind == CONV1X1:
+        return 2 * layer.in_ch * layer.out_ch * layer.h * layer.w
     return 0
 
 

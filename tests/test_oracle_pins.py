@@ -225,6 +225,34 @@ def test_conv_via_im2col_and_triple_loop(oracle_mod):
     assert np.allclose(out.reshape(H * W, O), ref, rtol=1e-12, atol=1e-12)
 
 
+# ----------------------------------------------------------------- pointwise conv
+def test_conv1x1_is_the_dense_layer_at_every_pixel_and_the_centre_tap_of_a_3x3(oracle_mod):
+    rng = np.random.default_rng(31)
+    H, W, C, O = 3, 5, 4, 6            # H != W, C != O
+    wb = rand_bits(rng, (O, C), 0.5); b = rng.standard_normal(O).astype(np.float32)
+    xb = rand_bits(rng, (H * W, C))
+    pw = Layer(synth.CONV1X1, C, O, h=H, w=W, relu=1, weight=wb, bias=b)
+    out = oracle_mod.forward_one([pw], xb.reshape(-1)).reshape(H * W, O)
+    # (a) the dense layer, one pixel at a time
+    dense = Layer(DENSE, C, O, relu=1, weight=wb, bias=b)
+    for p in range(H * W):
+        assert np.array_equal(out[p], oracle_mod.forward_one([dense], xb[p]))
+    # (b) numpy in float64
+    assert np.allclose(out, np.maximum(f64(xb) @ f64(wb).T + b, 0.0), rtol=1e-12, atol=1e-12)
+    # (c) a 3x3 conv whose only non-zero tap is the centre one
+    w3 = np.zeros((O, 3, 3, C), np.float32); w3[:, 1, 1, :] = synth.bf16_bits_to_f32(wb).reshape(O, C)
+    c3 = Layer(CONV3X3, C, O, h=H, w=W, relu=1, weight=synth.f32_to_bf16_bits(w3), bias=b)
+    assert np.array_equal(out.reshape(-1), oracle_mod.forward_one([c3], xb.reshape(-1)))
+    # and inside a chain: 3x3 -> 1x1 -> 1x1 -> pool -> dense against numpy
+    l0 = Layer(CONV3X3, C, C, h=H, w=W, relu=1, weight=rand_bits(rng, (C, 3, 3, C), 0.5), bias=None)
+    l2 = Layer(synth.CONV1X1, O, 2, h=H, w=W, relu=0, weight=rand_bits(rng, (2, O)), bias=None)
+    head = Layer(DENSE, 2, 3, relu=0, weight=rand_bits(rng, (3, 2)), bias=rng.standard_normal(3).astype(np.float32))
+    full = oracle_mod.forward_one([l0, pw, l2, Layer(GLOBAL_AVG_POOL, 2, 2, h=H, w=W), head], xb.reshape(-1))
+    a = np.maximum(brute_conv(f64(xb).reshape(H, W, C), f64(l0.weight), np.zeros(C)), 0.0).reshape(H * W, C)
+    a = np.maximum(a @ f64(wb).T + b, 0.0) @ f64(l2.weight).T
+    assert np.allclose(full, f64(head.weight) @ a.mean(axis=0) + head.bias, rtol=1e-10, atol=1e-10)
+
+
 # ----------------------------------------------------------------- identity shortcut (two-layer residual block)
 def test_shortcut_with_zero_weights_is_a_closed_form_of_the_block_input(oracle_mod):
     # block: a1 = relu(conv0(a0)); a2 = relu(conv1(a1) + b1 + a0).  With conv1's weights zero, a2 = relu(b1 + a0): it
