@@ -43,7 +43,7 @@ typedef enum {
     MT_ERR_NOT_RESIDENT = 10  /* (async) a request names a registered model whose weights are not on the device now */
 } mt_status;
 
-typedef enum { MT_DENSE = 0, MT_CONV3X3 = 1, MT_GLOBAL_AVG_POOL = 2 } mt_layer_kind;
+typedef enum { MT_DENSE = 0, MT_CONV3X3 = 1, MT_GLOBAL_AVG_POOL = 2, MT_CONV1X1 = 3 } mt_layer_kind;
 
 #define MT_MAX_LAYERS 8
 
@@ -52,6 +52,7 @@ typedef enum { MT_DENSE = 0, MT_CONV3X3 = 1, MT_GLOBAL_AVG_POOL = 2 } mt_layer_k
  *   MT_CONV3X3          NHWC, stride 1, zero pad 1, cross-correlation; W bf16 [out_ch][3][3][in_ch];
  *                       tap (ky,kx) reads pixel (y+ky-1, x+kx-1)
  *   MT_GLOBAL_AVG_POOL  mean over the h*w positions of each channel; no weights
+ *   MT_CONV1X1          pointwise conv, NHWC: the fully-connected layer applied at every pixel; W bf16 [out_ch][in_ch]
  * residual (MT_CONV3X3 only, the layer before it a conv too): the layer closes a two-layer residual block with an
  * identity shortcut, the building block of the network the paper uses as its running example (Sec. 1.1, resnet18):
  * a[l+1] = act(conv(a[l]) + b + a[l-1]), where a[l-1] is the INPUT of the layer before.  Tenants of one conv family
@@ -88,8 +89,9 @@ mt_status mt_shutdown(void);
  * untouched.  The row stride of the input buffer is the WIDEST registered model's input (mt_input_elems); a request of a
  * model with fewer inputs carries them at the start of its row and the rest of the row is never read.
  * Kernel limits (else MT_ERR_UNSUPPORTED): 1..MT_MAX_LAYERS layers; dense in_ch a multiple of 64;
- * conv in_ch == out_ch == 64, w <= 126; a pool must follow a conv; a dense layer may not precede a conv; residual
- * only on a conv layer that follows a conv layer.
+ * conv3x3 in_ch == out_ch == 64, w <= 126; conv1x1 in_ch a multiple of 64, between two conv layers (it follows a conv3x3
+ * or conv1x1 and is followed by one); a pool must follow a conv3x3; a dense layer may not precede a conv; residual only
+ * on a conv3x3 layer that follows a conv3x3 layer.
  * The call does not wait for the device: weights and biases in HOST memory are copied into the library's pinned
  * staging before it returns (the caller may free them at once), and the copy to the device and the re-layout run on
  * an internal stream, under whatever batches are in flight; the first mt_infer* / mt_prefetch that follows waits, on

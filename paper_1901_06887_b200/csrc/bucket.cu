@@ -21,9 +21,10 @@
 namespace mt {
 
 
-// Per layer: columns (v) and rows (m) of one dense work item, and the layer's kind (the same for every tenant of the
-// hosted family).
-struct LayerTileN { int v[8]; int m[8]; int kind[8]; };
+// Per layer: columns (v) and rows (m) of one dense work item, the layer's kind (the same for every tenant of the
+// hosted family) and, for dense layers, the matrix rows one request contributes (scale: 1, or H * W when the layer is a
+// pointwise conv, i.e. the dense layer applied at every pixel of the request's image).
+struct LayerTileN { int v[8]; int m[8]; int kind[8]; int scale[8]; };
 
 // Compact copy of what the bucketing passes need from the tenant table, one row of `ld` ints per field: row 0 =
 // alive flag, row 1 + l = out features of layer l.  (Reading these through the 328-byte ModelDev records costs one
@@ -130,14 +131,14 @@ __device__ __forceinline__ LayerHead load_head(Brief br, const LayerTileN& tn, i
     return h;
 }
 // Work units (tiles / strips) a tenant with c requests contributes to a layer.
-__device__ __forceinline__ int units_of(LayerHead h, int c, int rows_per_unit, int tile_n, int tile_m) {
+__device__ __forceinline__ int units_of(LayerHead h, int c, int rows_per_unit, int tile_n, int tile_m, int scale) {
     if (c <= 0) return 0;
-    if (h.kind == MT_DENSE) return ((c + tile_m - 1) / tile_m) * ((h.N + tile_n - 1) / tile_n);
+    if (h.kind == MT_DENSE) return ((c * scale + tile_m - 1) / tile_m) * ((h.N + tile_n - 1) / tile_n);
     if (h.kind == MT_CONV3X3) return ((c + tile_m - 1) / tile_m) * rows_per_unit;   // tile_m = images per unit
     return 0;
 }
 __device__ __forceinline__ int layer_units(Brief br, const LayerTileN& tn, int t, int l, int c, int rows_per_unit) {
-    return units_of(load_head(br, tn, t, l), c, rows_per_unit, tn.v[l], tn.m[l]);
+    return units_of(load_head(br, tn, t, l), c, rows_per_unit, tn.v[l], tn.m[l], tn.scale[l]);
 }
 
 // Offsets (exclusive scan of counts over the T + 1 buckets, offsets[T + 1] = n) and, per layer, the prefix sums of
@@ -174,7 +175,7 @@ __device__ __forceinline__ void scan_buckets(int T, Brief br, int n_layers, int 
         int units[MT_MAX_LAYERS];
 #pragma unroll
         for (int l = 0; l < MT_MAX_LAYERS; ++l)
-            units[l] = (l < n_layers && lo < hi_t) ? units_of(head[l], cnt[t_l[l]], rows_per_unit, tn.v[l], tn.m[l]) : 0;
+            units[l] = (l < n_layers && lo < hi_t) ? units_of(head[l], cnt[t_l[l]], rows_per_unit, tn.v[l], tn.m[l], tn.scale[l]) : 0;
         int urun[MT_MAX_LAYERS], utotal[MT_MAX_LAYERS];
         cta_excl_scan_vec(units, urun, utotal, s_vec, n_layers);
 #pragma unroll
@@ -269,7 +270,7 @@ struct ItemPtrs { WorkItem* v[8]; };
 // Work item `item` of dense layer l: (tenant, row tile, column tile) and what the executor needs to know about it.
 __device__ __forceinline__ WorkItem make_work_item(int item, int l, int T, const ModelDev* __restrict__ models,
                                                    const int32_t* order_row, const int32_t* __restrict__ offsets,
-                                                   const int32_t* __restrict__ prefix, int tile_m) {
+                                                   const int32_t* __restrict__ prefix, int tile_m, int row_scale) {
     int lo = 0, hi = T;   // largest rank r with prefix[r] <= item
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
@@ -277,7 +278,7 @@ __device__ __forceinline__ WorkItem make_work_item(int item, int l, int T, const
     }
     const int t = order_row[lo];               // lo is a rank in the layer's cost order
     const LayerDev& L = models[t].layer[l];
-    const int seg0 = offsets[t], n_t = offsets[t + 1] - seg0;
+    const int seg0 = offsets[t] * row_scale, n_t = (offsets[t + 1] - offsets[t]) * row_scale;   // matrix rows of the tenant
     const int m_tiles = (n_t + tile_m - 1) / tile_m;
     const int local = item - prefix[lo];
     // Order of a tenant's items: column tiles in groups of kColGroup, inside a group row tile by row tile.  Items in
@@ -364,7 +365,7 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
             int units[MT_MAX_LAYERS];
 #pragma unroll
             for (int l = 0; l < MT_MAX_LAYERS; ++l)
-                units[l] = (l < n_layers && lo < hi_t) ? units_of(head[l], s_cnt[t_l[l]], rows_per_unit, tn.v[l], tn.m[l]) : 0;
+                units[l] = (l < n_layers && lo < hi_t) ? units_of(head[l], s_cnt[t_l[l]], rows_per_unit, tn.v[l], tn.m[l], tn.scale[l]) : 0;
             int urun[MT_MAX_LAYERS], utotal[MT_MAX_LAYERS];
             cta_excl_scan_vec(units, urun, utotal, s_vec, n_layers);
 #pragma unroll
@@ -422,7 +423,7 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
         for (int t = threadIdx.x; t < T1; t += nthr) s_cnt[t] = prefix[t];
         __syncthreads();
         const int n_items = s_cnt[T];
-        for (int item = threadIdx.x; item < n_items; item += nthr) out[item] = make_work_item(item, l, T, models, br.order + (size_t)l * br.ld, offsets, s_cnt, tn.m[l]);
+        for (int item = threadIdx.x; item < n_items; item += nthr) out[item] = make_work_item(item, l, T, models, br.order + (size_t)l * br.ld, offsets, s_cnt, tn.m[l], tn.scale[l]);
         __syncthreads();
     }
 }
@@ -542,7 +543,7 @@ bucket_scatter_expand(const int32_t* __restrict__ ids, int n, int T, const Model
             const int first = blockIdx.x * blockDim.x + threadIdx.x, stride = gridDim.x * blockDim.x;
             int g = first + ((done > first) ? ((done - first + stride - 1) / stride) * stride : 0);
             for (; g < done + total; g += stride)
-                out[g - done] = make_work_item(g - done, l, T, models, row + T1, offsets, row, tn.m[l]);
+                out[g - done] = make_work_item(g - done, l, T, models, row + T1, offsets, row, tn.m[l], tn.scale[l]);
             done += total;
             ++q;
         }
@@ -556,7 +557,7 @@ bucket_scatter_expand(const int32_t* __restrict__ ids, int n, int T, const Model
         __syncthreads();
         const int total = s_next[T];
         for (int item = blockIdx.x * blockDim.x + threadIdx.x; item < total; item += gridDim.x * blockDim.x)
-            out[item] = make_work_item(item, l, T, models, br.order + (size_t)l * br.ld, offsets, s_next, tn.m[l]);
+            out[item] = make_work_item(item, l, T, models, br.order + (size_t)l * br.ld, offsets, s_next, tn.m[l], tn.scale[l]);
         __syncthreads();
     }
 }
@@ -624,13 +625,16 @@ void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
     const int n_hist_blocks = (a.n + kHistChunk - 1) / kHistChunk;
     const size_t smem = sizeof(int32_t) * (size_t)(a.T + 1);
     LayerTileN tn;
-    for (int l = 0; l < 8; ++l) { tn.v[l] = a.tile_n[l] > 0 ? a.tile_n[l] : BN; tn.m[l] = a.tile_m[l] > 0 ? a.tile_m[l] : BM; tn.kind[l] = a.kind[l]; }
+    for (int l = 0; l < 8; ++l) { tn.v[l] = a.tile_n[l] > 0 ? a.tile_n[l] : BN; tn.m[l] = a.tile_m[l] > 0 ? a.tile_m[l] : BM; tn.kind[l] = a.kind[l]; tn.scale[l] = a.row_scale[l] > 0 ? a.row_scale[l] : 1; }
     Brief br{a.brief, a.brief_ld, a.order};
     ItemPtrs ip;
     for (int l = 0; l < 8; ++l) ip.v[l] = a.items[l];
     // measured: one CTA wins up to a few hundred requests; beyond that its serial scatter and the item expansion
     // by a single CTA cost more than the extra launches of the multi-CTA path
-    if (a.n <= 512 && a.T + 1 <= 4096) {
+    // (a pointwise conv multiplies the rows, and with them the work items one CTA would have to expand)
+    int max_scale = 1;
+    for (int l = 0; l < 8; ++l) if (a.row_scale[l] > max_scale) max_scale = a.row_scale[l];
+    if (a.n <= 512 && a.T + 1 <= 4096 && (long long)a.n * max_scale <= 8192) {
         const int threads = (a.n <= 256) ? 256 : 1024;
         launch_pdl(bucket_single_cta, dim3(1), dim3(threads), 2 * smem, s, a.ids, a.n, a.T, a.models, br, a.n_layers, a.rows_per_unit, tn, a.counts,
                                                       a.offsets, a.tile_prefix, a.perm, a.inv, ip, a.status, a.grid_bar);

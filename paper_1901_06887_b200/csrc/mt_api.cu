@@ -28,8 +28,10 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// kind is the EXECUTOR's kind: a pointwise conv (MT_CONV1X1 at the interface) is a dense layer over the pixels of the
+// request's image, i.e. MT_DENSE with hw = H * W matrix rows per request (hw = 1 for a fully-connected layer).
 struct HostLayer {
-    int kind, in_ch, out_ch, h, w, relu, residual;
+    int kind, in_ch, out_ch, h, w, relu, residual, hw;
 };
 
 struct HostModel {
@@ -362,14 +364,21 @@ mt_status ensure_workspace(int n) {
     for (int b = 0; b < L; ++b) {
         const HostLayer& f = g.family[b];
         if (f.kind == MT_DENSE) {
+            // rows: one per request, or one per pixel of every request's image (pointwise conv)
+            const size_t rows = (size_t)cap * f.hw;
+            if (rows > (size_t)INT_MAX) return MT_ERR_UNSUPPORTED;
             g.act_ld[b] = g.width[b];
-            const size_t bytes = (size_t)cap * g.act_ld[b] * 2;
+            const size_t bytes = rows * g.act_ld[b] * 2;
             CU_OK(cudaMalloc(&g.act[b], bytes));
             CU_OK(cudaMemset(g.act[b], 0, bytes));
-            mt_status st = encode_2d(&g.act_map[b], g.act[b], g.act_ld[b], cap);
+            mt_status st = encode_2d(&g.act_map[b], g.act[b], g.act_ld[b], (int)rows);
             if (st != MT_OK) return st;
-            st = encode_2d(&g.act_map32[b], g.act[b], g.act_ld[b], cap, 32);
+            st = encode_2d(&g.act_map32[b], g.act[b], g.act_ld[b], (int)rows, 32);
             if (st != MT_OK) return st;
+            if (b > 0 && g.family[b - 1].kind == MT_CONV3X3) {      // a conv3x3 stores its 64-channel pixels here
+                st = encode_nhwc(&g.act_store_map[b], g.act[b], f.in_ch, f.w, f.h, cap, 32, 1, 32);
+                if (st != MT_OK) return st;
+            }
         } else {
             g.act_ld[b] = f.in_ch * f.h * f.w;
             if (b == 0) continue;   // the first conv layer reads the caller's buffer through perm
@@ -396,9 +405,10 @@ mt_status ensure_workspace(int n) {
     // work items of the dense layers: at most (row tiles + one ragged tile per tenant) x column tiles of the widest model
     for (int l = 0; l < L; ++l) {
         if (g.family[l].kind != MT_DENSE) continue;
-        const int out_w = std::max((l + 1 < L) ? g.width[l + 1] : 0, g.out_elems);   // hidden, or some tenant's last layer
+        int out_w = std::max((l + 1 < L) ? g.width[l + 1] : 0, g.out_elems);   // hidden, or some tenant's last layer
+        if (l + 1 < L && g.family[l + 1].kind != MT_DENSE) out_w = g.family[l + 1].in_ch;   // pointwise conv in front of a conv3x3
         const size_t col_tiles = (size_t)(out_w + BN - 1) / BN;    // bound for either tile width
-        g.items_cap[l] = ((size_t)cap / BM + (size_t)g.max_models + 1) * col_tiles;
+        g.items_cap[l] = ((size_t)cap * g.family[l].hw / BM + (size_t)g.max_models + 1) * col_tiles;
         CU_OK(cudaMalloc(&g.d_items[l], sizeof(WorkItem) * g.items_cap[l]));
     }
     g.cap_n = cap;
@@ -640,7 +650,7 @@ mt_status validate_layers(const mt_layer_desc* layers, int n_layers) {
     if (!layers || n_layers < 1 || n_layers > MT_MAX_LAYERS) return n_layers > MT_MAX_LAYERS ? MT_ERR_UNSUPPORTED : MT_ERR_INVALID_ARG;
     for (int l = 0; l < n_layers; ++l) {
         const mt_layer_desc& d = layers[l];
-        if (d.kind < MT_DENSE || d.kind > MT_GLOBAL_AVG_POOL) return MT_ERR_INVALID_ARG;
+        if (d.kind < MT_DENSE || d.kind > MT_CONV1X1) return MT_ERR_INVALID_ARG;
         if (d.in_ch <= 0 || d.out_ch <= 0) return MT_ERR_INVALID_ARG;
         if (d.kind != MT_GLOBAL_AVG_POOL && !d.weight) return MT_ERR_INVALID_ARG;
         // an identity shortcut joins a conv layer's output with the input of the conv layer before it
@@ -648,15 +658,27 @@ mt_status validate_layers(const mt_layer_desc* layers, int n_layers) {
         if (d.kind == MT_DENSE) {
             if (l > 0) {
                 const mt_layer_desc& p = layers[l - 1];
-                if (p.kind == MT_CONV3X3) return MT_ERR_UNSUPPORTED;   // needs a pool in between
+                if (p.kind == MT_CONV3X3 || p.kind == MT_CONV1X1) return MT_ERR_UNSUPPORTED;   // needs a pool in between
                 if (p.out_ch != d.in_ch) return MT_ERR_SHAPE;
             }
             if (d.in_ch % BK != 0) return MT_ERR_UNSUPPORTED;
+        } else if (d.kind == MT_CONV1X1) {
+            // the dense executor over the pixels of the image: it reads an activation tensor in bucketed order, so it
+            // follows a conv layer, and what follows it reads 64-channel (conv3x3) or 64-multiple (conv1x1) pixels
+            if (d.h <= 0 || d.w <= 0) return MT_ERR_INVALID_ARG;
+            if (l == 0 || l + 1 >= n_layers) return MT_ERR_UNSUPPORTED;
+            const mt_layer_desc& p = layers[l - 1];
+            if (p.kind != MT_CONV3X3 && p.kind != MT_CONV1X1) return MT_ERR_UNSUPPORTED;
+            if (p.out_ch != d.in_ch || p.h != d.h || p.w != d.w) return MT_ERR_SHAPE;
+            if (d.in_ch % BK != 0) return MT_ERR_UNSUPPORTED;
+            const int next = layers[l + 1].kind;
+            if (next != MT_CONV3X3 && next != MT_CONV1X1) return MT_ERR_UNSUPPORTED;   // the pool is fused into a conv3x3 only
         } else {
             if (d.h <= 0 || d.w <= 0) return MT_ERR_INVALID_ARG;
             if (l > 0) {
                 const mt_layer_desc& p = layers[l - 1];
-                if (p.kind != MT_CONV3X3) return MT_ERR_UNSUPPORTED;    // conv/pool only after a conv
+                // conv/pool only after a conv; the pool only after a conv3x3, whose epilogue does the summing
+                if (p.kind != MT_CONV3X3 && !(p.kind == MT_CONV1X1 && d.kind == MT_CONV3X3)) return MT_ERR_UNSUPPORTED;
                 if (p.out_ch != d.in_ch || p.h != d.h || p.w != d.w) return MT_ERR_SHAPE;
             } else if (d.kind == MT_GLOBAL_AVG_POOL) {
                 return MT_ERR_UNSUPPORTED;
@@ -671,9 +693,9 @@ mt_status validate_layers(const mt_layer_desc* layers, int n_layers) {
 
 int layer_in_elems(const HostLayer& l) { return l.kind == MT_DENSE ? l.in_ch : l.in_ch * l.h * l.w; }
 
-bool all_dense(const std::vector<HostLayer>& m) {
+bool all_dense(const std::vector<HostLayer>& m) {     // an MLP: fully-connected layers only
     for (const HostLayer& l : m)
-        if (l.kind != MT_DENSE) return false;
+        if (l.kind != MT_DENSE || l.hw != 1) return false;
     return true;
 }
 
@@ -690,7 +712,7 @@ mt_status check_family(const std::vector<HostLayer>& m) {
     if (m.size() != g.family.size()) return MT_ERR_SHAPE;
     for (size_t l = 0; l < m.size(); ++l) {
         const HostLayer &a = m[l], &f = g.family[l];
-        if (a.kind != f.kind) return MT_ERR_SHAPE;
+        if (a.kind != f.kind || a.hw != f.hw) return MT_ERR_SHAPE;
         if (a.kind != MT_DENSE && (a.in_ch != f.in_ch || a.out_ch != f.out_ch || a.h != f.h || a.w != f.w)) return MT_ERR_SHAPE;
     }
     return MT_OK;
@@ -850,6 +872,7 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             if (pool_head && l == L - 1) a.items[l] = nullptr;     // the pool + head launch needs no work items
         }
         a.item_grid = g.sm_count;
+        for (int l = 0; l < 8; ++l) a.row_scale[l] = (l < L && g.family[l].kind == MT_DENSE) ? g.family[l].hw : 1;
         a.block_hist = g.d_block_hist; a.counts = g.d_counts; a.offsets = g.d_offsets; a.tile_prefix = g.d_tile_prefix;
         a.perm = g.d_perm; a.inv = g.d_inv; a.status = g.d_status;
         launch_bucketing(a, s);
@@ -895,7 +918,8 @@ mt_status infer_device(const void* inputs, const int32_t* ids, int n, void* outp
             // a tenant's last layer (any launch, for a family of mixed depths) writes straight into the caller's buffer in
             // arrival order; the family's deepest launch also fills the rows of rejected requests
             a.out = last ? nullptr : g.act[l + 1];
-            a.ld_out = last ? 0 : g.act_ld[l + 1];
+            // (a pointwise conv in front of a conv3x3 writes that layer's 64-channel pixels)
+            a.ld_out = last ? 0 : (g.family[l + 1].kind == MT_DENSE ? g.act_ld[l + 1] : g.family[l + 1].in_ch);
             a.final_out = static_cast<float*>(outputs);
             a.ld_final = g.out_elems;
             a.nan_fill = last ? 1 : 0;
@@ -1241,9 +1265,11 @@ mt_status mt_register_model(const mt_layer_desc* layers, int32_t n_layers, int32
     }
     CU_OK(cudaSetDevice(g.device));
     std::vector<HostLayer> hl(n_layers);
-    for (int l = 0; l < n_layers; ++l)
+    for (int l = 0; l < n_layers; ++l) {
         hl[l] = {layers[l].kind, layers[l].in_ch, layers[l].out_ch, layers[l].h, layers[l].w, layers[l].relu ? 1 : 0,
-                 layers[l].residual ? 1 : 0};
+                 layers[l].residual ? 1 : 0, 1};
+        if (layers[l].kind == MT_CONV1X1) { hl[l].kind = MT_DENSE; hl[l].hw = layers[l].h * layers[l].w; }
+    }
     st = check_family(hl);
     if (st != MT_OK) return st;
     int id = -1;

@@ -49,6 +49,7 @@ struct BucketArgs {
     int tile_n[8];            // dense: output columns per work item of each layer (128 or 256)
     int tile_m[8];            // dense: rows per work item of each layer (128, or 256 for the CTA-pair executor);
                               // conv: images per work unit (1, or 2 for the CTA-pair executor)
+    int row_scale[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // dense: matrix rows per request (0 or 1: one; H * W for a pointwise conv)
     int32_t* block_hist;      // [ceil(n / kHistChunk)][T + 1]
     int32_t* counts;          // [T + 1]
     int32_t* offsets;         // [T + 2]
