@@ -24,7 +24,7 @@ namespace mt {
 // Per layer: columns (v) and rows (m) of one dense work item, the layer's kind (the same for every tenant of the
 // hosted family) and, for dense layers, the matrix rows one request contributes (scale: 1, or H * W when the layer is a
 // pointwise conv, i.e. the dense layer applied at every pixel of the request's image).
-struct LayerTileN { int v[8]; int m[8]; int kind[8]; int scale[8]; };
+struct LayerTileN { int v[8]; int m[8]; int kind[8]; };   // kind[l]: layer kind in the low byte, row scale above it
 
 // Compact copy of what the bucketing passes need from the tenant table, one row of `ld` ints per field: row 0 =
 // alive flag, row 1 + l = out features of layer l.  (Reading these through the 328-byte ModelDev records costs one
@@ -126,7 +126,7 @@ __device__ __forceinline__ void cta_excl_scan_vec(const int (&v)[MT_MAX_LAYERS],
 struct LayerHead { int kind, N; };
 __device__ __forceinline__ LayerHead load_head(Brief br, const LayerTileN& tn, int t, int l) {
     LayerHead h;
-    h.kind = tn.kind[l];
+    h.kind = tn.kind[l] & 0xff;
     h.N = __ldg(br.p + (size_t)(1 + l) * br.ld + t);
     return h;
 }
@@ -138,7 +138,7 @@ __device__ __forceinline__ int units_of(LayerHead h, int c, int rows_per_unit, i
     return 0;
 }
 __device__ __forceinline__ int layer_units(Brief br, const LayerTileN& tn, int t, int l, int c, int rows_per_unit) {
-    return units_of(load_head(br, tn, t, l), c, rows_per_unit, tn.v[l], tn.m[l], tn.scale[l]);
+    return units_of(load_head(br, tn, t, l), c, rows_per_unit, tn.v[l], tn.m[l], (tn.kind[l] >> 8));
 }
 
 // Offsets (exclusive scan of counts over the T + 1 buckets, offsets[T + 1] = n) and, per layer, the prefix sums of
@@ -175,7 +175,7 @@ __device__ __forceinline__ void scan_buckets(int T, Brief br, int n_layers, int 
         int units[MT_MAX_LAYERS];
 #pragma unroll
         for (int l = 0; l < MT_MAX_LAYERS; ++l)
-            units[l] = (l < n_layers && lo < hi_t) ? units_of(head[l], cnt[t_l[l]], rows_per_unit, tn.v[l], tn.m[l], tn.scale[l]) : 0;
+            units[l] = (l < n_layers && lo < hi_t) ? units_of(head[l], cnt[t_l[l]], rows_per_unit, tn.v[l], tn.m[l], (tn.kind[l] >> 8)) : 0;
         int urun[MT_MAX_LAYERS], utotal[MT_MAX_LAYERS];
         cta_excl_scan_vec(units, urun, utotal, s_vec, n_layers);
 #pragma unroll
@@ -365,7 +365,7 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
             int units[MT_MAX_LAYERS];
 #pragma unroll
             for (int l = 0; l < MT_MAX_LAYERS; ++l)
-                units[l] = (l < n_layers && lo < hi_t) ? units_of(head[l], s_cnt[t_l[l]], rows_per_unit, tn.v[l], tn.m[l], tn.scale[l]) : 0;
+                units[l] = (l < n_layers && lo < hi_t) ? units_of(head[l], s_cnt[t_l[l]], rows_per_unit, tn.v[l], tn.m[l], (tn.kind[l] >> 8)) : 0;
             int urun[MT_MAX_LAYERS], utotal[MT_MAX_LAYERS];
             cta_excl_scan_vec(units, urun, utotal, s_vec, n_layers);
 #pragma unroll
@@ -423,7 +423,7 @@ bucket_single_cta(const int32_t* __restrict__ ids, int n, int T, const ModelDev*
         for (int t = threadIdx.x; t < T1; t += nthr) s_cnt[t] = prefix[t];
         __syncthreads();
         const int n_items = s_cnt[T];
-        for (int item = threadIdx.x; item < n_items; item += nthr) out[item] = make_work_item(item, l, T, models, br.order + (size_t)l * br.ld, offsets, s_cnt, tn.m[l], tn.scale[l]);
+        for (int item = threadIdx.x; item < n_items; item += nthr) out[item] = make_work_item(item, l, T, models, br.order + (size_t)l * br.ld, offsets, s_cnt, tn.m[l], (tn.kind[l] >> 8));
         __syncthreads();
     }
 }
@@ -543,7 +543,7 @@ bucket_scatter_expand(const int32_t* __restrict__ ids, int n, int T, const Model
             const int first = blockIdx.x * blockDim.x + threadIdx.x, stride = gridDim.x * blockDim.x;
             int g = first + ((done > first) ? ((done - first + stride - 1) / stride) * stride : 0);
             for (; g < done + total; g += stride)
-                out[g - done] = make_work_item(g - done, l, T, models, row + T1, offsets, row, tn.m[l], tn.scale[l]);
+                out[g - done] = make_work_item(g - done, l, T, models, row + T1, offsets, row, tn.m[l], (tn.kind[l] >> 8));
             done += total;
             ++q;
         }
@@ -557,7 +557,7 @@ bucket_scatter_expand(const int32_t* __restrict__ ids, int n, int T, const Model
         __syncthreads();
         const int total = s_next[T];
         for (int item = blockIdx.x * blockDim.x + threadIdx.x; item < total; item += gridDim.x * blockDim.x)
-            out[item] = make_work_item(item, l, T, models, br.order + (size_t)l * br.ld, offsets, s_next, tn.m[l], tn.scale[l]);
+            out[item] = make_work_item(item, l, T, models, br.order + (size_t)l * br.ld, offsets, s_next, tn.m[l], (tn.kind[l] >> 8));
         __syncthreads();
     }
 }
@@ -625,7 +625,7 @@ void launch_bucketing(const BucketArgs& a, cudaStream_t s) {
     const int n_hist_blocks = (a.n + kHistChunk - 1) / kHistChunk;
     const size_t smem = sizeof(int32_t) * (size_t)(a.T + 1);
     LayerTileN tn;
-    for (int l = 0; l < 8; ++l) { tn.v[l] = a.tile_n[l] > 0 ? a.tile_n[l] : BN; tn.m[l] = a.tile_m[l] > 0 ? a.tile_m[l] : BM; tn.kind[l] = a.kind[l]; tn.scale[l] = a.row_scale[l] > 0 ? a.row_scale[l] : 1; }
+    for (int l = 0; l < 8; ++l) { tn.v[l] = a.tile_n[l] > 0 ? a.tile_n[l] : BN; tn.m[l] = a.tile_m[l] > 0 ? a.tile_m[l] : BM; tn.kind[l] = (a.kind[l] & 0xff) | ((a.row_scale[l] > 0 ? a.row_scale[l] : 1) << 8); }
     Brief br{a.brief, a.brief_ld, a.order};
     ItemPtrs ip;
     for (int l = 0; l < 8; ++l) ip.v[l] = a.items[l];
